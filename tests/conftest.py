@@ -1,0 +1,24 @@
+import os
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def pytest_configure(config):
+    config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
+
+
+@pytest.fixture(scope="session")
+def tiny_corpus():
+    from paper_1412_1576_b200 import synth
+    return synth.make("tiny", seed=0)
+
+
+@pytest.fixture(scope="session")
+def small_corpus():
+    from paper_1412_1576_b200 import synth
+    return synth.make("small", seed=0)

@@ -1,0 +1,360 @@
+"""Pins for the oracle's proposals, acceptance ratios, chain, counts and
+log-likelihood against what the paper's equations fix (CPU only)."""
+import math
+
+import numpy as np
+import pytest
+from scipy import stats
+
+from oracle import ldaref
+from paper_1412_1576_b200 import synth
+
+SEED = 1234
+
+
+def _dense_counts(c, z):
+    """Brute-force count tables from assignments (Section 3, Eq. 12)."""
+    w = c.word_ids.numpy()
+    off = c.doc_offsets.numpy()
+    D = off.size - 1
+    doc = np.repeat(np.arange(D), np.diff(off))
+    n_wk = np.zeros((c.V, c.K), np.int64)
+    n_dk = np.zeros((D, c.K), np.int64)
+    np.add.at(n_wk, (w, z), 1)
+    np.add.at(n_dk, (doc, z), 1)
+    return n_wk, n_dk, n_wk.sum(0), doc
+
+
+def _oracle(c, seed=SEED):
+    o = ldaref.Oracle(c.V, c.K, c.alpha, c.beta)
+    o.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    o.init(seed)
+    return o
+
+
+@pytest.fixture(scope="module")
+def tiny(tiny_corpus):
+    o = _oracle(tiny_corpus)
+    o.sweep(3, 2)   # move away from the uniform start so counts are uneven
+    z = o.get_assignments().copy()
+    return tiny_corpus, o, z, _dense_counts(tiny_corpus, z)
+
+
+def _toy(V=12, K=4, D=6, L=8, alpha=0.3, beta=0.2, seed=3):
+    c = synth.generate(V=V, K=K, D=D, length=("fixed", L), zipf_s=None, alpha=alpha, beta=beta,
+                       seed=seed)
+    o = _oracle(c, seed=99)
+    o.sweep(2, 2)
+    z = o.get_assignments().copy()
+    return c, o, z, _dense_counts(c, z)
+
+
+# ---- counts -------------------------------------------------------------------
+
+def test_counts_match_brute_force_and_invariants(tiny):
+    c, o, z, (n_wk, n_dk, n_k, doc) = tiny
+    assert np.array_equal(o.get_nk(), n_k)
+    off, top, cnt = o.get_csr(ldaref.NWK)
+    dense = np.zeros_like(n_wk)
+    for w in range(c.V):
+        seg = slice(off[w], off[w + 1])
+        assert np.all(np.diff(top[seg]) > 0)          # ascending, no duplicates
+        assert np.all(cnt[seg] > 0)
+        dense[w, top[seg]] = cnt[seg]
+    assert np.array_equal(dense, n_wk)
+    offd, topd, cntd = o.get_csr(ldaref.NDK)
+    dense_d = np.zeros_like(n_dk)
+    for d in range(n_dk.shape[0]):
+        seg = slice(offd[d], offd[d + 1])
+        assert np.all(np.diff(topd[seg]) > 0)
+        dense_d[d, topd[seg]] = cntd[seg]
+    assert np.array_equal(dense_d, n_dk)
+    # invariants: sum_k n_dk = n_d ; sum_d n_dk = n_k = sum_w n_wk ; sum_k n_k = N
+    assert np.array_equal(dense_d.sum(1), np.diff(c.doc_offsets.numpy()))
+    assert np.array_equal(dense_d.sum(0), n_k)
+    assert np.array_equal(dense.sum(0), n_k)
+    assert n_k.sum() == c.n_tokens
+
+
+def test_init_is_uniform_and_a_function_of_seed(tiny_corpus):
+    a, b, d = _oracle(tiny_corpus, 5), _oracle(tiny_corpus, 5), _oracle(tiny_corpus, 6)
+    za, zb, zd = a.get_assignments(), b.get_assignments(), d.get_assignments()
+    assert np.array_equal(za, zb) and not np.array_equal(za, zd)
+    assert za.min() >= 0 and za.max() < tiny_corpus.K
+    p = stats.chisquare(np.bincount(za, minlength=tiny_corpus.K)).pvalue
+    assert p > 1e-4
+
+
+# ---- proposals ------------------------------------------------------------------
+
+def _word_proposal_pmf_from_tables(tb, w, K, row_topics):
+    """Exact law of the oracle's word-proposal draw, from its stored tables."""
+    def table_pmf(thr32, alias):
+        n = len(thr32)
+        p = np.zeros(n)
+        for b in range(n):
+            keep = 1.0 if alias[b] == b else thr32[b] / 2.0 ** 32
+            p[b] += keep / n
+            if alias[b] != b:
+                p[alias[b]] += (1 - keep) / n
+        return p
+    lo, hi = tb["row_off"][w], tb["row_off"][w + 1]
+    mix = tb["mix32"][w] / 2.0 ** 32
+    pmf = (1 - mix) * table_pmf(tb["dn_thr32"], tb["dn_alias"])
+    if hi > lo:
+        ps = table_pmf(tb["sp_thr32"][lo:hi], tb["sp_alias"][lo:hi])
+        np.add.at(pmf, row_topics[lo:hi], mix * ps)
+    return pmf
+
+
+def test_word_proposal_tables_give_eq6(tiny):
+    c, o, z, (n_wk, n_dk, n_k, doc) = tiny
+    tb = o.get_tables()
+    _, top, _ = o.get_csr(ldaref.NWK)
+    Vb = c.V * c.beta
+    words = np.argsort(-n_wk.sum(1))[:25]
+    for w in words:
+        q = (n_wk[w] + c.beta) / (n_k + Vb)          # Eq. 6
+        q = q / q.sum()
+        pmf = _word_proposal_pmf_from_tables(tb, w, c.K, top)
+        assert abs(pmf.sum() - 1) < 1e-9
+        assert np.max(np.abs(pmf - q)) < 1e-7
+
+
+def test_word_proposal_draws_chi_square(tiny):
+    c, o, z, (n_wk, n_dk, n_k, doc) = tiny
+    rng = np.random.default_rng(11)
+    Vb = c.V * c.beta
+    n_draw = 100_000
+    for w in np.argsort(-n_wk.sum(1))[[0, 3, 40]]:
+        q = (n_wk[w] + c.beta) / (n_k + Vb)
+        q = q / q.sum()
+        r = rng.integers(0, 2 ** 32, (n_draw, 3))
+        h = np.zeros(c.K)
+        for a, b, cc in r:
+            h[o.word_proposal(int(w), int(a), int(b), int(cc))] += 1
+        keep = q * n_draw >= 5
+        obs = np.append(h[keep], h[~keep].sum())
+        exp = np.append(q[keep], q[~keep].sum()) * n_draw
+        if exp[-1] == 0:
+            obs, exp = obs[:-1], exp[:-1]
+        assert stats.chisquare(obs, exp).pvalue > 1e-4
+
+
+def test_doc_proposal_draws_chi_square(tiny):
+    c, o, z, (n_wk, n_dk, n_k, doc) = tiny
+    rng = np.random.default_rng(12)
+    n_draw = 100_000
+    for d in (0, 17, 133):
+        q = (n_dk[d] + c.alpha) / (n_dk[d].sum() + c.K * c.alpha)   # Eq. 9
+        r = rng.integers(0, 2 ** 32, (n_draw, 2))
+        h = np.zeros(c.K)
+        for a, b in r:
+            h[o.doc_proposal(d, int(a), int(b))] += 1
+        assert stats.chisquare(h, q * n_draw).pvalue > 1e-4
+
+
+def test_doc_proposal_branches():
+    """r0 chooses the term: low values copy z_dj, high values draw a uniform topic."""
+    c, o, z, (n_wk, n_dk, n_k, doc) = _toy()
+    off = c.doc_offsets.numpy()
+    d, n_d = 2, int(off[3] - off[2])
+    for r1 in (0, 2 ** 31, 2 ** 32 - 1):
+        j = (r1 * n_d) >> 32
+        assert o.doc_proposal(d, 0, r1) == z[off[d] + j]
+        assert o.doc_proposal(d, 2 ** 32 - 1, r1) == (r1 * c.K) >> 32
+    # branch boundary: copy iff u*(n_d + K*alpha) < n_d
+    edge = n_d / (n_d + c.K * c.alpha)
+    r_lo, r_hi = int(edge * 2 ** 32) - 2, int(edge * 2 ** 32) + 2
+    assert o.doc_proposal(d, r_lo, 0) == z[off[d]]
+    assert o.doc_proposal(d, r_hi, 0) == 0
+
+
+# ---- acceptance ratios ------------------------------------------------------------
+
+def _target(c, n_wk, n_dk, n_k, w, d, z0):
+    """Eq. 4 with the token's own count removed at z0."""
+    e = np.zeros(c.K)
+    e[z0] = 1
+    return (n_dk[d] - e + c.alpha) * (n_wk[w] - e + c.beta) / (n_k - e + c.V * c.beta)
+
+
+def test_acceptance_ratios_equal_p_q_quotients(tiny):
+    c, o, z, (n_wk, n_dk, n_k, doc) = tiny
+    rng = np.random.default_rng(13)
+    wid = c.word_ids.numpy()
+    Vb = c.V * c.beta
+    for i in rng.integers(0, c.n_tokens, 300):
+        w, d, z0 = wid[i], doc[i], z[i]
+        p = _target(c, n_wk, n_dk, n_k, w, d, z0)
+        qw = (n_wk[w] + c.beta) / (n_k + Vb)        # Eq. 6 (unnormalised)
+        qd = n_dk[d] + c.alpha                      # Eq. 9 (unnormalised)
+        s, t = rng.integers(0, c.K, 2)
+        # the chain only visits states with p(s) > 0; keep s there
+        if p[s] <= 0:
+            s = z0
+        for kind, q in ((0, qw), (1, qd)):
+            num, den = o.accept_ratio(int(i), int(s), int(t), kind)
+            want = p[t] * q[s] / (p[s] * q[t])      # Eq. 7 / Eq. 10
+            assert num / den == pytest.approx(want, rel=1e-11)
+            assert num >= 0 and den > 0
+
+
+# ---- the chain -------------------------------------------------------------------
+
+def _step_matrix(c, o, i, kind, prop_pmf):
+    K = c.K
+    P = np.zeros((K, K))
+    for s in range(K):
+        for t in range(K):
+            if t == s:
+                continue
+            num, den = o.accept_ratio(i, s, t, kind)
+            # accept iff u*den < num, u = r3/2^32 uniform on a 2^-32 grid
+            acc = 1.0 if num >= den else num / den
+            P[s, t] = prop_pmf[t] * acc
+        P[s, s] = 1 - P[s].sum()
+    return P
+
+
+def test_chain_transition_matrices_leave_eq4_invariant():
+    c, o, z, (n_wk, n_dk, n_k, doc) = _toy()
+    tb = o.get_tables()
+    _, top, _ = o.get_csr(ldaref.NWK)
+    wid = c.word_ids.numpy()
+    for i in (0, 7, 19, 33, 47):
+        w, d, z0 = wid[i], doc[i], z[i]
+        p = _target(c, n_wk, n_dk, n_k, w, d, z0)
+        assert np.all(p > 0)       # alpha, beta > 0 and counts >= own contribution
+        pi = p / p.sum()
+        q_word = _word_proposal_pmf_from_tables(tb, w, c.K, top)
+        q_doc = (n_dk[d] + c.alpha) / (n_dk[d].sum() + c.K * c.alpha)
+        for kind, q in ((0, q_word), (1, q_doc)):
+            P = _step_matrix(c, o, i, kind, q)
+            assert np.all(P >= -1e-12)
+            assert np.max(np.abs(pi @ P - pi)) < 1e-7
+            # detailed balance of each MH kernel
+            F = pi[:, None] * P
+            assert np.max(np.abs(F - F.T)) < 1e-7
+
+
+def test_chain_histogram_matches_gibbs_conditional():
+    """Many replicas of one token's chain (different Philox streams) land on Eq. 4."""
+    c, o, z, (n_wk, n_dk, n_k, doc) = _toy(V=10, K=5, D=5, L=10, seed=8)
+    wid = c.word_ids.numpy()
+    n_rep = 40_000
+    for i in (3, 28):
+        p = _target(c, n_wk, n_dk, n_k, wid[i], doc[i], z[i])
+        pi = p / p.sum()
+        h = np.zeros(c.K)
+        for rep in range(n_rep):
+            h[o.chain(i, 1000 + rep, 24)] += 1
+        assert stats.chisquare(h, pi * n_rep).pvalue > 1e-4
+
+
+def test_chain_with_zero_steps_keeps_state_and_one_step_is_word_proposal(tiny):
+    c, o, z, _ = tiny
+    wid = c.word_ids.numpy()
+    key = [SEED & 0xFFFFFFFF, SEED >> 32]
+    for i in (0, 5, 4242):
+        assert o.chain(i, 7, 0) == z[i]
+        r = ldaref.philox([i, 7, 0, 0], key)
+        t = o.word_proposal(int(wid[i]), int(r[0]), int(r[1]), int(r[2]))
+        got = o.chain(i, 7, 1)
+        if t == z[i]:
+            assert got == z[i]
+        else:
+            num, den = o.accept_ratio(i, int(z[i]), t, 0)
+            accept = (int(r[3]) / 2.0 ** 32) * den < num
+            assert got == (t if accept else z[i])
+
+
+def test_sweep_is_frozen_and_order_independent(tiny_corpus):
+    """Sampling tokens one by one from the sweep-start state equals the sweep."""
+    c = tiny_corpus
+    a, b = _oracle(c, 77), _oracle(c, 77)
+    a.sweep(2, 2)
+    b.sweep(1, 2)
+    toks = np.random.default_rng(0).permutation(c.n_tokens)[:3000]
+    picked = b.sample_tokens(toks, 2)
+    b.sweep(1, 2)
+    assert np.array_equal(picked, b.get_assignments()[toks])
+    assert np.array_equal(a.get_assignments(), b.get_assignments())
+    assert a.sweeps_done == 2
+
+
+# ---- log-likelihood -----------------------------------------------------------------
+
+def _sequential_joint(c, z):
+    """log p(w, z) by the chain rule of the two Polya urns (independent of the
+    closed form): p(z_i | earlier z of the doc) p(w_i | earlier (w, z))."""
+    wid = c.word_ids.numpy()
+    off = c.doc_offsets.numpy()
+    n_wk = np.zeros((c.V, c.K))
+    n_k = np.zeros(c.K)
+    lw = ld = 0.0
+    for d in range(off.size - 1):
+        n_dk = np.zeros(c.K)
+        for j, i in enumerate(range(off[d], off[d + 1])):
+            k, w = z[i], wid[i]
+            ld += math.log((n_dk[k] + c.alpha) / (j + c.K * c.alpha))
+            lw += math.log((n_wk[w, k] + c.beta) / (n_k[k] + c.V * c.beta))
+            n_dk[k] += 1
+            n_wk[w, k] += 1
+            n_k[k] += 1
+    return lw, ld
+
+
+def test_loglik_equals_sequential_urn_probability(tiny):
+    c, o, z, _ = tiny
+    total, lw, ld = o.loglik()
+    sw, sd = _sequential_joint(c, z)
+    assert lw == pytest.approx(sw, rel=1e-10)
+    assert ld == pytest.approx(sd, rel=1e-10)
+    assert total == pytest.approx(sw + sd, rel=1e-10)
+
+
+def test_loglik_single_topic_closed_form():
+    c = synth.generate(V=30, K=1, D=7, length=("fixed", 9), zipf_s=None, alpha=0.4, beta=0.05,
+                       seed=2)
+    o = _oracle(c)
+    total, lw, ld = o.loglik()
+    tf = np.bincount(c.word_ids.numpy(), minlength=c.V)
+    N = c.n_tokens
+    want_w = math.lgamma(c.V * c.beta) - math.lgamma(N + c.V * c.beta) + sum(
+        math.lgamma(n + c.beta) - math.lgamma(c.beta) for n in tf)
+    assert lw == pytest.approx(want_w, rel=1e-12)
+    assert ld == pytest.approx(0.0, abs=1e-9)     # one topic: p(z) = 1
+
+
+# ---- behaviour over sweeps (trend only) ------------------------------------------------
+
+def test_loglik_rises_towards_sequential_gibbs_level(tiny_corpus):
+    """The paper's claim is qualitative (cycle proposal close to Gibbs per
+    iteration); no number is printed, so this checks trend only."""
+    c = tiny_corpus
+    o = _oracle(c, 3)
+    ll0 = o.loglik()[0]
+    o.sweep(100, 2)     # frozen counts and two proposals per sweep mix more slowly per sweep
+    ll_mh = o.loglik()[0]
+    assert ll_mh > ll0 + 0.15 * abs(ll0)
+    # sequential collapsed Gibbs (Eq. 1), plain numpy
+    rng = np.random.default_rng(0)
+    wid = c.word_ids.numpy()
+    z = ldaref.Oracle(c.V, c.K, c.alpha, c.beta)
+    z.load_corpus(wid, c.doc_offsets.numpy())
+    z.init(3)
+    zz = z.get_assignments().copy()
+    n_wk, n_dk, n_k, doc = _dense_counts(c, zz)
+    n_wk, n_dk, n_k = n_wk.astype(float), n_dk.astype(float), n_k.astype(float)
+    for _ in range(30):
+        for i in range(c.n_tokens):
+            w, d, k = wid[i], doc[i], zz[i]
+            n_wk[w, k] -= 1; n_dk[d, k] -= 1; n_k[k] -= 1
+            p = (n_dk[d] + c.alpha) * (n_wk[w] + c.beta) / (n_k + c.V * c.beta)
+            k = rng.choice(c.K, p=p / p.sum())
+            zz[i] = k
+            n_wk[w, k] += 1; n_dk[d, k] += 1; n_k[k] += 1
+    z.set_assignments(zz, 3)
+    ll_gibbs = z.loglik()[0]
+    assert abs(ll_mh - ll_gibbs) < 0.05 * abs(ll_gibbs)
