@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the frozen-counts LightLDA sweep on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+A "step" is one whole sweep (alias tables, token MH kernel, count rebuild) over
+a synthetic corpus of the chosen workload.  Prints ONE JSON line on rank 0.
+``--impl reference`` times the CPU oracle instead (rank 0 only).
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "sampled tokens/sec per sweep"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=["tiny", "small", "mid", "large", "big"])
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the number of documents")
+    ap.add_argument("--mh-steps", type=int, default=2)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    return ap.parse_args()
+
+
+def hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.gpu)],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        try:
+            for ln in open(self.path):
+                f = [x.strip() for x in ln.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), f[5:9]):
+                    if val.lower() == "active":
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def workload_config(args):
+    from paper_1412_1576_b200 import synth
+    cfg = dict(synth.CONFIGS[args.workload])
+    cfg["D"] = max(1, int(round(cfg["D"] * args.scale)))
+    return cfg
+
+
+def algorithmic_bytes_per_token_sample(mh_steps: int, topic_bytes: int, rho_wk: float) -> float:
+    """Bytes the token MH kernel must move per token: streamed token record
+    (doc id, token id, z in, z out in both layouts), the doc-proposal's z reads,
+    one n_kd entry per lookup (own topic + one per proposal), and the word's row
+    and alias entries once per nonzero."""
+    T = topic_bytes
+    return 8 + 3 * T + T * (mh_steps // 2) + 4 * (mh_steps + 1) + 16.0 * rho_wk
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_1412_1576_b200 import binding, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    cfg = workload_config(args)
+    M = args.mh_steps
+    # independent replicas: every rank draws its own corpus of the same shape
+    t0 = time.time()
+    corpus = synth.generate(seed=args.seed + rank, device="cuda", **cfg)
+    torch.cuda.synchronize()
+    gen_s = time.time() - t0
+    N, D = corpus.n_tokens, corpus.n_docs
+    stream = torch.cuda.current_stream()
+    lda = binding.LightLDA(cfg["V"], cfg["K"], cfg["alpha"], cfg["beta"], stream=stream.cuda_stream)
+    torch.cuda.empty_cache()
+    t0 = time.time()
+    lda.load_corpus(corpus.word_ids, corpus.doc_offsets)
+    load_s = time.time() - t0
+    gen_stats = corpus.stats
+    del corpus
+    torch.cuda.empty_cache()
+    lda.init(1234 + rank)
+
+    for _ in range(args.warmup):
+        lda.sweep(1, M)
+    st0 = lda.stats()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    phases = dict(ms_alias_dense=0.0, ms_alias_sparse=0.0, ms_sample=0.0, ms_count_wk=0.0,
+                  ms_count_k=0.0, ms_count_dk=0.0, ms_total=0.0)
+    launches = 0
+    rho_sum = 0.0
+    barrier()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        lda.sweep(1, M)
+        s = lda._h and binding.lda_get_stats(lda._h)[1]
+        for k in phases:
+            phases[k] += getattr(s, k)
+        launches += s.kernel_launches
+        rho_sum += s.nnz_wk / max(N, 1)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        tot = torch.tensor([float(N)], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+        total_tokens = float(tot.item())
+    else:
+        total_tokens = float(N)
+    ms_per_step = ms / args.steps
+    value = total_tokens / (ms_per_step * 1e-3)
+    st1 = lda.stats()
+
+    # --- end to end through the host-buffer entry points -----------------------------------
+    e2e = None
+    if not args.no_e2e and args.e2e_steps > 0:
+        z_host = torch.empty(N, dtype=torch.int32).pin_memory()
+        binding.lda_get_assignments_ptr(lda._h, z_host.data_ptr())
+        barrier()
+        t0 = time.perf_counter()
+        ev0.record(stream)
+        ll = None
+        for i in range(args.e2e_steps):
+            rc = binding.lda_set_assignments_ptr(lda._h, z_host.data_ptr(), 1234 + rank,
+                                                 st1["sweeps_done"] + i)
+            assert rc == 0, binding.lda_last_error(lda._h)
+            lda.sweep(1, M)
+            rc = binding.lda_get_assignments_ptr(lda._h, z_host.data_ptr())
+            assert rc == 0
+            ll = lda.loglik()
+        ev1.record(stream)
+        barrier()
+        e_ms = ev0.elapsed_time(ev1)
+        wall_ms = (time.perf_counter() - t0) * 1e3
+        e_ms = max(e_ms, wall_ms)   # host-side work between calls counts too
+        if dist is not None:
+            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": total_tokens / (e_ms / args.e2e_steps * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": 4 * N, "d2h_bytes_per_step": 4 * N + 24,
+               "steps": args.e2e_steps, "loglik": ll[0] if ll else None,
+               "what": "lda_set_assignments(host z) + lda_sweep(1) + lda_get_assignments(host z) + lda_loglik"}
+        del z_host
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = hbm_peak()
+    topic_bytes = 4 if cfg["K"] > 65536 else 2
+    rho = rho_sum / args.steps
+    b_alg = algorithmic_bytes_per_token_sample(M, topic_bytes, rho)
+    sample_ms = phases["ms_sample"] / args.steps
+    achieved = b_alg * N / (sample_ms * 1e-3) / 1e9 if sample_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "k_sample", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                "algorithmic_bytes_per_token": b_alg, "avg_launch_ms": sample_ms,
+                "share_of_step": sample_ms / ms_per_step if ms_per_step else None}
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        try:
+            tr = json.load(open(prof)).get("k_sample", {})
+            if tr.get("workload") == args.workload and tr.get("mh_steps") == M:
+                roofline["traffic"] = tr["dram_bytes_per_token"] * N
+                roofline["traffic_source"] = tr.get("source")
+        except Exception:
+            pass
+
+    cpu = None
+    if not args.no_cpu:
+        cpu = cpu_baseline(args, args.cpu_seconds)
+
+    line = {
+        "metric": f"{METRIC} (mh_steps={M})", "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"{args.workload} LDA" + (f" x{args.scale}" if args.scale != 1.0 else ""),
+                   "V": cfg["V"], "K": cfg["K"], "D": D, "n_tokens": N, "mh_steps": M,
+                   "alpha": cfg["alpha"], "beta": cfg["beta"], "topic_bytes": topic_bytes,
+                   "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "l2": "inputs larger than L2" if N * 14 > 126e6 else "inputs fit in L2",
+                   "sweeps_timed": [st0["sweeps_done"], st0["sweeps_done"] + args.steps],
+                   "top10pct_vocab_token_share": gen_stats["top10pct_vocab_token_share"]},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+        "cpu_baseline": cpu,
+        "phases_ms_per_step": {k: v / args.steps for k, v in phases.items()},
+        "state": {"nnz_wk": st1["nnz_wk"], "nnz_dk": st1["nnz_dk"], "dense_words": st1["n_dense_words"],
+                  "device_bytes": st1["device_bytes"], "generate_s": gen_s, "load_s": load_s},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def _oracle_setup(args, scale_cap_tokens=40e6):
+    """The oracle on a bounded sample of the workload: the same generator with
+    fewer documents (same V, K, length law, priors)."""
+    from oracle import ldaref
+    from paper_1412_1576_b200 import synth
+    cfg = workload_config(args)
+    avg_len = {"fixed": lambda l: l[1], "poisson": lambda l: l[1], "lognormal": lambda l: l[1]}[cfg["length"][0]](cfg["length"])
+    d_cap = max(1, int(scale_cap_tokens / max(avg_len, 1)))
+    sample_scale = 1.0
+    if cfg["D"] > d_cap:
+        sample_scale = d_cap / cfg["D"]
+        cfg["D"] = d_cap
+    c = synth.generate(seed=args.seed, device="cpu", **cfg)
+    o = ldaref.Oracle(c.V, c.K, c.alpha, c.beta)
+    o.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    o.init(1234)
+    return o, c, sample_scale
+
+
+def cpu_baseline(args, seconds):
+    o, c, sample_scale = _oracle_setup(args)
+    M = args.mh_steps
+    n = min(c.n_tokens, 200_000)
+    t0 = time.perf_counter(); o.sweep_prefix(n, M); dt = time.perf_counter() - t0
+    n2 = int(min(c.n_tokens, max(n, n / max(dt, 1e-6) * seconds)))
+    t0 = time.perf_counter(); o.sweep_prefix(n2, M); dt = time.perf_counter() - t0
+    return {"value": n2 / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {n2} tokens of one sweep (tables already built) on the same generator "
+                      f"with {c.n_docs} documents ({c.n_tokens} tokens), mh_steps={M}"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    o, c, sample_scale = _oracle_setup(args, scale_cap_tokens=20e6)
+    M = args.mh_steps
+    n = min(c.n_tokens, 100_000)
+    t0 = time.perf_counter(); o.sweep_prefix(n, M); dt = time.perf_counter() - t0
+    budget = 60.0 / max(1, args.steps + args.warmup)
+    n_step = int(min(c.n_tokens, max(1000, n / max(dt, 1e-6) * budget)))
+    for _ in range(args.warmup):
+        o.sweep_prefix(n_step, M)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        o.sweep_prefix(n_step, M)
+    dt = time.perf_counter() - t0
+    value = n_step * args.steps / dt
+    sample = (f"each step = first {n_step} tokens of one oracle sweep on the same generator with "
+              f"{c.n_docs} documents ({c.n_tokens} tokens), mh_steps={M}")
+    cfg = workload_config(args)
+    line = {
+        "impl": "reference", "metric": f"{METRIC} (mh_steps={M})", "value": value, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload} LDA" + (f" x{args.scale}" if args.scale != 1.0 else ""),
+                   "V": cfg["V"], "K": cfg["K"], "mh_steps": M, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -1,0 +1,135 @@
+/*
+ * lda_b200.h -- C ABI of the B200 (sm_100a) LightLDA sweep library.
+ *
+ * The library runs the data-parallel hot path of the LightLDA sampler on one
+ * GPU: per sweep it rebuilds the word-proposal alias tables from the counts
+ * frozen at sweep start, runs `mh_steps` Metropolis-Hastings proposals per
+ * token (word-proposal on even steps, doc-proposal on odd steps) and rebuilds
+ * the count tables n_kw, n_k, n_kd from the new assignments.
+ *
+ * Conventions
+ *   - every function returns an int status: LDA_OK or a negative LDA_E* code;
+ *     nothing throws, exits or prints.  lda_last_error() gives a message.
+ *   - pointers are HOST pointers unless the parameter says DEVICE.
+ *   - the caller owns every buffer it passes; inputs are copied, so they may
+ *     be freed once the call returns.  The context owns all device memory it
+ *     allocates and frees it in lda_destroy().
+ *   - a context is bound to the CUDA device that is current in lda_create()
+ *     and to one stream (the legacy default stream unless lda_set_stream() is
+ *     called).  One host thread per context.
+ *   - all calls are synchronous: results are complete when they return.
+ *   - limits: n_tokens < 2^31, K <= 131072; bitlen(K-1) + bitlen(longest
+ *     document) <= 32 (n_kd entries are stored as one packed 32-bit word).
+ *
+ * There is no CPU fallback: every entry point that computes needs the GPU.
+ */
+#ifndef LDA_B200_H
+#define LDA_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LDA_OK 0
+#define LDA_EINVAL (-1)    /* NULL pointer, V/K <= 0, alpha/beta not finite and > 0, iters < 0, mh_steps < 1 */
+#define LDA_ERANGE (-2)    /* word id outside [0,V), bad offsets, sizes beyond the limits, capacity too small */
+#define LDA_ESTATE (-3)    /* call order: load before init, init before sweep */
+#define LDA_ENOMEM (-4)    /* host or device allocation failed */
+#define LDA_ECUDA (-5)     /* a CUDA call or launch failed */
+#define LDA_EINTERNAL (-6) /* a kernel raised the device error word (inconsistent tables) */
+
+#define LDA_NK 0
+#define LDA_NWK 1
+#define LDA_NDK 2
+
+typedef struct lda_ctx lda_ctx; /* opaque, owned by the library */
+
+/* Timings and counters of the most recent lda_sweep() call (all its iterations summed). */
+typedef struct lda_stats {
+    int64_t n_tokens, n_docs;
+    int64_t nnz_wk, nnz_dk;   /* nonzeros of n_kw and n_kd after the last rebuild */
+    int64_t n_dense_words;    /* words whose n_kw row is kept dense */
+    int64_t device_bytes;     /* device memory held by the context */
+    int64_t kernel_launches;  /* kernels launched by the last lda_sweep() */
+    int32_t sweeps_done;      /* sweeps since lda_init()/lda_set_assignments() */
+    int32_t iters;            /* iterations of the last lda_sweep() */
+    float ms_alias_dense;     /* dense smoothing table            (Section 4.2) */
+    float ms_alias_sparse;    /* per-word sparse alias tables     (Section 4.2) */
+    float ms_sample;          /* token MH kernel                  (Eq. 6-13)    */
+    float ms_count_wk;        /* n_kw rebuild                     (Section 3)   */
+    float ms_count_k;         /* n_k rebuild                                    */
+    float ms_count_dk;        /* n_kd rebuild                     (Eq. 12)      */
+    float ms_total;           /* first launch to last kernel end                */
+} lda_stats;
+
+/* Model dimensions and symmetric priors of the collapsed LDA model (Section 3,
+ * Eq. 1: alpha_k = alpha, beta_w = beta, beta-bar = V*beta). */
+int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out);
+
+/* Run all later work of this context on `cuda_stream` (a cudaStream_t); NULL = default stream. */
+int lda_set_stream(lda_ctx* ctx, void* cuda_stream);
+
+/* Tunables that never change results.  Must be set before lda_load_corpus().
+ *   "dense_frac"   fraction of the vocabulary (by term frequency) whose n_kw rows are dense (Section 5)
+ *   "dense_min_tf" words rarer than this stay sparse even inside dense_frac                          */
+int lda_set_option(lda_ctx* ctx, const char* key, double value);
+
+/* Corpus in document order: token i has word word_ids[i]; document d owns tokens
+ * [doc_offsets[d], doc_offsets[d+1]); doc_offsets has n_docs+1 entries, [0] = 0,
+ * [n_docs] = n_tokens; empty documents are legal.  Builds the word-sorted token
+ * layout once (Section 6, item 3) and chooses the dense/sparse class of every
+ * word (Section 5).  Both arrays are HOST memory. */
+int lda_load_corpus(lda_ctx* ctx, const int32_t* word_ids, int64_t n_tokens,
+                    const int64_t* doc_offsets, int64_t n_docs);
+
+/* Same, with both arrays in DEVICE memory of the context's GPU. */
+int lda_load_corpus_device(lda_ctx* ctx, const int32_t* word_ids_dev, int64_t n_tokens,
+                           const int64_t* doc_offsets_dev, int64_t n_docs);
+
+/* z_i uniform on {0..K-1} from Philox4x32-10 keyed by `seed`, counter
+ * (token, 0, 0, 1); builds n_kw, n_k, n_kd (Section 3, Eq. 12); sweep counter = 0. */
+int lda_init(lda_ctx* ctx, uint64_t seed);
+
+/* Warm start (Section 6: counts are re-initialised from z).  z has n_tokens
+ * entries in the caller's document order, each in [0,K). */
+int lda_set_assignments(lda_ctx* ctx, const int32_t* z, uint64_t seed, uint32_t sweep);
+
+/* `iters` frozen-counts sweeps of `mh_steps` proposals per token (Section 4.2-4.3,
+ * Eq. 6-13; Section 6 "immutable model").  Randomness: one Philox block per
+ * (token, sweep, step), counter (token, sweep, step, 0). */
+int lda_sweep(lda_ctx* ctx, int32_t iters, int32_t mh_steps);
+
+/* Collapsed joint log p(w,z): word part + document part (Section 7.2, Figure 11).
+ * Any output pointer may be NULL. */
+int lda_loglik(lda_ctx* ctx, double* total, double* word_ll, double* doc_ll);
+
+/* Count tables as CSR, topics ascending inside a row.
+ *   LDA_NK : counts[0..K) dense, `capacity` >= K; row_offsets/topics unused.
+ *   LDA_NWK: V rows; LDA_NDK: n_docs rows.  row_offsets has rows+1 entries.
+ * With topics == counts == row_offsets == NULL only *nnz_out is written. */
+int lda_get_counts(lda_ctx* ctx, int which, int64_t* row_offsets, int32_t* topics,
+                   int32_t* counts, int64_t capacity, int64_t* nnz_out);
+
+/* Current assignments, n_tokens entries in the caller's document order. */
+int lda_get_assignments(lda_ctx* ctx, int32_t* z_out);
+
+/* Word-proposal tables built from the current counts (Section 4.2): per-word sparse
+ * alias tables indexed like the LDA_NWK rows (split point as a 32-bit fraction,
+ * alias as an item index inside the row), per-word mixture thresholds [V], the
+ * dense table [K] and the dense term's fixed-point mass.  Any pointer may be NULL. */
+int lda_get_tables(lda_ctx* ctx, uint32_t* sp_thr32, int32_t* sp_alias, int64_t capacity,
+                   uint32_t* mix32, uint32_t* dn_thr32, int32_t* dn_alias, uint64_t* dense_mass);
+
+int lda_get_stats(lda_ctx* ctx, lda_stats* out);
+
+/* Message of the last failure on this context (library-owned, valid until the next call). */
+const char* lda_last_error(const lda_ctx* ctx);
+
+void lda_destroy(lda_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LDA_B200_H */

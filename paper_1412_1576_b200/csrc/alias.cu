@@ -1,0 +1,246 @@
+// Word-proposal tables (Section 4.2): the word-proposal (n_kw + beta)/(n_k + V*beta)
+// is sampled as a mixture of a sparse term over the word's nonzero n_kw (one alias
+// table per word, O(K_w) to build) and a dense term beta/(n_k + V*beta) whose alias
+// table is shared by all words.
+//
+// Alias construction is cooperative (a warp for short rows, a CTA for long ones)
+// and exact in integers, so the table is a function of the counts alone:
+//   - fixed-point weights wt_i = floor(weight_i * 2^44), W44 = sum wt_i;
+//   - pre-shift sh = max(0, bitlen(W44) + bitlen(n) - 62), w_i = wt_i >> sh, W = sum w_i;
+//   - bin capacity W, item i brings a_i = n * w_i; a_i <= W is "light", else "heavy";
+//   - with D_l = deficits of the lights before light l (ascending item order) and
+//     E_m = surpluses of heavies 0..m, light l is filled by heavy #{m : E_m <= D_l};
+//     heavy m keeps W + E_m - D_lam with lam = min{l : D_l >= E_m} and is filled by
+//     heavy m+1 (or is full).
+// This is the closed form of "fill lights in order from the current heavy item; an
+// exhausted heavy item becomes a bin topped up by the next heavy item".
+#include "lda_device.cuh"
+#include "lda_internal.cuh"
+
+namespace lda {
+
+typedef unsigned long long ull;
+
+template <bool BLOCK>
+struct Group {
+    ull* smem;  // CTA groups only: >= 33 entries
+    __device__ __forceinline__ int rank() const { return BLOCK ? (int)threadIdx.x : (int)(threadIdx.x & 31); }
+    __device__ __forceinline__ int size() const { return BLOCK ? (int)blockDim.x : 32; }
+    __device__ __forceinline__ void sync() const
+    {
+        if (BLOCK) __syncthreads(); else __syncwarp();
+    }
+    __device__ __forceinline__ ull reduce(ull v) const
+    {
+        if (BLOCK) return block_reduce_sum<ull>(v, smem);
+        return warp_reduce_sum<ull>(v);
+    }
+    __device__ __forceinline__ ull scan_excl(ull v, ull& total) const
+    {
+        if (BLOCK) return block_scan_excl<ull>(v, smem, total);
+        const ull incl = warp_scan_incl<ull>(v);
+        total = __shfl_sync(0xffffffffu, incl, 31);
+        return incl - v;
+    }
+};
+
+__device__ __forceinline__ uint32_t to_frac32(ull part, ull whole)
+{
+    int sh = bit_length(whole) - 32;
+    if (sh < 0) sh = 0;
+    const ull q = ((part >> sh) << 32) / (whole >> sh);
+    return q > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)q;
+}
+
+// Builds one table of n items.  weight(i) gives the fixed-point weight of item i.
+// sc_w, sc_de, sc_item: scratch of n entries each, private to this row.
+// Returns W44 (the sum of the fixed-point weights) to every thread of the group.
+template <bool BLOCK, class Weight>
+__device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, ull* sc_w, ull* sc_de,
+                               uint32_t* sc_item, uint32_t* out_thr, uint32_t* out_idx, int* err)
+{
+    const int r = g.rank(), gs = g.size();
+    ull s = 0;
+    for (int32_t i = r; i < n; i += gs) {
+        const ull wt = weight(i);
+        sc_w[i] = wt;
+        s += wt;
+    }
+    const ull W44 = g.reduce(s);
+    int sh = bit_length(W44) + bit_length((ull)n) - 62;
+    if (sh < 0) sh = 0;
+    s = 0;
+    for (int32_t i = r; i < n; i += gs) s += sc_w[i] >> sh;
+    const ull W = g.reduce(s);
+    if (W == 0) {
+        if (r == 0) atomicOr(err, ERR_ALIAS);
+        return W44;
+    }
+    uint32_t L = 0, H = 0;
+    ull d_sum = 0, e_sum = 0;
+    for (int32_t i0 = 0; i0 < n; i0 += gs) {
+        const int32_t i = i0 + r;
+        const bool valid = i < n;
+        const ull a = valid ? (ull)n * (sc_w[i] >> sh) : 0;
+        const bool light = valid && a <= W, heavy = valid && a > W;
+        const ull def = light ? W - a : 0, sur = heavy ? a - W : 0;
+        ull c_tot, d_tot, e_tot;
+        const ull c_pre = g.scan_excl((light ? 1ull : 0ull) | (heavy ? (1ull << 32) : 0ull), c_tot);
+        const ull d_pre = g.scan_excl(def, d_tot);
+        const ull e_pre = g.scan_excl(sur, e_tot);
+        if (valid) sc_w[i] = a;
+        if (light) {
+            const uint32_t l = L + (uint32_t)c_pre;
+            sc_de[l] = d_sum + d_pre;
+            sc_item[l] = (uint32_t)i;
+        }
+        if (heavy) {
+            const uint32_t m = H + (uint32_t)(c_pre >> 32);
+            sc_de[n - 1 - m] = e_sum + e_pre + sur;
+            sc_item[n - 1 - m] = (uint32_t)i;
+        }
+        L += (uint32_t)c_tot;
+        H += (uint32_t)(c_tot >> 32);
+        d_sum += d_tot;
+        e_sum += e_tot;
+    }
+    g.sync();
+    for (uint32_t l = r; l < L; l += gs) {
+        const uint32_t i = sc_item[l];
+        const ull a = sc_w[i];
+        uint32_t al = i;
+        if (a != W) {
+            const ull D = sc_de[l];
+            uint32_t lo = 0, hi = H;  // number of heavies with E_m <= D
+            while (lo < hi) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (sc_de[n - 1 - mid] <= D) lo = mid + 1; else hi = mid;
+            }
+            if (lo >= H) { atomicOr(err, ERR_ALIAS); lo = H ? H - 1 : 0; }
+            al = H ? sc_item[n - 1 - lo] : i;
+        }
+        out_thr[i] = to_frac32(a, W);
+        out_idx[i] = al;
+    }
+    for (uint32_t m = r; m < H; m += gs) {
+        const uint32_t i = sc_item[n - 1 - m];
+        const ull E = sc_de[n - 1 - m];
+        uint32_t lo = 0, hi = L;  // first light l with D_l >= E; l == L stands for the total deficit
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (sc_de[mid] >= E) hi = mid; else lo = mid + 1;
+        }
+        const ull Dl = lo < L ? sc_de[lo] : d_sum;
+        const ull thr = W + E - Dl;
+        uint32_t al = i;
+        if (thr != W) {
+            if (m + 1 >= H) atomicOr(err, ERR_ALIAS);
+            else al = sc_item[n - 1 - (m + 1)];
+        }
+        out_thr[i] = to_frac32(thr, W);
+        out_idx[i] = al;
+    }
+    return W44;
+}
+
+constexpr double FIXED_ONE = 17592186044416.0;  // 2^44
+
+struct DenseWeight {
+    const int32_t* nk;
+    double beta, Vbeta;
+    __device__ __forceinline__ ull operator()(int32_t k) const
+    {
+        const double den = __dadd_rn((double)nk[k], Vbeta);
+        return __double2ull_rz(__dmul_rn(__ddiv_rn(beta, den), FIXED_ONE));
+    }
+};
+
+struct SparseWeight {
+    const uint32_t* topic;
+    const uint32_t* count;
+    const int32_t* nk;
+    double Vbeta;
+    __device__ __forceinline__ ull operator()(int32_t i) const
+    {
+        const double den = __dadd_rn((double)nk[topic[i]], Vbeta);
+        return __double2ull_rz(__dmul_rn(__ddiv_rn((double)count[i], den), FIXED_ONE));
+    }
+};
+
+__global__ void __launch_bounds__(1024) k_alias_dense(View v, ull* sc)
+{
+    __shared__ ull smem[33];
+    Group<true> g{smem};
+    const int32_t K = v.K;
+    DenseWeight wf{v.nk, v.beta, v.Vbeta};
+    const ull B = build_alias_row<true>(g, K, wf, sc, sc + K, (uint32_t*)(sc + 2 * (size_t)K), v.dn_thr,
+                                        v.dn_idx, v.err);
+    if (threadIdx.x == 0) *v.dense_mass = B;
+}
+
+__device__ __forceinline__ uint32_t mixture_threshold(ull S, ull B)
+{
+    if (S == 0) return 0;
+    return to_frac32(S, S + B);
+}
+
+// One warp per word, rows of at most ALIAS_WARP_MAX items.
+__global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, ull* sc_de, uint32_t* sc_item)
+{
+    Group<false> g{nullptr};
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    const ull B = *v.dense_mass;
+    for (int32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < v.V; w += warps) {
+        const int32_t n = v.wk_nnz[w];
+        if (n > ALIAS_WARP_MAX) continue;
+        if (n == 0) {
+            if ((threadIdx.x & 31) == 0) v.mix32[w] = 0;
+            continue;
+        }
+        const int32_t r0 = v.row_start[w];
+        SparseWeight wf{v.wk_topic + r0, v.wk_count + r0, v.nk, v.Vbeta};
+        const ull S = build_alias_row<false>(g, n, wf, sc_w + r0, sc_de + r0, sc_item + r0, v.al_thr + r0,
+                                             v.al_idx + r0, v.err);
+        if ((threadIdx.x & 31) == 0) v.mix32[w] = mixture_threshold(S, B);
+        __syncwarp();
+    }
+}
+
+// One CTA per word whose row can be longer than ALIAS_WARP_MAX.
+__global__ void __launch_bounds__(256)
+k_alias_sparse_block(View v, const int32_t* __restrict__ words, ull* sc_w, ull* sc_de, uint32_t* sc_item)
+{
+    __shared__ ull smem[33];
+    Group<true> g{smem};
+    const int32_t w = words[blockIdx.x];
+    const int32_t n = v.wk_nnz[w];
+    if (n <= ALIAS_WARP_MAX) return;
+    const int32_t r0 = v.row_start[w];
+    SparseWeight wf{v.wk_topic + r0, v.wk_count + r0, v.nk, v.Vbeta};
+    const ull S = build_alias_row<true>(g, n, wf, sc_w + r0, sc_de + r0, sc_item + r0, v.al_thr + r0,
+                                        v.al_idx + r0, v.err);
+    if (threadIdx.x == 0) v.mix32[w] = mixture_threshold(S, *v.dense_mass);
+}
+
+int launch_alias_dense(Ctx& c)
+{
+    k_alias_dense<<<1, 1024, 0, c.stream>>>(c.v, c.sc_dense);
+    return 1;
+}
+
+int launch_alias_sparse(Ctx& c)
+{
+    int launches = 0;
+    int grid = (int)(((int64_t)c.V * 32 + 255) / 256);
+    if (grid > 148 * 16) grid = 148 * 16;
+    k_alias_sparse_warp<<<grid, 256, 0, c.stream>>>(c.v, c.sc_w, c.sc_de, c.sc_item);
+    ++launches;
+    if (c.n_alias_big) {
+        k_alias_sparse_block<<<c.n_alias_big, 256, 0, c.stream>>>(c.v, c.alias_big, c.sc_w, c.sc_de,
+                                                                 c.sc_item);
+        ++launches;
+    }
+    return launches;
+}
+
+}  // namespace lda

@@ -1,0 +1,658 @@
+// C ABI of the library: argument checks, device memory, work lists, launch order.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "lda_internal.cuh"
+
+namespace lda {
+void set_hist_smem_limits();
+
+void* dev_alloc(Ctx& c, size_t bytes)
+{
+    void* p = nullptr;
+    if (bytes == 0) bytes = 16;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    c.allocs.push_back(p);
+    c.device_bytes += (int64_t)bytes;
+    return p;
+}
+
+void dev_free_all(Ctx& c)
+{
+    for (void* p : c.allocs) cudaFree(p);
+    c.allocs.clear();
+    c.device_bytes = 0;
+}
+
+static int fail(Ctx* c, int code, const char* msg)
+{
+    if (c) c->err = msg;
+    return code;
+}
+
+static int cuda_fail(Ctx* c, const char* where)
+{
+    cudaError_t e = cudaGetLastError();
+    if (c) c->err = std::string(where) + ": " + cudaGetErrorString(e);
+    return LDA_ECUDA;
+}
+
+// Reads and clears the device error word.
+static int read_err(Ctx& c, int* bits)
+{
+    if (cudaMemcpyAsync(bits, c.v.err, sizeof(int), cudaMemcpyDeviceToHost, c.stream) != cudaSuccess ||
+        cudaStreamSynchronize(c.stream) != cudaSuccess)
+        return cuda_fail(&c, "reading the device error word");
+    if (*bits) cudaMemsetAsync(c.v.err, 0, sizeof(int), c.stream);
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail(&c, "kernel launch");
+    return LDA_OK;
+}
+
+static int check_device(Ctx& c)
+{
+    if (cudaSetDevice(c.device) != cudaSuccess) return cuda_fail(&c, "cudaSetDevice");
+    return LDA_OK;
+}
+
+template <typename T>
+static T* upload(Ctx& c, const std::vector<T>& h)
+{
+    T* d = (T*)dev_alloc(c, h.size() * sizeof(T));
+    if (d && !h.empty() &&
+        cudaMemcpyAsync(d, h.data(), h.size() * sizeof(T), cudaMemcpyHostToDevice, c.stream) != cudaSuccess)
+        return nullptr;
+    return d;
+}
+
+static void free_corpus(Ctx& c)
+{
+    int* err = c.v.err;
+    // the error word is allocated in lda_create and outlives corpora
+    std::vector<void*> keep;
+    for (void* p : c.allocs)
+        if (p == (void*)err) keep.push_back(p); else cudaFree(p);
+    c.allocs = keep;
+    c.device_bytes = keep.empty() ? 0 : 16;
+    View nv{};
+    nv.V = c.V; nv.K = c.K; nv.alpha = c.alpha; nv.beta = c.beta;
+    nv.Vbeta = (double)c.V * c.beta;
+    nv.Kalpha = (double)c.K * c.alpha;
+    nv.err = err;
+    c.v = nv;
+    c.loaded = c.inited = c.tables_valid = false;
+    c.N = c.D = 0;
+}
+
+static int rebuild_counts(Ctx& c, int64_t* launches)
+{
+    int n = launch_count_wk(c);
+    n += launch_count_k(c);
+    n += launch_count_dk(c);
+    if (launches) *launches += n;
+    c.tables_valid = false;
+    return LDA_OK;
+}
+
+static int ensure_tables(Ctx& c)
+{
+    if (c.tables_valid) return LDA_OK;
+    launch_alias_dense(c);
+    launch_alias_sparse(c);
+    int bits = 0;
+    int rc = read_err(c, &bits);
+    if (rc) return rc;
+    if (bits) return fail(&c, LDA_EINTERNAL, "alias construction raised the device error word");
+    c.tables_valid = true;
+    return LDA_OK;
+}
+
+static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const int64_t* doc_off,
+                       int64_t n_docs)
+{
+    free_corpus(c);
+    c.N = n_tokens;
+    c.D = n_docs;
+    View& v = c.v;
+    v.N = (int32_t)n_tokens;
+    v.D = (int32_t)n_docs;
+    const int32_t V = c.V, K = c.K;
+    const int32_t N = v.N, D = v.D;
+
+    int64_t max_len = 0;
+    for (int64_t d = 0; d < n_docs; ++d) max_len = std::max(max_len, doc_off[d + 1] - doc_off[d]);
+    int tb = 1;
+    while ((1ll << tb) < (long long)K) ++tb;
+    int cb = 1;
+    while ((1ll << cb) <= max_len) ++cb;
+    if (tb + cb > 32) {
+        free_corpus(c);
+        return fail(&c, LDA_ERANGE, "bits(K-1) + bits(longest document) exceeds 32");
+    }
+    v.topic_bits = tb;
+    v.count_bits = cb;
+
+    int rc = build_layout(c, words_dev, doc_off);
+    if (rc != LDA_OK) { free_corpus(c); return fail(&c, rc, "building the word-sorted layout failed"); }
+    int bits = 0;
+    rc = read_err(c, &bits);
+    if (rc) { free_corpus(c); return rc; }
+    if (bits & ERR_WORD_RANGE) { free_corpus(c); return fail(&c, LDA_ERANGE, "word id outside [0,V)"); }
+
+    std::vector<int32_t> word_off((size_t)V + 1);
+    if (cudaMemcpy(word_off.data(), v.word_off, ((size_t)V + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        free_corpus(c);
+        return cuda_fail(&c, "copying word offsets");
+    }
+
+    // --- dense / sparse class of every word (Section 5) ---------------------------------
+    std::vector<int32_t> tf((size_t)V);
+    for (int32_t w = 0; w < V; ++w) tf[w] = word_off[w + 1] - word_off[w];
+    int32_t tf_cut = INT32_MAX;
+    const int64_t n_top = (int64_t)std::floor(c.dense_frac * (double)V);
+    if (n_top > 0) {
+        std::vector<int32_t> tmp(tf);
+        const size_t nth = (size_t)std::min<int64_t>(n_top, V) - 1;
+        std::nth_element(tmp.begin(), tmp.begin() + nth, tmp.end(), std::greater<int32_t>());
+        tf_cut = std::max<int32_t>(tmp[nth], (int32_t)std::max(1.0, c.dense_min_tf));
+    }
+    std::vector<int32_t> dense_slot((size_t)V, -1), dense_words, row_start((size_t)V + 1), alias_big;
+    std::vector<int32_t> hist_chunks, word_tiles;
+    int64_t cap_total = 0;
+    for (int32_t w = 0; w < V; ++w) {
+        row_start[w] = (int32_t)cap_total;
+        const int32_t cap = std::min(tf[w], K);
+        cap_total += cap;
+        if (cap > ALIAS_WARP_MAX) alias_big.push_back(w);
+        if (tf[w] > SORT_TILE || (tf[w] > 0 && tf[w] >= tf_cut)) {
+            dense_slot[w] = (int32_t)dense_words.size();
+            dense_words.push_back(w);
+            for (int32_t o = 0; o < tf[w]; o += HIST_CHUNK) {
+                hist_chunks.push_back(w);
+                hist_chunks.push_back(word_off[w] + o);
+                hist_chunks.push_back(std::min(HIST_CHUNK, tf[w] - o));
+            }
+        }
+    }
+    row_start[V] = (int32_t)cap_total;
+    // tiles of consecutive sparse words: <= SORT_TILE tokens and <= SORT_TILE words each
+    {
+        int32_t s0 = 0, tok = 0;
+        auto close = [&](int32_t s1) {
+            if (s1 > s0) { word_tiles.push_back(s0); word_tiles.push_back(s1); }
+        };
+        for (int32_t w = 0; w < V; ++w) {
+            if (dense_slot[w] >= 0) { close(w); s0 = w + 1; tok = 0; continue; }
+            if (tok + tf[w] > SORT_TILE || w - s0 >= SORT_TILE) { close(w); s0 = w; tok = 0; }
+            tok += tf[w];
+        }
+        close(V);
+    }
+    std::vector<int32_t> doc_tiles, long_docs;
+    {
+        int32_t s0 = 0;
+        int64_t tok = 0;
+        auto close = [&](int32_t s1) {
+            if (s1 > s0) { doc_tiles.push_back(s0); doc_tiles.push_back(s1); }
+        };
+        for (int32_t d = 0; d < D; ++d) {
+            const int64_t len = doc_off[d + 1] - doc_off[d];
+            if (len > SORT_TILE) { close(d); s0 = d + 1; tok = 0; long_docs.push_back(d); continue; }
+            if (tok + len > SORT_TILE || d - s0 >= SORT_TILE) { close(d); s0 = d; tok = 0; }
+            tok += len;
+        }
+        close(D);
+    }
+    c.n_word_tiles = (int32_t)(word_tiles.size() / 2);
+    c.n_doc_tiles = (int32_t)(doc_tiles.size() / 2);
+    c.n_dense = (int32_t)dense_words.size();
+    c.n_hist_chunks = (int32_t)(hist_chunks.size() / 3);
+    c.n_long_docs = (int32_t)long_docs.size();
+    c.n_alias_big = (int32_t)alias_big.size();
+
+    const size_t n1 = (size_t)std::max<int64_t>(N, 1), cap1 = (size_t)std::max<int64_t>(cap_total, 1);
+    const size_t zt = c.wide_topics ? 4 : 2;
+    bool ok = true;
+    auto A = [&](size_t bytes) { void* p = dev_alloc(c, bytes); ok = ok && p; return p; };
+    for (int b = 0; b < 2; ++b) { v.zw[b] = A(n1 * zt); v.zd[b] = A(n1 * zt); }
+    v.row_start = upload(c, row_start);
+    v.dense_slot = upload(c, dense_slot);
+    c.word_tiles = upload(c, word_tiles);
+    c.doc_tiles = upload(c, doc_tiles);
+    c.dense_words = upload(c, dense_words);
+    c.hist_chunks = upload(c, hist_chunks);
+    c.long_docs = upload(c, long_docs);
+    c.alias_big = upload(c, alias_big);
+    ok = ok && v.row_start && v.dense_slot && c.word_tiles && c.doc_tiles && c.dense_words &&
+         c.hist_chunks && c.long_docs && c.alias_big;
+    v.wk_nnz = (int32_t*)A((size_t)V * 4);
+    v.wk_topic = (uint32_t*)A(cap1 * 4);
+    v.wk_count = (uint32_t*)A(cap1 * 4);
+    v.dense_rows = (int32_t*)A(std::max<size_t>((size_t)c.n_dense * K, 1) * 4);
+    v.al_thr = (uint32_t*)A(cap1 * 4);
+    v.al_idx = (uint32_t*)A(cap1 * 4);
+    v.mix32 = (uint32_t*)A((size_t)V * 4);
+    v.dn_thr = (uint32_t*)A((size_t)K * 4);
+    v.dn_idx = (uint32_t*)A((size_t)K * 4);
+    v.dense_mass = (unsigned long long*)A(8);
+    v.nk = (int32_t*)A((size_t)K * 4);
+    v.dk_pairs = (uint32_t*)A(n1 * 4);
+    v.dk_nnz = (int32_t*)A((size_t)std::max<int32_t>(D, 1) * 4);
+    c.sc_w = (unsigned long long*)A(cap1 * 8);
+    c.sc_de = (unsigned long long*)A(cap1 * 8);
+    c.sc_item = (uint32_t*)A(cap1 * 4);
+    c.sc_dense = (unsigned long long*)A((size_t)K * 8 * 3);
+    c.red = (double*)A(sizeof(double) * 2 * 592);
+    c.red_i = (int64_t*)A(16);
+    if (!ok) { free_corpus(c); return fail(&c, LDA_ENOMEM, "device allocation failed"); }
+    cudaMemsetAsync(v.wk_nnz, 0, (size_t)V * 4, c.stream);
+    cudaMemsetAsync(v.dk_nnz, 0, (size_t)std::max<int32_t>(D, 1) * 4, c.stream);
+    cudaMemsetAsync(v.mix32, 0, (size_t)V * 4, c.stream);
+    cudaMemsetAsync(v.nk, 0, (size_t)K * 4, c.stream);
+    if (cudaStreamSynchronize(c.stream) != cudaSuccess) { free_corpus(c); return cuda_fail(&c, "load"); }
+    c.stats = lda_stats{};
+    c.stats.n_tokens = N;
+    c.stats.n_docs = D;
+    c.stats.n_dense_words = c.n_dense;
+    c.loaded = true;
+    return LDA_OK;
+}
+
+static int validate_offsets(Ctx* c, int64_t n_tokens, const int64_t* doc_off, int64_t n_docs)
+{
+    if (n_tokens >= 2147483648ll || n_docs >= 2147483647ll) return fail(c, LDA_ERANGE, "n_tokens and n_docs must be below 2^31");
+    if (doc_off[0] != 0 || doc_off[n_docs] != n_tokens)
+        return fail(c, LDA_ERANGE, "doc_offsets must start at 0 and end at n_tokens");
+    for (int64_t d = 0; d < n_docs; ++d)
+        if (doc_off[d + 1] < doc_off[d]) return fail(c, LDA_ERANGE, "doc_offsets must be non-decreasing");
+    return LDA_OK;
+}
+
+}  // namespace lda
+
+using namespace lda;
+
+struct lda_ctx {
+    Ctx c;
+};
+
+extern "C" {
+
+int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
+{
+    if (!out) return LDA_EINVAL;
+    *out = nullptr;
+    if (V <= 0 || K <= 0 || !(alpha > 0) || !(beta > 0) || !std::isfinite(alpha) || !std::isfinite(beta))
+        return LDA_EINVAL;
+    if (K > 131072) return LDA_ERANGE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LDA_ECUDA; }
+    lda_ctx* h = new (std::nothrow) lda_ctx();
+    if (!h) return LDA_ENOMEM;
+    Ctx& c = h->c;
+    c.V = V; c.K = K; c.alpha = alpha; c.beta = beta; c.device = dev;
+    c.wide_topics = K > 65536;
+    c.v.V = V; c.v.K = K; c.v.alpha = alpha; c.v.beta = beta;
+    c.v.Vbeta = (double)V * beta;
+    c.v.Kalpha = (double)K * alpha;
+    c.v.err = (int*)dev_alloc(c, 16);
+    if (!c.v.err || cudaMemset(c.v.err, 0, 16) != cudaSuccess) {
+        dev_free_all(c);
+        delete h;
+        cudaGetLastError();
+        return LDA_ECUDA;
+    }
+    for (int i = 0; i < 8; ++i)
+        if (cudaEventCreate(&c.ev[i]) != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(c.ev[j]);
+            dev_free_all(c);
+            delete h;
+            cudaGetLastError();
+            return LDA_ECUDA;
+        }
+    c.have_events = true;
+    set_hist_smem_limits();
+    *out = h;
+    return LDA_OK;
+}
+
+void lda_destroy(lda_ctx* h)
+{
+    if (!h) return;
+    Ctx& c = h->c;
+    cudaSetDevice(c.device);
+    cudaStreamSynchronize(c.stream);
+    if (c.have_events)
+        for (int i = 0; i < 8; ++i) cudaEventDestroy(c.ev[i]);
+    dev_free_all(c);
+    cudaGetLastError();
+    delete h;
+}
+
+const char* lda_last_error(const lda_ctx* h) { return h ? h->c.err.c_str() : "null context"; }
+
+int lda_set_stream(lda_ctx* h, void* cuda_stream)
+{
+    if (!h) return LDA_EINVAL;
+    cudaStreamSynchronize(h->c.stream);
+    h->c.stream = (cudaStream_t)cuda_stream;
+    return LDA_OK;
+}
+
+int lda_set_option(lda_ctx* h, const char* key, double value)
+{
+    if (!h || !key) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (c.loaded) return fail(&c, LDA_ESTATE, "options must be set before lda_load_corpus");
+    if (!std::strcmp(key, "dense_frac")) {
+        if (!(value >= 0.0 && value <= 1.0)) return fail(&c, LDA_EINVAL, "dense_frac must be in [0,1]");
+        c.dense_frac = value;
+        return LDA_OK;
+    }
+    if (!std::strcmp(key, "dense_min_tf")) {
+        if (!(value >= 1.0)) return fail(&c, LDA_EINVAL, "dense_min_tf must be >= 1");
+        c.dense_min_tf = value;
+        return LDA_OK;
+    }
+    return fail(&c, LDA_EINVAL, "unknown option");
+}
+
+int lda_load_corpus(lda_ctx* h, const int32_t* word_ids, int64_t n_tokens, const int64_t* doc_offsets,
+                    int64_t n_docs)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!doc_offsets || n_tokens < 0 || n_docs < 0 || (n_tokens > 0 && !word_ids))
+        return fail(&c, LDA_EINVAL, "null pointer or negative size");
+    int rc = validate_offsets(&c, n_tokens, doc_offsets, n_docs);
+    if (rc) return rc;
+    if ((rc = check_device(c))) return rc;
+    int32_t* wd = nullptr;
+    if (cudaMalloc(&wd, (size_t)std::max<int64_t>(n_tokens, 1) * 4) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(&c, LDA_ENOMEM, "device allocation failed");
+    }
+    if (n_tokens > 0 &&
+        cudaMemcpyAsync(wd, word_ids, (size_t)n_tokens * 4, cudaMemcpyHostToDevice, c.stream) != cudaSuccess) {
+        cudaFree(wd);
+        return cuda_fail(&c, "copying word ids");
+    }
+    rc = load_common(c, wd, n_tokens, doc_offsets, n_docs);
+    cudaStreamSynchronize(c.stream);
+    cudaFree(wd);
+    return rc;
+}
+
+int lda_load_corpus_device(lda_ctx* h, const int32_t* word_ids_dev, int64_t n_tokens,
+                           const int64_t* doc_offsets_dev, int64_t n_docs)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!doc_offsets_dev || n_tokens < 0 || n_docs < 0 || (n_tokens > 0 && !word_ids_dev))
+        return fail(&c, LDA_EINVAL, "null pointer or negative size");
+    if (n_docs >= 2147483647ll) return fail(&c, LDA_ERANGE, "n_docs must be below 2^31");
+    int rc = check_device(c);
+    if (rc) return rc;
+    std::vector<int64_t> off((size_t)n_docs + 1);
+    if (cudaMemcpy(off.data(), doc_offsets_dev, ((size_t)n_docs + 1) * 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return cuda_fail(&c, "copying doc offsets");
+    if ((rc = validate_offsets(&c, n_tokens, off.data(), n_docs))) return rc;
+    return load_common(c, word_ids_dev, n_tokens, off.data(), n_docs);
+}
+
+int lda_init(lda_ctx* h, uint64_t seed)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!c.loaded) return fail(&c, LDA_ESTATE, "lda_init before lda_load_corpus");
+    int rc = check_device(c);
+    if (rc) return rc;
+    c.seed = seed;
+    c.sweep = 0;
+    c.cur = 0;
+    launch_init(c);
+    rebuild_counts(c, nullptr);
+    int bits = 0;
+    if ((rc = read_err(c, &bits))) return rc;
+    if (bits) return fail(&c, LDA_EINTERNAL, "count rebuild raised the device error word");
+    c.inited = true;
+    return LDA_OK;
+}
+
+int lda_set_assignments(lda_ctx* h, const int32_t* z, uint64_t seed, uint32_t sweep)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!c.loaded) return fail(&c, LDA_ESTATE, "lda_set_assignments before lda_load_corpus");
+    if (c.N > 0 && !z) return fail(&c, LDA_EINVAL, "null assignments");
+    int rc = check_device(c);
+    if (rc) return rc;
+    int32_t* zdev = nullptr;
+    if (cudaMalloc(&zdev, (size_t)std::max<int64_t>(c.N, 1) * 4) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(&c, LDA_ENOMEM, "device allocation failed");
+    }
+    if (c.N > 0 && cudaMemcpyAsync(zdev, z, (size_t)c.N * 4, cudaMemcpyHostToDevice, c.stream) != cudaSuccess) {
+        cudaFree(zdev);
+        return cuda_fail(&c, "copying assignments");
+    }
+    c.cur = 0;
+    launch_spread_assignments(c, zdev);
+    int bits = 0;
+    rc = read_err(c, &bits);
+    cudaFree(zdev);
+    if (rc) return rc;
+    if (bits & ERR_TOPIC_RANGE) { c.inited = false; return fail(&c, LDA_ERANGE, "assignment outside [0,K)"); }
+    c.seed = seed;
+    c.sweep = sweep;
+    rebuild_counts(c, nullptr);
+    if ((rc = read_err(c, &bits))) return rc;
+    if (bits) return fail(&c, LDA_EINTERNAL, "count rebuild raised the device error word");
+    c.inited = true;
+    return LDA_OK;
+}
+
+int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (iters < 0 || mh_steps < 1) return fail(&c, LDA_EINVAL, "iters must be >= 0 and mh_steps >= 1");
+    if (!c.inited) return fail(&c, LDA_ESTATE, "lda_sweep before lda_init");
+    int rc = check_device(c);
+    if (rc) return rc;
+    lda_stats& s = c.stats;
+    s.ms_alias_dense = s.ms_alias_sparse = s.ms_sample = s.ms_count_wk = s.ms_count_k = s.ms_count_dk =
+        s.ms_total = 0.f;
+    s.kernel_launches = 0;
+    s.iters = iters;
+    for (int32_t it = 0; it < iters; ++it) {
+        int64_t n = 0;
+        cudaEventRecord(c.ev[0], c.stream);
+        n += launch_alias_dense(c);
+        cudaEventRecord(c.ev[1], c.stream);
+        n += launch_alias_sparse(c);
+        cudaEventRecord(c.ev[2], c.stream);
+        n += launch_sample(c, mh_steps);
+        c.cur ^= 1;
+        cudaEventRecord(c.ev[3], c.stream);
+        n += launch_count_wk(c);
+        cudaEventRecord(c.ev[4], c.stream);
+        n += launch_count_k(c);
+        cudaEventRecord(c.ev[5], c.stream);
+        n += launch_count_dk(c);
+        cudaEventRecord(c.ev[6], c.stream);
+        c.tables_valid = false;
+        c.sweep += 1;
+        int bits = 0;
+        if ((rc = read_err(c, &bits))) return rc;
+        if (bits) {
+            c.err = "a kernel raised the device error word: " + std::to_string(bits);
+            return LDA_EINTERNAL;
+        }
+        float ms[7] = {0};
+        for (int i = 0; i < 6; ++i) cudaEventElapsedTime(&ms[i], c.ev[i], c.ev[i + 1]);
+        cudaEventElapsedTime(&ms[6], c.ev[0], c.ev[6]);
+        s.ms_alias_dense += ms[0]; s.ms_alias_sparse += ms[1]; s.ms_sample += ms[2];
+        s.ms_count_wk += ms[3]; s.ms_count_k += ms[4]; s.ms_count_dk += ms[5]; s.ms_total += ms[6];
+        s.kernel_launches += n;
+    }
+    return LDA_OK;
+}
+
+int lda_loglik(lda_ctx* h, double* total, double* word_ll, double* doc_ll)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!c.inited) return fail(&c, LDA_ESTATE, "lda_loglik before lda_init");
+    int rc = check_device(c);
+    if (rc) return rc;
+    double out[3];
+    if (launch_loglik(c, out) < 0) return cuda_fail(&c, "log-likelihood");
+    if (total) *total = out[0];
+    if (word_ll) *word_ll = out[1];
+    if (doc_ll) *doc_ll = out[2];
+    return LDA_OK;
+}
+
+int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics, int32_t* counts,
+                   int64_t capacity, int64_t* nnz_out)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!c.inited) return fail(&c, LDA_ESTATE, "lda_get_counts before lda_init");
+    int rc = check_device(c);
+    if (rc) return rc;
+    const View& v = c.v;
+    cudaStreamSynchronize(c.stream);
+    if (which == LDA_NK) {
+        if (nnz_out) *nnz_out = c.K;
+        if (counts) {
+            if (capacity < c.K) return fail(&c, LDA_ERANGE, "capacity below K");
+            if (cudaMemcpy(counts, v.nk, (size_t)c.K * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+                return cuda_fail(&c, "copying n_k");
+        }
+        return LDA_OK;
+    }
+    if (which != LDA_NWK && which != LDA_NDK) return fail(&c, LDA_EINVAL, "unknown table");
+    const bool words = which == LDA_NWK;
+    const int64_t rows = words ? c.V : c.D;
+    std::vector<int32_t> nnz((size_t)std::max<int64_t>(rows, 1)), start((size_t)rows + 1);
+    if (rows && cudaMemcpy(nnz.data(), words ? v.wk_nnz : v.dk_nnz, (size_t)rows * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return cuda_fail(&c, "copying row sizes");
+    if (cudaMemcpy(start.data(), words ? v.row_start : v.doc_off, ((size_t)rows + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return cuda_fail(&c, "copying row starts");
+    int64_t total = 0;
+    for (int64_t r = 0; r < rows; ++r) total += nnz[(size_t)r];
+    if (nnz_out) *nnz_out = total;
+    if (!row_offsets && !topics && !counts) return LDA_OK;
+    if (capacity < total) return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros");
+    const size_t cap = (size_t)start[(size_t)rows];
+    std::vector<uint32_t> a(std::max<size_t>(cap, 1)), b;
+    if (words) {
+        b.resize(std::max<size_t>(cap, 1));
+        if (cap && (cudaMemcpy(a.data(), v.wk_topic, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+                    cudaMemcpy(b.data(), v.wk_count, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess))
+            return cuda_fail(&c, "copying n_kw rows");
+    } else if (cap && cudaMemcpy(a.data(), v.dk_pairs, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        return cuda_fail(&c, "copying n_kd rows");
+    }
+    const uint32_t cmask = (1u << v.count_bits) - 1u;
+    int64_t o = 0;
+    for (int64_t r = 0; r < rows; ++r) {
+        if (row_offsets) row_offsets[r] = o;
+        const size_t s0 = (size_t)start[(size_t)r];
+        for (int32_t j = 0; j < nnz[(size_t)r]; ++j, ++o) {
+            if (words) {
+                if (topics) topics[o] = (int32_t)a[s0 + j];
+                if (counts) counts[o] = (int32_t)b[s0 + j];
+            } else {
+                if (topics) topics[o] = (int32_t)(a[s0 + j] >> v.count_bits);
+                if (counts) counts[o] = (int32_t)(a[s0 + j] & cmask);
+            }
+        }
+    }
+    if (row_offsets) row_offsets[rows] = o;
+    return LDA_OK;
+}
+
+int lda_get_assignments(lda_ctx* h, int32_t* z_out)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!c.inited) return fail(&c, LDA_ESTATE, "lda_get_assignments before lda_init");
+    if (c.N > 0 && !z_out) return fail(&c, LDA_EINVAL, "null output");
+    if (c.N == 0) return LDA_OK;
+    int rc = check_device(c);
+    if (rc) return rc;
+    int32_t* zdev = nullptr;
+    if (cudaMalloc(&zdev, (size_t)c.N * 4) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(&c, LDA_ENOMEM, "device allocation failed");
+    }
+    launch_export_assignments(c, zdev);
+    cudaError_t e = cudaMemcpyAsync(z_out, zdev, (size_t)c.N * 4, cudaMemcpyDeviceToHost, c.stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
+    cudaFree(zdev);
+    if (e != cudaSuccess) return cuda_fail(&c, "copying assignments");
+    return LDA_OK;
+}
+
+int lda_get_tables(lda_ctx* h, uint32_t* sp_thr32, int32_t* sp_alias, int64_t capacity, uint32_t* mix32,
+                   uint32_t* dn_thr32, int32_t* dn_alias, uint64_t* dense_mass)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!c.inited) return fail(&c, LDA_ESTATE, "lda_get_tables before lda_init");
+    int rc = check_device(c);
+    if (rc) return rc;
+    if ((rc = ensure_tables(c))) return rc;
+    const View& v = c.v;
+    const size_t V = (size_t)c.V, K = (size_t)c.K;
+    if (mix32 && cudaMemcpy(mix32, v.mix32, V * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail(&c, "copy");
+    if (dn_thr32 && cudaMemcpy(dn_thr32, v.dn_thr, K * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail(&c, "copy");
+    if (dn_alias && cudaMemcpy(dn_alias, v.dn_idx, K * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail(&c, "copy");
+    if (dense_mass && cudaMemcpy(dense_mass, v.dense_mass, 8, cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail(&c, "copy");
+    if (!sp_thr32 && !sp_alias) return LDA_OK;
+    std::vector<int32_t> nnz(V), start(V + 1);
+    if (cudaMemcpy(nnz.data(), v.wk_nnz, V * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(start.data(), v.row_start, (V + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return cuda_fail(&c, "copy");
+    int64_t total = 0;
+    for (size_t w = 0; w < V; ++w) total += nnz[w];
+    if (capacity < total) return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros");
+    const size_t cap = (size_t)start[V];
+    std::vector<uint32_t> a(std::max<size_t>(cap, 1)), b(std::max<size_t>(cap, 1));
+    if (cap && (cudaMemcpy(a.data(), v.al_thr, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+                cudaMemcpy(b.data(), v.al_idx, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess))
+        return cuda_fail(&c, "copy");
+    int64_t o = 0;
+    for (size_t w = 0; w < V; ++w)
+        for (int32_t j = 0; j < nnz[w]; ++j, ++o) {
+            if (sp_thr32) sp_thr32[o] = a[(size_t)start[w] + j];
+            if (sp_alias) sp_alias[o] = (int32_t)b[(size_t)start[w] + j];
+        }
+    return LDA_OK;
+}
+
+int lda_get_stats(lda_ctx* h, lda_stats* out)
+{
+    if (!h || !out) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (c.inited) {
+        if (check_device(c)) return LDA_ECUDA;
+        int64_t a = 0, b = 0;
+        launch_count_nnz(c, &a, &b);
+        c.stats.nnz_wk = a;
+        c.stats.nnz_dk = b;
+    }
+    c.stats.device_bytes = c.device_bytes;
+    c.stats.sweeps_done = (int32_t)c.sweep;
+    *out = c.stats;
+    return LDA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,362 @@
+// Count-table rebuild from the assignments (Section 3: n_kw, n_k; Eq. 12: n_kd).
+//
+// Both n_kw (segments = words over the word-sorted z) and n_kd (segments =
+// documents over the document-order z) are "per contiguous segment, the sorted
+// list of (topic, count)".  Two paths, chosen per segment at load time:
+//   - short segments: whole segments are packed into tiles of <= SORT_TILE
+//     tokens; one CTA sorts the tile's (segment, topic) keys in shared memory
+//     and run-length encodes them;
+//   - long segments (hot words, very long documents): shared-memory histogram
+//     over a window of topics, merged into the word's dense row (words) or
+//     compacted directly (documents).
+// No per-token global atomics: a CTA touches global counters once per bin it
+// actually filled.
+#include "lda_device.cuh"
+#include "lda_internal.cuh"
+
+namespace lda {
+
+struct EmitWord {
+    const int32_t* row_start;
+    uint32_t* topic;
+    uint32_t* count;
+    int32_t* nnz;
+    __device__ __forceinline__ void entry(int32_t seg, int32_t rank, uint32_t k, uint32_t n) const
+    {
+        const int32_t slot = row_start[seg] + rank;
+        topic[slot] = k;
+        count[slot] = n;
+    }
+    __device__ __forceinline__ void rows(int32_t seg, int32_t n) const { nnz[seg] = n; }
+};
+
+struct EmitDoc {
+    const int32_t* doc_off;
+    uint32_t* pairs;
+    int32_t* nnz;
+    int count_bits;
+    __device__ __forceinline__ void entry(int32_t seg, int32_t rank, uint32_t k, uint32_t n) const
+    {
+        pairs[doc_off[seg] + rank] = (k << count_bits) | n;
+    }
+    __device__ __forceinline__ void rows(int32_t seg, int32_t n) const { nnz[seg] = n; }
+};
+
+// One CTA per tile of whole segments [s0, s1) holding <= SORT_TILE tokens and
+// <= SORT_TILE segments.
+template <typename T, class Emit>
+__global__ void __launch_bounds__(256)
+k_seg_count_sorted(const int32_t* __restrict__ tiles, const int32_t* __restrict__ seg_off,
+                   const T* __restrict__ z, int topic_bits, int32_t K, Emit emit, int* err)
+{
+    __shared__ uint32_t keys[SORT_TILE];
+    __shared__ int32_t soff[SORT_TILE + 1];
+    __shared__ int32_t hidx[SORT_TILE + 1];
+    __shared__ int32_t headpos[SORT_TILE + 1];
+    __shared__ int32_t scan_tmp[33];
+
+    const int tid = threadIdx.x;
+    const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
+    const int32_t nseg = s1 - s0;
+    const int32_t base = seg_off[s0];
+    const int32_t cnt = seg_off[s1] - base;
+    for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = seg_off[s0 + j] - base;
+    int npad = 1;
+    while (npad < cnt) npad <<= 1;
+    __syncthreads();
+    if (cnt == 0) {
+        for (int j = tid; j < nseg; j += blockDim.x) emit.rows(s0 + j, 0);
+        return;
+    }
+    for (int j = tid; j < npad; j += blockDim.x) {
+        uint32_t key = 0xFFFFFFFFu;
+        if (j < cnt) {
+            int lo = 0, hi = nseg;  // last segment with soff[seg] <= j
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (soff[mid] <= j) lo = mid; else hi = mid;
+            }
+            const uint32_t k = (uint32_t)z[base + j];
+            if (k >= (uint32_t)K) atomicOr(err, ERR_TOPIC_RANGE);
+            key = ((uint32_t)lo << topic_bits) | k;
+        }
+        keys[j] = key;
+    }
+    __syncthreads();
+    // bitonic sort, ascending
+    for (int size = 2; size <= npad; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int t = tid; t < (npad >> 1); t += blockDim.x) {
+                const int i = ((t & ~(stride - 1)) << 1) | (t & (stride - 1));
+                const int j = i | stride;
+                const bool up = ((i & size) == 0);
+                const uint32_t a = keys[i], b = keys[j];
+                if ((a > b) == up) { keys[i] = b; keys[j] = a; }
+            }
+            __syncthreads();
+        }
+    }
+    // head flags -> exclusive scan (8 consecutive entries per thread)
+    constexpr int PER = SORT_TILE / 256;
+    int32_t flags[PER];
+    int32_t local = 0;
+#pragma unroll
+    for (int q = 0; q < PER; ++q) {
+        const int j = tid * PER + q;
+        flags[q] = (j < cnt && (j == 0 || keys[j] != keys[j - 1])) ? 1 : 0;
+        local += flags[q];
+    }
+    int32_t total;
+    int32_t run = block_scan_excl<int32_t>(local, scan_tmp, total);
+#pragma unroll
+    for (int q = 0; q < PER; ++q) {
+        const int j = tid * PER + q;
+        if (j < cnt) {
+            hidx[j] = run;
+            if (flags[q]) headpos[run] = j;
+            run += flags[q];
+        }
+    }
+    if (tid == 0) { hidx[cnt] = total; headpos[total] = cnt; }
+    __syncthreads();
+    const uint32_t kmask = (1u << topic_bits) - 1u;
+    for (int h = tid; h < total; h += blockDim.x) {
+        const int j = headpos[h];
+        const uint32_t key = keys[j];
+        const int32_t seg = (int32_t)(key >> topic_bits);
+        const int32_t rank = h - hidx[soff[seg]];
+        emit.entry(s0 + seg, rank, key & kmask, (uint32_t)(headpos[h + 1] - j));
+    }
+    for (int j = tid; j < nseg; j += blockDim.x) emit.rows(s0 + j, hidx[soff[j + 1]] - hidx[soff[j]]);
+}
+
+// Hot words: one CTA per chunk of a word's tokens; histogram of a window of
+// topics in shared memory, merged into the word's dense row with one global
+// add per nonzero bin.
+template <typename T>
+__global__ void __launch_bounds__(512)
+k_hist_chunks(const int32_t* __restrict__ chunks, const T* __restrict__ z,
+              const int32_t* __restrict__ dense_slot, int32_t* __restrict__ dense_rows, int32_t K,
+              int32_t window, int* err)
+{
+    extern __shared__ int32_t bins[];
+    const int32_t w = chunks[3 * blockIdx.x], first = chunks[3 * blockIdx.x + 1],
+                  cnt = chunks[3 * blockIdx.x + 2];
+    int32_t* row = dense_rows + (size_t)dense_slot[w] * K;
+    for (int32_t k0 = 0; k0 < K; k0 += window) {
+        const int32_t nb = min(window, K - k0);
+        for (int b = threadIdx.x; b < nb; b += blockDim.x) bins[b] = 0;
+        __syncthreads();
+        for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
+            const uint32_t k = (uint32_t)z[first + j];
+            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+            const uint32_t b = k - (uint32_t)k0;
+            if (b < (uint32_t)nb) atomicAdd(&bins[b], 1);
+        }
+        __syncthreads();
+        for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+            const int32_t n = bins[b];
+            if (n) atomicAdd(&row[k0 + b], n);
+        }
+        __syncthreads();
+    }
+}
+
+// Dense row -> sorted (topic, count) row, one CTA per dense word.
+__global__ void __launch_bounds__(256)
+k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restrict__ dense_slot,
+                const int32_t* __restrict__ dense_rows, const int32_t* __restrict__ row_start,
+                uint32_t* __restrict__ wk_topic, uint32_t* __restrict__ wk_count,
+                int32_t* __restrict__ wk_nnz, int32_t K, int* err)
+{
+    __shared__ int32_t scan_tmp[33];
+    const int32_t w = dense_words[blockIdx.x];
+    const int32_t* row = dense_rows + (size_t)dense_slot[w] * K;
+    const int32_t out0 = row_start[w], cap = row_start[w + 1] - out0;
+    int32_t done = 0;
+    for (int32_t k0 = 0; k0 < K; k0 += blockDim.x) {
+        const int32_t k = k0 + threadIdx.x;
+        const int32_t n = (k < K) ? row[k] : 0;
+        int32_t total;
+        const int32_t pos = block_scan_excl<int32_t>(n > 0 ? 1 : 0, scan_tmp, total);
+        if (n > 0) {
+            if (done + pos < cap) {
+                wk_topic[out0 + done + pos] = (uint32_t)k;
+                wk_count[out0 + done + pos] = (uint32_t)n;
+            } else {
+                atomicOr(err, ERR_ROW_OVERFLOW);
+            }
+        }
+        done += total;
+    }
+    if (threadIdx.x == 0) wk_nnz[w] = done;
+}
+
+// Documents longer than a sort tile: one CTA per document, windowed histogram,
+// compacted straight into the document's row.
+template <typename T>
+__global__ void __launch_bounds__(512)
+k_long_docs(const int32_t* __restrict__ long_docs, const int32_t* __restrict__ doc_off,
+            const T* __restrict__ z, uint32_t* __restrict__ pairs, int32_t* __restrict__ dk_nnz,
+            int32_t K, int32_t window, int count_bits, int* err)
+{
+    extern __shared__ int32_t bins[];
+    __shared__ int32_t scan_tmp[33];
+    const int32_t d = long_docs[blockIdx.x];
+    const int32_t first = doc_off[d], cnt = doc_off[d + 1] - first;
+    int32_t done = 0;
+    for (int32_t k0 = 0; k0 < K; k0 += window) {
+        const int32_t nb = min(window, K - k0);
+        for (int b = threadIdx.x; b < nb; b += blockDim.x) bins[b] = 0;
+        __syncthreads();
+        for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
+            const uint32_t k = (uint32_t)z[first + j];
+            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+            const uint32_t b = k - (uint32_t)k0;
+            if (b < (uint32_t)nb) atomicAdd(&bins[b], 1);
+        }
+        __syncthreads();
+        for (int32_t b0 = 0; b0 < nb; b0 += blockDim.x) {
+            const int32_t b = b0 + threadIdx.x;
+            const int32_t n = (b < nb) ? bins[b] : 0;
+            int32_t total;
+            const int32_t pos = block_scan_excl<int32_t>(n > 0 ? 1 : 0, scan_tmp, total);
+            if (n > 0) pairs[first + done + pos] = ((uint32_t)(k0 + b) << count_bits) | (uint32_t)n;
+            done += total;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) dk_nnz[d] = done;
+}
+
+// n_k: histogram of all assignments, CTA-private shared-memory bins.
+template <typename T>
+__global__ void __launch_bounds__(512)
+k_count_k(const T* __restrict__ z, int32_t n, int32_t* __restrict__ nk, int32_t K, int32_t window,
+          int* err)
+{
+    extern __shared__ int32_t bins[];
+    const int64_t per = ((int64_t)n + gridDim.x - 1) / gridDim.x;
+    const int64_t lo = per * blockIdx.x, hi = min((int64_t)n, lo + per);
+    for (int32_t k0 = 0; k0 < K; k0 += window) {
+        const int32_t nb = min(window, K - k0);
+        for (int b = threadIdx.x; b < nb; b += blockDim.x) bins[b] = 0;
+        __syncthreads();
+        for (int64_t j = lo + threadIdx.x; j < hi; j += blockDim.x) {
+            const uint32_t k = (uint32_t)z[j];
+            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+            const uint32_t b = k - (uint32_t)k0;
+            if (b < (uint32_t)nb) atomicAdd(&bins[b], 1);
+        }
+        __syncthreads();
+        for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+            const int32_t v = bins[b];
+            if (v) atomicAdd(&nk[k0 + b], v);
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void k_sum_i32(const int32_t* __restrict__ a, int64_t n, unsigned long long* out)
+{
+    __shared__ unsigned long long tmp[32];
+    unsigned long long s = 0;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+         i += (int64_t)gridDim.x * blockDim.x)
+        s += (unsigned long long)a[i];
+    s = block_reduce_sum<unsigned long long>(s, tmp);
+    if (threadIdx.x == 0 && s) atomicAdd(out, s);
+}
+
+static int hist_window(const Ctx& c) { return c.K < HIST_BINS ? c.K : HIST_BINS; }
+
+template <typename T>
+static int count_wk_t(Ctx& c)
+{
+    View& v = c.v;
+    int launches = 0;
+    const T* z = (const T*)v.zw[c.cur];
+    if (c.n_word_tiles) {
+        EmitWord e{v.row_start, v.wk_topic, v.wk_count, v.wk_nnz};
+        k_seg_count_sorted<T, EmitWord><<<c.n_word_tiles, 256, 0, c.stream>>>(
+            c.word_tiles, v.word_off, z, v.topic_bits, c.K, e, v.err);
+        ++launches;
+    }
+    if (c.n_dense) {
+        cudaMemsetAsync(v.dense_rows, 0, (size_t)c.n_dense * c.K * 4, c.stream);
+        const int win = hist_window(c);
+        k_hist_chunks<T><<<c.n_hist_chunks, 512, (size_t)win * 4, c.stream>>>(
+            c.hist_chunks, z, v.dense_slot, v.dense_rows, c.K, win, v.err);
+        k_compact_dense<<<c.n_dense, 256, 0, c.stream>>>(c.dense_words, v.dense_slot, v.dense_rows,
+                                                         v.row_start, v.wk_topic, v.wk_count,
+                                                         v.wk_nnz, c.K, v.err);
+        launches += 2;
+    }
+    return launches;
+}
+
+template <typename T>
+static int count_k_t(Ctx& c)
+{
+    View& v = c.v;
+    cudaMemsetAsync(v.nk, 0, (size_t)c.K * 4, c.stream);
+    if (c.N == 0) return 0;
+    const int win = hist_window(c);
+    int grid = (int)((c.N + 65535) / 65536);
+    if (grid > 148 * 4) grid = 148 * 4;
+    if (grid < 1) grid = 1;
+    k_count_k<T><<<grid, 512, (size_t)win * 4, c.stream>>>((const T*)v.zw[c.cur], (int32_t)c.N, v.nk,
+                                                          c.K, win, v.err);
+    return 1;
+}
+
+template <typename T>
+static int count_dk_t(Ctx& c)
+{
+    View& v = c.v;
+    int launches = 0;
+    const T* z = (const T*)v.zd[c.cur];
+    if (c.n_doc_tiles) {
+        EmitDoc e{v.doc_off, v.dk_pairs, v.dk_nnz, v.count_bits};
+        k_seg_count_sorted<T, EmitDoc><<<c.n_doc_tiles, 256, 0, c.stream>>>(
+            c.doc_tiles, v.doc_off, z, v.topic_bits, c.K, e, v.err);
+        ++launches;
+    }
+    if (c.n_long_docs) {
+        const int win = hist_window(c);
+        k_long_docs<T><<<c.n_long_docs, 512, (size_t)win * 4, c.stream>>>(
+            c.long_docs, v.doc_off, z, v.dk_pairs, v.dk_nnz, c.K, win, v.count_bits, v.err);
+        ++launches;
+    }
+    return launches;
+}
+
+int launch_count_wk(Ctx& c) { return c.wide_topics ? count_wk_t<int32_t>(c) : count_wk_t<uint16_t>(c); }
+int launch_count_k(Ctx& c) { return c.wide_topics ? count_k_t<int32_t>(c) : count_k_t<uint16_t>(c); }
+int launch_count_dk(Ctx& c) { return c.wide_topics ? count_dk_t<int32_t>(c) : count_dk_t<uint16_t>(c); }
+
+int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host)
+{
+    unsigned long long* acc = (unsigned long long*)c.red_i;
+    cudaMemsetAsync(acc, 0, 16, c.stream);
+    k_sum_i32<<<296, 256, 0, c.stream>>>(c.v.wk_nnz, c.V, acc);
+    if (c.D) k_sum_i32<<<296, 256, 0, c.stream>>>(c.v.dk_nnz, c.D, acc + 1);
+    unsigned long long h[2] = {0, 0};
+    cudaMemcpyAsync(h, acc, 16, cudaMemcpyDeviceToHost, c.stream);
+    cudaStreamSynchronize(c.stream);
+    *nnz_wk_host = (int64_t)h[0];
+    *nnz_dk_host = (int64_t)h[1];
+    return 2;
+}
+
+void set_hist_smem_limits()
+{
+    cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
+    cudaFuncSetAttribute(k_hist_chunks<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
+    cudaFuncSetAttribute(k_long_docs<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
+    cudaFuncSetAttribute(k_long_docs<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
+    cudaFuncSetAttribute(k_count_k<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
+    cudaFuncSetAttribute(k_count_k<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
+}
+
+}  // namespace lda

@@ -1,0 +1,118 @@
+// One-time corpus layout (Section 6, item 3: token-topic pairs are sorted by
+// word once, so that the tokens of a word -- and of a slice of words -- are
+// contiguous).  Tokens are sorted stably by word id, so inside a word they
+// stay in document order.  The sort itself uses CUB's device radix sort: it
+// runs once per corpus, outside the per-sweep path.
+#include <cub/device/device_radix_sort.cuh>
+
+#include "lda_device.cuh"
+#include "lda_internal.cuh"
+
+namespace lda {
+
+__global__ void k_check_words_iota(const int32_t* __restrict__ words, uint32_t* __restrict__ iota,
+                                   int32_t n, int32_t V, int* err)
+{
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        iota[i] = (uint32_t)i;
+        const int32_t w = words[i];
+        if (w < 0 || w >= V) atomicOr(err, ERR_WORD_RANGE);
+    }
+}
+
+// word_off[w] = first position whose word is >= w (positions are word-sorted).
+__global__ void k_word_offsets(const int32_t* __restrict__ sorted_words, int32_t n, int32_t V,
+                               int32_t* __restrict__ word_off)
+{
+    const int32_t w = blockIdx.x * blockDim.x + threadIdx.x;
+    if (w > V) return;
+    int32_t lo = 0, hi = n;
+    while (lo < hi) {
+        const int32_t mid = lo + ((hi - lo) >> 1);
+        if (sorted_words[mid] < w) lo = mid + 1; else hi = mid;
+    }
+    word_off[w] = lo;
+}
+
+// Document of every token in word-sorted order: the last d with doc_off[d] <= orig.
+__global__ void k_token_docs(const uint32_t* __restrict__ tok_orig, const int32_t* __restrict__ doc_off,
+                             int32_t n, int32_t D, int32_t* __restrict__ tok_doc)
+{
+    for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < n;
+         p += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t i = (int32_t)tok_orig[p];
+        int32_t lo = 0, hi = D;  // find first d in [0,D] with doc_off[d] > i
+        while (lo < hi) {
+            const int32_t mid = lo + ((hi - lo) >> 1);
+            if (doc_off[mid + 1] <= i) lo = mid + 1; else hi = mid;
+        }
+        tok_doc[p] = lo;
+    }
+}
+
+int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_host)
+{
+    const int32_t N = (int32_t)c.N, D = (int32_t)c.D, V = c.V;
+    cudaStream_t st = c.stream;
+    const size_t n1 = (size_t)(N > 0 ? N : 1);
+
+    int32_t* tok_doc = (int32_t*)dev_alloc(c, n1 * 4);
+    uint32_t* tok_orig = (uint32_t*)dev_alloc(c, n1 * 4);
+    int32_t* word_off = (int32_t*)dev_alloc(c, ((size_t)V + 1) * 4);
+    int32_t* doc_off = (int32_t*)dev_alloc(c, ((size_t)D + 1) * 4);
+    if (!tok_doc || !tok_orig || !word_off || !doc_off) return LDA_ENOMEM;
+
+    std::vector<int32_t> doc32((size_t)D + 1);
+    for (int64_t d = 0; d <= D; ++d) doc32[(size_t)d] = (int32_t)doc_off_host[d];
+    if (cudaMemcpyAsync(doc_off, doc32.data(), ((size_t)D + 1) * 4, cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+        return LDA_ECUDA;
+
+    // transient buffers of the sort
+    int32_t* keys_out = nullptr;
+    uint32_t* iota = nullptr;
+    void* temp = nullptr;
+    size_t temp_bytes = 0;
+    int rc = LDA_OK;
+    do {
+        if (cudaMalloc(&keys_out, n1 * 4) != cudaSuccess || cudaMalloc(&iota, n1 * 4) != cudaSuccess) {
+            rc = LDA_ENOMEM;
+            break;
+        }
+        if (N > 0) {
+            k_check_words_iota<<<1184, 256, 0, st>>>(word_ids_dev, iota, N, V, c.v.err);
+            int end_bit = 1;
+            while (end_bit < 31 && (1ll << end_bit) < (long long)V) ++end_bit;
+            if (cub::DeviceRadixSort::SortPairs(nullptr, temp_bytes, word_ids_dev, keys_out, iota,
+                                                tok_orig, N, 0, end_bit, st) != cudaSuccess) {
+                rc = LDA_ECUDA;
+                break;
+            }
+            if (cudaMalloc(&temp, temp_bytes ? temp_bytes : 1) != cudaSuccess) {
+                rc = LDA_ENOMEM;
+                break;
+            }
+            if (cub::DeviceRadixSort::SortPairs(temp, temp_bytes, word_ids_dev, keys_out, iota,
+                                                tok_orig, N, 0, end_bit, st) != cudaSuccess) {
+                rc = LDA_ECUDA;
+                break;
+            }
+            k_token_docs<<<1184, 256, 0, st>>>(tok_orig, doc_off, N, D, tok_doc);
+        }
+        k_word_offsets<<<(V + 1 + 255) / 256, 256, 0, st>>>(keys_out, N, V, word_off);
+        if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess)
+            rc = LDA_ECUDA;
+    } while (0);
+    cudaFree(keys_out);
+    cudaFree(iota);
+    cudaFree(temp);
+    if (rc != LDA_OK) return rc;
+    c.v.tok_doc = tok_doc;
+    c.v.tok_orig = tok_orig;
+    c.v.word_off = word_off;
+    c.v.doc_off = doc_off;
+    return LDA_OK;
+}
+
+}  // namespace lda

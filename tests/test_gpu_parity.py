@@ -1,0 +1,225 @@
+"""CUDA path against the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import ldaref
+from paper_1412_1576_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+SEED = 20260
+
+
+def _pair(c, seed=SEED, options=None):
+    g = binding.LightLDA(c.V, c.K, c.alpha, c.beta, options=options)
+    g.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    g.init(seed)
+    o = ldaref.Oracle(c.V, c.K, c.alpha, c.beta)
+    o.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    o.init(seed)
+    return g, o
+
+
+def _assert_same_counts(g, o):
+    assert np.array_equal(g.get_nk(), o.get_nk())
+    for which in (binding.LDA_NWK, binding.LDA_NDK):
+        a, b = g.get_csr(which), o.get_csr(which)
+        assert np.array_equal(a[0], b[0])
+        assert np.array_equal(a[1], b[1])
+        assert np.array_equal(a[2], b[2])
+
+
+def _assert_same_tables(g, o):
+    a, b = g.get_tables(), o.get_tables()
+    assert a["dense_mass"] == b["dense_mass"]
+    for k in ("dn_thr32", "dn_alias", "mix32", "sp_thr32", "sp_alias"):
+        assert np.array_equal(a[k], b[k]), k
+
+
+def _toy(V, K, D, L, alpha=0.3, beta=0.2, seed=3, length=None):
+    return synth.generate(V=V, K=K, D=D, length=length or ("fixed", L), zipf_s=None, alpha=alpha,
+                          beta=beta, seed=seed)
+
+
+def test_init_and_counts_tiny(tiny_corpus):
+    g, o = _pair(tiny_corpus)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_counts(g, o)
+
+
+def test_tables_bit_equal_tiny(tiny_corpus):
+    g, o = _pair(tiny_corpus)
+    _assert_same_tables(g, o)
+    o.sweep(2, 2)
+    g.set_assignments(o.get_assignments(), SEED, 2)
+    _assert_same_counts(g, o)
+    _assert_same_tables(g, o)
+
+
+def test_sweeps_bit_equal_tiny(tiny_corpus):
+    """fp64 acceptance in the same operation order: every token agrees, every sweep."""
+    g, o = _pair(tiny_corpus)
+    for sweep in range(20):
+        g.sweep(1, 2)
+        o.sweep(1, 2)
+        assert np.array_equal(g.get_assignments(), o.get_assignments()), sweep
+    _assert_same_counts(g, o)
+    lg, lo = g.loglik(), o.loglik()
+    for a, b in zip(lg, lo):
+        assert a == pytest.approx(b, rel=1e-10)
+
+
+@pytest.mark.parametrize("mh_steps", [1, 3, 4])
+def test_other_step_counts_tiny(tiny_corpus, mh_steps):
+    g, o = _pair(tiny_corpus, seed=7)
+    g.sweep(3, mh_steps)
+    o.sweep(3, mh_steps)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+
+
+def test_small_config_sweeps_counts_tables_loglik(small_corpus):
+    """~2M tokens: many tiles, ragged tails, dense and sparse words, hot-word histogram path."""
+    c = small_corpus
+    g, o = _pair(c)
+    st = g.stats()
+    assert 0 < st["n_dense_words"] < c.V
+    _assert_same_counts(g, o)
+    _assert_same_tables(g, o)
+    for sweep in range(3):
+        g.sweep(1, 2)
+        o.sweep(1, 2)
+        zg, zo = g.get_assignments(), o.get_assignments()
+        agree = float(np.mean(zg == zo))
+        assert agree >= 0.999, (sweep, agree)
+        assert np.array_equal(zg, zo), sweep
+    _assert_same_counts(g, o)
+    _assert_same_tables(g, o)
+    for a, b in zip(g.loglik(), o.loglik()):
+        assert a == pytest.approx(b, rel=1e-10)
+
+
+def test_small_config_loglik_trajectory_50_sweeps(small_corpus):
+    """Free-running 50 sweeps: log-likelihood within 0.5 % of the oracle's at every sweep."""
+    c = small_corpus
+    g, o = _pair(c, seed=99)
+    for sweep in range(50):
+        g.sweep(1, 2)
+        o.sweep(1, 2)
+        if sweep % 7 == 0 or sweep == 49:
+            a, b = g.loglik()[0], o.loglik()[0]
+            assert abs(a - b) <= 0.005 * abs(b), (sweep, a, b)
+    assert float(np.mean(g.get_assignments() == o.get_assignments())) >= 0.999
+
+
+def test_counts_consistent_with_own_assignments(small_corpus):
+    """The library's tables equal a brute-force recount of its own z (bit exact)."""
+    c = small_corpus
+    g = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
+    g.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    g.init(5)
+    g.sweep(4, 2)
+    z = g.get_assignments()
+    w = c.word_ids.numpy().astype(np.int64)
+    off = c.doc_offsets.numpy()
+    doc = np.repeat(np.arange(off.size - 1), np.diff(off))
+    assert np.array_equal(g.get_nk(), np.bincount(z, minlength=c.K))
+    for which, seg, rows in ((binding.LDA_NWK, w, c.V), (binding.LDA_NDK, doc, off.size - 1)):
+        ro, top, cnt = g.get_csr(which)
+        key = seg * c.K + z
+        uk, uc = np.unique(key, return_counts=True)
+        assert np.array_equal(uk // c.K * 0 + top, uk % c.K)
+        assert np.array_equal(cnt, uc)
+        assert np.array_equal(ro, np.searchsorted(uk // c.K, np.arange(rows + 1)))
+
+
+@pytest.mark.parametrize("dense_frac", [0.0, 1.0])
+def test_dense_sparse_split_is_invisible(tiny_corpus, dense_frac):
+    """Section 5: the hybrid row storage must not change any result."""
+    c = tiny_corpus
+    g, o = _pair(c, seed=11, options={"dense_frac": dense_frac, "dense_min_tf": 1})
+    g.sweep(3, 2)
+    o.sweep(3, 2)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_counts(g, o)
+    _assert_same_tables(g, o)
+
+
+def test_wide_topics_and_long_documents():
+    """K > 65536 uses 32-bit topic storage; documents longer than a sort tile use the histogram path."""
+    c = synth.generate(V=300, K=70_000, D=40, length=("fixed", 100), zipf_s=1.0, alpha=0.01, beta=0.01,
+                       seed=4)
+    g, o = _pair(c, seed=3)
+    _assert_same_counts(g, o)
+    g.sweep(2, 2)
+    o.sweep(2, 2)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_counts(g, o)
+    c2 = synth.generate(V=50, K=40, D=6, length=("fixed", 5000), zipf_s=1.0, alpha=0.1, beta=0.01, seed=5)
+    g, o = _pair(c2, seed=3)
+    _assert_same_counts(g, o)
+    _assert_same_tables(g, o)
+    g.sweep(2, 4)
+    o.sweep(2, 4)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_counts(g, o)
+
+
+def test_edge_cases():
+    # empty documents, a single token, one topic, absent words
+    w = np.array([3, 3, 0, 7, 7, 7], np.int32)
+    off = np.array([0, 0, 2, 2, 3, 6, 6], np.int64)
+    for K in (1, 2, 5):
+        g = binding.LightLDA(9, K, 0.5, 0.1)
+        g.load_corpus(w, off)
+        g.init(1)
+        o = ldaref.Oracle(9, K, 0.5, 0.1)
+        o.load_corpus(w, off)
+        o.init(1)
+        g.sweep(3, 2)
+        o.sweep(3, 2)
+        assert np.array_equal(g.get_assignments(), o.get_assignments())
+        _assert_same_counts(g, o)
+        for a, b in zip(g.loglik(), o.loglik()):
+            assert a == pytest.approx(b, rel=1e-10, abs=1e-9)
+    # empty corpus
+    g = binding.LightLDA(4, 3, 0.5, 0.1)
+    g.load_corpus(np.zeros(0, np.int32), np.zeros(1, np.int64))
+    g.init(0)
+    g.sweep(2, 2)
+    assert g.get_assignments().size == 0
+
+
+def test_error_paths():
+    g = binding.LightLDA(4, 3, 0.5, 0.1)
+    with pytest.raises(binding.LdaError) as e:
+        g.sweep(1, 2)
+    assert e.value.status == binding.LDA_ESTATE
+    with pytest.raises(binding.LdaError) as e:
+        g.load_corpus(np.array([0, 9], np.int32), np.array([0, 2], np.int64))
+    assert e.value.status == binding.LDA_ERANGE
+    with pytest.raises(binding.LdaError) as e:
+        g.load_corpus(np.array([0, 1], np.int32), np.array([0, 3], np.int64))
+    assert e.value.status == binding.LDA_ERANGE
+    g.load_corpus(np.array([0, 1], np.int32), np.array([0, 2], np.int64))
+    with pytest.raises(binding.LdaError) as e:
+        g.set_assignments(np.array([0, 5], np.int32), 0)
+    assert e.value.status == binding.LDA_ERANGE
+    g.init(0)
+    with pytest.raises(binding.LdaError) as e:
+        g.sweep(1, 0)
+    assert e.value.status == binding.LDA_EINVAL
+    g.sweep(1, 2)   # the context is still usable after the refused calls
+
+
+def test_device_resident_load_matches_host_load(tiny_corpus):
+    import torch
+    c = tiny_corpus
+    a = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
+    a.load_corpus(c.word_ids.cuda(), c.doc_offsets.cuda())
+    a.init(9)
+    b = binding.LightLDA(c.V, c.K, c.alpha, c.beta, stream=torch.cuda.current_stream().cuda_stream)
+    b.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    b.init(9)
+    a.sweep(2, 2)
+    b.sweep(2, 2)
+    assert np.array_equal(a.get_assignments(), b.get_assignments())
