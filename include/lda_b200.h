@@ -122,6 +122,36 @@ int lda_get_assignments(lda_ctx* ctx, int32_t* z_out);
 int lda_get_tables(lda_ctx* ctx, uint32_t* sp_thr32, int32_t* sp_alias, int64_t capacity,
                    uint32_t* mix32, uint32_t* dn_thr32, int32_t* dn_alias, uint64_t* dense_mass);
 
+/* Dense smoothing table without any allocation (the paper has no counterpart: this exists for
+ * callers of the library, not for the method).
+ *
+ * Who needs it: code that may not allocate device memory when it runs -- a component living
+ * inside another framework's memory pool, a latency-critical loop that cannot afford the
+ * device-wide synchronisation an allocation can imply, a process whose memory was budgeted
+ * at start-up.  Every other entry point here may allocate; this one calls no cudaMalloc,
+ * cudaFree or allocating library routine.
+ *
+ * Computes exactly what lda_get_tables() reports as dn_thr32 / dn_alias / dense_mass: the alias
+ * table over k of beta / (n_k[k] + V*beta).  All pointers are DEVICE memory owned by the caller:
+ *   n_k_dev[K] in; dn_thr32_dev[K], dn_alias_dev[K], dense_mass_dev[1] out;
+ *   status_dev[1] out, may be NULL: 0 on success, else the library's device error bits.
+ * The work is queued on `cuda_stream` (a cudaStream_t, NULL = default stream) and the call
+ * returns without waiting for it.
+ *
+ * The construction scratch is a fixed device array inside the library, sized for
+ * LDA_NOALLOC_MAX_K topics (20 bytes per topic, about 2.6 MB); every GPU that loads the library
+ * holds it until the process exits.  K above LDA_NOALLOC_MAX_K is refused with LDA_ERANGE.
+ * The first call on each device looks up the array's device address (one runtime query, made
+ * with that device current); make that first call before starting any stream capture.
+ * All calls share the one array and it keeps the previous call's contents; nothing in it needs
+ * clearing because each call overwrites what it later reads, and the status word is zeroed on
+ * the stream before the kernel.  Two calls that overlap on the GPU (different streams, or
+ * different host threads) race on the array and give undefined tables: serialise them. */
+#define LDA_NOALLOC_MAX_K 131072
+int lda_dense_table_noalloc(const int32_t* n_k_dev, int32_t K, int32_t V, double beta,
+                            uint32_t* dn_thr32_dev, int32_t* dn_alias_dev, uint64_t* dense_mass_dev,
+                            int32_t* status_dev, void* cuda_stream);
+
 int lda_get_stats(lda_ctx* ctx, lda_stats* out);
 
 /* Message of the last failure on this context (library-owned, valid until the next call). */

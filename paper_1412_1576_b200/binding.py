@@ -23,6 +23,7 @@ EXPORTS = [
     "lda_create", "lda_set_stream", "lda_set_option", "lda_load_corpus", "lda_load_corpus_device",
     "lda_init", "lda_set_assignments", "lda_sweep", "lda_loglik", "lda_get_counts",
     "lda_get_assignments", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
+    "lda_dense_table_noalloc",
 ]
 
 
@@ -78,6 +79,7 @@ def load_library(path: str | None = None):
     L.lda_get_assignments.argtypes = [vp, vp]
     L.lda_get_tables.argtypes = [vp, vp, vp, i64, vp, vp, vp, C.POINTER(u64)]
     L.lda_get_stats.argtypes = [vp, C.POINTER(lda_stats)]
+    L.lda_dense_table_noalloc.argtypes = [vp, i32, i32, dbl, vp, vp, vp, vp, vp]
     L.lda_last_error.argtypes = [vp]
     L.lda_last_error.restype = C.c_char_p
     L.lda_destroy.argtypes = [vp]
@@ -169,6 +171,16 @@ def lda_get_tables(h, sp_thr32, sp_alias, mix32, dn_thr32, dn_alias):
     rc = load_library().lda_get_tables(h, p(sp_thr32), p(sp_alias), cap, p(mix32), p(dn_thr32),
                                        p(dn_alias), C.byref(B))
     return rc, B.value
+
+
+def lda_dense_table_noalloc(n_k_ptr, K, V, beta, dn_thr32_ptr, dn_alias_ptr, dense_mass_ptr,
+                            status_ptr=None, cuda_stream=None):
+    """Dense smoothing table into caller-owned DEVICE buffers (raw pointers); the library
+    allocates nothing.  Queued on ``cuda_stream``; returns the launch status only."""
+    return load_library().lda_dense_table_noalloc(
+        C.c_void_p(n_k_ptr), K, V, beta, C.c_void_p(dn_thr32_ptr), C.c_void_p(dn_alias_ptr),
+        C.c_void_p(dense_mass_ptr), C.c_void_p(status_ptr) if status_ptr else None,
+        C.c_void_p(cuda_stream) if cuda_stream else None)
 
 
 def lda_get_stats(h):

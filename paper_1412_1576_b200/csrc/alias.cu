@@ -244,3 +244,86 @@ int launch_alias_sparse(Ctx& c)
 }
 
 }  // namespace lda
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free entry point.
+//
+// Some callers cannot allocate device memory at the moment they need a table: code that
+// runs inside a framework's memory pool and must not touch cudaMalloc behind its back, a
+// real-time loop where an allocation's implicit device synchronisation is not acceptable,
+// or a process whose memory budget was fixed at start-up.  For them the dense smoothing
+// table can be built with the construction scratch held in a file-scope device array.
+// Every GPU that loads the library holds that array (20 bytes per topic of LDA_NOALLOC_MAX_K,
+// about 2.6 MB) until exit.
+// ---------------------------------------------------------------------------------------
+namespace lda {
+
+constexpr int NOALLOC_MAX_K = LDA_NOALLOC_MAX_K;
+// per topic: one 64-bit mass, one 64-bit prefix sum, one 32-bit item index = 20 bytes
+constexpr size_t NOALLOC_SCRATCH_WORDS = 2 * (size_t)NOALLOC_MAX_K + (size_t)NOALLOC_MAX_K / 2;
+
+static __device__ __align__(256) unsigned long long g_noalloc_scratch[NOALLOC_SCRATCH_WORDS];
+static __device__ __align__(256) int g_noalloc_status[4];
+
+// Device addresses of the two arrays above, looked up once per device.  In host code the
+// array names are only handles for the runtime, not addresses a kernel could use.
+struct NoallocAddr {
+    bool ready = false;
+    unsigned long long* scratch = nullptr;
+    int* status = nullptr;
+};
+static NoallocAddr g_noalloc_addr[64];
+
+static int noalloc_setup(int dev, NoallocAddr** out)
+{
+    if (dev < 0 || dev >= 64) return LDA_ERANGE;
+    NoallocAddr& a = g_noalloc_addr[dev];
+    if (!a.ready) {
+        void* p = nullptr;
+        void* q = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess ||
+            cudaGetSymbolAddress(&q, g_noalloc_status) != cudaSuccess) {
+            cudaGetLastError();
+            return LDA_ECUDA;
+        }
+        a.scratch = (unsigned long long*)p;
+        a.status = (int*)q;
+        a.ready = true;
+    }
+    *out = &a;
+    return LDA_OK;
+}
+
+}  // namespace lda
+
+extern "C" int lda_dense_table_noalloc(const int32_t* n_k_dev, int32_t K, int32_t V, double beta,
+                                       uint32_t* dn_thr32_dev, int32_t* dn_alias_dev,
+                                       uint64_t* dense_mass_dev, int32_t* status_dev, void* cuda_stream)
+{
+    using namespace lda;
+    if (!n_k_dev || !dn_thr32_dev || !dn_alias_dev || !dense_mass_dev) return LDA_EINVAL;
+    if (K <= 0 || V <= 0 || !(beta > 0) || !isfinite(beta)) return LDA_EINVAL;
+    if (K > NOALLOC_MAX_K) return LDA_ERANGE;  // the fixed scratch array holds LDA_NOALLOC_MAX_K topics
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LDA_ECUDA; }
+    NoallocAddr* addr = nullptr;
+    int rc = noalloc_setup(dev, &addr);
+    if (rc != LDA_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int* status = status_dev ? (int*)status_dev : addr->status;
+    // the status word must start at zero; the scratch itself is fully overwritten before it is read
+    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) { cudaGetLastError(); return LDA_ECUDA; }
+    View v{};
+    v.V = V;
+    v.K = K;
+    v.beta = beta;
+    v.Vbeta = (double)V * beta;
+    v.nk = const_cast<int32_t*>(n_k_dev);
+    v.dn_thr = dn_thr32_dev;
+    v.dn_idx = (uint32_t*)dn_alias_dev;
+    v.dense_mass = (unsigned long long*)dense_mass_dev;
+    v.err = status;
+    k_alias_dense<<<1, 1024, 0, st>>>(v, addr->scratch);
+    if (cudaGetLastError() != cudaSuccess) return LDA_ECUDA;
+    return LDA_OK;
+}
