@@ -19,7 +19,7 @@
  *     called).  One host thread per context.
  *   - all calls are synchronous: results are complete when they return.
  *   - limits: n_tokens < 2^31, K <= 131072; bitlen(K-1) + bitlen(longest
- *     document) <= 32 (n_kd entries are stored as one packed 32-bit word).
+ *     document + 1) <= 32 (n_kd entries are stored as one packed 32-bit word).
  *
  * There is no CPU fallback: every entry point that computes needs the GPU.
  */

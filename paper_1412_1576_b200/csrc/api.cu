@@ -127,8 +127,8 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     for (int64_t d = 0; d < n_docs; ++d) max_len = std::max(max_len, doc_off[d + 1] - doc_off[d]);
     int tb = 1;
     while ((1ll << tb) < (long long)K) ++tb;
-    int cb = 1;
-    while ((1ll << cb) <= max_len) ++cb;
+    int cb = 1;  // a count never has all bits set, so no entry equals the empty-slot marker
+    while ((1ll << cb) <= max_len + 1) ++cb;
     if (tb + cb > 32) {
         free_corpus(c);
         return fail(&c, LDA_ERANGE, "bits(K-1) + bits(longest document) exceeds 32");
@@ -240,8 +240,7 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     v.dn_idx = (uint32_t*)A((size_t)K * 4);
     v.dense_mass = (unsigned long long*)A(8);
     v.nk = (int32_t*)A((size_t)K * 4);
-    v.dk_pairs = (uint32_t*)A(n1 * 4);
-    v.dk_nnz = (int32_t*)A((size_t)std::max<int32_t>(D, 1) * 4);
+    v.dk_slots = (uint32_t*)A(n1 * 8);
     c.sc_w = (unsigned long long*)A(cap1 * 8);
     c.sc_de = (unsigned long long*)A(cap1 * 8);
     c.sc_item = (uint32_t*)A(cap1 * 4);
@@ -250,7 +249,6 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.red_i = (int64_t*)A(16);
     if (!ok) { free_corpus(c); return fail(&c, LDA_ENOMEM, "device allocation failed"); }
     cudaMemsetAsync(v.wk_nnz, 0, (size_t)V * 4, c.stream);
-    cudaMemsetAsync(v.dk_nnz, 0, (size_t)std::max<int32_t>(D, 1) * 4, c.stream);
     cudaMemsetAsync(v.mix32, 0, (size_t)V * 4, c.stream);
     cudaMemsetAsync(v.nk, 0, (size_t)K * 4, c.stream);
     if (cudaStreamSynchronize(c.stream) != cudaSuccess) { free_corpus(c); return cuda_fail(&c, "load"); }
@@ -537,13 +535,43 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
         }
         return LDA_OK;
     }
-    if (which != LDA_NWK && which != LDA_NDK) return fail(&c, LDA_EINVAL, "unknown table");
-    const bool words = which == LDA_NWK;
-    const int64_t rows = words ? c.V : c.D;
-    std::vector<int32_t> nnz((size_t)std::max<int64_t>(rows, 1)), start((size_t)rows + 1);
-    if (rows && cudaMemcpy(nnz.data(), words ? v.wk_nnz : v.dk_nnz, (size_t)rows * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+    if (which == LDA_NDK) {
+        // every document's table is copied out and its filled slots sorted by topic on the host
+        std::vector<int32_t> start((size_t)c.D + 1);
+        if (cudaMemcpy(start.data(), v.doc_off, ((size_t)c.D + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+            return cuda_fail(&c, "copying document offsets");
+        std::vector<uint32_t> slots((size_t)std::max<int64_t>(2 * c.N, 1));
+        if (c.N && cudaMemcpy(slots.data(), v.dk_slots, (size_t)c.N * 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+            return cuda_fail(&c, "copying n_kd tables");
+        int64_t total = 0;
+        for (uint32_t e : slots) total += (c.N && e != DK_EMPTY);
+        if (nnz_out) *nnz_out = total;
+        if (!row_offsets && !topics && !counts) return LDA_OK;
+        if (capacity < total) return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros");
+        const uint32_t cmask = (1u << v.count_bits) - 1u;
+        std::vector<uint32_t> row;
+        int64_t o = 0;
+        for (int64_t d = 0; d < c.D; ++d) {
+            if (row_offsets) row_offsets[d] = o;
+            row.clear();
+            for (int64_t j = 2 * (int64_t)start[(size_t)d]; j < 2 * (int64_t)start[(size_t)d + 1]; ++j)
+                if (slots[(size_t)j] != DK_EMPTY) row.push_back(slots[(size_t)j]);
+            std::sort(row.begin(), row.end());
+            for (uint32_t e : row) {
+                if (topics) topics[o] = (int32_t)(e >> v.count_bits);
+                if (counts) counts[o] = (int32_t)(e & cmask);
+                ++o;
+            }
+        }
+        if (row_offsets) row_offsets[c.D] = o;
+        return LDA_OK;
+    }
+    if (which != LDA_NWK) return fail(&c, LDA_EINVAL, "unknown table");
+    const int64_t rows = c.V;
+    std::vector<int32_t> nnz((size_t)rows), start((size_t)rows + 1);
+    if (cudaMemcpy(nnz.data(), v.wk_nnz, (size_t)rows * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
         return cuda_fail(&c, "copying row sizes");
-    if (cudaMemcpy(start.data(), words ? v.row_start : v.doc_off, ((size_t)rows + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+    if (cudaMemcpy(start.data(), v.row_start, ((size_t)rows + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
         return cuda_fail(&c, "copying row starts");
     int64_t total = 0;
     for (int64_t r = 0; r < rows; ++r) total += nnz[(size_t)r];
@@ -551,28 +579,17 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
     if (!row_offsets && !topics && !counts) return LDA_OK;
     if (capacity < total) return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros");
     const size_t cap = (size_t)start[(size_t)rows];
-    std::vector<uint32_t> a(std::max<size_t>(cap, 1)), b;
-    if (words) {
-        b.resize(std::max<size_t>(cap, 1));
-        if (cap && (cudaMemcpy(a.data(), v.wk_topic, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
-                    cudaMemcpy(b.data(), v.wk_count, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess))
-            return cuda_fail(&c, "copying n_kw rows");
-    } else if (cap && cudaMemcpy(a.data(), v.dk_pairs, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
-        return cuda_fail(&c, "copying n_kd rows");
-    }
-    const uint32_t cmask = (1u << v.count_bits) - 1u;
+    std::vector<uint32_t> a(std::max<size_t>(cap, 1)), b(std::max<size_t>(cap, 1));
+    if (cap && (cudaMemcpy(a.data(), v.wk_topic, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+                cudaMemcpy(b.data(), v.wk_count, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess))
+        return cuda_fail(&c, "copying n_kw rows");
     int64_t o = 0;
     for (int64_t r = 0; r < rows; ++r) {
         if (row_offsets) row_offsets[r] = o;
         const size_t s0 = (size_t)start[(size_t)r];
         for (int32_t j = 0; j < nnz[(size_t)r]; ++j, ++o) {
-            if (words) {
-                if (topics) topics[o] = (int32_t)a[s0 + j];
-                if (counts) counts[o] = (int32_t)b[s0 + j];
-            } else {
-                if (topics) topics[o] = (int32_t)(a[s0 + j] >> v.count_bits);
-                if (counts) counts[o] = (int32_t)(a[s0 + j] & cmask);
-            }
+            if (topics) topics[o] = (int32_t)a[s0 + j];
+            if (counts) counts[o] = (int32_t)b[s0 + j];
         }
     }
     if (row_offsets) row_offsets[rows] = o;

@@ -1,16 +1,16 @@
 // Count-table rebuild from the assignments (Section 3: n_kw, n_k; Eq. 12: n_kd).
 //
-// Both n_kw (segments = words over the word-sorted z) and n_kd (segments =
-// documents over the document-order z) are "per contiguous segment, the sorted
-// list of (topic, count)".  Two paths, chosen per segment at load time:
-//   - short segments: whole segments are packed into tiles of <= SORT_TILE
-//     tokens; one CTA sorts the tile's (segment, topic) keys in shared memory
-//     and run-length encodes them;
-//   - long segments (hot words, very long documents): shared-memory histogram
-//     over a window of topics, merged into the word's dense row (words) or
-//     compacted directly (documents).
+// n_kw (segments = words over the word-sorted z): per word, the sorted list of
+// (topic, count).  Two paths, chosen per word at load time:
+//   - tail words: whole words are packed into tiles of <= SORT_TILE tokens; one
+//     CTA sorts the tile's (word, topic) keys in shared memory and run-length
+//     encodes them;
+//   - hot words: shared-memory histogram over a window of topics, merged into
+//     the word's dense row, then compacted into the sorted row.
+// n_kd (segments = documents over the document-order z): per document an
+// open-addressing table built by insertion in shared memory.
 // No per-token global atomics: a CTA touches global counters once per bin it
-// actually filled.
+// actually filled (documents longer than a tile are the one exception).
 #include "lda_device.cuh"
 #include "lda_internal.cuh"
 
@@ -26,18 +26,6 @@ struct EmitWord {
         const int32_t slot = row_start[seg] + rank;
         topic[slot] = k;
         count[slot] = n;
-    }
-    __device__ __forceinline__ void rows(int32_t seg, int32_t n) const { nnz[seg] = n; }
-};
-
-struct EmitDoc {
-    const int32_t* doc_off;
-    uint32_t* pairs;
-    int32_t* nnz;
-    int count_bits;
-    __device__ __forceinline__ void entry(int32_t seg, int32_t rank, uint32_t k, uint32_t n) const
-    {
-        pairs[doc_off[seg] + rank] = (k << count_bits) | n;
     }
     __device__ __forceinline__ void rows(int32_t seg, int32_t n) const { nnz[seg] = n; }
 };
@@ -192,41 +180,73 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
     if (threadIdx.x == 0) wk_nnz[w] = done;
 }
 
-// Documents longer than a sort tile: one CTA per document, windowed histogram,
-// compacted straight into the document's row.
+// n_kd as per-document open-addressing tables (Section 5, fn. 5: capacity twice the number of
+// tokens, so the load factor stays <= 0.5).  One CTA per tile of whole documents holding
+// <= SORT_TILE tokens: the tile's tables are built in shared memory by insertion (claim a slot
+// with compare-and-swap, then add one to its count bits) and written out in one coalesced pass.
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_off,
+           const T* __restrict__ z, uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
+{
+    __shared__ uint32_t slots[2 * SORT_TILE];
+    __shared__ int32_t soff[SORT_TILE + 1];
+    const int tid = threadIdx.x;
+    const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
+    const int32_t nseg = s1 - s0;
+    const int32_t base = doc_off[s0];
+    const int32_t cnt = doc_off[s1] - base;
+    if (cnt == 0) return;
+    for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = doc_off[s0 + j] - base;
+    for (int j = tid; j < 2 * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
+    __syncthreads();
+    for (int j = tid; j < cnt; j += blockDim.x) {
+        int lo = 0, hi = nseg;  // last document with soff[doc] <= j
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (soff[mid] <= j) lo = mid; else hi = mid;
+        }
+        const uint32_t k = (uint32_t)z[base + j];
+        if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+        const uint32_t cap = 2u * (uint32_t)(soff[lo + 1] - soff[lo]);
+        uint32_t* tab = slots + 2 * soff[lo];
+        uint32_t h = __umulhi(k * DK_HASH, cap);
+        const uint32_t fresh = k << count_bits;
+        for (uint32_t probe = 0; probe < cap; ++probe) {
+            const uint32_t prev = atomicCAS(&tab[h], DK_EMPTY, fresh);
+            if (prev == DK_EMPTY || (prev >> count_bits) == k) { atomicAdd(&tab[h], 1u); break; }
+            if (++h == cap) h = 0;
+        }
+    }
+    __syncthreads();
+    uint32_t* out = slots_out + 2 * (size_t)base;
+    for (int j = tid; j < 2 * cnt; j += blockDim.x) out[j] = slots[j];
+}
+
+// Documents longer than a tile: one CTA per document, the same insertion straight in global memory.
 template <typename T>
 __global__ void __launch_bounds__(512)
-k_long_docs(const int32_t* __restrict__ long_docs, const int32_t* __restrict__ doc_off,
-            const T* __restrict__ z, uint32_t* __restrict__ pairs, int32_t* __restrict__ dk_nnz,
-            int32_t K, int32_t window, int count_bits, int* err)
+k_long_doc_hash(const int32_t* __restrict__ long_docs, const int32_t* __restrict__ doc_off,
+                const T* __restrict__ z, uint32_t* __restrict__ slots_out, int count_bits, int32_t K,
+                int* err)
 {
-    extern __shared__ int32_t bins[];
-    __shared__ int32_t scan_tmp[33];
     const int32_t d = long_docs[blockIdx.x];
     const int32_t first = doc_off[d], cnt = doc_off[d + 1] - first;
-    int32_t done = 0;
-    for (int32_t k0 = 0; k0 < K; k0 += window) {
-        const int32_t nb = min(window, K - k0);
-        for (int b = threadIdx.x; b < nb; b += blockDim.x) bins[b] = 0;
-        __syncthreads();
-        for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-            const uint32_t k = (uint32_t)z[first + j];
-            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
-            const uint32_t b = k - (uint32_t)k0;
-            if (b < (uint32_t)nb) atomicAdd(&bins[b], 1);
+    const uint32_t cap = 2u * (uint32_t)cnt;
+    uint32_t* tab = slots_out + 2 * (size_t)first;
+    for (uint32_t j = threadIdx.x; j < cap; j += blockDim.x) tab[j] = DK_EMPTY;
+    __syncthreads();
+    for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
+        const uint32_t k = (uint32_t)z[first + j];
+        if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+        uint32_t h = __umulhi(k * DK_HASH, cap);
+        const uint32_t fresh = k << count_bits;
+        for (uint32_t probe = 0; probe < cap; ++probe) {
+            const uint32_t prev = atomicCAS(&tab[h], DK_EMPTY, fresh);
+            if (prev == DK_EMPTY || (prev >> count_bits) == k) { atomicAdd(&tab[h], 1u); break; }
+            if (++h == cap) h = 0;
         }
-        __syncthreads();
-        for (int32_t b0 = 0; b0 < nb; b0 += blockDim.x) {
-            const int32_t b = b0 + threadIdx.x;
-            const int32_t n = (b < nb) ? bins[b] : 0;
-            int32_t total;
-            const int32_t pos = block_scan_excl<int32_t>(n > 0 ? 1 : 0, scan_tmp, total);
-            if (n > 0) pairs[first + done + pos] = ((uint32_t)(k0 + b) << count_bits) | (uint32_t)n;
-            done += total;
-        }
-        __syncthreads();
     }
-    if (threadIdx.x == 0) dk_nnz[d] = done;
 }
 
 // n_k: histogram of all assignments, CTA-private shared-memory bins.
@@ -264,6 +284,17 @@ __global__ void k_sum_i32(const int32_t* __restrict__ a, int64_t n, unsigned lon
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
          i += (int64_t)gridDim.x * blockDim.x)
         s += (unsigned long long)a[i];
+    s = block_reduce_sum<unsigned long long>(s, tmp);
+    if (threadIdx.x == 0 && s) atomicAdd(out, s);
+}
+
+__global__ void k_count_filled(const uint32_t* __restrict__ slots, int64_t n, unsigned long long* out)
+{
+    __shared__ unsigned long long tmp[32];
+    unsigned long long s = 0;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+         i += (int64_t)gridDim.x * blockDim.x)
+        s += slots[i] != DK_EMPTY;
     s = block_reduce_sum<unsigned long long>(s, tmp);
     if (threadIdx.x == 0 && s) atomicAdd(out, s);
 }
@@ -317,15 +348,13 @@ static int count_dk_t(Ctx& c)
     int launches = 0;
     const T* z = (const T*)v.zd[c.cur];
     if (c.n_doc_tiles) {
-        EmitDoc e{v.doc_off, v.dk_pairs, v.dk_nnz, v.count_bits};
-        k_seg_count_sorted<T, EmitDoc><<<c.n_doc_tiles, 256, 0, c.stream>>>(
-            c.doc_tiles, v.doc_off, z, v.topic_bits, c.K, e, v.err);
+        k_doc_hash<T><<<c.n_doc_tiles, 256, 0, c.stream>>>(c.doc_tiles, v.doc_off, z, v.dk_slots,
+                                                          v.count_bits, c.K, v.err);
         ++launches;
     }
     if (c.n_long_docs) {
-        const int win = hist_window(c);
-        k_long_docs<T><<<c.n_long_docs, 512, (size_t)win * 4, c.stream>>>(
-            c.long_docs, v.doc_off, z, v.dk_pairs, v.dk_nnz, c.K, win, v.count_bits, v.err);
+        k_long_doc_hash<T><<<c.n_long_docs, 512, 0, c.stream>>>(c.long_docs, v.doc_off, z, v.dk_slots,
+                                                               v.count_bits, c.K, v.err);
         ++launches;
     }
     return launches;
@@ -340,7 +369,7 @@ int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host)
     unsigned long long* acc = (unsigned long long*)c.red_i;
     cudaMemsetAsync(acc, 0, 16, c.stream);
     k_sum_i32<<<296, 256, 0, c.stream>>>(c.v.wk_nnz, c.V, acc);
-    if (c.D) k_sum_i32<<<296, 256, 0, c.stream>>>(c.v.dk_nnz, c.D, acc + 1);
+    if (c.N) k_count_filled<<<592, 256, 0, c.stream>>>(c.v.dk_slots, 2 * c.N, acc + 1);
     unsigned long long h[2] = {0, 0};
     cudaMemcpyAsync(h, acc, 16, cudaMemcpyDeviceToHost, c.stream);
     cudaStreamSynchronize(c.stream);
@@ -353,8 +382,6 @@ void set_hist_smem_limits()
 {
     cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
     cudaFuncSetAttribute(k_hist_chunks<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
-    cudaFuncSetAttribute(k_long_docs<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
-    cudaFuncSetAttribute(k_long_docs<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
     cudaFuncSetAttribute(k_count_k<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
     cudaFuncSetAttribute(k_count_k<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
 }

@@ -35,9 +35,10 @@ __global__ void k_word_offsets(const int32_t* __restrict__ sorted_words, int32_t
     word_off[w] = lo;
 }
 
-// Document of every token in word-sorted order: the last d with doc_off[d] <= orig.
+// Document of every token in word-sorted order (the last d with doc_off[d] <= orig), stored as
+// (first token of the document, document length) so the sampler streams it instead of gathering.
 __global__ void k_token_docs(const uint32_t* __restrict__ tok_orig, const int32_t* __restrict__ doc_off,
-                             int32_t n, int32_t D, int32_t* __restrict__ tok_doc)
+                             int32_t n, int32_t D, uint2* __restrict__ tok_dinfo)
 {
     for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < n;
          p += (int64_t)gridDim.x * blockDim.x) {
@@ -47,7 +48,8 @@ __global__ void k_token_docs(const uint32_t* __restrict__ tok_orig, const int32_
             const int32_t mid = lo + ((hi - lo) >> 1);
             if (doc_off[mid + 1] <= i) lo = mid + 1; else hi = mid;
         }
-        tok_doc[p] = lo;
+        const int32_t d0 = doc_off[lo];
+        tok_dinfo[p] = make_uint2((uint32_t)d0, (uint32_t)(doc_off[lo + 1] - d0));
     }
 }
 
@@ -57,11 +59,11 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
     cudaStream_t st = c.stream;
     const size_t n1 = (size_t)(N > 0 ? N : 1);
 
-    int32_t* tok_doc = (int32_t*)dev_alloc(c, n1 * 4);
+    uint2* tok_dinfo = (uint2*)dev_alloc(c, n1 * 8);
     uint32_t* tok_orig = (uint32_t*)dev_alloc(c, n1 * 4);
     int32_t* word_off = (int32_t*)dev_alloc(c, ((size_t)V + 1) * 4);
     int32_t* doc_off = (int32_t*)dev_alloc(c, ((size_t)D + 1) * 4);
-    if (!tok_doc || !tok_orig || !word_off || !doc_off) return LDA_ENOMEM;
+    if (!tok_dinfo || !tok_orig || !word_off || !doc_off) return LDA_ENOMEM;
 
     std::vector<int32_t> doc32((size_t)D + 1);
     for (int64_t d = 0; d <= D; ++d) doc32[(size_t)d] = (int32_t)doc_off_host[d];
@@ -98,7 +100,7 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
                 rc = LDA_ECUDA;
                 break;
             }
-            k_token_docs<<<1184, 256, 0, st>>>(tok_orig, doc_off, N, D, tok_doc);
+            k_token_docs<<<1184, 256, 0, st>>>(tok_orig, doc_off, N, D, tok_dinfo);
         }
         k_word_offsets<<<(V + 1 + 255) / 256, 256, 0, st>>>(keys_out, N, V, word_off);
         if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess)
@@ -108,7 +110,7 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
     cudaFree(iota);
     cudaFree(temp);
     if (rc != LDA_OK) return rc;
-    c.v.tok_doc = tok_doc;
+    c.v.tok_dinfo = tok_dinfo;
     c.v.tok_orig = tok_orig;
     c.v.word_off = word_off;
     c.v.doc_off = doc_off;

@@ -19,6 +19,8 @@ enum : int {
     ERR_ALIAS = 16,       // alias construction met an impossible state
 };
 
+constexpr uint32_t DK_EMPTY = 0xFFFFFFFFu;
+constexpr uint32_t DK_HASH = 0x9E3779B1u;
 constexpr int SORT_TILE = 2048;      // tokens per segmented-sort tile (one CTA)
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (bins)
 constexpr int HIST_CHUNK = 16384;    // tokens per CTA in the histogram path
@@ -32,7 +34,7 @@ struct View {
     int topic_bits;  // bits of K-1
     int count_bits;  // low bits of a packed n_kd entry that hold the count
     // tokens in word-sorted order
-    const int32_t* tok_doc;
+    const uint2* tok_dinfo;  // per token: (first token of its document, document length)
     const uint32_t* tok_orig;
     void* zw[2];  // assignments in word-sorted order (topic type: u16 or i32)
     void* zd[2];  // assignments in the caller's document order
@@ -53,9 +55,10 @@ struct View {
     uint32_t* dn_idx;  // [K]
     unsigned long long* dense_mass;
     int32_t* nk;  // [K]
-    // n_kd: row d lives at dk_pairs[doc_off[d] ...], entries (topic << count_bits) | count, ascending
-    uint32_t* dk_pairs;
-    int32_t* dk_nnz;  // [D]
+    // n_kd: document d owns the open-addressing table dk_slots[2*doc_off[d] .. 2*doc_off[d+1])
+    // (capacity twice the document length, load <= 0.5); a slot is (topic << count_bits) | count
+    // or DK_EMPTY; topic k starts probing at umulhi(k * DK_HASH, capacity), linear, wrapping.
+    uint32_t* dk_slots;
     int* err;
 };
 

@@ -24,18 +24,18 @@ __device__ __forceinline__ int32_t lookup_wk(const View& v, int32_t dslot, int32
     return (lo < nnz && __ldg(v.wk_topic + r0 + lo) == k) ? (int32_t)__ldg(v.wk_count + r0 + lo) : 0;
 }
 
-// n_kd lookup in the document's packed, topic-sorted row.
-__device__ __forceinline__ int32_t lookup_dk(const View& v, int32_t d0, int32_t nnz, uint32_t k)
+// n_kd lookup in the document's open-addressing table (capacity 2*n_d, linear probing).
+__device__ __forceinline__ int32_t lookup_dk(const View& v, const uint32_t* __restrict__ tab, uint32_t cap,
+                                             uint32_t k)
 {
-    const uint32_t key = k << v.count_bits;
-    int32_t lo = 0, hi = nnz;
-    while (lo < hi) {
-        const int32_t mid = (lo + hi) >> 1;
-        if (__ldg(v.dk_pairs + d0 + mid) < key) lo = mid + 1; else hi = mid;
+    uint32_t h = __umulhi(k * DK_HASH, cap);
+    for (uint32_t probe = 0; probe < cap; ++probe) {
+        const uint32_t e = __ldg(tab + h);
+        if (e == DK_EMPTY) return 0;
+        if ((e >> v.count_bits) == k) return (int32_t)(e & ((1u << v.count_bits) - 1u));
+        if (++h == cap) h = 0;
     }
-    if (lo >= nnz) return 0;
-    const uint32_t e = __ldg(v.dk_pairs + d0 + lo);
-    return (e >> v.count_bits) == k ? (int32_t)(e & ((1u << v.count_bits) - 1u)) : 0;
+    return 0;
 }
 
 template <typename T>
@@ -67,19 +67,20 @@ k_sample(View v, const T* __restrict__ zw_cur, const T* __restrict__ zd_cur, T* 
             if (__ldg(v.word_off + mid) <= p) lo = mid; else hi = mid;
         }
         const int32_t w = lo;
-        const int32_t d = __ldg(v.tok_doc + p);
+        const uint2 dinfo = __ldg(v.tok_dinfo + p);
         const uint32_t tok = __ldg(v.tok_orig + p);
         const uint32_t z0 = (uint32_t)zw_cur[p];
 
         const int32_t r0 = __ldg(v.row_start + w), wnnz = __ldg(v.wk_nnz + w);
         const int32_t dslot = __ldg(v.dense_slot + w);
         const uint32_t mix = __ldg(v.mix32 + w);
-        const int32_t d0 = __ldg(v.doc_off + d), n_d = __ldg(v.doc_off + d + 1) - d0;
-        const int32_t dnnz = __ldg(v.dk_nnz + d);
+        const int32_t d0 = (int32_t)dinfo.x, n_d = (int32_t)dinfo.y;
+        const uint32_t* dtab = v.dk_slots + 2 * (size_t)dinfo.x;
+        const uint32_t dcap = 2u * dinfo.y;
 
         // counts at the current state s (start: s = z0, where all three are >= 1)
         uint32_t s = z0;
-        int32_t n_sd = lookup_dk(v, d0, dnnz, s);
+        int32_t n_sd = lookup_dk(v, dtab, dcap, s);
         int32_t n_sw = lookup_wk(v, dslot, r0, wnnz, s);
         int32_t n_s = __ldg(v.nk + s);
         if (n_sd < 1 || n_sw < 1 || n_s < 1) atomicOr(v.err, ERR_COUNT_ZERO);
@@ -113,7 +114,7 @@ k_sample(View v, const T* __restrict__ zw_cur, const T* __restrict__ zd_cur, T* 
             }
             if (t == s) continue;
             if (n_tw < 0) n_tw = lookup_wk(v, dslot, r0, wnnz, t);
-            const int32_t n_td = lookup_dk(v, d0, dnnz, t);
+            const int32_t n_td = lookup_dk(v, dtab, dcap, t);
             const int32_t n_t = __ldg(v.nk + t);
             const int32_t e_s = (s == z0), e_t = (t == z0);
             // Eq. 8 (word step) / Eq. 11 (doc step), products taken left to right
