@@ -52,12 +52,24 @@ __device__ __forceinline__ uint32_t to_frac32(ull part, ull whole)
     return q > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)q;
 }
 
+// One bin in the form the MH kernel reads with a single load.  With `topic` (a word's sorted
+// row) the second word holds the topics of the bin's own item and of its alias item, 16 bits
+// each; without it (the dense table, whose items are the topics) it holds the alias.
+__device__ __forceinline__ void store_packed_bin(uint2* out_pk, const uint32_t* topic, uint32_t i, uint32_t thr32,
+                                                 uint32_t al)
+{
+    if (!out_pk) return;
+    out_pk[i] = make_uint2(thr32, topic ? (topic[i] | (topic[al] << 16)) : al);
+}
+
 // Builds one table of n items.  weight(i) gives the fixed-point weight of item i.
 // sc_w, sc_de, sc_item: scratch of n entries each, private to this row.
+// out_pk (may be null) receives the packed form of every bin, see store_packed_bin().
 // Returns W44 (the sum of the fixed-point weights) to every thread of the group.
 template <bool BLOCK, class Weight>
 __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, ull* sc_w, ull* sc_de,
-                               uint32_t* sc_item, uint32_t* out_thr, uint32_t* out_idx, int* err)
+                               uint32_t* sc_item, uint32_t* out_thr, uint32_t* out_idx, uint2* out_pk,
+                               const uint32_t* pk_topic, int* err)
 {
     const int r = g.rank(), gs = g.size();
     ull s = 0;
@@ -119,8 +131,10 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
             if (lo >= H) { atomicOr(err, ERR_ALIAS); lo = H ? H - 1 : 0; }
             al = H ? sc_item[n - 1 - lo] : i;
         }
-        out_thr[i] = to_frac32(a, W);
+        const uint32_t thr32 = to_frac32(a, W);
+        out_thr[i] = thr32;
         out_idx[i] = al;
+        store_packed_bin(out_pk, pk_topic, i, thr32, al);
     }
     for (uint32_t m = r; m < H; m += gs) {
         const uint32_t i = sc_item[n - 1 - m];
@@ -137,8 +151,10 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
             if (m + 1 >= H) atomicOr(err, ERR_ALIAS);
             else al = sc_item[n - 1 - (m + 1)];
         }
-        out_thr[i] = to_frac32(thr, W);
+        const uint32_t thr32 = to_frac32(thr, W);
+        out_thr[i] = thr32;
         out_idx[i] = al;
+        store_packed_bin(out_pk, pk_topic, i, thr32, al);
     }
     return W44;
 }
@@ -174,7 +190,7 @@ __global__ void __launch_bounds__(1024) k_alias_dense(View v, ull* sc)
     const int32_t K = v.K;
     DenseWeight wf{v.nk, v.beta, v.Vbeta};
     const ull B = build_alias_row<true>(g, K, wf, sc, sc + K, (uint32_t*)(sc + 2 * (size_t)K), v.dn_thr,
-                                        v.dn_idx, v.err);
+                                        v.dn_idx, v.dn_pk, nullptr, v.err);
     if (threadIdx.x == 0) *v.dense_mass = B;
 }
 
@@ -200,7 +216,8 @@ __global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, ul
         const int32_t r0 = v.row_start[w];
         SparseWeight wf{v.wk_topic + r0, v.wk_count + r0, v.nk, v.Vbeta};
         const ull S = build_alias_row<false>(g, n, wf, sc_w + r0, sc_de + r0, sc_item + r0, v.al_thr + r0,
-                                             v.al_idx + r0, v.err);
+                                             v.al_idx + r0, v.al_pk ? v.al_pk + r0 : nullptr,
+                                             v.wk_topic + r0, v.err);
         if ((threadIdx.x & 31) == 0) v.mix32[w] = mixture_threshold(S, B);
         __syncwarp();
     }
@@ -218,7 +235,8 @@ k_alias_sparse_block(View v, const int32_t* __restrict__ words, ull* sc_w, ull* 
     const int32_t r0 = v.row_start[w];
     SparseWeight wf{v.wk_topic + r0, v.wk_count + r0, v.nk, v.Vbeta};
     const ull S = build_alias_row<true>(g, n, wf, sc_w + r0, sc_de + r0, sc_item + r0, v.al_thr + r0,
-                                        v.al_idx + r0, v.err);
+                                        v.al_idx + r0, v.al_pk ? v.al_pk + r0 : nullptr, v.wk_topic + r0,
+                                        v.err);
     if (threadIdx.x == 0) v.mix32[w] = mixture_threshold(S, *v.dense_mass);
 }
 

@@ -8,6 +8,7 @@
 
 namespace lda {
 void set_hist_smem_limits();
+void set_sample_smem_limits();
 
 void* dev_alloc(Ctx& c, size_t bytes)
 {
@@ -82,11 +83,57 @@ static void free_corpus(Ctx& c)
     nv.V = c.V; nv.K = c.K; nv.alpha = c.alpha; nv.beta = c.beta;
     nv.Vbeta = (double)c.V * c.beta;
     nv.Kalpha = (double)c.K * c.alpha;
+    nv.dense_stride = (c.K + 3) & ~3;
     nv.err = err;
     c.v = nv;
     c.loaded = c.inited = c.tables_valid = false;
     c.N = c.D = 0;
+    c.side_steps = 0;
 }
+
+}  // namespace lda
+
+// Buffers the passes of the MH step hand results to each other in; sized by the number of steps.
+int lda::ensure_exchange(Ctx& c, int mh_steps)
+{
+    if (c.N == 0 || (mh_steps <= c.side_steps && c.v.dside)) return LDA_OK;
+    auto drop = [&](void* p) {
+        if (!p) return;
+        for (size_t i = 0; i < c.allocs.size(); ++i)
+            if (c.allocs[i] == p) { c.allocs.erase(c.allocs.begin() + i); break; }
+        cudaFree(p);
+    };
+    auto bytes_for = [&](int steps, size_t& prop_b, size_t& side_b, int& stride) {
+        const size_t zt = c.wide_topics ? 4 : 2, n = (size_t)c.N;
+        stride = (1 + steps + 3) & ~3;
+        prop_b = zt * (((size_t)steps + 1) / 2) * n;
+        side_b = 4 * (size_t)stride * n;
+    };
+    cudaStreamSynchronize(c.stream);
+    size_t pb = 0, sb = 0;
+    int stride = 0;
+    if (c.side_steps) {
+        bytes_for(c.side_steps, pb, sb, stride);
+        c.device_bytes -= (int64_t)(pb + sb);
+    }
+    drop(c.v.prop);
+    drop(c.v.dside);
+    c.v.prop = nullptr;
+    c.v.dside = nullptr;
+    c.side_steps = 0;
+    bytes_for(mh_steps, pb, sb, stride);
+    c.v.prop = dev_alloc(c, pb);
+    c.v.dside = (uint32_t*)dev_alloc(c, sb);
+    if (!c.v.prop || !c.v.dside) {
+        c.err = "device allocation failed";
+        return LDA_ENOMEM;
+    }
+    c.v.side_stride = stride;
+    c.side_steps = mh_steps;
+    return LDA_OK;
+}
+
+namespace lda {
 
 static int rebuild_counts(Ctx& c, int64_t* launches)
 {
@@ -192,6 +239,30 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         }
         close(V);
     }
+    // MH kernel work lists: a hot word (more tokens than a tail tile holds; it has a dense row by
+    // the rule above) is cut into runs of HOT_TILE tokens, tail words are packed whole into tiles
+    std::vector<int32_t> hot_tiles, cold_tiles;
+    {
+        static_assert(COLD_TILE >= SORT_TILE, "every word longer than a tail tile must have a dense row");
+        int32_t s0 = 0, tok = 0;
+        auto close = [&](int32_t s1) {
+            if (s1 > s0 && tok > 0) { cold_tiles.push_back(s0); cold_tiles.push_back(s1); }
+        };
+        for (int32_t w = 0; w < V; ++w) {
+            if (tf[w] > COLD_TILE) {
+                close(w); s0 = w + 1; tok = 0;
+                for (int32_t o = 0; o < tf[w]; o += HOT_TILE) {
+                    hot_tiles.push_back(w);
+                    hot_tiles.push_back(word_off[w] + o);
+                    hot_tiles.push_back(std::min(HOT_TILE, tf[w] - o));
+                }
+                continue;
+            }
+            if (tok + tf[w] > COLD_TILE || w - s0 >= COLD_WORDS) { close(w); s0 = w; tok = 0; }
+            tok += tf[w];
+        }
+        close(V);
+    }
     std::vector<int32_t> doc_tiles, long_docs;
     {
         int32_t s0 = 0;
@@ -213,12 +284,16 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.n_hist_chunks = (int32_t)(hist_chunks.size() / 3);
     c.n_long_docs = (int32_t)long_docs.size();
     c.n_alias_big = (int32_t)alias_big.size();
+    c.n_hot_tiles = (int32_t)(hot_tiles.size() / 3);
+    c.n_cold_tiles = (int32_t)(cold_tiles.size() / 2);
 
     const size_t n1 = (size_t)std::max<int64_t>(N, 1), cap1 = (size_t)std::max<int64_t>(cap_total, 1);
     const size_t zt = c.wide_topics ? 4 : 2;
     bool ok = true;
     auto A = [&](size_t bytes) { void* p = dev_alloc(c, bytes); ok = ok && p; return p; };
-    for (int b = 0; b < 2; ++b) { v.zw[b] = A(n1 * zt); v.zd[b] = A(n1 * zt); }
+    v.zw = A(n1 * zt);
+    v.zbm = A(n1 * zt);
+    v.rec = (uint32_t*)A(n1 * 4 + 16);  // + one aligned group of four words past the last record
     v.row_start = upload(c, row_start);
     v.dense_slot = upload(c, dense_slot);
     c.word_tiles = upload(c, word_tiles);
@@ -227,20 +302,24 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.hist_chunks = upload(c, hist_chunks);
     c.long_docs = upload(c, long_docs);
     c.alias_big = upload(c, alias_big);
+    c.hot_tiles = upload(c, hot_tiles);
+    c.cold_tiles = upload(c, cold_tiles);
     ok = ok && v.row_start && v.dense_slot && c.word_tiles && c.doc_tiles && c.dense_words &&
-         c.hist_chunks && c.long_docs && c.alias_big;
+         c.hist_chunks && c.long_docs && c.alias_big && c.hot_tiles && c.cold_tiles;
     v.wk_nnz = (int32_t*)A((size_t)V * 4);
     v.wk_topic = (uint32_t*)A(cap1 * 4);
     v.wk_count = (uint32_t*)A(cap1 * 4);
-    v.dense_rows = (int32_t*)A(std::max<size_t>((size_t)c.n_dense * K, 1) * 4);
+    v.dense_rows = (int32_t*)A(std::max<size_t>((size_t)c.n_dense * v.dense_stride, 1) * 4);
     v.al_thr = (uint32_t*)A(cap1 * 4);
     v.al_idx = (uint32_t*)A(cap1 * 4);
+    v.al_pk = c.wide_topics ? nullptr : (uint2*)A(cap1 * 8);
+    v.dn_pk = (uint2*)A((size_t)K * 8);
     v.mix32 = (uint32_t*)A((size_t)V * 4);
     v.dn_thr = (uint32_t*)A((size_t)K * 4);
     v.dn_idx = (uint32_t*)A((size_t)K * 4);
     v.dense_mass = (unsigned long long*)A(8);
     v.nk = (int32_t*)A((size_t)K * 4);
-    v.dk_slots = (uint32_t*)A(n1 * 8);
+    v.dk_slots = (uint32_t*)A(n1 * 8 + 16);
     c.sc_w = (unsigned long long*)A(cap1 * 8);
     c.sc_de = (unsigned long long*)A(cap1 * 8);
     c.sc_item = (uint32_t*)A(cap1 * 4);
@@ -297,6 +376,7 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
     c.v.V = V; c.v.K = K; c.v.alpha = alpha; c.v.beta = beta;
     c.v.Vbeta = (double)V * beta;
     c.v.Kalpha = (double)K * alpha;
+    c.v.dense_stride = (K + 3) & ~3;
     c.v.err = (int*)dev_alloc(c, 16);
     if (!c.v.err || cudaMemset(c.v.err, 0, 16) != cudaSuccess) {
         dev_free_all(c);
@@ -314,6 +394,7 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
         }
     c.have_events = true;
     set_hist_smem_limits();
+    set_sample_smem_limits();
     *out = h;
     return LDA_OK;
 }
@@ -411,7 +492,6 @@ int lda_init(lda_ctx* h, uint64_t seed)
     if (rc) return rc;
     c.seed = seed;
     c.sweep = 0;
-    c.cur = 0;
     launch_init(c);
     rebuild_counts(c, nullptr);
     int bits = 0;
@@ -438,7 +518,6 @@ int lda_set_assignments(lda_ctx* h, const int32_t* z, uint64_t seed, uint32_t sw
         cudaFree(zdev);
         return cuda_fail(&c, "copying assignments");
     }
-    c.cur = 0;
     launch_spread_assignments(c, zdev);
     int bits = 0;
     rc = read_err(c, &bits);
@@ -462,6 +541,7 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
     if (!c.inited) return fail(&c, LDA_ESTATE, "lda_sweep before lda_init");
     int rc = check_device(c);
     if (rc) return rc;
+    if ((rc = ensure_exchange(c, mh_steps))) return rc;
     lda_stats& s = c.stats;
     s.ms_alias_dense = s.ms_alias_sparse = s.ms_sample = s.ms_count_wk = s.ms_count_k = s.ms_count_dk =
         s.ms_total = 0.f;
@@ -475,7 +555,6 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
         n += launch_alias_sparse(c);
         cudaEventRecord(c.ev[2], c.stream);
         n += launch_sample(c, mh_steps);
-        c.cur ^= 1;
         cudaEventRecord(c.ev[3], c.stream);
         n += launch_count_wk(c);
         cudaEventRecord(c.ev[4], c.stream);

@@ -8,7 +8,8 @@
 //   - hot words: shared-memory histogram over a window of topics, merged into
 //     the word's dense row, then compacted into the sorted row.
 // n_kd (segments = documents over the document-order z): per document an
-// open-addressing table built by insertion in shared memory.
+// open-addressing table built by insertion in shared memory, plus one record
+// (topic, its n_kd) per token.
 // No per-token global atomics: a CTA touches global counters once per bin it
 // actually filled (documents longer than a tile are the one exception).
 #include "lda_device.cuh"
@@ -125,12 +126,12 @@ template <typename T>
 __global__ void __launch_bounds__(512)
 k_hist_chunks(const int32_t* __restrict__ chunks, const T* __restrict__ z,
               const int32_t* __restrict__ dense_slot, int32_t* __restrict__ dense_rows, int32_t K,
-              int32_t window, int* err)
+              int32_t stride, int32_t window, int* err)
 {
     extern __shared__ int32_t bins[];
     const int32_t w = chunks[3 * blockIdx.x], first = chunks[3 * blockIdx.x + 1],
                   cnt = chunks[3 * blockIdx.x + 2];
-    int32_t* row = dense_rows + (size_t)dense_slot[w] * K;
+    int32_t* row = dense_rows + (size_t)dense_slot[w] * stride;
     for (int32_t k0 = 0; k0 < K; k0 += window) {
         const int32_t nb = min(window, K - k0);
         for (int b = threadIdx.x; b < nb; b += blockDim.x) bins[b] = 0;
@@ -155,11 +156,11 @@ __global__ void __launch_bounds__(256)
 k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restrict__ dense_slot,
                 const int32_t* __restrict__ dense_rows, const int32_t* __restrict__ row_start,
                 uint32_t* __restrict__ wk_topic, uint32_t* __restrict__ wk_count,
-                int32_t* __restrict__ wk_nnz, int32_t K, int* err)
+                int32_t* __restrict__ wk_nnz, int32_t K, int32_t stride, int* err)
 {
     __shared__ int32_t scan_tmp[33];
     const int32_t w = dense_words[blockIdx.x];
-    const int32_t* row = dense_rows + (size_t)dense_slot[w] * K;
+    const int32_t* row = dense_rows + (size_t)dense_slot[w] * stride;
     const int32_t out0 = row_start[w], cap = row_start[w + 1] - out0;
     int32_t done = 0;
     for (int32_t k0 = 0; k0 < K; k0 += blockDim.x) {
@@ -180,72 +181,122 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
     if (threadIdx.x == 0) wk_nnz[w] = done;
 }
 
-// n_kd as per-document open-addressing tables (Section 5, fn. 5: capacity twice the number of
-// tokens, so the load factor stays <= 0.5).  One CTA per tile of whole documents holding
-// <= SORT_TILE tokens: the tile's tables are built in shared memory by insertion (claim a slot
-// with compare-and-swap, then add one to its count bits) and written out in one coalesced pass.
+// n_kd as per-document open-addressing tables (layout and probe order: DkProbe).  One CTA per
+// tile of whole documents holding <= SORT_TILE tokens: the tile's tables are built in shared
+// memory by insertion (claim a slot with compare-and-swap, then add one to its count bits) and
+// written out in one coalesced pass.  Every token's record (topic, n_kd of its topic in its
+// document) is written next to it, so that the MH step gets both in one read.
+//
+// `tab` points at the copy of global slot `a0`; slot x of the global array is tab[x - a0].
+__device__ __forceinline__ void dk_insert(uint32_t* tab, uint32_t a0, const DkProbe& pr, uint32_t k, int count_bits)
+{
+    const uint32_t fresh = k << count_bits;
+    uint32_t g = pr.first(k);
+    for (uint32_t n = 0; n < pr.g_cnt; ++n, g = pr.next(g)) {
+#pragma unroll
+        for (uint32_t l = 0; l < 4; ++l) {
+            const uint32_t slot = 4u * g + l;
+            if (!pr.inside(slot)) continue;
+            const uint32_t prev = atomicCAS(&tab[slot - a0], DK_EMPTY, fresh);
+            if (prev == DK_EMPTY || (prev >> count_bits) == k) {
+                atomicAdd(&tab[slot - a0], 1u);
+                return;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t dk_find(const uint32_t* tab, uint32_t a0, const DkProbe& pr, uint32_t k,
+                                            int count_bits)
+{
+    uint32_t g = pr.first(k);
+    for (uint32_t n = 0; n < pr.g_cnt; ++n, g = pr.next(g)) {
+#pragma unroll
+        for (uint32_t l = 0; l < 4; ++l) {
+            const uint32_t slot = 4u * g + l;
+            if (!pr.inside(slot)) continue;
+            const uint32_t e = tab[slot - a0];
+            if (e == DK_EMPTY) return k << count_bits;
+            if ((e >> count_bits) == k) return e;
+        }
+    }
+    return k << count_bits;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
-k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_off,
-           const T* __restrict__ z, uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
+k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_off, const T* __restrict__ zbm,
+           const uint32_t* __restrict__ bm_of_tok, uint32_t* __restrict__ rec, uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
 {
-    __shared__ uint32_t slots[2 * SORT_TILE];
+    __shared__ uint32_t slots[2 * SORT_TILE + 4];
     __shared__ int32_t soff[SORT_TILE + 1];
+    __shared__ uint32_t topic[SORT_TILE];
     const int tid = threadIdx.x;
     const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
     const int32_t nseg = s1 - s0;
     const int32_t base = doc_off[s0];
     const int32_t cnt = doc_off[s1] - base;
     if (cnt == 0) return;
+    const uint32_t a0 = (2u * (uint32_t)base) & ~3u;        // global slot kept in slots[0]
+    const uint32_t lead = 2u * (uint32_t)base - a0;         // 0 or 2
+    // the tile's documents lie in one or two blocks of the block-major order: these reads hit L2
+    for (int j = tid; j < cnt; j += blockDim.x) topic[j] = (uint32_t)__ldcg(zbm + __ldcs(bm_of_tok + base + j));
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = doc_off[s0 + j] - base;
-    for (int j = tid; j < 2 * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
+    for (int j = tid; j < 2 * cnt + 4; j += blockDim.x) slots[j] = DK_EMPTY;
     __syncthreads();
-    for (int j = tid; j < cnt; j += blockDim.x) {
-        int lo = 0, hi = nseg;  // last document with soff[doc] <= j
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (soff[mid] <= j) lo = mid; else hi = mid;
-        }
-        const uint32_t k = (uint32_t)z[base + j];
-        if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
-        const uint32_t cap = 2u * (uint32_t)(soff[lo + 1] - soff[lo]);
-        uint32_t* tab = slots + 2 * soff[lo];
-        uint32_t h = __umulhi(k * DK_HASH, cap);
-        const uint32_t fresh = k << count_bits;
-        for (uint32_t probe = 0; probe < cap; ++probe) {
-            const uint32_t prev = atomicCAS(&tab[h], DK_EMPTY, fresh);
-            if (prev == DK_EMPTY || (prev >> count_bits) == k) { atomicAdd(&tab[h], 1u); break; }
-            if (++h == cap) h = 0;
+    int32_t my_doc[SORT_TILE / 256];  // document (relative to the tile) of each of this thread's tokens
+#pragma unroll
+    for (int q = 0; q < SORT_TILE / 256; ++q) {
+        const int j = tid + q * 256;
+        my_doc[q] = -1;
+        if (j < cnt) {
+            int lo = 0, hi = nseg;  // last document with soff[doc] <= j
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (soff[mid] <= j) lo = mid; else hi = mid;
+            }
+            const uint32_t k = topic[j];
+            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+            my_doc[q] = lo;
+            const DkProbe pr((uint32_t)(base + soff[lo]), (uint32_t)(soff[lo + 1] - soff[lo]));
+            dk_insert(slots, a0, pr, k, count_bits);
         }
     }
     __syncthreads();
     uint32_t* out = slots_out + 2 * (size_t)base;
-    for (int j = tid; j < 2 * cnt; j += blockDim.x) out[j] = slots[j];
+    for (int j = tid; j < 2 * cnt; j += blockDim.x) out[j] = slots[lead + j];
+#pragma unroll
+    for (int q = 0; q < SORT_TILE / 256; ++q) {
+        const int j = tid + q * 256;
+        const int32_t lo = my_doc[q];
+        if (lo >= 0) {
+            const DkProbe pr((uint32_t)(base + soff[lo]), (uint32_t)(soff[lo + 1] - soff[lo]));
+            rec[base + j] = dk_find(slots, a0, pr, topic[j], count_bits);
+        }
+    }
 }
 
 // Documents longer than a tile: one CTA per document, the same insertion straight in global memory.
 template <typename T>
 __global__ void __launch_bounds__(512)
 k_long_doc_hash(const int32_t* __restrict__ long_docs, const int32_t* __restrict__ doc_off,
-                const T* __restrict__ z, uint32_t* __restrict__ slots_out, int count_bits, int32_t K,
-                int* err)
+                const T* __restrict__ zbm, const uint32_t* __restrict__ bm_of_tok, uint32_t* __restrict__ rec,
+                uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
 {
     const int32_t d = long_docs[blockIdx.x];
     const int32_t first = doc_off[d], cnt = doc_off[d + 1] - first;
-    const uint32_t cap = 2u * (uint32_t)cnt;
-    uint32_t* tab = slots_out + 2 * (size_t)first;
-    for (uint32_t j = threadIdx.x; j < cap; j += blockDim.x) tab[j] = DK_EMPTY;
+    const DkProbe pr((uint32_t)first, (uint32_t)cnt);
+    for (uint32_t j = threadIdx.x; j < 2u * (uint32_t)cnt; j += blockDim.x) slots_out[pr.t0 + j] = DK_EMPTY;
     __syncthreads();
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-        const uint32_t k = (uint32_t)z[first + j];
+        const uint32_t k = (uint32_t)zbm[bm_of_tok[first + j]];
         if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
-        uint32_t h = __umulhi(k * DK_HASH, cap);
-        const uint32_t fresh = k << count_bits;
-        for (uint32_t probe = 0; probe < cap; ++probe) {
-            const uint32_t prev = atomicCAS(&tab[h], DK_EMPTY, fresh);
-            if (prev == DK_EMPTY || (prev >> count_bits) == k) { atomicAdd(&tab[h], 1u); break; }
-            if (++h == cap) h = 0;
-        }
+        dk_insert(slots_out, 0u, pr, k, count_bits);
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
+        const uint32_t k = (uint32_t)zbm[bm_of_tok[first + j]];
+        if (k < (uint32_t)K) rec[first + j] = dk_find(slots_out, 0u, pr, k, count_bits);
     }
 }
 
@@ -306,7 +357,7 @@ static int count_wk_t(Ctx& c)
 {
     View& v = c.v;
     int launches = 0;
-    const T* z = (const T*)v.zw[c.cur];
+    const T* z = (const T*)v.zw;
     if (c.n_word_tiles) {
         EmitWord e{v.row_start, v.wk_topic, v.wk_count, v.wk_nnz};
         k_seg_count_sorted<T, EmitWord><<<c.n_word_tiles, 256, 0, c.stream>>>(
@@ -314,13 +365,13 @@ static int count_wk_t(Ctx& c)
         ++launches;
     }
     if (c.n_dense) {
-        cudaMemsetAsync(v.dense_rows, 0, (size_t)c.n_dense * c.K * 4, c.stream);
+        cudaMemsetAsync(v.dense_rows, 0, (size_t)c.n_dense * v.dense_stride * 4, c.stream);
         const int win = hist_window(c);
         k_hist_chunks<T><<<c.n_hist_chunks, 512, (size_t)win * 4, c.stream>>>(
-            c.hist_chunks, z, v.dense_slot, v.dense_rows, c.K, win, v.err);
+            c.hist_chunks, z, v.dense_slot, v.dense_rows, c.K, v.dense_stride, win, v.err);
         k_compact_dense<<<c.n_dense, 256, 0, c.stream>>>(c.dense_words, v.dense_slot, v.dense_rows,
                                                          v.row_start, v.wk_topic, v.wk_count,
-                                                         v.wk_nnz, c.K, v.err);
+                                                         v.wk_nnz, c.K, v.dense_stride, v.err);
         launches += 2;
     }
     return launches;
@@ -336,7 +387,7 @@ static int count_k_t(Ctx& c)
     int grid = (int)((c.N + 65535) / 65536);
     if (grid > 148 * 4) grid = 148 * 4;
     if (grid < 1) grid = 1;
-    k_count_k<T><<<grid, 512, (size_t)win * 4, c.stream>>>((const T*)v.zw[c.cur], (int32_t)c.N, v.nk,
+    k_count_k<T><<<grid, 512, (size_t)win * 4, c.stream>>>((const T*)v.zw, (int32_t)c.N, v.nk,
                                                           c.K, win, v.err);
     return 1;
 }
@@ -346,14 +397,14 @@ static int count_dk_t(Ctx& c)
 {
     View& v = c.v;
     int launches = 0;
-    const T* z = (const T*)v.zd[c.cur];
+    const T* zbm = (const T*)v.zbm;
     if (c.n_doc_tiles) {
-        k_doc_hash<T><<<c.n_doc_tiles, 256, 0, c.stream>>>(c.doc_tiles, v.doc_off, z, v.dk_slots,
+        k_doc_hash<T><<<c.n_doc_tiles, 256, 0, c.stream>>>(c.doc_tiles, v.doc_off, zbm, v.bm_of_tok, v.rec, v.dk_slots,
                                                           v.count_bits, c.K, v.err);
         ++launches;
     }
     if (c.n_long_docs) {
-        k_long_doc_hash<T><<<c.n_long_docs, 512, 0, c.stream>>>(c.long_docs, v.doc_off, z, v.dk_slots,
+        k_long_doc_hash<T><<<c.n_long_docs, 512, 0, c.stream>>>(c.long_docs, v.doc_off, zbm, v.bm_of_tok, v.rec, v.dk_slots,
                                                                v.count_bits, c.K, v.err);
         ++launches;
     }

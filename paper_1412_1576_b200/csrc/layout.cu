@@ -35,6 +35,33 @@ __global__ void k_word_offsets(const int32_t* __restrict__ sorted_words, int32_t
     word_off[w] = lo;
 }
 
+// Keys of the block-major order: the block of a token is the high part of its document-order index.
+__global__ void k_block_keys(const uint32_t* __restrict__ tok_orig, int32_t n, int shift,
+                             uint32_t* __restrict__ keys, uint32_t* __restrict__ iota)
+{
+    for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < n;
+         p += (int64_t)gridDim.x * blockDim.x) {
+        keys[p] = tok_orig[p] >> shift;
+        iota[p] = (uint32_t)p;
+    }
+}
+
+// Static token records copied into block-major order, so the document-side pass streams them.
+__global__ void k_gather_block_major(const uint32_t* __restrict__ order, const uint2* __restrict__ tok_dinfo,
+                                     const uint32_t* __restrict__ tok_orig, int32_t n,
+                                     uint2* __restrict__ dinfo_bm, uint32_t* __restrict__ tok_bm,
+                                     uint32_t* __restrict__ inv, uint32_t* __restrict__ bm_of_tok)
+{
+    for (int64_t m = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; m < n;
+         m += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t p = order[m];
+        dinfo_bm[m] = tok_dinfo[p];
+        tok_bm[m] = tok_orig[p];
+        inv[p] = (uint32_t)m;
+        bm_of_tok[tok_orig[p]] = (uint32_t)m;
+    }
+}
+
 // Document of every token in word-sorted order (the last d with doc_off[d] <= orig), stored as
 // (first token of the document, document length) so the sampler streams it instead of gathering.
 __global__ void k_token_docs(const uint32_t* __restrict__ tok_orig, const int32_t* __restrict__ doc_off,
@@ -59,11 +86,15 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
     cudaStream_t st = c.stream;
     const size_t n1 = (size_t)(N > 0 ? N : 1);
 
-    uint2* tok_dinfo = (uint2*)dev_alloc(c, n1 * 8);
     uint32_t* tok_orig = (uint32_t*)dev_alloc(c, n1 * 4);
+    uint32_t* order = (uint32_t*)dev_alloc(c, n1 * 4);
+    uint32_t* inv = (uint32_t*)dev_alloc(c, n1 * 4);
+    uint32_t* bm_of_tok = (uint32_t*)dev_alloc(c, n1 * 4);
+    uint2* dinfo_bm = (uint2*)dev_alloc(c, n1 * 8);
+    uint32_t* tok_bm = (uint32_t*)dev_alloc(c, n1 * 4);
     int32_t* word_off = (int32_t*)dev_alloc(c, ((size_t)V + 1) * 4);
     int32_t* doc_off = (int32_t*)dev_alloc(c, ((size_t)D + 1) * 4);
-    if (!tok_dinfo || !tok_orig || !word_off || !doc_off) return LDA_ENOMEM;
+    if (!tok_orig || !order || !inv || !bm_of_tok || !dinfo_bm || !tok_bm || !word_off || !doc_off) return LDA_ENOMEM;
 
     std::vector<int32_t> doc32((size_t)D + 1);
     for (int64_t d = 0; d <= D; ++d) doc32[(size_t)d] = (int32_t)doc_off_host[d];
@@ -74,11 +105,15 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
     // transient buffers of the sort
     int32_t* keys_out = nullptr;
     uint32_t* iota = nullptr;
+    uint32_t* keys_blk = nullptr;
+    uint2* tok_dinfo = nullptr;
     void* temp = nullptr;
-    size_t temp_bytes = 0;
+    void* temp2 = nullptr;
+    size_t temp_bytes = 0, temp2_bytes = 0;
     int rc = LDA_OK;
     do {
-        if (cudaMalloc(&keys_out, n1 * 4) != cudaSuccess || cudaMalloc(&iota, n1 * 4) != cudaSuccess) {
+        if (cudaMalloc(&keys_out, n1 * 4) != cudaSuccess || cudaMalloc(&iota, n1 * 4) != cudaSuccess ||
+            cudaMalloc(&keys_blk, n1 * 4) != cudaSuccess || cudaMalloc(&tok_dinfo, n1 * 8) != cudaSuccess) {
             rc = LDA_ENOMEM;
             break;
         }
@@ -101,16 +136,47 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
                 break;
             }
             k_token_docs<<<1184, 256, 0, st>>>(tok_orig, doc_off, N, D, tok_dinfo);
+            // block-major order: tokens sorted by (block of their document-order index, word-sorted
+            // position); a stable sort of the positions by block
+            uint32_t* keys_tmp = reinterpret_cast<uint32_t*>(keys_out);  // the word keys are no longer needed
+            k_block_keys<<<1184, 256, 0, st>>>(tok_orig, N, c.block_shift, keys_blk, iota);
+            int blk_bits = 1;
+            while (blk_bits < 32 && (((long long)N - 1) >> c.block_shift) >= (1ll << blk_bits)) ++blk_bits;
+            if (cub::DeviceRadixSort::SortPairs(nullptr, temp2_bytes, keys_blk, keys_tmp, iota, order, N, 0,
+                                                blk_bits, st) != cudaSuccess) {
+                rc = LDA_ECUDA;
+                break;
+            }
+            if (cudaMalloc(&temp2, temp2_bytes ? temp2_bytes : 1) != cudaSuccess) {
+                rc = LDA_ENOMEM;
+                break;
+            }
+            // the word offsets are taken from keys_out first: the next sort overwrites it
+            k_word_offsets<<<(V + 1 + 255) / 256, 256, 0, st>>>(keys_out, N, V, word_off);
+            if (cub::DeviceRadixSort::SortPairs(temp2, temp2_bytes, keys_blk, keys_tmp, iota, order, N, 0,
+                                                blk_bits, st) != cudaSuccess) {
+                rc = LDA_ECUDA;
+                break;
+            }
+            k_gather_block_major<<<1184, 256, 0, st>>>(order, tok_dinfo, tok_orig, N, dinfo_bm, tok_bm, inv, bm_of_tok);
+        } else {
+            k_word_offsets<<<(V + 1 + 255) / 256, 256, 0, st>>>(keys_out, N, V, word_off);
         }
-        k_word_offsets<<<(V + 1 + 255) / 256, 256, 0, st>>>(keys_out, N, V, word_off);
         if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess)
             rc = LDA_ECUDA;
     } while (0);
     cudaFree(keys_out);
     cudaFree(iota);
+    cudaFree(keys_blk);
+    cudaFree(tok_dinfo);
     cudaFree(temp);
+    cudaFree(temp2);
     if (rc != LDA_OK) return rc;
-    c.v.tok_dinfo = tok_dinfo;
+    c.v.order = order;
+    c.v.inv = inv;
+    c.v.bm_of_tok = bm_of_tok;
+    c.v.dinfo_bm = dinfo_bm;
+    c.v.tok_bm = tok_bm;
     c.v.tok_orig = tok_orig;
     c.v.word_off = word_off;
     c.v.doc_off = doc_off;

@@ -25,6 +25,49 @@ __device__ __forceinline__ uint32_t scale_to_range(uint32_t r, uint32_t n) { ret
 
 __device__ __forceinline__ int bit_length(unsigned long long x) { return 64 - __clzll((long long)x); }
 
+// --- n_kd tables --------------------------------------------------------------------------------
+// Document d owns slots [t0, t1) = [2*doc_off[d], 2*doc_off[d+1]) of one global slot array (twice
+// its length, so the load factor stays <= 0.5; Section 5, fn. 5).  A slot is
+// (topic << count_bits) | count, or DK_EMPTY_SLOT.  The table is bucketed by aligned groups of
+// four slots (one 16-byte read): topic k starts at group DkProbe::first() and tries the group's
+// slots that lie inside [t0, t1) in order, then the next group, wrapping to the table's first
+// group.  An empty slot met on the way means "absent".
+constexpr uint32_t DK_EMPTY_SLOT = 0xFFFFFFFFu;
+constexpr uint32_t DK_HASH_MULT = 0x9E3779B1u;
+
+struct DkProbe {
+    uint32_t t0, t1;          // the table's slot range
+    uint32_t g_first, g_cnt;  // first group (slot index / 4) and number of groups it touches
+    __device__ __forceinline__ DkProbe(uint32_t doc_first_token, uint32_t doc_len)
+        : t0(2u * doc_first_token), t1(2u * (doc_first_token + doc_len))
+    {
+        g_first = t0 >> 2;
+        g_cnt = ((t1 - 1u) >> 2) - g_first + 1u;
+    }
+    __device__ __forceinline__ uint32_t first(uint32_t k) const { return g_first + __umulhi(k * DK_HASH_MULT, g_cnt); }
+    __device__ __forceinline__ uint32_t next(uint32_t g) const { return g + 1u - g_first == g_cnt ? g_first : g + 1u; }
+    __device__ __forceinline__ bool inside(uint32_t slot) const { return slot >= t0 && slot < t1; }
+};
+
+// Looks topic k up in one group of four slots `q` (group index g).  Returns true when the search
+// is over (found, or an empty slot proves absence) and sets `entry` (0 when absent).
+__device__ __forceinline__ bool dk_match_group(const DkProbe& pr, uint32_t g, const uint4& q, uint32_t k,
+                                               int count_bits, uint32_t& entry)
+{
+    const uint32_t qv[4] = {q.x, q.y, q.z, q.w};
+    bool done = false;
+    entry = 0;
+#pragma unroll
+    for (uint32_t l = 0; l < 4; ++l) {
+        const uint32_t e = qv[l];
+        if (!done && pr.inside(4u * g + l)) {
+            if (e == DK_EMPTY_SLOT) done = true;
+            else if ((e >> count_bits) == k) { entry = e; done = true; }
+        }
+    }
+    return done;
+}
+
 template <typename T>
 __device__ __forceinline__ T warp_reduce_sum(T v)
 {

@@ -17,14 +17,17 @@ enum : int {
     ERR_ROW_OVERFLOW = 4, // a count row needed more entries than its capacity
     ERR_TOPIC_RANGE = 8,  // an assignment outside [0,K)
     ERR_ALIAS = 16,       // alias construction met an impossible state
+    ERR_STAGE = 32,       // a bulk copy into shared memory did not complete within its wait limit
 };
 
-constexpr uint32_t DK_EMPTY = 0xFFFFFFFFu;
-constexpr uint32_t DK_HASH = 0x9E3779B1u;
+constexpr uint32_t DK_EMPTY = 0xFFFFFFFFu;  // == DK_EMPTY_SLOT of the device helpers
 constexpr int SORT_TILE = 2048;      // tokens per segmented-sort tile (one CTA)
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (bins)
 constexpr int HIST_CHUNK = 16384;    // tokens per CTA in the histogram path
-constexpr int SAMPLE_TILE = 1024;    // tokens per CTA in the MH kernel
+constexpr int HOT_TILE = 8192;       // MH kernel: tokens of one hot word per CTA
+constexpr int COLD_TILE = 2048;      // MH kernel: tokens of a tile of whole tail words
+constexpr int COLD_WORDS = 512;      // MH kernel: words per tail tile
+constexpr int HOT_STAGE_MAX_K = 16384;  // dense rows up to this many topics are staged in shared memory
 constexpr int ALIAS_WARP_MAX = 256;  // rows up to this many items are built by one warp
 
 // Everything a kernel needs, passed by value.
@@ -33,11 +36,28 @@ struct View {
     double alpha, beta, Vbeta, Kalpha;
     int topic_bits;  // bits of K-1
     int count_bits;  // low bits of a packed n_kd entry that hold the count
-    // tokens in word-sorted order
-    const uint2* tok_dinfo;  // per token: (first token of its document, document length)
-    const uint32_t* tok_orig;
-    void* zw[2];  // assignments in word-sorted order (topic type: u16 or i32)
-    void* zd[2];  // assignments in the caller's document order
+    // tokens in word-sorted order (position p)
+    const uint32_t* tok_orig;  // index of the token in the caller's document order
+    // the same tokens in block-major order (index m): sorted by (block of the document-order
+    // index, word-sorted position), so that a pass in this order touches one block of the
+    // document-side tables at a time -- small enough to stay in L2 -- while still walking runs of
+    // consecutive word-sorted positions
+    const uint32_t* order;    // [N] word-sorted position of the m-th token
+    const uint32_t* inv;      // [N] block-major index of the token at word-sorted position p
+    const uint2* dinfo_bm;    // [N] (first token of its document, document length)
+    const uint32_t* tok_bm;   // [N] document-order index
+    const uint32_t* bm_of_tok;  // [N] block-major index of the token with document-order index i
+    // per-sweep exchange buffers between the word-order and the document-order passes
+    void* prop;        // [word steps][N] block-major: topics proposed by the word-proposals (topic type)
+    uint32_t* dside;   // [N][side_stride] block-major: own record, then per step (topic << count_bits) | n_kd
+    int32_t side_stride;  // words per token in dside: 1 + steps, rounded up to a multiple of 4
+    // assignments (topic type: u16 or i32) after the last MH step or initialisation
+    void* zw;   // word-sorted order: read by the n_kw / n_k rebuild
+    void* zbm;  // block-major order: read (through bm_of_tok) by the n_kd rebuild
+    // Sweep-start state in document order: rec[i] = (z_i << count_bits) | n_kd[d][z_i], a token's
+    // topic together with that topic's count in its document, so the doc-proposal (Eq. 12) gets
+    // the proposed topic and its n_kd in one read.  Written by the n_kd rebuild.
+    uint32_t* rec;
     const int32_t* word_off;  // [V+1] token range of each word in word-sorted order
     const int32_t* doc_off;   // [D+1]
     // n_kw: every word has a sorted (topic, count) row of fixed capacity; hot words also a dense row
@@ -46,18 +66,21 @@ struct View {
     uint32_t* wk_topic;        // [row_start[V]]
     uint32_t* wk_count;
     const int32_t* dense_slot;  // [V] index of the word's dense row or -1
-    int32_t* dense_rows;        // [n_dense * K]
+    int32_t* dense_rows;        // [n_dense * dense_stride]
+    int32_t dense_stride;       // K rounded up to a multiple of 4 (rows start 16-byte aligned)
     // word-proposal tables
     uint32_t* al_thr;  // split point of each sparse bin as a 32-bit fraction
     uint32_t* al_idx;  // alias item of each sparse bin
+    uint2* al_pk;      // 16-bit topics only: bin as (split point, topic of the bin's item | topic of
+                       // its alias item << 16), so a draw costs one read
     uint32_t* mix32;   // [V] share of the sparse term
     uint32_t* dn_thr;  // [K]
     uint32_t* dn_idx;  // [K]
+    uint2* dn_pk;      // [K] (split point, alias) of the dense table in one word pair
     unsigned long long* dense_mass;
     int32_t* nk;  // [K]
     // n_kd: document d owns the open-addressing table dk_slots[2*doc_off[d] .. 2*doc_off[d+1])
-    // (capacity twice the document length, load <= 0.5); a slot is (topic << count_bits) | count
-    // or DK_EMPTY; topic k starts probing at umulhi(k * DK_HASH, capacity), linear, wrapping.
+    // (capacity twice the document length, load <= 0.5); layout and probe order: DkProbe.
     uint32_t* dk_slots;
     int* err;
 };
@@ -68,23 +91,26 @@ struct Ctx {
     int device = 0;
     cudaStream_t stream = nullptr;
     bool wide_topics = false;  // false: 16-bit topic storage, true: 32-bit
+    int block_shift = 21;  // log2 of the tokens per block of the block-major order
+    int side_steps = 0;    // number of steps the exchange buffers are allocated for
     double dense_frac = 0.05;
     double dense_min_tf = 64;
     bool loaded = false, inited = false, tables_valid = false;
-    int cur = 0;  // which of the two z buffers is current
     uint64_t seed = 0;
     uint32_t sweep = 0;
     int64_t N = 0, D = 0;
     View v{};
     // host-side work lists (device copies below)
     int32_t n_word_tiles = 0, n_doc_tiles = 0, n_dense = 0, n_hist_chunks = 0, n_long_docs = 0,
-            n_alias_big = 0;
+            n_alias_big = 0, n_hot_tiles = 0, n_cold_tiles = 0;
     int32_t* word_tiles = nullptr;   // [n_word_tiles*2] word ranges sorted per CTA
     int32_t* doc_tiles = nullptr;    // [n_doc_tiles*2]
     int32_t* dense_words = nullptr;  // [n_dense]
     int32_t* hist_chunks = nullptr;  // [n_hist_chunks*3] (word, first token, count)
     int32_t* long_docs = nullptr;    // [n_long_docs]
     int32_t* alias_big = nullptr;    // [n_alias_big] words whose row can exceed ALIAS_WARP_MAX
+    int32_t* hot_tiles = nullptr;    // [n_hot_tiles*3] (word, first token, count): MH kernel, hot words
+    int32_t* cold_tiles = nullptr;   // [n_cold_tiles*2] word ranges of whole tail words: MH kernel
     // alias-construction scratch
     unsigned long long* sc_w = nullptr;   // [row capacity total] scaled masses
     unsigned long long* sc_de = nullptr;  // deficits prefix (front) / surpluses prefix (back)
@@ -110,7 +136,8 @@ int launch_count_k(Ctx& c);
 int launch_count_dk(Ctx& c);
 int launch_alias_dense(Ctx& c);
 int launch_alias_sparse(Ctx& c);
-int launch_sample(Ctx& c, int mh_steps);
+int launch_sample(Ctx& c, int mh_steps);   // all passes of the MH step; needs ensure_exchange()
+int ensure_exchange(Ctx& c, int mh_steps);  // (re)allocates View::prop / View::dside; LDA_* status
 int launch_loglik(Ctx& c, double* out3_host);
 int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host);
 

@@ -1,183 +1,505 @@
-// Token Metropolis-Hastings kernel (Section 4.2-4.3) and the assignment
-// initialisation / import / export kernels.
+// Token Metropolis-Hastings step (Section 4.2-4.3) and the assignment initialisation / import /
+// export kernels.
 //
-// One thread owns one token for the whole chain.  Everything it reads is the
-// sweep-start state (Section 6: the model is immutable while sampled), it writes
-// only its own two output slots, so the result does not depend on scheduling.
+// Everything a token's chain reads is the sweep-start state (Section 6: the model is immutable
+// while sampled) and a thread writes only its own output slots, so the result does not depend
+// on scheduling.  Because the counts are frozen, a proposal never depends on the chain's current
+// state.  The step is therefore split into passes that each stay on one side of the model:
+//   1. word order : draw the word-proposals (alias bins of the word staged per tile);
+//   2. block-major: gather the document side -- own record, doc-proposals, n_kd at every
+//                   proposed topic -- one L2-sized block of documents at a time;
+//   3. word order : accept/reject chain in registers, n_kw rows staged in shared memory (hot
+//                   words: the dense row, by one bulk asynchronous copy; tail words: the sorted rows
+//                   of a tile of whole words);
+// Pass 3 leaves the new assignments in word order (for the n_kw / n_k rebuild) and in block-major
+// order, from where the n_kd rebuild picks them up block by block.
+// A random access to HBM costs far more than the bytes it returns: pass 2 turns the document-side
+// gathers into L2 hits, passes 1 and 3 stream, and whatever crosses between the two orders moves
+// in runs of consecutive positions.
 #include "lda_device.cuh"
 #include "lda_internal.cuh"
 
 namespace lda {
 
 constexpr double INV_2_32 = 1.0 / 4294967296.0;
+#ifndef LDA_HOT_THREADS
+#define LDA_HOT_THREADS 512
+#endif
+constexpr int HOT_THREADS = LDA_HOT_THREADS;
+constexpr int COLD_THREADS = 256;
+constexpr int STAGE_WAIT_LIMIT = 1 << 20;
 
-// n_kw lookup: dense row if the word has one, else binary search in its sorted row.
-__device__ __forceinline__ int32_t lookup_wk(const View& v, int32_t dslot, int32_t r0, int32_t nnz,
-                                             uint32_t k)
+// --- shared-memory barrier and bulk-copy primitives ------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void* bar, uint32_t arrivals)
 {
-    if (dslot >= 0) return __ldg(v.dense_rows + (size_t)dslot * v.K + k);
-    int32_t lo = 0, hi = nnz;
-    while (lo < hi) {
-        const int32_t mid = (lo + hi) >> 1;
-        if (__ldg(v.wk_topic + r0 + mid) < k) lo = mid + 1; else hi = mid;
-    }
-    return (lo < nnz && __ldg(v.wk_topic + r0 + lo) == k) ? (int32_t)__ldg(v.wk_count + r0 + lo) : 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// n_kd lookup in the document's open-addressing table (capacity 2*n_d, linear probing).
-__device__ __forceinline__ int32_t lookup_dk(const View& v, const uint32_t* __restrict__ tab, uint32_t cap,
-                                             uint32_t k)
+__device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes)
 {
-    uint32_t h = __umulhi(k * DK_HASH, cap);
-    for (uint32_t probe = 0; probe < cap; ++probe) {
-        const uint32_t e = __ldg(tab + h);
-        if (e == DK_EMPTY) return 0;
-        if ((e >> v.count_bits) == k) return (int32_t)(e & ((1u << v.count_bits) - 1u));
-        if (++h == cap) h = 0;
-    }
-    return 0;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
 }
 
+// Global -> shared bulk copy; both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, void* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst_smem)),
+                 "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+// Waits for the barrier's phase `parity`; gives up after `limit` polls and returns false.
+__device__ __forceinline__ bool mbar_wait_bounded(void* bar, uint32_t parity, int limit)
+{
+    uint32_t done = 0;
+    for (int i = 0; i < limit && !done; ++i)
+        asm volatile(
+            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+            : "=r"(done)
+            : "r"(smem_addr(bar)), "r"(parity)
+            : "memory");
+    return done != 0;
+}
+
+// --- document side ---------------------------------------------------------------------------
+// Group g (four slots, 16 bytes, aligned) of the n_kd slot array.
+__device__ __forceinline__ uint4 load_group(const uint32_t* __restrict__ slots, uint32_t g)
+{
+    return __ldcg(reinterpret_cast<const uint4*>(slots) + g);
+}
+
+__device__ __forceinline__ uint32_t quad_word(const uint4& q, uint32_t lane)
+{
+    return lane == 0 ? q.x : lane == 1 ? q.y : lane == 2 ? q.z : q.w;
+}
+
+// n_kd[k] as a packed entry (0 when absent).  `q` is the first group of the probe sequence,
+// already loaded; further groups are read only when that one is full of other topics.
+__device__ __forceinline__ uint32_t lookup_dk(const uint32_t* __restrict__ slots, const DkProbe& pr, uint32_t g,
+                                              uint4 q, uint32_t k, int count_bits)
+{
+    uint32_t entry;
+    for (uint32_t n = 1; !dk_match_group(pr, g, q, k, count_bits, entry) && n < pr.g_cnt; ++n) {
+        g = pr.next(g);
+        q = load_group(slots, g);
+    }
+    return entry;
+}
+
+// --- word side -------------------------------------------------------------------------------
+// What a word-proposal draw keeps between issuing its table read and using the result.
+struct Draw {
+    uint2 e;      // the bin read from global memory (hot words; dense term of tail words)
+    uint32_t b;   // bin index
+    uint32_t rz;  // the alias coin
+    bool sparse;  // sparse term (the word's own table) or dense smoothing term
+};
+
+// A hot word: dense n_kw row (in shared memory when STAGED), alias bins read from global memory.
+template <bool STAGED, bool PACKED>
+struct HotTile {
+    struct Ref {};
+    const int32_t* row;
+    const uint2* pk;          // PACKED: the word's bins
+    const uint32_t* thr;      // otherwise the three separate arrays
+    const uint32_t* idx;
+    const uint32_t* topic;
+    int32_t nnz;
+    uint32_t mix;
+    void* bar;   // STAGED: barrier the bulk copy of the row completes on
+    bool ready;  // the row has landed
+    __device__ __forceinline__ Ref ref(int32_t) const { return Ref{}; }
+    // Called before the first lookup: the row must have landed by then.
+    __device__ __forceinline__ void prepare(const View& v)
+    {
+        if (STAGED && !ready) {
+            if (!mbar_wait_bounded(bar, 0, STAGE_WAIT_LIMIT)) atomicOr(v.err, ERR_STAGE);
+            ready = true;
+        }
+    }
+    __device__ __forceinline__ int32_t count(const Ref&, uint32_t k) const
+    {
+        return STAGED ? row[k] : __ldg(row + k);
+    }
+    __device__ __forceinline__ Draw draw_issue(const Ref&, const View& v, const uint4& r) const
+    {
+        Draw d;
+        d.sparse = r.x < mix;
+        d.rz = r.z;
+        d.b = scale_to_range(r.y, d.sparse ? (uint32_t)nnz : (uint32_t)v.K);
+        if (PACKED) {
+            d.e = __ldg((d.sparse ? pk : v.dn_pk) + d.b);
+        } else if (d.sparse) {
+            const uint32_t al = __ldg(idx + d.b);
+            const uint32_t item = (al == d.b || r.z < __ldg(thr + d.b)) ? d.b : al;
+            d.e = make_uint2(0u, __ldg(topic + item));
+        } else {
+            d.e = __ldg(v.dn_pk + d.b);
+        }
+        return d;
+    }
+    __device__ __forceinline__ void draw_finish(const Ref&, const Draw& d, uint32_t& t, int32_t& n_tw) const
+    {
+        if (d.sparse) {
+            if (PACKED) t = (d.rz < d.e.x) ? (d.e.y & 0xFFFFu) : (d.e.y >> 16);
+            else t = d.e.y;
+        } else {
+            t = (d.e.y == d.b || d.rz < d.e.x) ? d.b : d.e.y;
+        }
+        n_tw = -1;  // looked up with the other counts
+    }
+};
+
+// A tile of tail words: sorted n_kw rows and alias bins in shared memory.
+struct ColdTile {
+    struct Ref {
+        int32_t rs, nnz;  // the word's row inside the tile's arrays
+        uint32_t mix;
+    };
+    const int32_t* woff;  // [nw+1] first token of each word, relative to the tile
+    const int32_t* rs;    // [nw+1] first row slot of each word, relative to the tile
+    const int32_t* nnz;
+    const uint32_t* mix;
+    const uint32_t* topic;
+    const uint32_t* cnt;
+    const uint32_t* thr;
+    const uint32_t* idx;
+    int32_t nw;
+    __device__ __forceinline__ Ref ref(int32_t q) const
+    {
+        int32_t lo = 0, hi = nw;  // last word with woff[word] <= q
+        while (hi - lo > 1) {
+            const int32_t mid = (lo + hi) >> 1;
+            if (woff[mid] <= q) lo = mid; else hi = mid;
+        }
+        return Ref{rs[lo], nnz[lo], mix[lo]};
+    }
+    __device__ __forceinline__ void prepare(const View&) {}
+    __device__ __forceinline__ int32_t count(const Ref& w, uint32_t k) const
+    {
+        int32_t lo = 0, hi = w.nnz;
+        while (lo < hi) {
+            const int32_t mid = (lo + hi) >> 1;
+            if (topic[w.rs + mid] < k) lo = mid + 1; else hi = mid;
+        }
+        return (lo < w.nnz && topic[w.rs + lo] == k) ? (int32_t)cnt[w.rs + lo] : 0;
+    }
+    __device__ __forceinline__ Draw draw_issue(const Ref& w, const View& v, const uint4& r) const
+    {
+        Draw d;
+        d.sparse = r.x < w.mix;
+        d.rz = r.z;
+        d.b = scale_to_range(r.y, d.sparse ? (uint32_t)w.nnz : (uint32_t)v.K);
+        d.e = make_uint2(0u, 0u);
+        if (!d.sparse) d.e = __ldg(v.dn_pk + d.b);
+        return d;
+    }
+    __device__ __forceinline__ void draw_finish(const Ref& w, const Draw& d, uint32_t& t, int32_t& n_tw) const
+    {
+        if (d.sparse) {
+            const uint32_t al = idx[w.rs + d.b];
+            const uint32_t item = (al == d.b || d.rz < thr[w.rs + d.b]) ? d.b : al;
+            t = topic[w.rs + item];
+            n_tw = (int32_t)cnt[w.rs + item];
+        } else {
+            t = (d.e.y == d.b || d.rz < d.e.x) ? d.b : d.e.y;
+            n_tw = -1;
+        }
+    }
+};
+
+// --- pass 1: word-proposals (word order) ---------------------------------------------------------
+// Draws the topic proposed by every word-proposal step (even steps, Eq. 6) of the tile's tokens.
+// A proposal depends on (token, sweep, step) and the frozen tables only, never on the chain's
+// state, so all of them can be drawn before anything is accepted.
+template <typename T, class Tile>
+__device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, const int32_t p_begin,
+                                               const int32_t p_end, const int32_t nthreads, const uint2 key,
+                                               const uint32_t sweep, const int32_t mh_steps)
+{
+    T* prop = reinterpret_cast<T*>(v.prop);
+    for (int32_t p = p_begin + (int32_t)threadIdx.x; p < p_end; p += nthreads) {
+        const uint32_t tok = __ldcs(v.tok_orig + p);
+        const uint32_t at = __ldcs(v.inv + p);  // the document-side pass reads block-major
+        const typename Tile::Ref w = tile.ref(p - p_begin);
+        for (int32_t m = 0; m < mh_steps; m += 2) {
+            const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)m, 0u), key);
+            const Draw d = tile.draw_issue(w, v, r);
+            uint32_t t;
+            int32_t n_tw;
+            tile.draw_finish(w, d, t, n_tw);
+            __stcs(prop + (size_t)(m >> 1) * v.N + at, (T)t);
+        }
+    }
+}
+
+// --- pass 2: document side (block-major order) -----------------------------------------------------
+// For every token: its own record, the doc-proposals (odd steps, Eq. 9 / Eq. 12) and n_kd at every
+// proposed topic.  The tokens come in block-major order, so the records and tables read here
+// belong to one block of documents at a time and are served from L2; the results go to the
+// token's word-sorted position.
 template <typename T>
 __global__ void __launch_bounds__(256)
-k_sample(View v, const T* __restrict__ zw_cur, const T* __restrict__ zd_cur, T* __restrict__ zw_nxt,
-         T* __restrict__ zd_nxt, uint2 key, uint32_t sweep, int32_t mh_steps)
+k_doc_side(View v, uint2 key, uint32_t sweep, int32_t mh_steps)
 {
-    __shared__ int32_t w_lo_s, w_hi_s;
-    const int32_t p0 = blockIdx.x * SAMPLE_TILE;
-    const int32_t p1 = min(v.N, p0 + SAMPLE_TILE);
-    if (threadIdx.x < 2) {
-        // word of the tile's first / last token: last w with word_off[w] <= p
-        const int32_t p = threadIdx.x == 0 ? p0 : p1 - 1;
-        int32_t lo = 0, hi = v.V;
-        while (hi - lo > 1) {
-            const int32_t mid = (lo + hi) >> 1;
-            if (__ldg(v.word_off + mid) <= p) lo = mid; else hi = mid;
+    const int cb = v.count_bits;
+    const T* prop = reinterpret_cast<const T*>(v.prop);
+    const double Ka = v.Kalpha;
+    const size_t N = (size_t)v.N;
+    const int lane = threadIdx.x & 31;
+    // all lanes of a warp run the same number of iterations and meet again after every phase;
+    // lanes past the end repeat the last token and store nothing
+    for (int64_t m0 = blockIdx.x * (int64_t)blockDim.x + threadIdx.x - lane; m0 < v.N;
+         m0 += (int64_t)gridDim.x * blockDim.x) {
+        const bool valid = m0 + lane < v.N;
+        const int64_t m = valid ? m0 + lane : v.N - 1;
+        const uint2 dinfo = __ldcs(v.dinfo_bm + m);
+        const uint32_t tok = __ldcs(v.tok_bm + m);
+        const uint32_t own = __ldcg(v.rec + tok);
+        const DkProbe pr(dinfo.x, dinfo.y);
+        const double n_d = (double)dinfo.y;
+        uint32_t* out = v.dside + (size_t)m * v.side_stride;
+        if (valid) __stcs(out, own);
+        for (int32_t st = 0; st < mh_steps; st += 2) {
+            // word-proposal of step st (drawn by pass 1): first group of its n_kd lookup
+            const uint32_t t1 = (uint32_t)__ldcs(prop + (size_t)(st >> 1) * N + m);
+            const uint32_t g1 = pr.first(t1);
+            const uint4 q1 = load_group(v.dk_slots, g1);
+            // doc-proposal of step st+1 (Eq. 9, Eq. 12): the record of a random token of the
+            // document, or a uniform topic with probability K*alpha / (n_d + K*alpha) and then
+            // the first group of its n_kd lookup -- one read either way
+            const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)(st + 1), 0u), key);
+            const double uu = __dmul_rn((double)r.x, INV_2_32);
+            const bool copy = __dmul_rn(uu, __dadd_rn(n_d, Ka)) < n_d;
+            const uint32_t t2 = scale_to_range(r.y, (uint32_t)v.K);
+            const uint32_t g2 = pr.first(t2);
+            const uint32_t j = dinfo.x + scale_to_range(r.y, dinfo.y);
+            const uint4 q2 = copy ? load_group(v.rec, j >> 2) : load_group(v.dk_slots, g2);
+            __syncwarp();
+            const uint32_t e1 = lookup_dk(v.dk_slots, pr, g1, q1, t1, cb);
+            __syncwarp();
+            uint32_t out2 = quad_word(q2, j & 3u);
+            if (!copy) {
+                const uint32_t e2 = lookup_dk(v.dk_slots, pr, g2, q2, t2, cb);
+                out2 = e2 ? e2 : t2 << cb;
+            }
+            __syncwarp();
+            if (valid) {
+                __stcs(out + 1 + st, e1 ? e1 : t1 << cb);
+                if (st + 1 < mh_steps) __stcs(out + 2 + st, out2);
+            }
         }
-        if (threadIdx.x == 0) w_lo_s = lo; else w_hi_s = lo;
+        __syncwarp();
+    }
+}
+
+// --- pass 3: accept / reject (word order) -----------------------------------------------------------
+// Runs the chain of every token of the tile: everything the document side contributes was
+// gathered by pass 2, the word side comes from the tile's staged rows.
+template <typename T, int CH, class Tile>
+__device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const int32_t p_begin, const int32_t p_end,
+                                              const int32_t nthreads, const uint2 key, const uint32_t sweep,
+                                              const int32_t mh_steps)
+{
+    const int cb = v.count_bits;
+    const uint32_t cmask = (1u << cb) - 1u;
+    const double alpha = v.alpha, beta = v.beta, Vb = v.Vbeta;
+    static_assert(CH % 2 == 0, "a group of steps starts on a word-proposal");
+    const size_t N = (size_t)v.N;
+    T* zw = reinterpret_cast<T*>(v.zw);
+    bool bad = false;
+    for (int32_t p = p_begin + (int32_t)threadIdx.x; p < p_end; p += nthreads) {
+        const uint32_t tok = __ldcs(v.tok_orig + p);
+        const uint32_t at = __ldcs(v.inv + p);
+        const uint32_t* side = v.dside + (size_t)at * v.side_stride;  // what pass 2 gathered for this token
+        const uint32_t own = __ldcs(side);
+        const typename Tile::Ref w = tile.ref(p - p_begin);
+        uint32_t z0 = 0, s = 0;
+        int32_t n_sd = 0, n_sw = 0, n_s = 0;
+        for (int32_t m0 = 0; m0 < mh_steps; m0 += CH) {
+            uint32_t e[CH], ua[CH];
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                e[i] = 0;
+                ua[i] = 0;
+                if (m0 + i < mh_steps) {
+                    e[i] = __ldcs(side + 1 + m0 + i);
+                    ua[i] = philox4x32_10(make_uint4(tok, sweep, (uint32_t)(m0 + i), 0u), key).w;
+                }
+            }
+            if (m0 == 0) {
+                // counts at the start state s = z0, where all three are >= 1
+                tile.prepare(v);
+                z0 = s = own >> cb;
+                n_sd = (int32_t)(own & cmask);
+                n_sw = tile.count(w, z0);
+                n_s = __ldg(v.nk + z0);
+                bad = bad || n_sd < 1 || n_sw < 1 || n_s < 1;
+            }
+            // counts at the proposed topics, all read before the first acceptance test
+            uint32_t t[CH];
+            int32_t n_tw[CH], n_t[CH];
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                t[i] = e[i] >> cb;
+                n_tw[i] = tile.count(w, t[i]);
+                n_t[i] = __ldg(v.nk + t[i]);
+            }
+            // Eq. 8 (word steps) / Eq. 11 (doc steps), products taken left to right
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                const bool live = m0 + i < mh_steps && t[i] != s;
+                const int32_t n_td = (int32_t)(e[i] & cmask);
+                const int32_t e_s = (s == z0), e_t = (t[i] == z0);
+                double num = __dadd_rn((double)(n_td - e_t), alpha);
+                num = __dmul_rn(num, __dadd_rn((double)(n_tw[i] - e_t), beta));
+                num = __dmul_rn(num, __dadd_rn((double)(n_s - e_s), Vb));
+                double den = __dadd_rn((double)(n_sd - e_s), alpha);
+                den = __dmul_rn(den, __dadd_rn((double)(n_sw - e_s), beta));
+                den = __dmul_rn(den, __dadd_rn((double)(n_t[i] - e_t), Vb));
+                if ((i & 1) == 0) {
+                    num = __dmul_rn(num, __dadd_rn((double)n_sw, beta));
+                    num = __dmul_rn(num, __dadd_rn((double)n_t[i], Vb));
+                    den = __dmul_rn(den, __dadd_rn((double)n_tw[i], beta));
+                    den = __dmul_rn(den, __dadd_rn((double)n_s, Vb));
+                } else {
+                    num = __dmul_rn(num, __dadd_rn((double)n_sd, alpha));
+                    den = __dmul_rn(den, __dadd_rn((double)n_td, alpha));
+                }
+                const double u = __dmul_rn((double)ua[i], INV_2_32);
+                if (live && __dmul_rn(u, den) < num) {
+                    s = t[i];
+                    n_sd = n_td;
+                    n_sw = n_tw[i];
+                    n_s = n_t[i];
+                }
+            }
+        }
+        __stcs(zw + p, (T)s);
+        __stcs(reinterpret_cast<T*>(v.zbm) + at, (T)s);
+    }
+    if (bad) atomicOr(v.err, ERR_COUNT_ZERO);
+}
+
+// Hot words: tile = (word, first token, count).  ACCEPT = false: pass 1, true: pass 3.
+template <typename T, int CH, bool STAGED, bool ACCEPT>
+__global__ void __launch_bounds__(HOT_THREADS)
+k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
+{
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    __shared__ __align__(8) unsigned long long bar;
+    constexpr bool PACKED = sizeof(T) == 2;
+    const int32_t w = tiles[3 * blockIdx.x], p0 = tiles[3 * blockIdx.x + 1], cnt = tiles[3 * blockIdx.x + 2];
+    const int32_t* row_g = v.dense_rows + (size_t)__ldg(v.dense_slot + w) * v.dense_stride;
+    int32_t* row_s = reinterpret_cast<int32_t*>(dyn_smem);
+    if (STAGED && ACCEPT) {
+        if (threadIdx.x == 0) {
+            const uint32_t bytes = (uint32_t)v.dense_stride * 4u;
+            mbar_init(&bar, 1);
+            mbar_expect_tx(&bar, bytes);
+            bulk_copy_g2s(row_s, row_g, bytes, &bar);
+        }
+        __syncthreads();
+    }
+    const int32_t r0 = __ldg(v.row_start + w);
+    HotTile<STAGED && ACCEPT, PACKED> tile;
+    tile.row = (STAGED && ACCEPT) ? row_s : row_g;
+    tile.pk = v.al_pk + r0;
+    tile.thr = v.al_thr + r0;
+    tile.idx = v.al_idx + r0;
+    tile.topic = v.wk_topic + r0;
+    tile.nnz = __ldg(v.wk_nnz + w);
+    tile.mix = __ldg(v.mix32 + w);
+    tile.bar = &bar;
+    tile.ready = !(STAGED && ACCEPT);
+    if (ACCEPT) accept_tokens<T, CH>(v, tile, p0, p0 + cnt, HOT_THREADS, key, sweep, mh_steps);
+    else propose_tokens<T>(v, tile, p0, p0 + cnt, HOT_THREADS, key, sweep, mh_steps);
+    // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one
+}
+
+// Tail words: tile = range of whole words [w0, w1) with at most COLD_TILE tokens.
+template <typename T, int CH, bool ACCEPT>
+__global__ void __launch_bounds__(COLD_THREADS)
+k_word_cold(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
+{
+    __shared__ int32_t woff_s[COLD_WORDS + 1];  // first token of each word, relative to the tile
+    __shared__ int32_t rs_s[COLD_WORDS + 1];    // first row slot of each word, relative to the tile
+    __shared__ int32_t nnz_s[COLD_WORDS];
+    __shared__ uint32_t mix_s[COLD_WORDS];
+    __shared__ uint32_t topic_s[COLD_TILE], count_s[COLD_TILE], thr_s[COLD_TILE], idx_s[COLD_TILE];
+    const int tid = threadIdx.x;
+    const int32_t w0 = tiles[2 * blockIdx.x], w1 = tiles[2 * blockIdx.x + 1];
+    const int32_t nw = w1 - w0;
+    const int32_t p0 = __ldg(v.word_off + w0), cnt = __ldg(v.word_off + w1) - p0;
+    const int32_t e0 = __ldg(v.row_start + w0), ne = __ldg(v.row_start + w1) - e0;
+    if (cnt == 0) return;
+    for (int j = tid; j <= nw; j += COLD_THREADS) {
+        woff_s[j] = __ldg(v.word_off + w0 + j) - p0;
+        rs_s[j] = __ldg(v.row_start + w0 + j) - e0;
+    }
+    for (int j = tid; j < nw; j += COLD_THREADS) {
+        nnz_s[j] = __ldg(v.wk_nnz + w0 + j);
+        mix_s[j] = __ldg(v.mix32 + w0 + j);
+    }
+    for (int j = tid; j < ne; j += COLD_THREADS) {
+        topic_s[j] = __ldcs(v.wk_topic + e0 + j);
+        if (ACCEPT) {
+            count_s[j] = __ldcs(v.wk_count + e0 + j);
+        } else {
+            thr_s[j] = __ldcs(v.al_thr + e0 + j);
+            idx_s[j] = __ldcs(v.al_idx + e0 + j);
+        }
     }
     __syncthreads();
-    const int32_t w_lo = w_lo_s, w_hi = w_hi_s;
-    const double alpha = v.alpha, beta = v.beta, Vb = v.Vbeta, Ka = v.Kalpha;
-
-    for (int32_t p = p0 + threadIdx.x; p < p1; p += blockDim.x) {
-        int32_t lo = w_lo, hi = w_hi + 1;
-        while (hi - lo > 1) {
-            const int32_t mid = (lo + hi) >> 1;
-            if (__ldg(v.word_off + mid) <= p) lo = mid; else hi = mid;
-        }
-        const int32_t w = lo;
-        const uint2 dinfo = __ldg(v.tok_dinfo + p);
-        const uint32_t tok = __ldg(v.tok_orig + p);
-        const uint32_t z0 = (uint32_t)zw_cur[p];
-
-        const int32_t r0 = __ldg(v.row_start + w), wnnz = __ldg(v.wk_nnz + w);
-        const int32_t dslot = __ldg(v.dense_slot + w);
-        const uint32_t mix = __ldg(v.mix32 + w);
-        const int32_t d0 = (int32_t)dinfo.x, n_d = (int32_t)dinfo.y;
-        const uint32_t* dtab = v.dk_slots + 2 * (size_t)dinfo.x;
-        const uint32_t dcap = 2u * dinfo.y;
-
-        // counts at the current state s (start: s = z0, where all three are >= 1)
-        uint32_t s = z0;
-        int32_t n_sd = lookup_dk(v, dtab, dcap, s);
-        int32_t n_sw = lookup_wk(v, dslot, r0, wnnz, s);
-        int32_t n_s = __ldg(v.nk + s);
-        if (n_sd < 1 || n_sw < 1 || n_s < 1) atomicOr(v.err, ERR_COUNT_ZERO);
-
-        for (int32_t m = 0; m < mh_steps; ++m) {
-            const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)m, 0u), key);
-            uint32_t t;
-            int32_t n_tw = -1;
-            const bool word_step = (m & 1) == 0;
-            if (word_step) {
-                // word-proposal (Eq. 6): sparse term with probability mix/2^32, else dense term
-                if (r.x < mix) {
-                    const uint32_t b = scale_to_range(r.y, (uint32_t)wnnz);
-                    const uint32_t al = __ldg(v.al_idx + r0 + b);
-                    const uint32_t item = (al == b || r.z < __ldg(v.al_thr + r0 + b)) ? b : al;
-                    t = __ldg(v.wk_topic + r0 + item);
-                    n_tw = (int32_t)__ldg(v.wk_count + r0 + item);
-                } else {
-                    const uint32_t b = scale_to_range(r.y, (uint32_t)v.K);
-                    const uint32_t al = __ldg(v.dn_idx + b);
-                    t = (al == b || r.z < __ldg(v.dn_thr + b)) ? b : al;
-                }
-            } else {
-                // doc-proposal (Eq. 9, Eq. 12): copy the topic of a random token of the document,
-                // or a uniform topic with probability K*alpha / (n_d + K*alpha)
-                const double u = __dmul_rn((double)r.x, INV_2_32);
-                if (__dmul_rn(u, __dadd_rn((double)n_d, Ka)) < (double)n_d)
-                    t = (uint32_t)zd_cur[d0 + scale_to_range(r.y, (uint32_t)n_d)];
-                else
-                    t = scale_to_range(r.y, (uint32_t)v.K);
-            }
-            if (t == s) continue;
-            if (n_tw < 0) n_tw = lookup_wk(v, dslot, r0, wnnz, t);
-            const int32_t n_td = lookup_dk(v, dtab, dcap, t);
-            const int32_t n_t = __ldg(v.nk + t);
-            const int32_t e_s = (s == z0), e_t = (t == z0);
-            // Eq. 8 (word step) / Eq. 11 (doc step), products taken left to right
-            double num = __dadd_rn((double)(n_td - e_t), alpha);
-            num = __dmul_rn(num, __dadd_rn((double)(n_tw - e_t), beta));
-            num = __dmul_rn(num, __dadd_rn((double)(n_s - e_s), Vb));
-            double den = __dadd_rn((double)(n_sd - e_s), alpha);
-            den = __dmul_rn(den, __dadd_rn((double)(n_sw - e_s), beta));
-            den = __dmul_rn(den, __dadd_rn((double)(n_t - e_t), Vb));
-            if (word_step) {
-                num = __dmul_rn(num, __dadd_rn((double)n_sw, beta));
-                num = __dmul_rn(num, __dadd_rn((double)n_t, Vb));
-                den = __dmul_rn(den, __dadd_rn((double)n_tw, beta));
-                den = __dmul_rn(den, __dadd_rn((double)n_s, Vb));
-            } else {
-                num = __dmul_rn(num, __dadd_rn((double)n_sd, alpha));
-                den = __dmul_rn(den, __dadd_rn((double)n_td, alpha));
-            }
-            const double ua = __dmul_rn((double)r.w, INV_2_32);
-            if (__dmul_rn(ua, den) < num) {
-                s = t;
-                n_sd = n_td;
-                n_sw = n_tw;
-                n_s = n_t;
-            }
-        }
-        zw_nxt[p] = (T)s;
-        zd_nxt[tok] = (T)s;
-    }
+    ColdTile tile{woff_s, rs_s, nnz_s, mix_s, topic_s, count_s, thr_s, idx_s, nw};
+    if (ACCEPT) accept_tokens<T, CH>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
+    else propose_tokens<T>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
 }
 
 // z_i uniform on {0..K-1}: Philox counter (token, 0, 0, 1), word 0.
 template <typename T>
-__global__ void k_init(View v, T* __restrict__ zw, T* __restrict__ zd, uint2 key)
+__global__ void k_init(View v, uint2 key)
 {
+    T* zw = reinterpret_cast<T*>(v.zw);
+    T* zbm = reinterpret_cast<T*>(v.zbm);
     for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < v.N;
          p += (int64_t)gridDim.x * blockDim.x) {
         const uint32_t tok = v.tok_orig[p];
         const uint4 r = philox4x32_10(make_uint4(tok, 0u, 0u, 1u), key);
         const T z = (T)scale_to_range(r.x, (uint32_t)v.K);
         zw[p] = z;
-        zd[tok] = z;
+        zbm[v.inv[p]] = z;
     }
 }
 
 template <typename T>
-__global__ void k_spread(View v, const int32_t* __restrict__ z_in, T* __restrict__ zw, T* __restrict__ zd)
+__global__ void k_spread(View v, const int32_t* __restrict__ z_in)
 {
+    T* zw = reinterpret_cast<T*>(v.zw);
+    T* zbm = reinterpret_cast<T*>(v.zbm);
     for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < v.N;
          p += (int64_t)gridDim.x * blockDim.x) {
-        const int32_t a = z_in[p];
-        if (a < 0 || a >= v.K) atomicOr(v.err, ERR_TOPIC_RANGE);
-        zd[p] = (T)a;
-        zw[p] = (T)z_in[v.tok_orig[p]];
+        int32_t a = z_in[v.tok_orig[p]];
+        if (a < 0 || a >= v.K) {
+            atomicOr(v.err, ERR_TOPIC_RANGE);
+            a = 0;
+        }
+        zw[p] = (T)a;
+        zbm[v.inv[p]] = (T)a;
     }
 }
 
-template <typename T>
-__global__ void k_export(int32_t n, const T* __restrict__ zd, int32_t* __restrict__ out)
+__global__ void k_export(View v, int32_t* __restrict__ out)
 {
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < v.N;
          i += (int64_t)gridDim.x * blockDim.x)
-        out[i] = (int32_t)zd[i];
+        out[i] = (int32_t)(v.rec[i] >> v.count_bits);
 }
 
 static int grid_for(int64_t n, int block)
@@ -187,22 +509,73 @@ static int grid_for(int64_t n, int block)
     return g < 1 ? 1 : (int)g;
 }
 
+template <typename T, int CH>
+static int sample_tc(Ctx& c, int mh_steps)
+{
+    const View& v = c.v;
+    const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
+    const bool staged = c.K <= HOT_STAGE_MAX_K;
+    const int side_grid = 148 * 8;
+    int launches = 0;
+    // pass 1: word-proposals
+    if (c.n_hot_tiles) {
+        k_word_hot<T, CH, false, false><<<c.n_hot_tiles, HOT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key, c.sweep,
+                                                                                    mh_steps);
+        ++launches;
+    }
+    if (c.n_cold_tiles) {
+        k_word_cold<T, CH, false><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
+                                                                                mh_steps);
+        ++launches;
+    }
+    // pass 2: document side
+    k_doc_side<T><<<side_grid, 256, 0, c.stream>>>(v, key, c.sweep, mh_steps);
+    ++launches;
+    // pass 3: accept / reject
+    if (c.n_hot_tiles) {
+        if (staged)
+            k_word_hot<T, CH, true, true><<<c.n_hot_tiles, HOT_THREADS, (size_t)v.dense_stride * 4, c.stream>>>(
+                v, c.hot_tiles, key, c.sweep, mh_steps);
+        else
+            k_word_hot<T, CH, false, true><<<c.n_hot_tiles, HOT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
+                                                                                       c.sweep, mh_steps);
+        ++launches;
+    }
+    if (c.n_cold_tiles) {
+        k_word_cold<T, CH, true><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
+                                                                               mh_steps);
+        ++launches;
+    }
+    return launches;
+}
+
+// The accept/reject pass handles proposals in groups of two (mh_steps <= 2) or four.
 template <typename T>
 static int sample_t(Ctx& c, int mh_steps)
 {
-    if (c.N == 0) return 0;
-    View& v = c.v;
-    const int nxt = c.cur ^ 1;
-    const int grid = (int)((c.N + SAMPLE_TILE - 1) / SAMPLE_TILE);
-    const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
-    k_sample<T><<<grid, 256, 0, c.stream>>>(v, (const T*)v.zw[c.cur], (const T*)v.zd[c.cur],
-                                            (T*)v.zw[nxt], (T*)v.zd[nxt], key, c.sweep, mh_steps);
-    return 1;
+    return mh_steps <= 2 ? sample_tc<T, 2>(c, mh_steps) : sample_tc<T, 4>(c, mh_steps);
 }
 
+// Reads the records and tables of the sweep-start state; writes zw and zbm.
 int launch_sample(Ctx& c, int mh_steps)
 {
+    if (c.N == 0) return 0;
     return c.wide_topics ? sample_t<int32_t>(c, mh_steps) : sample_t<uint16_t>(c, mh_steps);
+}
+
+template <typename T, int CH>
+static void set_hot_limit()
+{
+    cudaFuncSetAttribute(k_word_hot<T, CH, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         HOT_STAGE_MAX_K * 4);
+}
+
+void set_sample_smem_limits()
+{
+    set_hot_limit<uint16_t, 2>();
+    set_hot_limit<uint16_t, 4>();
+    set_hot_limit<int32_t, 2>();
+    set_hot_limit<int32_t, 4>();
 }
 
 int launch_init(Ctx& c)
@@ -210,10 +583,8 @@ int launch_init(Ctx& c)
     if (c.N == 0) return 0;
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     const int g = grid_for(c.N, 256);
-    if (c.wide_topics)
-        k_init<int32_t><<<g, 256, 0, c.stream>>>(c.v, (int32_t*)c.v.zw[c.cur], (int32_t*)c.v.zd[c.cur], key);
-    else
-        k_init<uint16_t><<<g, 256, 0, c.stream>>>(c.v, (uint16_t*)c.v.zw[c.cur], (uint16_t*)c.v.zd[c.cur], key);
+    if (c.wide_topics) k_init<int32_t><<<g, 256, 0, c.stream>>>(c.v, key);
+    else k_init<uint16_t><<<g, 256, 0, c.stream>>>(c.v, key);
     return 1;
 }
 
@@ -221,21 +592,15 @@ int launch_spread_assignments(Ctx& c, const int32_t* z_dev)
 {
     if (c.N == 0) return 0;
     const int g = grid_for(c.N, 256);
-    if (c.wide_topics)
-        k_spread<int32_t><<<g, 256, 0, c.stream>>>(c.v, z_dev, (int32_t*)c.v.zw[c.cur], (int32_t*)c.v.zd[c.cur]);
-    else
-        k_spread<uint16_t><<<g, 256, 0, c.stream>>>(c.v, z_dev, (uint16_t*)c.v.zw[c.cur], (uint16_t*)c.v.zd[c.cur]);
+    if (c.wide_topics) k_spread<int32_t><<<g, 256, 0, c.stream>>>(c.v, z_dev);
+    else k_spread<uint16_t><<<g, 256, 0, c.stream>>>(c.v, z_dev);
     return 1;
 }
 
 int launch_export_assignments(Ctx& c, int32_t* z_dev)
 {
     if (c.N == 0) return 0;
-    const int g = grid_for(c.N, 256);
-    if (c.wide_topics)
-        k_export<int32_t><<<g, 256, 0, c.stream>>>((int32_t)c.N, (const int32_t*)c.v.zd[c.cur], z_dev);
-    else
-        k_export<uint16_t><<<g, 256, 0, c.stream>>>((int32_t)c.N, (const uint16_t*)c.v.zd[c.cur], z_dev);
+    k_export<<<grid_for(c.N, 256), 256, 0, c.stream>>>(c.v, z_dev);
     return 1;
 }
 
