@@ -437,6 +437,11 @@ int lda_set_option(lda_ctx* h, const char* key, double value)
         c.dense_min_tf = value;
         return LDA_OK;
     }
+    if (!std::strcmp(key, "block_log2")) {
+        if (!(value >= 10.0 && value <= 30.0)) return fail(&c, LDA_EINVAL, "block_log2 must be in [10,30]");
+        c.block_shift = (int)value;
+        return LDA_OK;
+    }
     return fail(&c, LDA_EINVAL, "unknown option");
 }
 

@@ -188,7 +188,10 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
 // document) is written next to it, so that the MH step gets both in one read.
 //
 // `tab` points at the copy of global slot `a0`; slot x of the global array is tab[x - a0].
-__device__ __forceinline__ void dk_insert(uint32_t* tab, uint32_t a0, const DkProbe& pr, uint32_t k, int count_bits)
+// Returns the global slot the topic lives in (or 0xFFFFFFFF if the table had no room, which the
+// load factor rules out).
+__device__ __forceinline__ uint32_t dk_insert(uint32_t* tab, uint32_t a0, const DkProbe& pr, uint32_t k,
+                                              int count_bits)
 {
     const uint32_t fresh = k << count_bits;
     uint32_t g = pr.first(k);
@@ -200,10 +203,11 @@ __device__ __forceinline__ void dk_insert(uint32_t* tab, uint32_t a0, const DkPr
             const uint32_t prev = atomicCAS(&tab[slot - a0], DK_EMPTY, fresh);
             if (prev == DK_EMPTY || (prev >> count_bits) == k) {
                 atomicAdd(&tab[slot - a0], 1u);
-                return;
+                return slot;
             }
         }
     }
+    return 0xFFFFFFFFu;
 }
 
 __device__ __forceinline__ uint32_t dk_find(const uint32_t* tab, uint32_t a0, const DkProbe& pr, uint32_t k,
@@ -244,35 +248,25 @@ k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_of
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = doc_off[s0 + j] - base;
     for (int j = tid; j < 2 * cnt + 4; j += blockDim.x) slots[j] = DK_EMPTY;
     __syncthreads();
-    int32_t my_doc[SORT_TILE / 256];  // document (relative to the tile) of each of this thread's tokens
-#pragma unroll
-    for (int q = 0; q < SORT_TILE / 256; ++q) {
-        const int j = tid + q * 256;
-        my_doc[q] = -1;
-        if (j < cnt) {
-            int lo = 0, hi = nseg;  // last document with soff[doc] <= j
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (soff[mid] <= j) lo = mid; else hi = mid;
-            }
+    // one warp per document: its lanes insert the document's tokens and note where each topic landed
+    const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    for (int d = warp; d < nseg; d += nwarps) {
+        const int32_t first = soff[d], len = soff[d + 1] - first;
+        const DkProbe pr((uint32_t)(base + first), (uint32_t)len);
+        for (int j = first + lane; j < first + len; j += 32) {
             const uint32_t k = topic[j];
-            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
-            my_doc[q] = lo;
-            const DkProbe pr((uint32_t)(base + soff[lo]), (uint32_t)(soff[lo + 1] - soff[lo]));
-            dk_insert(slots, a0, pr, k, count_bits);
+            uint32_t slot = 0xFFFFFFFFu;
+            if (k < (uint32_t)K) slot = dk_insert(slots, a0, pr, k, count_bits);
+            if (slot == 0xFFFFFFFFu) atomicOr(err, k < (uint32_t)K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
+            topic[j] = slot;
         }
     }
     __syncthreads();
     uint32_t* out = slots_out + 2 * (size_t)base;
     for (int j = tid; j < 2 * cnt; j += blockDim.x) out[j] = slots[lead + j];
-#pragma unroll
-    for (int q = 0; q < SORT_TILE / 256; ++q) {
-        const int j = tid + q * 256;
-        const int32_t lo = my_doc[q];
-        if (lo >= 0) {
-            const DkProbe pr((uint32_t)(base + soff[lo]), (uint32_t)(soff[lo + 1] - soff[lo]));
-            rec[base + j] = dk_find(slots, a0, pr, topic[j], count_bits);
-        }
+    for (int j = tid; j < cnt; j += blockDim.x) {
+        const uint32_t slot = topic[j];
+        if (slot != 0xFFFFFFFFu) rec[base + j] = slots[slot - a0];
     }
 }
 

@@ -27,6 +27,10 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 #endif
 constexpr int HOT_THREADS = LDA_HOT_THREADS;
 constexpr int COLD_THREADS = 256;
+#ifndef LDA_DOC_SIDE_TILE
+#define LDA_DOC_SIDE_TILE 2048
+#endif
+constexpr int DOC_SIDE_TILE = LDA_DOC_SIDE_TILE;  // tokens per CTA of the document-side pass
 constexpr int STAGE_WAIT_LIMIT = 1 << 20;
 
 // --- shared-memory barrier and bulk-copy primitives ------------------------------------------
@@ -253,11 +257,13 @@ k_doc_side(View v, uint2 key, uint32_t sweep, int32_t mh_steps)
     const double Ka = v.Kalpha;
     const size_t N = (size_t)v.N;
     const int lane = threadIdx.x & 31;
-    // all lanes of a warp run the same number of iterations and meet again after every phase;
-    // lanes past the end repeat the last token and store nothing
-    for (int64_t m0 = blockIdx.x * (int64_t)blockDim.x + threadIdx.x - lane; m0 < v.N;
-         m0 += (int64_t)gridDim.x * blockDim.x) {
-        const bool valid = m0 + lane < v.N;
+    // A CTA takes DOC_SIDE_TILE consecutive tokens; CTAs start in index order, so the ones running at
+    // any moment work on neighbouring tokens, i.e. on the same block of documents.
+    // All lanes of a warp run the same number of iterations and meet again after every phase;
+    // lanes past the end repeat the last token and store nothing.
+    const int64_t tile_end = min((int64_t)v.N, (blockIdx.x + 1) * (int64_t)DOC_SIDE_TILE);
+    for (int64_t m0 = blockIdx.x * (int64_t)DOC_SIDE_TILE + threadIdx.x - lane; m0 < tile_end; m0 += blockDim.x) {
+        const bool valid = m0 + lane < tile_end;
         const int64_t m = valid ? m0 + lane : v.N - 1;
         const uint2 dinfo = __ldcs(v.dinfo_bm + m);
         const uint32_t tok = __ldcs(v.tok_bm + m);
@@ -515,7 +521,7 @@ static int sample_tc(Ctx& c, int mh_steps)
     const View& v = c.v;
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     const bool staged = c.K <= HOT_STAGE_MAX_K;
-    const int side_grid = 148 * 8;
+    const int side_grid = (int)((c.N + DOC_SIDE_TILE - 1) / DOC_SIDE_TILE);
     int launches = 0;
     // pass 1: word-proposals
     if (c.n_hot_tiles) {
