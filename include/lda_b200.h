@@ -57,11 +57,14 @@ typedef struct lda_stats {
     int32_t iters;            /* iterations of the last lda_sweep() */
     float ms_alias_dense;     /* dense smoothing table            (Section 4.2) */
     float ms_alias_sparse;    /* per-word sparse alias tables     (Section 4.2) */
-    float ms_sample;          /* token MH kernel                  (Eq. 6-13)    */
+    float ms_sample;          /* token MH step, all passes        (Eq. 6-13)    */
     float ms_count_wk;        /* n_kw rebuild                     (Section 3)   */
     float ms_count_k;         /* n_k rebuild                                    */
     float ms_count_dk;        /* n_kd rebuild                     (Eq. 12)      */
     float ms_total;           /* first launch to last kernel end                */
+    float ms_propose;         /* MH step, pass 1: word-proposals   (part of ms_sample) */
+    float ms_doc_side;        /* MH step, pass 2: document side    (part of ms_sample) */
+    float ms_accept;          /* MH step, pass 3: accept / reject  (part of ms_sample) */
 } lda_stats;
 
 /* Model dimensions and symmetric priors of the collapsed LDA model (Section 3,
@@ -73,7 +76,10 @@ int lda_set_stream(lda_ctx* ctx, void* cuda_stream);
 
 /* Tunables that never change results.  Must be set before lda_load_corpus().
  *   "dense_frac"   fraction of the vocabulary (by term frequency) whose n_kw rows are dense (Section 5)
- *   "dense_min_tf" words rarer than this stay sparse even inside dense_frac                          */
+ *   "dense_min_tf" words rarer than this stay sparse even inside dense_frac
+ *   "block_log2"   log2 of the tokens per block of documents in the block-major token order that the
+ *                  document-side pass of the MH step walks (default 21: the records and n_kd tables
+ *                  of one block, 12 bytes per token, stay in L2 while the pass is on it)             */
 int lda_set_option(lda_ctx* ctx, const char* key, double value);
 
 /* Corpus in document order: token i has word word_ids[i]; document d owns tokens

@@ -34,7 +34,8 @@ class lda_stats(C.Structure):
         ("sweeps_done", C.c_int32), ("iters", C.c_int32),
         ("ms_alias_dense", C.c_float), ("ms_alias_sparse", C.c_float), ("ms_sample", C.c_float),
         ("ms_count_wk", C.c_float), ("ms_count_k", C.c_float), ("ms_count_dk", C.c_float),
-        ("ms_total", C.c_float),
+        ("ms_total", C.c_float), ("ms_propose", C.c_float), ("ms_doc_side", C.c_float),
+        ("ms_accept", C.c_float),
     ]
 
     def as_dict(self):

@@ -384,7 +384,7 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
         cudaGetLastError();
         return LDA_ECUDA;
     }
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 10; ++i)
         if (cudaEventCreate(&c.ev[i]) != cudaSuccess) {
             for (int j = 0; j < i; ++j) cudaEventDestroy(c.ev[j]);
             dev_free_all(c);
@@ -406,7 +406,7 @@ void lda_destroy(lda_ctx* h)
     cudaSetDevice(c.device);
     cudaStreamSynchronize(c.stream);
     if (c.have_events)
-        for (int i = 0; i < 8; ++i) cudaEventDestroy(c.ev[i]);
+        for (int i = 0; i < 10; ++i) cudaEventDestroy(c.ev[i]);
     dev_free_all(c);
     cudaGetLastError();
     delete h;
@@ -549,7 +549,7 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
     if ((rc = ensure_exchange(c, mh_steps))) return rc;
     lda_stats& s = c.stats;
     s.ms_alias_dense = s.ms_alias_sparse = s.ms_sample = s.ms_count_wk = s.ms_count_k = s.ms_count_dk =
-        s.ms_total = 0.f;
+        s.ms_total = s.ms_propose = s.ms_doc_side = s.ms_accept = 0.f;
     s.kernel_launches = 0;
     s.iters = iters;
     for (int32_t it = 0; it < iters; ++it) {
@@ -578,6 +578,13 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
         float ms[7] = {0};
         for (int i = 0; i < 6; ++i) cudaEventElapsedTime(&ms[i], c.ev[i], c.ev[i + 1]);
         cudaEventElapsedTime(&ms[6], c.ev[0], c.ev[6]);
+        if (c.N > 0) {
+            float a = 0.f, b = 0.f, d = 0.f;
+            cudaEventElapsedTime(&a, c.ev[2], c.ev[8]);
+            cudaEventElapsedTime(&b, c.ev[8], c.ev[9]);
+            cudaEventElapsedTime(&d, c.ev[9], c.ev[3]);
+            s.ms_propose += a; s.ms_doc_side += b; s.ms_accept += d;
+        }
         s.ms_alias_dense += ms[0]; s.ms_alias_sparse += ms[1]; s.ms_sample += ms[2];
         s.ms_count_wk += ms[3]; s.ms_count_k += ms[4]; s.ms_count_dk += ms[5]; s.ms_total += ms[6];
         s.kernel_launches += n;

@@ -122,7 +122,7 @@ struct Ctx {
     int64_t device_bytes = 0;
     lda_stats stats{};
     int64_t launches = 0;
-    cudaEvent_t ev[8] = {};
+    cudaEvent_t ev[10] = {};  // 0..6 bracket the phases of a sweep, 8 and 9 the passes of the MH step
     bool have_events = false;
     std::string err;
 };

@@ -535,9 +535,11 @@ static int sample_tc(Ctx& c, int mh_steps)
         ++launches;
     }
     // pass 2: document side
+    cudaEventRecord(c.ev[8], c.stream);
     k_doc_side<T><<<side_grid, 256, 0, c.stream>>>(v, key, c.sweep, mh_steps);
     ++launches;
     // pass 3: accept / reject
+    cudaEventRecord(c.ev[9], c.stream);
     if (c.n_hot_tiles) {
         if (staged)
             k_word_hot<T, CH, true, true><<<c.n_hot_tiles, HOT_THREADS, (size_t)v.dense_stride * 4, c.stream>>>(
