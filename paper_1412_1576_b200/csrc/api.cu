@@ -105,7 +105,7 @@ int lda::ensure_exchange(Ctx& c, int mh_steps)
     };
     auto bytes_for = [&](int steps, size_t& prop_b, size_t& side_b, int& stride) {
         const size_t zt = c.wide_topics ? 4 : 2, n = (size_t)c.N;
-        stride = (1 + steps + 3) & ~3;
+        stride = (1 + steps + steps / 2 + 3) & ~3;  // own, one word per step, one uniform per doc step
         prop_b = zt * (((size_t)steps + 1) / 2) * n;
         side_b = 4 * (size_t)stride * n;
     };
@@ -272,8 +272,8 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         };
         for (int32_t d = 0; d < D; ++d) {
             const int64_t len = doc_off[d + 1] - doc_off[d];
-            if (len > SORT_TILE) { close(d); s0 = d + 1; tok = 0; long_docs.push_back(d); continue; }
-            if (tok + len > SORT_TILE || d - s0 >= SORT_TILE) { close(d); s0 = d; tok = 0; }
+            if (len > DOC_TILE) { close(d); s0 = d + 1; tok = 0; long_docs.push_back(d); continue; }
+            if (tok + len > DOC_TILE || d - s0 >= DOC_TILE) { close(d); s0 = d; tok = 0; }
             tok += len;
         }
         close(D);
@@ -318,8 +318,8 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     v.dn_thr = (uint32_t*)A((size_t)K * 4);
     v.dn_idx = (uint32_t*)A((size_t)K * 4);
     v.dense_mass = (unsigned long long*)A(8);
-    v.nk = (int32_t*)A((size_t)K * 4);
-    v.dk_slots = (uint32_t*)A(n1 * 8 + 16);
+    v.nk = (int32_t*)A((size_t)v.dense_stride * 4);  // padded like a dense row: copied in 16-byte units
+    v.dk_slots = (uint32_t*)A(n1 * 16 + 32);  // four slots per token, + one group past the end
     c.sc_w = (unsigned long long*)A(cap1 * 8);
     c.sc_de = (unsigned long long*)A(cap1 * 8);
     c.sc_item = (uint32_t*)A(cap1 * 4);
@@ -631,8 +631,9 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
         std::vector<int32_t> start((size_t)c.D + 1);
         if (cudaMemcpy(start.data(), v.doc_off, ((size_t)c.D + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
             return cuda_fail(&c, "copying document offsets");
-        std::vector<uint32_t> slots((size_t)std::max<int64_t>(2 * c.N, 1));
-        if (c.N && cudaMemcpy(slots.data(), v.dk_slots, (size_t)c.N * 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+        const int64_t spt = 4;  // slots per token (DK_SLOTS_PER_TOKEN of the device code)
+        std::vector<uint32_t> slots((size_t)std::max<int64_t>(spt * c.N, 1));
+        if (c.N && cudaMemcpy(slots.data(), v.dk_slots, (size_t)c.N * 4 * (size_t)spt, cudaMemcpyDeviceToHost) != cudaSuccess)
             return cuda_fail(&c, "copying n_kd tables");
         int64_t total = 0;
         for (uint32_t e : slots) total += (c.N && e != DK_EMPTY);
@@ -645,7 +646,7 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
         for (int64_t d = 0; d < c.D; ++d) {
             if (row_offsets) row_offsets[d] = o;
             row.clear();
-            for (int64_t j = 2 * (int64_t)start[(size_t)d]; j < 2 * (int64_t)start[(size_t)d + 1]; ++j)
+            for (int64_t j = spt * (int64_t)start[(size_t)d]; j < spt * (int64_t)start[(size_t)d + 1]; ++j)
                 if (slots[(size_t)j] != DK_EMPTY) row.push_back(slots[(size_t)j]);
             std::sort(row.begin(), row.end());
             for (uint32_t e : row) {

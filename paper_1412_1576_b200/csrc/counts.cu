@@ -187,44 +187,28 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
 // written out in one coalesced pass.  Every token's record (topic, n_kd of its topic in its
 // document) is written next to it, so that the MH step gets both in one read.
 //
-// `tab` points at the copy of global slot `a0`; slot x of the global array is tab[x - a0].
-// Returns the global slot the topic lives in (or 0xFFFFFFFF if the table had no room, which the
-// load factor rules out).
-__device__ __forceinline__ uint32_t dk_insert(uint32_t* tab, uint32_t a0, const DkProbe& pr, uint32_t k,
+// `tab` points at the copy of group `g0`; slot l of group g is tab[(g - g0) * 8 + l].
+// Returns the index into `tab` the topic lives at (or 0xFFFFFFFF if the table had no room,
+// which the load factor rules out).
+__device__ __forceinline__ uint32_t dk_insert(uint32_t* tab, uint32_t g0, const DkProbe& pr, uint32_t k,
                                               int count_bits)
 {
     const uint32_t fresh = k << count_bits;
     uint32_t g = pr.first(k);
     for (uint32_t n = 0; n < pr.g_cnt; ++n, g = pr.next(g)) {
+        const uint32_t lanes = pr.lanes(g);
 #pragma unroll
-        for (uint32_t l = 0; l < 4; ++l) {
-            const uint32_t slot = 4u * g + l;
-            if (!pr.inside(slot)) continue;
-            const uint32_t prev = atomicCAS(&tab[slot - a0], DK_EMPTY, fresh);
+        for (uint32_t l = 0; l < DK_GROUP; ++l) {
+            if (!((lanes >> l) & 1u)) continue;
+            const uint32_t at = (g - g0) * DK_GROUP + l;
+            const uint32_t prev = atomicCAS(&tab[at], DK_EMPTY, fresh);
             if (prev == DK_EMPTY || (prev >> count_bits) == k) {
-                atomicAdd(&tab[slot - a0], 1u);
-                return slot;
+                atomicAdd(&tab[at], 1u);
+                return at;
             }
         }
     }
     return 0xFFFFFFFFu;
-}
-
-__device__ __forceinline__ uint32_t dk_find(const uint32_t* tab, uint32_t a0, const DkProbe& pr, uint32_t k,
-                                            int count_bits)
-{
-    uint32_t g = pr.first(k);
-    for (uint32_t n = 0; n < pr.g_cnt; ++n, g = pr.next(g)) {
-#pragma unroll
-        for (uint32_t l = 0; l < 4; ++l) {
-            const uint32_t slot = 4u * g + l;
-            if (!pr.inside(slot)) continue;
-            const uint32_t e = tab[slot - a0];
-            if (e == DK_EMPTY) return k << count_bits;
-            if ((e >> count_bits) == k) return e;
-        }
-    }
-    return k << count_bits;
 }
 
 template <typename T>
@@ -232,21 +216,21 @@ __global__ void __launch_bounds__(256)
 k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_off, const T* __restrict__ zbm,
            const uint32_t* __restrict__ bm_of_tok, uint32_t* __restrict__ rec, uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
 {
-    __shared__ uint32_t slots[2 * SORT_TILE + 4];
-    __shared__ int32_t soff[SORT_TILE + 1];
-    __shared__ uint32_t topic[SORT_TILE];
+    __shared__ uint32_t slots[DK_SLOTS_PER_TOKEN * DOC_TILE + DK_GROUP];
+    __shared__ int32_t soff[DOC_TILE + 1];
+    __shared__ uint32_t topic[DOC_TILE];
     const int tid = threadIdx.x;
     const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
     const int32_t nseg = s1 - s0;
     const int32_t base = doc_off[s0];
     const int32_t cnt = doc_off[s1] - base;
     if (cnt == 0) return;
-    const uint32_t a0 = (2u * (uint32_t)base) & ~3u;        // global slot kept in slots[0]
-    const uint32_t lead = 2u * (uint32_t)base - a0;         // 0 or 2
+    const uint32_t g0 = (uint32_t)base >> 1;                    // group kept in slots[0..8)
+    const uint32_t lead = ((uint32_t)base & 1u) ? 4u : 0u;      // the tile's first slot inside that group
     // the tile's documents lie in one or two blocks of the block-major order: these reads hit L2
     for (int j = tid; j < cnt; j += blockDim.x) topic[j] = (uint32_t)__ldcg(zbm + __ldcs(bm_of_tok + base + j));
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = doc_off[s0 + j] - base;
-    for (int j = tid; j < 2 * cnt + 4; j += blockDim.x) slots[j] = DK_EMPTY;
+    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt + DK_GROUP; j += blockDim.x) slots[j] = DK_EMPTY;
     __syncthreads();
     // one warp per document: its lanes insert the document's tokens and note where each topic landed
     const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -256,17 +240,17 @@ k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_of
         for (int j = first + lane; j < first + len; j += 32) {
             const uint32_t k = topic[j];
             uint32_t slot = 0xFFFFFFFFu;
-            if (k < (uint32_t)K) slot = dk_insert(slots, a0, pr, k, count_bits);
+            if (k < (uint32_t)K) slot = dk_insert(slots, g0, pr, k, count_bits);
             if (slot == 0xFFFFFFFFu) atomicOr(err, k < (uint32_t)K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
             topic[j] = slot;
         }
     }
     __syncthreads();
-    uint32_t* out = slots_out + 2 * (size_t)base;
-    for (int j = tid; j < 2 * cnt; j += blockDim.x) out[j] = slots[lead + j];
+    uint32_t* out = slots_out + DK_SLOTS_PER_TOKEN * (size_t)base;
+    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) out[j] = slots[lead + j];
     for (int j = tid; j < cnt; j += blockDim.x) {
         const uint32_t slot = topic[j];
-        if (slot != 0xFFFFFFFFu) rec[base + j] = slots[slot - a0];
+        if (slot != 0xFFFFFFFFu) rec[base + j] = slots[slot];
     }
 }
 
@@ -280,17 +264,21 @@ k_long_doc_hash(const int32_t* __restrict__ long_docs, const int32_t* __restrict
     const int32_t d = long_docs[blockIdx.x];
     const int32_t first = doc_off[d], cnt = doc_off[d + 1] - first;
     const DkProbe pr((uint32_t)first, (uint32_t)cnt);
-    for (uint32_t j = threadIdx.x; j < 2u * (uint32_t)cnt; j += blockDim.x) slots_out[pr.t0 + j] = DK_EMPTY;
+    uint32_t* tab = slots_out + (size_t)pr.g_first * DK_GROUP;  // the table's first group
+    uint32_t* mine = slots_out + DK_SLOTS_PER_TOKEN * (size_t)first;
+    for (uint32_t j = threadIdx.x; j < (uint32_t)DK_SLOTS_PER_TOKEN * (uint32_t)cnt; j += blockDim.x) mine[j] = DK_EMPTY;
     __syncthreads();
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
         const uint32_t k = (uint32_t)zbm[bm_of_tok[first + j]];
-        if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
-        dk_insert(slots_out, 0u, pr, k, count_bits);
+        uint32_t at = 0xFFFFFFFFu;
+        if (k < (uint32_t)K) at = dk_insert(tab, pr.g_first, pr, k, count_bits);
+        if (at == 0xFFFFFFFFu) atomicOr(err, k < (uint32_t)K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
+        rec[first + j] = at;  // parked here until every insertion is done
     }
     __syncthreads();
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-        const uint32_t k = (uint32_t)zbm[bm_of_tok[first + j]];
-        if (k < (uint32_t)K) rec[first + j] = dk_find(slots_out, 0u, pr, k, count_bits);
+        const uint32_t at = rec[first + j];
+        if (at != 0xFFFFFFFFu) rec[first + j] = tab[at];
     }
 }
 
@@ -414,7 +402,7 @@ int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host)
     unsigned long long* acc = (unsigned long long*)c.red_i;
     cudaMemsetAsync(acc, 0, 16, c.stream);
     k_sum_i32<<<296, 256, 0, c.stream>>>(c.v.wk_nnz, c.V, acc);
-    if (c.N) k_count_filled<<<592, 256, 0, c.stream>>>(c.v.dk_slots, 2 * c.N, acc + 1);
+    if (c.N) k_count_filled<<<592, 256, 0, c.stream>>>(c.v.dk_slots, (int64_t)DK_SLOTS_PER_TOKEN * c.N, acc + 1);
     unsigned long long h[2] = {0, 0};
     cudaMemcpyAsync(h, acc, 16, cudaMemcpyDeviceToHost, c.stream);
     cudaStreamSynchronize(c.stream);

@@ -26,41 +26,54 @@ __device__ __forceinline__ uint32_t scale_to_range(uint32_t r, uint32_t n) { ret
 __device__ __forceinline__ int bit_length(unsigned long long x) { return 64 - __clzll((long long)x); }
 
 // --- n_kd tables --------------------------------------------------------------------------------
-// Document d owns slots [t0, t1) = [2*doc_off[d], 2*doc_off[d+1]) of one global slot array (twice
-// its length, so the load factor stays <= 0.5; Section 5, fn. 5).  A slot is
-// (topic << count_bits) | count, or DK_EMPTY_SLOT.  The table is bucketed by aligned groups of
-// four slots (one 16-byte read): topic k starts at group DkProbe::first() and tries the group's
-// slots that lie inside [t0, t1) in order, then the next group, wrapping to the table's first
-// group.  An empty slot met on the way means "absent".
+// Document d owns slots [4*doc_off[d], 4*doc_off[d+1]) of one global slot array: four slots per
+// token, so the load factor stays <= 0.25 (Section 5, fn. 5 asks for at least twice the number
+// of entries).  A slot is (topic << count_bits) | count, or DK_EMPTY_SLOT.  The table is
+// bucketed by aligned groups of eight slots (one 32-byte sector): topic k starts at group
+// DkProbe::first(k) and tries the group's slots that belong to the document in order, then the
+// next group, wrapping to the table's first group.  An empty slot met on the way means "absent".
+// At this load a lookup almost never needs a second group.
 constexpr uint32_t DK_EMPTY_SLOT = 0xFFFFFFFFu;
 constexpr uint32_t DK_HASH_MULT = 0x9E3779B1u;
+constexpr int DK_SLOTS_PER_TOKEN = 4;
+constexpr int DK_GROUP = 8;
 
 struct DkProbe {
-    uint32_t t0, t1;          // the table's slot range
-    uint32_t g_first, g_cnt;  // first group (slot index / 4) and number of groups it touches
+    uint32_t g_first, g_cnt;  // first group (slot index / 8) and number of groups the table touches
+    bool head_half, tail_half;  // the table starts / ends in the middle of a group
     __device__ __forceinline__ DkProbe(uint32_t doc_first_token, uint32_t doc_len)
-        : t0(2u * doc_first_token), t1(2u * (doc_first_token + doc_len))
     {
-        g_first = t0 >> 2;
-        g_cnt = ((t1 - 1u) >> 2) - g_first + 1u;
+        const uint32_t end = doc_first_token + doc_len;  // tokens; the document is not empty
+        g_first = doc_first_token >> 1;
+        g_cnt = ((end - 1u) >> 1) - g_first + 1u;
+        head_half = doc_first_token & 1u;
+        tail_half = end & 1u;
     }
     __device__ __forceinline__ uint32_t first(uint32_t k) const { return g_first + __umulhi(k * DK_HASH_MULT, g_cnt); }
     __device__ __forceinline__ uint32_t next(uint32_t g) const { return g + 1u - g_first == g_cnt ? g_first : g + 1u; }
-    __device__ __forceinline__ bool inside(uint32_t slot) const { return slot >= t0 && slot < t1; }
+    // bit l set: slot l of group g belongs to this table
+    __device__ __forceinline__ uint32_t lanes(uint32_t g) const
+    {
+        uint32_t m = 0xFFu;
+        if (head_half && g == g_first) m &= 0xF0u;
+        if (tail_half && g + 1u - g_first == g_cnt) m &= 0x0Fu;
+        return m;
+    }
 };
 
-// Looks topic k up in one group of four slots `q` (group index g).  Returns true when the search
-// is over (found, or an empty slot proves absence) and sets `entry` (0 when absent).
-__device__ __forceinline__ bool dk_match_group(const DkProbe& pr, uint32_t g, const uint4& q, uint32_t k,
-                                               int count_bits, uint32_t& entry)
+// Looks topic k up in group g, whose eight slots are (qa, qb).  Returns true when the search is
+// over (found, or an empty slot proves absence) and sets `entry` (0 when absent).
+__device__ __forceinline__ bool dk_match_group(const DkProbe& pr, uint32_t g, const uint4& qa, const uint4& qb,
+                                               uint32_t k, int count_bits, uint32_t& entry)
 {
-    const uint32_t qv[4] = {q.x, q.y, q.z, q.w};
+    const uint32_t qv[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+    const uint32_t lanes = pr.lanes(g);
     bool done = false;
     entry = 0;
 #pragma unroll
-    for (uint32_t l = 0; l < 4; ++l) {
+    for (uint32_t l = 0; l < 8; ++l) {
         const uint32_t e = qv[l];
-        if (!done && pr.inside(4u * g + l)) {
+        if (!done && ((lanes >> l) & 1u)) {
             if (e == DK_EMPTY_SLOT) done = true;
             else if ((e >> count_bits) == k) { entry = e; done = true; }
         }

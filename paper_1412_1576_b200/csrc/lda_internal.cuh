@@ -22,6 +22,7 @@ enum : int {
 
 constexpr uint32_t DK_EMPTY = 0xFFFFFFFFu;  // == DK_EMPTY_SLOT of the device helpers
 constexpr int SORT_TILE = 2048;      // tokens per segmented-sort tile (one CTA)
+constexpr int DOC_TILE = 1024;       // tokens per tile of whole documents in the n_kd rebuild (one CTA)
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (bins)
 constexpr int HIST_CHUNK = 16384;    // tokens per CTA in the histogram path
 constexpr int HOT_TILE = 8192;       // MH kernel: tokens of one hot word per CTA
@@ -49,8 +50,9 @@ struct View {
     const uint32_t* bm_of_tok;  // [N] block-major index of the token with document-order index i
     // per-sweep exchange buffers between the word-order and the document-order passes
     void* prop;        // [word steps][N] block-major: topics proposed by the word-proposals (topic type)
-    uint32_t* dside;   // [N][side_stride] block-major: own record, then per step (topic << count_bits) | n_kd
-    int32_t side_stride;  // words per token in dside: 1 + steps, rounded up to a multiple of 4
+    uint32_t* dside;   // [N][side_stride] block-major: own record, per step (topic << count_bits) | n_kd,
+                       // per doc step its acceptance uniform
+    int32_t side_stride;  // words per token in dside, a multiple of 4
     // assignments (topic type: u16 or i32) after the last MH step or initialisation
     void* zw;   // word-sorted order: read by the n_kw / n_k rebuild
     void* zbm;  // block-major order: read (through bm_of_tok) by the n_kd rebuild
@@ -79,8 +81,8 @@ struct View {
     uint2* dn_pk;      // [K] (split point, alias) of the dense table in one word pair
     unsigned long long* dense_mass;
     int32_t* nk;  // [K]
-    // n_kd: document d owns the open-addressing table dk_slots[2*doc_off[d] .. 2*doc_off[d+1])
-    // (capacity twice the document length, load <= 0.5); layout and probe order: DkProbe.
+    // n_kd: document d owns the open-addressing table dk_slots[4*doc_off[d] .. 4*doc_off[d+1])
+    // (four slots per token, load <= 0.25); layout and probe order: DkProbe.
     uint32_t* dk_slots;
     int* err;
 };

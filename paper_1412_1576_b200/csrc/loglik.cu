@@ -34,8 +34,8 @@ __global__ void __launch_bounds__(256) k_ll_doc(View v, double lg_alpha, double*
     const uint32_t cmask = (1u << v.count_bits) - 1u;
     double s = 0.0;
     for (int32_t d = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; d < v.D; d += warps) {
-        const int32_t d0 = v.doc_off[d], n = 2 * (v.doc_off[d + 1] - d0);
-        const uint32_t* tab = v.dk_slots + 2 * (size_t)d0;
+        const int32_t d0 = v.doc_off[d], n = DK_SLOTS_PER_TOKEN * (v.doc_off[d + 1] - d0);
+        const uint32_t* tab = v.dk_slots + DK_SLOTS_PER_TOKEN * (size_t)d0;
         for (int32_t j = lane; j < n; j += 32) {
             const uint32_t e = tab[j];
             if (e != DK_EMPTY) s += lgamma((double)(e & cmask) + v.alpha) - lg_alpha;

@@ -72,24 +72,27 @@ __device__ __forceinline__ bool mbar_wait_bounded(void* bar, uint32_t parity, in
 }
 
 // --- document side ---------------------------------------------------------------------------
-// Group g (four slots, 16 bytes, aligned) of the n_kd slot array.
-__device__ __forceinline__ uint4 load_group(const uint32_t* __restrict__ slots, uint32_t g)
-{
-    return __ldcg(reinterpret_cast<const uint4*>(slots) + g);
-}
+struct Group8 {
+    uint4 a, b;
+};
 
-__device__ __forceinline__ uint32_t quad_word(const uint4& q, uint32_t lane)
+// Group g (eight slots, one aligned 32-byte sector) of the n_kd slot array.
+__device__ __forceinline__ Group8 load_group(const uint32_t* __restrict__ slots, uint32_t g)
 {
-    return lane == 0 ? q.x : lane == 1 ? q.y : lane == 2 ? q.z : q.w;
+    const uint4* p = reinterpret_cast<const uint4*>(slots) + 2 * (size_t)g;
+    Group8 q;
+    q.a = __ldcg(p);
+    q.b = __ldcg(p + 1);
+    return q;
 }
 
 // n_kd[k] as a packed entry (0 when absent).  `q` is the first group of the probe sequence,
 // already loaded; further groups are read only when that one is full of other topics.
 __device__ __forceinline__ uint32_t lookup_dk(const uint32_t* __restrict__ slots, const DkProbe& pr, uint32_t g,
-                                              uint4 q, uint32_t k, int count_bits)
+                                              Group8 q, uint32_t k, int count_bits)
 {
     uint32_t entry;
-    for (uint32_t n = 1; !dk_match_group(pr, g, q, k, count_bits, entry) && n < pr.g_cnt; ++n) {
+    for (uint32_t n = 1; !dk_match_group(pr, g, q.a, q.b, k, count_bits, entry) && n < pr.g_cnt; ++n) {
         g = pr.next(g);
         q = load_group(slots, g);
     }
@@ -110,6 +113,7 @@ template <bool STAGED, bool PACKED>
 struct HotTile {
     struct Ref {};
     const int32_t* row;
+    const int32_t* nk_tab;    // n_k: shared memory when STAGED, else global
     const uint2* pk;          // PACKED: the word's bins
     const uint32_t* thr;      // otherwise the three separate arrays
     const uint32_t* idx;
@@ -131,6 +135,7 @@ struct HotTile {
     {
         return STAGED ? row[k] : __ldg(row + k);
     }
+    __device__ __forceinline__ int32_t nk(uint32_t k) const { return STAGED ? nk_tab[k] : __ldg(nk_tab + k); }
     __device__ __forceinline__ Draw draw_issue(const Ref&, const View& v, const uint4& r) const
     {
         Draw d;
@@ -175,6 +180,8 @@ struct ColdTile {
     const uint32_t* thr;
     const uint32_t* idx;
     int32_t nw;
+    const int32_t* nk_tab;  // n_k in global memory
+    __device__ __forceinline__ int32_t nk(uint32_t k) const { return __ldg(nk_tab + k); }
     __device__ __forceinline__ Ref ref(int32_t q) const
     {
         int32_t lo = 0, hi = nw;  // last word with woff[word] <= q
@@ -276,7 +283,7 @@ k_doc_side(View v, uint2 key, uint32_t sweep, int32_t mh_steps)
             // word-proposal of step st (drawn by pass 1): first group of its n_kd lookup
             const uint32_t t1 = (uint32_t)__ldcs(prop + (size_t)(st >> 1) * N + m);
             const uint32_t g1 = pr.first(t1);
-            const uint4 q1 = load_group(v.dk_slots, g1);
+            const Group8 q1 = load_group(v.dk_slots, g1);
             // doc-proposal of step st+1 (Eq. 9, Eq. 12): the record of a random token of the
             // document, or a uniform topic with probability K*alpha / (n_d + K*alpha) and then
             // the first group of its n_kd lookup -- one read either way
@@ -286,11 +293,14 @@ k_doc_side(View v, uint2 key, uint32_t sweep, int32_t mh_steps)
             const uint32_t t2 = scale_to_range(r.y, (uint32_t)v.K);
             const uint32_t g2 = pr.first(t2);
             const uint32_t j = dinfo.x + scale_to_range(r.y, dinfo.y);
-            const uint4 q2 = copy ? load_group(v.rec, j >> 2) : load_group(v.dk_slots, g2);
+            const uint32_t e_copy = copy ? __ldcg(v.rec + j) : 0u;
+            Group8 q2;
+            q2.a = q2.b = make_uint4(DK_EMPTY, DK_EMPTY, DK_EMPTY, DK_EMPTY);
+            if (!copy) q2 = load_group(v.dk_slots, g2);
             __syncwarp();
             const uint32_t e1 = lookup_dk(v.dk_slots, pr, g1, q1, t1, cb);
             __syncwarp();
-            uint32_t out2 = quad_word(q2, j & 3u);
+            uint32_t out2 = e_copy;
             if (!copy) {
                 const uint32_t e2 = lookup_dk(v.dk_slots, pr, g2, q2, t2, cb);
                 out2 = e2 ? e2 : t2 << cb;
@@ -298,7 +308,10 @@ k_doc_side(View v, uint2 key, uint32_t sweep, int32_t mh_steps)
             __syncwarp();
             if (valid) {
                 __stcs(out + 1 + st, e1 ? e1 : t1 << cb);
-                if (st + 1 < mh_steps) __stcs(out + 2 + st, out2);
+                if (st + 1 < mh_steps) {
+                    __stcs(out + 2 + st, out2);
+                    __stcs(out + 1 + mh_steps + (st >> 1), r.w);  // the step's acceptance uniform
+                }
             }
         }
         __syncwarp();
@@ -336,7 +349,10 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 ua[i] = 0;
                 if (m0 + i < mh_steps) {
                     e[i] = __ldcs(side + 1 + m0 + i);
-                    ua[i] = philox4x32_10(make_uint4(tok, sweep, (uint32_t)(m0 + i), 0u), key).w;
+                    // acceptance uniform: word 3 of the step's Philox block; pass 2 already drew the
+                    // doc steps' blocks and left that word beside the gathered counts
+                    ua[i] = (i & 1) ? __ldcs(side + 1 + mh_steps + ((m0 + i) >> 1))
+                                    : philox4x32_10(make_uint4(tok, sweep, (uint32_t)(m0 + i), 0u), key).w;
                 }
             }
             if (m0 == 0) {
@@ -345,7 +361,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 z0 = s = own >> cb;
                 n_sd = (int32_t)(own & cmask);
                 n_sw = tile.count(w, z0);
-                n_s = __ldg(v.nk + z0);
+                n_s = tile.nk(z0);
                 bad = bad || n_sd < 1 || n_sw < 1 || n_s < 1;
             }
             // counts at the proposed topics, all read before the first acceptance test
@@ -355,7 +371,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
             for (int i = 0; i < CH; ++i) {
                 t[i] = e[i] >> cb;
                 n_tw[i] = tile.count(w, t[i]);
-                n_t[i] = __ldg(v.nk + t[i]);
+                n_t[i] = tile.nk(t[i]);
             }
             // Eq. 8 (word steps) / Eq. 11 (doc steps), products taken left to right
 #pragma unroll
@@ -404,18 +420,22 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     const int32_t w = tiles[3 * blockIdx.x], p0 = tiles[3 * blockIdx.x + 1], cnt = tiles[3 * blockIdx.x + 2];
     const int32_t* row_g = v.dense_rows + (size_t)__ldg(v.dense_slot + w) * v.dense_stride;
     int32_t* row_s = reinterpret_cast<int32_t*>(dyn_smem);
+    int32_t* nk_s = row_s + v.dense_stride;
     if (STAGED && ACCEPT) {
         if (threadIdx.x == 0) {
+            // the word's dense n_kw row and n_k, one bulk copy each, both signalling the same barrier
             const uint32_t bytes = (uint32_t)v.dense_stride * 4u;
             mbar_init(&bar, 1);
-            mbar_expect_tx(&bar, bytes);
+            mbar_expect_tx(&bar, 2u * bytes);
             bulk_copy_g2s(row_s, row_g, bytes, &bar);
+            bulk_copy_g2s(nk_s, v.nk, bytes, &bar);
         }
         __syncthreads();
     }
     const int32_t r0 = __ldg(v.row_start + w);
     HotTile<STAGED && ACCEPT, PACKED> tile;
     tile.row = (STAGED && ACCEPT) ? row_s : row_g;
+    tile.nk_tab = (STAGED && ACCEPT) ? nk_s : v.nk;
     tile.pk = v.al_pk + r0;
     tile.thr = v.al_thr + r0;
     tile.idx = v.al_idx + r0;
@@ -463,7 +483,7 @@ k_word_cold(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep
         }
     }
     __syncthreads();
-    ColdTile tile{woff_s, rs_s, nnz_s, mix_s, topic_s, count_s, thr_s, idx_s, nw};
+    ColdTile tile{woff_s, rs_s, nnz_s, mix_s, topic_s, count_s, thr_s, idx_s, nw, v.nk};
     if (ACCEPT) accept_tokens<T, CH>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
     else propose_tokens<T>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
 }
@@ -542,7 +562,7 @@ static int sample_tc(Ctx& c, int mh_steps)
     cudaEventRecord(c.ev[9], c.stream);
     if (c.n_hot_tiles) {
         if (staged)
-            k_word_hot<T, CH, true, true><<<c.n_hot_tiles, HOT_THREADS, (size_t)v.dense_stride * 4, c.stream>>>(
+            k_word_hot<T, CH, true, true><<<c.n_hot_tiles, HOT_THREADS, (size_t)v.dense_stride * 8, c.stream>>>(
                 v, c.hot_tiles, key, c.sweep, mh_steps);
         else
             k_word_hot<T, CH, false, true><<<c.n_hot_tiles, HOT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
@@ -575,7 +595,7 @@ template <typename T, int CH>
 static void set_hot_limit()
 {
     cudaFuncSetAttribute(k_word_hot<T, CH, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         HOT_STAGE_MAX_K * 4);
+                         HOT_STAGE_MAX_K * 8);
 }
 
 void set_sample_smem_limits()
