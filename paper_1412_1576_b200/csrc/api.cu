@@ -86,7 +86,7 @@ static void free_corpus(Ctx& c)
     nv.dense_stride = (c.K + 3) & ~3;
     nv.err = err;
     c.v = nv;
-    c.loaded = c.inited = c.tables_valid = false;
+    c.loaded = c.inited = c.tables_valid = c.dk_valid = false;
     c.N = c.D = 0;
     c.side_steps = 0;
 }
@@ -139,9 +139,22 @@ static int rebuild_counts(Ctx& c, int64_t* launches)
 {
     int n = launch_count_wk(c);
     n += launch_count_k(c);
-    n += launch_count_dk(c);
     if (launches) *launches += n;
     c.tables_valid = false;
+    c.dk_valid = false;
+    return LDA_OK;
+}
+
+// The n_kd tables in device memory (the exported form; the MH step builds its own per tile).
+static int ensure_dk(Ctx& c)
+{
+    if (c.dk_valid) return LDA_OK;
+    launch_count_dk(c);
+    int bits = 0;
+    int rc = read_err(c, &bits);
+    if (rc) return rc;
+    if (bits) return fail(&c, LDA_EINTERNAL, "the n_kd rebuild raised the device error word");
+    c.dk_valid = true;
     return LDA_OK;
 }
 
@@ -565,9 +578,9 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
         cudaEventRecord(c.ev[4], c.stream);
         n += launch_count_k(c);
         cudaEventRecord(c.ev[5], c.stream);
-        n += launch_count_dk(c);
-        cudaEventRecord(c.ev[6], c.stream);
+        cudaEventRecord(c.ev[6], c.stream);  // n_kd is rebuilt inside the next MH step, per tile
         c.tables_valid = false;
+        c.dk_valid = false;
         c.sweep += 1;
         int bits = 0;
         if ((rc = read_err(c, &bits))) return rc;
@@ -599,6 +612,7 @@ int lda_loglik(lda_ctx* h, double* total, double* word_ll, double* doc_ll)
     if (!c.inited) return fail(&c, LDA_ESTATE, "lda_loglik before lda_init");
     int rc = check_device(c);
     if (rc) return rc;
+    if ((rc = ensure_dk(c))) return rc;
     double out[3];
     if (launch_loglik(c, out) < 0) return cuda_fail(&c, "log-likelihood");
     if (total) *total = out[0];
@@ -627,6 +641,7 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
         return LDA_OK;
     }
     if (which == LDA_NDK) {
+        if ((rc = ensure_dk(c))) return rc;
         // every document's table is copied out and its filled slots sorted by topic on the host
         std::vector<int32_t> start((size_t)c.D + 1);
         if (cudaMemcpy(start.data(), v.doc_off, ((size_t)c.D + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
@@ -753,6 +768,7 @@ int lda_get_stats(lda_ctx* h, lda_stats* out)
     Ctx& c = h->c;
     if (c.inited) {
         if (check_device(c)) return LDA_ECUDA;
+        if (ensure_dk(c)) return LDA_ECUDA;
         int64_t a = 0, b = 0;
         launch_count_nnz(c, &a, &b);
         c.stats.nnz_wk = a;

@@ -187,30 +187,6 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
 // written out in one coalesced pass.  Every token's record (topic, n_kd of its topic in its
 // document) is written next to it, so that the MH step gets both in one read.
 //
-// `tab` points at the copy of group `g0`; slot l of group g is tab[(g - g0) * 8 + l].
-// Returns the index into `tab` the topic lives at (or 0xFFFFFFFF if the table had no room,
-// which the load factor rules out).
-__device__ __forceinline__ uint32_t dk_insert(uint32_t* tab, uint32_t g0, const DkProbe& pr, uint32_t k,
-                                              int count_bits)
-{
-    const uint32_t fresh = k << count_bits;
-    uint32_t g = pr.first(k);
-    for (uint32_t n = 0; n < pr.g_cnt; ++n, g = pr.next(g)) {
-        const uint32_t lanes = pr.lanes(g);
-#pragma unroll
-        for (uint32_t l = 0; l < DK_GROUP; ++l) {
-            if (!((lanes >> l) & 1u)) continue;
-            const uint32_t at = (g - g0) * DK_GROUP + l;
-            const uint32_t prev = atomicCAS(&tab[at], DK_EMPTY, fresh);
-            if (prev == DK_EMPTY || (prev >> count_bits) == k) {
-                atomicAdd(&tab[at], 1u);
-                return at;
-            }
-        }
-    }
-    return 0xFFFFFFFFu;
-}
-
 template <typename T>
 __global__ void __launch_bounds__(256)
 k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_off, const T* __restrict__ zbm,

@@ -46,37 +46,15 @@ __global__ void k_block_keys(const uint32_t* __restrict__ tok_orig, int32_t n, i
     }
 }
 
-// Static token records copied into block-major order, so the document-side pass streams them.
-__global__ void k_gather_block_major(const uint32_t* __restrict__ order, const uint2* __restrict__ tok_dinfo,
-                                     const uint32_t* __restrict__ tok_orig, int32_t n,
-                                     uint2* __restrict__ dinfo_bm, uint32_t* __restrict__ tok_bm,
-                                     uint32_t* __restrict__ inv, uint32_t* __restrict__ bm_of_tok)
+// The block-major index of every token, by word-sorted position and by document-order index.
+__global__ void k_block_major_maps(const uint32_t* __restrict__ order, const uint32_t* __restrict__ tok_orig,
+                                   int32_t n, uint32_t* __restrict__ inv, uint32_t* __restrict__ bm_of_tok)
 {
     for (int64_t m = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; m < n;
          m += (int64_t)gridDim.x * blockDim.x) {
         const uint32_t p = order[m];
-        dinfo_bm[m] = tok_dinfo[p];
-        tok_bm[m] = tok_orig[p];
         inv[p] = (uint32_t)m;
         bm_of_tok[tok_orig[p]] = (uint32_t)m;
-    }
-}
-
-// Document of every token in word-sorted order (the last d with doc_off[d] <= orig), stored as
-// (first token of the document, document length) so the sampler streams it instead of gathering.
-__global__ void k_token_docs(const uint32_t* __restrict__ tok_orig, const int32_t* __restrict__ doc_off,
-                             int32_t n, int32_t D, uint2* __restrict__ tok_dinfo)
-{
-    for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < n;
-         p += (int64_t)gridDim.x * blockDim.x) {
-        const int32_t i = (int32_t)tok_orig[p];
-        int32_t lo = 0, hi = D;  // find first d in [0,D] with doc_off[d] > i
-        while (lo < hi) {
-            const int32_t mid = lo + ((hi - lo) >> 1);
-            if (doc_off[mid + 1] <= i) lo = mid + 1; else hi = mid;
-        }
-        const int32_t d0 = doc_off[lo];
-        tok_dinfo[p] = make_uint2((uint32_t)d0, (uint32_t)(doc_off[lo + 1] - d0));
     }
 }
 
@@ -87,14 +65,11 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
     const size_t n1 = (size_t)(N > 0 ? N : 1);
 
     uint32_t* tok_orig = (uint32_t*)dev_alloc(c, n1 * 4);
-    uint32_t* order = (uint32_t*)dev_alloc(c, n1 * 4);
     uint32_t* inv = (uint32_t*)dev_alloc(c, n1 * 4);
     uint32_t* bm_of_tok = (uint32_t*)dev_alloc(c, n1 * 4);
-    uint2* dinfo_bm = (uint2*)dev_alloc(c, n1 * 8);
-    uint32_t* tok_bm = (uint32_t*)dev_alloc(c, n1 * 4);
     int32_t* word_off = (int32_t*)dev_alloc(c, ((size_t)V + 1) * 4);
     int32_t* doc_off = (int32_t*)dev_alloc(c, ((size_t)D + 1) * 4);
-    if (!tok_orig || !order || !inv || !bm_of_tok || !dinfo_bm || !tok_bm || !word_off || !doc_off) return LDA_ENOMEM;
+    if (!tok_orig || !inv || !bm_of_tok || !word_off || !doc_off) return LDA_ENOMEM;
 
     std::vector<int32_t> doc32((size_t)D + 1);
     for (int64_t d = 0; d <= D; ++d) doc32[(size_t)d] = (int32_t)doc_off_host[d];
@@ -106,14 +81,14 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
     int32_t* keys_out = nullptr;
     uint32_t* iota = nullptr;
     uint32_t* keys_blk = nullptr;
-    uint2* tok_dinfo = nullptr;
+    uint32_t* order = nullptr;
     void* temp = nullptr;
     void* temp2 = nullptr;
     size_t temp_bytes = 0, temp2_bytes = 0;
     int rc = LDA_OK;
     do {
         if (cudaMalloc(&keys_out, n1 * 4) != cudaSuccess || cudaMalloc(&iota, n1 * 4) != cudaSuccess ||
-            cudaMalloc(&keys_blk, n1 * 4) != cudaSuccess || cudaMalloc(&tok_dinfo, n1 * 8) != cudaSuccess) {
+            cudaMalloc(&keys_blk, n1 * 4) != cudaSuccess || cudaMalloc(&order, n1 * 4) != cudaSuccess) {
             rc = LDA_ENOMEM;
             break;
         }
@@ -135,7 +110,6 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
                 rc = LDA_ECUDA;
                 break;
             }
-            k_token_docs<<<1184, 256, 0, st>>>(tok_orig, doc_off, N, D, tok_dinfo);
             // block-major order: tokens sorted by (block of their document-order index, word-sorted
             // position); a stable sort of the positions by block
             uint32_t* keys_tmp = reinterpret_cast<uint32_t*>(keys_out);  // the word keys are no longer needed
@@ -158,7 +132,7 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
                 rc = LDA_ECUDA;
                 break;
             }
-            k_gather_block_major<<<1184, 256, 0, st>>>(order, tok_dinfo, tok_orig, N, dinfo_bm, tok_bm, inv, bm_of_tok);
+            k_block_major_maps<<<1184, 256, 0, st>>>(order, tok_orig, N, inv, bm_of_tok);
         } else {
             k_word_offsets<<<(V + 1 + 255) / 256, 256, 0, st>>>(keys_out, N, V, word_off);
         }
@@ -168,15 +142,12 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
     cudaFree(keys_out);
     cudaFree(iota);
     cudaFree(keys_blk);
-    cudaFree(tok_dinfo);
+    cudaFree(order);
     cudaFree(temp);
     cudaFree(temp2);
     if (rc != LDA_OK) return rc;
-    c.v.order = order;
     c.v.inv = inv;
     c.v.bm_of_tok = bm_of_tok;
-    c.v.dinfo_bm = dinfo_bm;
-    c.v.tok_bm = tok_bm;
     c.v.tok_orig = tok_orig;
     c.v.word_off = word_off;
     c.v.doc_off = doc_off;

@@ -81,6 +81,43 @@ __device__ __forceinline__ bool dk_match_group(const DkProbe& pr, uint32_t g, co
     return done;
 }
 
+// `tab` points at the copy of group `g0`; slot l of group g is tab[(g - g0) * 8 + l].
+// Returns the index into `tab` the topic lives at (or 0xFFFFFFFF if the table had no room,
+// which the load factor rules out).
+__device__ __forceinline__ uint32_t dk_insert(uint32_t* tab, uint32_t g0, const DkProbe& pr, uint32_t k,
+                                              int count_bits)
+{
+    const uint32_t fresh = k << count_bits;
+    uint32_t g = pr.first(k);
+    for (uint32_t n = 0; n < pr.g_cnt; ++n, g = pr.next(g)) {
+        const uint32_t lanes = pr.lanes(g);
+#pragma unroll
+        for (uint32_t l = 0; l < DK_GROUP; ++l) {
+            if (!((lanes >> l) & 1u)) continue;
+            const uint32_t at = (g - g0) * DK_GROUP + l;
+            const uint32_t prev = atomicCAS(&tab[at], DK_EMPTY_SLOT, fresh);
+            if (prev == DK_EMPTY_SLOT || (prev >> count_bits) == k) {
+                atomicAdd(&tab[at], 1u);
+                return at;
+            }
+        }
+    }
+    return 0xFFFFFFFFu;
+}
+
+// n_kd[k] as a packed entry (0 when absent) from a table held as in dk_insert(); `tab` is 16-byte
+// aligned.
+__device__ __forceinline__ uint32_t dk_lookup(const uint32_t* tab, uint32_t g0, const DkProbe& pr, uint32_t k,
+                                              int count_bits)
+{
+    uint32_t g = pr.first(k), entry = 0;
+    for (uint32_t n = 0; n < pr.g_cnt; ++n, g = pr.next(g)) {
+        const uint4* q = reinterpret_cast<const uint4*>(tab + (size_t)(g - g0) * DK_GROUP);
+        if (dk_match_group(pr, g, q[0], q[1], k, count_bits, entry)) break;
+    }
+    return entry;
+}
+
 template <typename T>
 __device__ __forceinline__ T warp_reduce_sum(T v)
 {

@@ -39,14 +39,10 @@ struct View {
     int count_bits;  // low bits of a packed n_kd entry that hold the count
     // tokens in word-sorted order (position p)
     const uint32_t* tok_orig;  // index of the token in the caller's document order
-    // the same tokens in block-major order (index m): sorted by (block of the document-order
-    // index, word-sorted position), so that a pass in this order touches one block of the
-    // document-side tables at a time -- small enough to stay in L2 -- while still walking runs of
-    // consecutive word-sorted positions
-    const uint32_t* order;    // [N] word-sorted position of the m-th token
-    const uint32_t* inv;      // [N] block-major index of the token at word-sorted position p
-    const uint2* dinfo_bm;    // [N] (first token of its document, document length)
-    const uint32_t* tok_bm;   // [N] document-order index
+    // block-major order (index m): the tokens sorted by (block of the document-order index,
+    // word-sorted position).  Buffers in this order are reached from word order in runs of
+    // consecutive positions and from document order within one L2-sized block at a time.
+    const uint32_t* inv;        // [N] block-major index of the token at word-sorted position p
     const uint32_t* bm_of_tok;  // [N] block-major index of the token with document-order index i
     // per-sweep exchange buffers between the word-order and the document-order passes
     void* prop;        // [word steps][N] block-major: topics proposed by the word-proposals (topic type)
@@ -55,10 +51,9 @@ struct View {
     int32_t side_stride;  // words per token in dside, a multiple of 4
     // assignments (topic type: u16 or i32) after the last MH step or initialisation
     void* zw;   // word-sorted order: read by the n_kw / n_k rebuild
-    void* zbm;  // block-major order: read (through bm_of_tok) by the n_kd rebuild
-    // Sweep-start state in document order: rec[i] = (z_i << count_bits) | n_kd[d][z_i], a token's
-    // topic together with that topic's count in its document, so the doc-proposal (Eq. 12) gets
-    // the proposed topic and its n_kd in one read.  Written by the n_kd rebuild.
+    void* zbm;  // block-major order: read (through bm_of_tok) by everything that works per document
+    // Document order, valid after launch_count_dk() only (the exported form of n_kd):
+    // rec[i] = (z_i << count_bits) | n_kd[d][z_i].
     uint32_t* rec;
     const int32_t* word_off;  // [V+1] token range of each word in word-sorted order
     const int32_t* doc_off;   // [D+1]
@@ -98,6 +93,7 @@ struct Ctx {
     double dense_frac = 0.05;
     double dense_min_tf = 64;
     bool loaded = false, inited = false, tables_valid = false;
+    bool dk_valid = false;  // dk_slots / rec hold the n_kd tables of the current assignments
     uint64_t seed = 0;
     uint32_t sweep = 0;
     int64_t N = 0, D = 0;
@@ -139,6 +135,7 @@ int launch_count_dk(Ctx& c);
 int launch_alias_dense(Ctx& c);
 int launch_alias_sparse(Ctx& c);
 int launch_sample(Ctx& c, int mh_steps);   // all passes of the MH step; needs ensure_exchange()
+int launch_doc_side(Ctx& c, int mh_steps);  // pass 2 of the MH step
 int ensure_exchange(Ctx& c, int mh_steps);  // (re)allocates View::prop / View::dside; LDA_* status
 int launch_loglik(Ctx& c, double* out3_host);
 int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host);

@@ -6,16 +6,17 @@
 // on scheduling.  Because the counts are frozen, a proposal never depends on the chain's current
 // state.  The step is therefore split into passes that each stay on one side of the model:
 //   1. word order : draw the word-proposals (alias bins of the word staged per tile);
-//   2. block-major: gather the document side -- own record, doc-proposals, n_kd at every
-//                   proposed topic -- one L2-sized block of documents at a time;
+//   2. doc order  : the document side -- own record, doc-proposals, n_kd at every proposed topic --
+//                   from per-document tables built in shared memory (docside.cu);
 //   3. word order : accept/reject chain in registers, n_kw rows staged in shared memory (hot
 //                   words: the dense row, by one bulk asynchronous copy; tail words: the sorted rows
 //                   of a tile of whole words);
 // Pass 3 leaves the new assignments in word order (for the n_kw / n_k rebuild) and in block-major
-// order, from where the n_kd rebuild picks them up block by block.
-// A random access to HBM costs far more than the bytes it returns: pass 2 turns the document-side
-// gathers into L2 hits, passes 1 and 3 stream, and whatever crosses between the two orders moves
-// in runs of consecutive positions.
+// order, where the next document-side pass picks them up.
+// A random access to HBM costs far more than the bytes it returns.  The passes exchange their
+// results through buffers in block-major order (tokens sorted by block of documents, then by
+// word-order position): the word-order passes reach them in runs of consecutive positions, the
+// document-order pass within one L2-sized block at a time.
 #include "lda_device.cuh"
 #include "lda_internal.cuh"
 
@@ -27,10 +28,6 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 #endif
 constexpr int HOT_THREADS = LDA_HOT_THREADS;
 constexpr int COLD_THREADS = 256;
-#ifndef LDA_DOC_SIDE_TILE
-#define LDA_DOC_SIDE_TILE 2048
-#endif
-constexpr int DOC_SIDE_TILE = LDA_DOC_SIDE_TILE;  // tokens per CTA of the document-side pass
 constexpr int STAGE_WAIT_LIMIT = 1 << 20;
 
 // --- shared-memory barrier and bulk-copy primitives ------------------------------------------
@@ -69,34 +66,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(void* bar, uint32_t parity, in
             : "r"(smem_addr(bar)), "r"(parity)
             : "memory");
     return done != 0;
-}
-
-// --- document side ---------------------------------------------------------------------------
-struct Group8 {
-    uint4 a, b;
-};
-
-// Group g (eight slots, one aligned 32-byte sector) of the n_kd slot array.
-__device__ __forceinline__ Group8 load_group(const uint32_t* __restrict__ slots, uint32_t g)
-{
-    const uint4* p = reinterpret_cast<const uint4*>(slots) + 2 * (size_t)g;
-    Group8 q;
-    q.a = __ldcg(p);
-    q.b = __ldcg(p + 1);
-    return q;
-}
-
-// n_kd[k] as a packed entry (0 when absent).  `q` is the first group of the probe sequence,
-// already loaded; further groups are read only when that one is full of other topics.
-__device__ __forceinline__ uint32_t lookup_dk(const uint32_t* __restrict__ slots, const DkProbe& pr, uint32_t g,
-                                              Group8 q, uint32_t k, int count_bits)
-{
-    uint32_t entry;
-    for (uint32_t n = 1; !dk_match_group(pr, g, q.a, q.b, k, count_bits, entry) && n < pr.g_cnt; ++n) {
-        g = pr.next(g);
-        q = load_group(slots, g);
-    }
-    return entry;
 }
 
 // --- word side -------------------------------------------------------------------------------
@@ -247,74 +216,6 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
             tile.draw_finish(w, d, t, n_tw);
             __stcs(prop + (size_t)(m >> 1) * v.N + at, (T)t);
         }
-    }
-}
-
-// --- pass 2: document side (block-major order) -----------------------------------------------------
-// For every token: its own record, the doc-proposals (odd steps, Eq. 9 / Eq. 12) and n_kd at every
-// proposed topic.  The tokens come in block-major order, so the records and tables read here
-// belong to one block of documents at a time and are served from L2; the results go to the
-// token's word-sorted position.
-template <typename T>
-__global__ void __launch_bounds__(256)
-k_doc_side(View v, uint2 key, uint32_t sweep, int32_t mh_steps)
-{
-    const int cb = v.count_bits;
-    const T* prop = reinterpret_cast<const T*>(v.prop);
-    const double Ka = v.Kalpha;
-    const size_t N = (size_t)v.N;
-    const int lane = threadIdx.x & 31;
-    // A CTA takes DOC_SIDE_TILE consecutive tokens; CTAs start in index order, so the ones running at
-    // any moment work on neighbouring tokens, i.e. on the same block of documents.
-    // All lanes of a warp run the same number of iterations and meet again after every phase;
-    // lanes past the end repeat the last token and store nothing.
-    const int64_t tile_end = min((int64_t)v.N, (blockIdx.x + 1) * (int64_t)DOC_SIDE_TILE);
-    for (int64_t m0 = blockIdx.x * (int64_t)DOC_SIDE_TILE + threadIdx.x - lane; m0 < tile_end; m0 += blockDim.x) {
-        const bool valid = m0 + lane < tile_end;
-        const int64_t m = valid ? m0 + lane : v.N - 1;
-        const uint2 dinfo = __ldcs(v.dinfo_bm + m);
-        const uint32_t tok = __ldcs(v.tok_bm + m);
-        const uint32_t own = __ldcg(v.rec + tok);
-        const DkProbe pr(dinfo.x, dinfo.y);
-        const double n_d = (double)dinfo.y;
-        uint32_t* out = v.dside + (size_t)m * v.side_stride;
-        if (valid) __stcs(out, own);
-        for (int32_t st = 0; st < mh_steps; st += 2) {
-            // word-proposal of step st (drawn by pass 1): first group of its n_kd lookup
-            const uint32_t t1 = (uint32_t)__ldcs(prop + (size_t)(st >> 1) * N + m);
-            const uint32_t g1 = pr.first(t1);
-            const Group8 q1 = load_group(v.dk_slots, g1);
-            // doc-proposal of step st+1 (Eq. 9, Eq. 12): the record of a random token of the
-            // document, or a uniform topic with probability K*alpha / (n_d + K*alpha) and then
-            // the first group of its n_kd lookup -- one read either way
-            const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)(st + 1), 0u), key);
-            const double uu = __dmul_rn((double)r.x, INV_2_32);
-            const bool copy = __dmul_rn(uu, __dadd_rn(n_d, Ka)) < n_d;
-            const uint32_t t2 = scale_to_range(r.y, (uint32_t)v.K);
-            const uint32_t g2 = pr.first(t2);
-            const uint32_t j = dinfo.x + scale_to_range(r.y, dinfo.y);
-            const uint32_t e_copy = copy ? __ldcg(v.rec + j) : 0u;
-            Group8 q2;
-            q2.a = q2.b = make_uint4(DK_EMPTY, DK_EMPTY, DK_EMPTY, DK_EMPTY);
-            if (!copy) q2 = load_group(v.dk_slots, g2);
-            __syncwarp();
-            const uint32_t e1 = lookup_dk(v.dk_slots, pr, g1, q1, t1, cb);
-            __syncwarp();
-            uint32_t out2 = e_copy;
-            if (!copy) {
-                const uint32_t e2 = lookup_dk(v.dk_slots, pr, g2, q2, t2, cb);
-                out2 = e2 ? e2 : t2 << cb;
-            }
-            __syncwarp();
-            if (valid) {
-                __stcs(out + 1 + st, e1 ? e1 : t1 << cb);
-                if (st + 1 < mh_steps) {
-                    __stcs(out + 2 + st, out2);
-                    __stcs(out + 1 + mh_steps + (st >> 1), r.w);  // the step's acceptance uniform
-                }
-            }
-        }
-        __syncwarp();
     }
 }
 
@@ -521,11 +422,13 @@ __global__ void k_spread(View v, const int32_t* __restrict__ z_in)
     }
 }
 
+template <typename T>
 __global__ void k_export(View v, int32_t* __restrict__ out)
 {
+    const T* zbm = reinterpret_cast<const T*>(v.zbm);
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < v.N;
          i += (int64_t)gridDim.x * blockDim.x)
-        out[i] = (int32_t)(v.rec[i] >> v.count_bits);
+        out[i] = (int32_t)zbm[v.bm_of_tok[i]];
 }
 
 static int grid_for(int64_t n, int block)
@@ -541,7 +444,6 @@ static int sample_tc(Ctx& c, int mh_steps)
     const View& v = c.v;
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     const bool staged = c.K <= HOT_STAGE_MAX_K;
-    const int side_grid = (int)((c.N + DOC_SIDE_TILE - 1) / DOC_SIDE_TILE);
     int launches = 0;
     // pass 1: word-proposals
     if (c.n_hot_tiles) {
@@ -556,8 +458,7 @@ static int sample_tc(Ctx& c, int mh_steps)
     }
     // pass 2: document side
     cudaEventRecord(c.ev[8], c.stream);
-    k_doc_side<T><<<side_grid, 256, 0, c.stream>>>(v, key, c.sweep, mh_steps);
-    ++launches;
+    launches += launch_doc_side(c, mh_steps);
     // pass 3: accept / reject
     cudaEventRecord(c.ev[9], c.stream);
     if (c.n_hot_tiles) {
@@ -628,7 +529,8 @@ int launch_spread_assignments(Ctx& c, const int32_t* z_dev)
 int launch_export_assignments(Ctx& c, int32_t* z_dev)
 {
     if (c.N == 0) return 0;
-    k_export<<<grid_for(c.N, 256), 256, 0, c.stream>>>(c.v, z_dev);
+    if (c.wide_topics) k_export<int32_t><<<grid_for(c.N, 256), 256, 0, c.stream>>>(c.v, z_dev);
+    else k_export<uint16_t><<<grid_for(c.N, 256), 256, 0, c.stream>>>(c.v, z_dev);
     return 1;
 }
 
