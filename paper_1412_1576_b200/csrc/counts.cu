@@ -181,7 +181,7 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
     if (threadIdx.x == 0) wk_nnz[w] = done;
 }
 
-// n_kd as per-document open-addressing tables (layout and probe order: DkProbe).  One CTA per
+// n_kd as per-document open-addressing tables (layout and probe order: dk_insert in lda_device.cuh).  One CTA per
 // tile of whole documents holding <= SORT_TILE tokens: the tile's tables are built in shared
 // memory by insertion (claim a slot with compare-and-swap, then add one to its count bits) and
 // written out in one coalesced pass.  Every token's record (topic, n_kd of its topic in its
@@ -192,7 +192,7 @@ __global__ void __launch_bounds__(256)
 k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_off, const T* __restrict__ zbm,
            const uint32_t* __restrict__ bm_of_tok, uint32_t* __restrict__ rec, uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
 {
-    __shared__ uint32_t slots[DK_SLOTS_PER_TOKEN * DOC_TILE + DK_GROUP];
+    __shared__ uint32_t slots[DK_SLOTS_PER_TOKEN * DOC_TILE];
     __shared__ int32_t soff[DOC_TILE + 1];
     __shared__ uint32_t topic[DOC_TILE];
     const int tid = threadIdx.x;
@@ -201,29 +201,29 @@ k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_of
     const int32_t base = doc_off[s0];
     const int32_t cnt = doc_off[s1] - base;
     if (cnt == 0) return;
-    const uint32_t g0 = (uint32_t)base >> 1;                    // group kept in slots[0..8)
-    const uint32_t lead = ((uint32_t)base & 1u) ? 4u : 0u;      // the tile's first slot inside that group
     // the tile's documents lie in one or two blocks of the block-major order: these reads hit L2
     for (int j = tid; j < cnt; j += blockDim.x) topic[j] = (uint32_t)__ldcg(zbm + __ldcs(bm_of_tok + base + j));
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = doc_off[s0 + j] - base;
-    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt + DK_GROUP; j += blockDim.x) slots[j] = DK_EMPTY;
+    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
     __syncthreads();
     // one warp per document: its lanes insert the document's tokens and note where each topic landed
     const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     for (int d = warp; d < nseg; d += nwarps) {
         const int32_t first = soff[d], len = soff[d + 1] - first;
-        const DkProbe pr((uint32_t)(base + first), (uint32_t)len);
+        if (len == 0) continue;
         for (int j = first + lane; j < first + len; j += 32) {
             const uint32_t k = topic[j];
             uint32_t slot = 0xFFFFFFFFu;
-            if (k < (uint32_t)K) slot = dk_insert(slots, g0, pr, k, count_bits);
+            if (k < (uint32_t)K)
+                slot = dk_insert(slots + DK_SLOTS_PER_TOKEN * first, DK_SLOTS_PER_TOKEN * (uint32_t)len, k, count_bits);
             if (slot == 0xFFFFFFFFu) atomicOr(err, k < (uint32_t)K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
+            else slot += DK_SLOTS_PER_TOKEN * (uint32_t)first;
             topic[j] = slot;
         }
     }
     __syncthreads();
     uint32_t* out = slots_out + DK_SLOTS_PER_TOKEN * (size_t)base;
-    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) out[j] = slots[lead + j];
+    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) out[j] = slots[j];
     for (int j = tid; j < cnt; j += blockDim.x) {
         const uint32_t slot = topic[j];
         if (slot != 0xFFFFFFFFu) rec[base + j] = slots[slot];
@@ -239,15 +239,14 @@ k_long_doc_hash(const int32_t* __restrict__ long_docs, const int32_t* __restrict
 {
     const int32_t d = long_docs[blockIdx.x];
     const int32_t first = doc_off[d], cnt = doc_off[d + 1] - first;
-    const DkProbe pr((uint32_t)first, (uint32_t)cnt);
-    uint32_t* tab = slots_out + (size_t)pr.g_first * DK_GROUP;  // the table's first group
-    uint32_t* mine = slots_out + DK_SLOTS_PER_TOKEN * (size_t)first;
-    for (uint32_t j = threadIdx.x; j < (uint32_t)DK_SLOTS_PER_TOKEN * (uint32_t)cnt; j += blockDim.x) mine[j] = DK_EMPTY;
+    const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)cnt;
+    uint32_t* tab = slots_out + DK_SLOTS_PER_TOKEN * (size_t)first;
+    for (uint32_t j = threadIdx.x; j < cap; j += blockDim.x) tab[j] = DK_EMPTY;
     __syncthreads();
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
         const uint32_t k = (uint32_t)zbm[bm_of_tok[first + j]];
         uint32_t at = 0xFFFFFFFFu;
-        if (k < (uint32_t)K) at = dk_insert(tab, pr.g_first, pr, k, count_bits);
+        if (k < (uint32_t)K) at = dk_insert(tab, cap, k, count_bits);
         if (at == 0xFFFFFFFFu) atomicOr(err, k < (uint32_t)K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
         rec[first + j] = at;  // parked here until every insertion is done
     }

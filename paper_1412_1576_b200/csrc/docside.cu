@@ -22,14 +22,14 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 
 // Everything pass 3 needs from the document side for one token, written at the token's
 // block-major index `bm`.
-//   tab, g0 : the document's table (see dk_insert)
-//   slot_at : table index of the slot holding the topic of the document's j-th token
+//   tab     : the document's table, 4 * doc_len slots
+//   slot_at : slot holding the topic of the document's j-th token
 template <typename T, class SlotAt>
-__device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* tab, uint32_t g0, const DkProbe& pr,
-                                               uint32_t tok, uint32_t doc_len, uint32_t own, uint32_t t_first,
-                                               uint32_t bm, const SlotAt& slot_at, uint2 key, uint32_t sweep,
-                                               int32_t mh_steps)
+__device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* tab, uint32_t tok, uint32_t doc_len,
+                                               uint32_t own, uint32_t t_first, uint32_t bm, const SlotAt& slot_at,
+                                               uint2 key, uint32_t sweep, int32_t mh_steps)
 {
+    const uint32_t cap = DK_SLOTS_PER_TOKEN * doc_len;
     const int cb = v.count_bits;
     const T* prop = reinterpret_cast<const T*>(v.prop);
     const size_t N = (size_t)v.N;
@@ -46,7 +46,7 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
     for (int32_t st = 0; st < mh_steps; st += 2) {
         // word-proposal of step st: n_kd at the topic pass 1 drew
         const uint32_t t1 = st == 0 ? t_first : (uint32_t)__ldcg(prop + (size_t)(st >> 1) * N + bm);
-        const uint32_t e1 = dk_lookup(tab, g0, pr, t1, cb);
+        const uint32_t e1 = dk_lookup(tab, cap, t1, cb);
         put(1 + st, e1 ? e1 : t1 << cb);
         if (st + 1 < mh_steps) {
             // doc-proposal of step st+1
@@ -57,7 +57,7 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
                 o2 = tab[slot_at(scale_to_range(r.y, doc_len))];
             } else {
                 const uint32_t t2 = scale_to_range(r.y, (uint32_t)v.K);
-                const uint32_t e2 = dk_lookup(tab, g0, pr, t2, cb);
+                const uint32_t e2 = dk_lookup(tab, cap, t2, cb);
                 o2 = e2 ? e2 : t2 << cb;
             }
             put(2 + st, o2);
@@ -71,7 +71,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
 {
-    __shared__ __align__(16) uint32_t slots[DK_SLOTS_PER_TOKEN * DOC_TILE + DK_GROUP];
+    __shared__ uint32_t slots[DK_SLOTS_PER_TOKEN * DOC_TILE];
     __shared__ int32_t soff[DOC_TILE + 1];
     __shared__ uint32_t topic[DOC_TILE];   // a token's topic, later the table index of its slot
     __shared__ uint32_t bm_s[DOC_TILE];    // a token's block-major index
@@ -84,7 +84,6 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     if (cnt == 0) return;
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
     const T* prop = reinterpret_cast<const T*>(v.prop);
-    const uint32_t g0 = (uint32_t)base >> 1;  // group kept in slots[0..8)
     for (int j = tid; j < cnt; j += blockDim.x) {
         const uint32_t bm = __ldcs(v.bm_of_tok + base + j);
         bm_s[j] = bm;
@@ -92,17 +91,18 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
         t1_s[j] = (uint32_t)__ldcg(prop + bm);
     }
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = v.doc_off[s0 + j] - base;
-    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt + DK_GROUP; j += blockDim.x) slots[j] = DK_EMPTY;
+    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
     __syncthreads();
     const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     for (int d = warp; d < nseg; d += nwarps) {
         const int32_t first = soff[d], len = soff[d + 1] - first;
         if (len == 0) continue;
-        const DkProbe pr((uint32_t)(base + first), (uint32_t)len);
+        uint32_t* tab = slots + DK_SLOTS_PER_TOKEN * first;
+        const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)len;
         for (int j = first + lane; j < first + len; j += 32) {
             const uint32_t k = topic[j];
             uint32_t at = 0xFFFFFFFFu;
-            if (k < (uint32_t)v.K) at = dk_insert(slots, g0, pr, k, v.count_bits);
+            if (k < (uint32_t)v.K) at = dk_insert(tab, cap, k, v.count_bits);
             if (at == 0xFFFFFFFFu) {
                 atomicOr(v.err, k < (uint32_t)v.K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
                 at = 0;
@@ -113,8 +113,8 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
         const uint32_t* slot_of = topic + first;
         auto slot_at = [slot_of](uint32_t j) { return slot_of[j]; };
         for (int j = first + lane; j < first + len; j += 32)
-            doc_side_token<T>(v, slots, g0, pr, (uint32_t)(base + j), (uint32_t)len, slots[topic[j]], t1_s[j], bm_s[j],
-                              slot_at, key, sweep, mh_steps);
+            doc_side_token<T>(v, tab, (uint32_t)(base + j), (uint32_t)len, tab[topic[j]], t1_s[j], bm_s[j], slot_at,
+                              key, sweep, mh_steps);
     }
 }
 
@@ -127,18 +127,17 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
 {
     const int32_t d = long_docs[blockIdx.x];
     const int32_t first = v.doc_off[d], cnt = v.doc_off[d + 1] - first;
-    const DkProbe pr((uint32_t)first, (uint32_t)cnt);
+    const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)cnt;
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
     const T* prop = reinterpret_cast<const T*>(v.prop);
-    uint32_t* tab = v.dk_slots + (size_t)pr.g_first * DK_GROUP;  // the table's first group
-    uint32_t* mine = v.dk_slots + DK_SLOTS_PER_TOKEN * (size_t)first;
+    uint32_t* tab = v.dk_slots + DK_SLOTS_PER_TOKEN * (size_t)first;
     uint32_t* slot_of = v.rec + first;
-    for (uint32_t j = threadIdx.x; j < (uint32_t)DK_SLOTS_PER_TOKEN * (uint32_t)cnt; j += blockDim.x) mine[j] = DK_EMPTY;
+    for (uint32_t j = threadIdx.x; j < cap; j += blockDim.x) tab[j] = DK_EMPTY;
     __syncthreads();
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
         const uint32_t k = (uint32_t)zbm[v.bm_of_tok[first + j]];
         uint32_t at = 0xFFFFFFFFu;
-        if (k < (uint32_t)v.K) at = dk_insert(tab, pr.g_first, pr, k, v.count_bits);
+        if (k < (uint32_t)v.K) at = dk_insert(tab, cap, k, v.count_bits);
         if (at == 0xFFFFFFFFu) {
             atomicOr(v.err, k < (uint32_t)v.K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
             at = 0;
@@ -149,8 +148,8 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
     auto slot_at = [slot_of](uint32_t j) { return slot_of[j]; };
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
         const uint32_t bm = v.bm_of_tok[first + j];
-        doc_side_token<T>(v, tab, pr.g_first, pr, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]],
-                          (uint32_t)prop[bm], bm, slot_at, key, sweep, mh_steps);
+        doc_side_token<T>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)prop[bm], bm,
+                          slot_at, key, sweep, mh_steps);
     }
 }
 

@@ -77,7 +77,7 @@ struct View {
     unsigned long long* dense_mass;
     int32_t* nk;  // [K]
     // n_kd: document d owns the open-addressing table dk_slots[4*doc_off[d] .. 4*doc_off[d+1])
-    // (four slots per token, load <= 0.25); layout and probe order: DkProbe.
+    // (four slots per token, load <= 0.25); layout and probe order: dk_insert in lda_device.cuh.
     uint32_t* dk_slots;
     int* err;
 };
