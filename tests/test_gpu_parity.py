@@ -164,6 +164,31 @@ def test_wide_topics_and_long_documents():
     _assert_same_counts(g, o)
 
 
+def test_hot_words_with_unstaged_rows_and_odd_step_counts():
+    """K above the shared-memory staging limit with words hot enough to get their own tiles, and
+    step counts that end on a word-proposal or exceed one group of four."""
+    c = synth.generate(V=40, K=20_000, D=300, length=("fixed", 400), zipf_s=1.0, alpha=0.05, beta=0.01, seed=8)
+    g, o = _pair(c, seed=5)
+    for mh_steps in (2, 5, 3):
+        g.sweep(1, mh_steps)
+        o.sweep(1, mh_steps)
+        assert np.array_equal(g.get_assignments(), o.get_assignments()), mh_steps
+    _assert_same_counts(g, o)
+
+
+@pytest.mark.parametrize("block_log2", [10, 14])
+def test_block_size_is_invisible(small_corpus, block_log2):
+    """The block-major exchange order is a layout choice: any block size gives the same sweep."""
+    c = small_corpus
+    g, o = _pair(c, seed=3, options={"block_log2": block_log2})
+    g.sweep(2, 4)
+    o.sweep(2, 4)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_counts(g, o)
+    for a, b in zip(g.loglik(), o.loglik()):
+        assert a == pytest.approx(b, rel=1e-10)
+
+
 def test_edge_cases():
     # empty documents, a single token, one topic, absent words
     w = np.array([3, 3, 0, 7, 7, 7], np.int32)
