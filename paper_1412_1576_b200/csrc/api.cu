@@ -9,6 +9,7 @@
 namespace lda {
 void set_hist_smem_limits();
 void set_sample_smem_limits();
+void set_doc_smem_limits();
 
 void* dev_alloc(Ctx& c, size_t bytes)
 {
@@ -276,8 +277,22 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         }
         close(V);
     }
+    // document tiles: the smallest tile shape that leaves at most 5 % of the tokens in documents
+    // too long for a tile (those get a CTA of their own and a table in device memory)
     std::vector<int32_t> doc_tiles, long_docs;
     {
+        int shape = DOC_TILE_SHAPES - 1;
+        for (int sft = 0; sft < DOC_TILE_SHAPES; ++sft) {
+            int64_t over = 0;
+            for (int32_t d = 0; d < D; ++d) {
+                const int64_t len = doc_off[d + 1] - doc_off[d];
+                if (len > DOC_TILE_TOKENS[sft]) over += len;
+            }
+            if (over * 20 <= (int64_t)N) { shape = sft; break; }
+        }
+        c.doc_tile = DOC_TILE_TOKENS[shape];
+        c.doc_threads = DOC_TILE_THREADS[shape];
+        const int32_t tile = c.doc_tile;
         int32_t s0 = 0;
         int64_t tok = 0;
         auto close = [&](int32_t s1) {
@@ -285,8 +300,8 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         };
         for (int32_t d = 0; d < D; ++d) {
             const int64_t len = doc_off[d + 1] - doc_off[d];
-            if (len > DOC_TILE) { close(d); s0 = d + 1; tok = 0; long_docs.push_back(d); continue; }
-            if (tok + len > DOC_TILE || d - s0 >= DOC_TILE) { close(d); s0 = d; tok = 0; }
+            if (len > tile) { close(d); s0 = d + 1; tok = 0; long_docs.push_back(d); continue; }
+            if (tok + len > tile || d - s0 >= tile) { close(d); s0 = d; tok = 0; }
             tok += len;
         }
         close(D);
@@ -408,6 +423,7 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
     c.have_events = true;
     set_hist_smem_limits();
     set_sample_smem_limits();
+    set_doc_smem_limits();
     *out = h;
     return LDA_OK;
 }

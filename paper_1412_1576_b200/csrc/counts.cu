@@ -188,13 +188,15 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
 // document) is written next to it, so that the MH step gets both in one read.
 //
 template <typename T>
-__global__ void __launch_bounds__(256)
-k_doc_hash(const int32_t* __restrict__ tiles, const int32_t* __restrict__ doc_off, const T* __restrict__ zbm,
-           const uint32_t* __restrict__ bm_of_tok, uint32_t* __restrict__ rec, uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
+__global__ void __launch_bounds__(1024)
+k_doc_hash(const int32_t* __restrict__ tiles, int32_t cap, const int32_t* __restrict__ doc_off,
+           const T* __restrict__ zbm, const uint32_t* __restrict__ bm_of_tok, uint32_t* __restrict__ rec,
+           uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
 {
-    __shared__ uint32_t slots[DK_SLOTS_PER_TOKEN * DOC_TILE];
-    __shared__ int32_t soff[DOC_TILE + 1];
-    __shared__ uint32_t topic[DOC_TILE];
+    extern __shared__ __align__(16) uint32_t doc_smem[];  // carved up for tiles of `cap` tokens
+    uint32_t* slots = doc_smem;
+    int32_t* soff = reinterpret_cast<int32_t*>(slots + DK_SLOTS_PER_TOKEN * cap);
+    uint32_t* topic = reinterpret_cast<uint32_t*>(soff + cap + 1);
     const int tid = threadIdx.x;
     const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
     const int32_t nseg = s1 - s0;
@@ -356,8 +358,8 @@ static int count_dk_t(Ctx& c)
     int launches = 0;
     const T* zbm = (const T*)v.zbm;
     if (c.n_doc_tiles) {
-        k_doc_hash<T><<<c.n_doc_tiles, 256, 0, c.stream>>>(c.doc_tiles, v.doc_off, zbm, v.bm_of_tok, v.rec, v.dk_slots,
-                                                          v.count_bits, c.K, v.err);
+        k_doc_hash<T><<<c.n_doc_tiles, c.doc_threads, doc_tile_smem_bytes(c.doc_tile), c.stream>>>(
+            c.doc_tiles, c.doc_tile, v.doc_off, zbm, v.bm_of_tok, v.rec, v.dk_slots, v.count_bits, c.K, v.err);
         ++launches;
     }
     if (c.n_long_docs) {
@@ -388,6 +390,9 @@ int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host)
 
 void set_hist_smem_limits()
 {
+    const int doc_bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
+    cudaFuncSetAttribute(k_doc_hash<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
+    cudaFuncSetAttribute(k_doc_hash<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
     cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
     cudaFuncSetAttribute(k_hist_chunks<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
     cudaFuncSetAttribute(k_count_k<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);

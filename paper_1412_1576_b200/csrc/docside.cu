@@ -3,8 +3,8 @@
 // The sweep-start n_kd of a document (Eq. 12) is a function of that document's assignments
 // alone, so the tile's tables are built where they are used: in shared memory, by insertion
 // (Section 5's hashed rows: claim a slot with compare-and-swap, then add one to its count), and
-// thrown away afterwards.  One warp owns one document at a time: it builds the table and then,
-// for every token of the document, gathers what the accept/reject pass needs from this side:
+// thrown away afterwards.  Every token then gathers what the accept/reject pass needs from this
+// side:
 //   - the token's own (topic, n_kd) record,
 //   - for every word-proposal (drawn by pass 1): n_kd at the proposed topic,
 //   - for every doc-proposal (Eq. 9, Eq. 12): the Philox block of the step, the proposed topic
@@ -67,15 +67,19 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
     __stcs(reinterpret_cast<uint4*>(out), make_uint4(own, w1, w2, w3));
 }
 
+// `cap` = tokens a tile can hold (the shared-memory carve-up); small tiles keep many CTAs per SM,
+// which is what hides the gathers of the first phase.
 template <typename T>
-__global__ void __launch_bounds__(256)
-k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
+__global__ void __launch_bounds__(1024)
+k_doc_tile(View v, const int32_t* __restrict__ tiles, int32_t cap, uint2 key, uint32_t sweep, int32_t mh_steps)
 {
-    __shared__ uint32_t slots[DK_SLOTS_PER_TOKEN * DOC_TILE];
-    __shared__ int32_t soff[DOC_TILE + 1];
-    __shared__ uint32_t topic[DOC_TILE];   // a token's topic, later the table index of its slot
-    __shared__ uint32_t bm_s[DOC_TILE];    // a token's block-major index
-    __shared__ uint32_t t1_s[DOC_TILE];    // the first word-proposal's topic
+    extern __shared__ __align__(16) uint32_t doc_smem[];
+    uint32_t* slots = doc_smem;                                  // [4 * cap] the tile's tables
+    int32_t* soff = reinterpret_cast<int32_t*>(slots + DK_SLOTS_PER_TOKEN * cap);  // [cap + 1] document offsets
+    uint32_t* topic = reinterpret_cast<uint32_t*>(soff + cap + 1);  // [cap] a token's topic, later its slot
+    uint32_t* bm_s = topic + cap;                                // [cap] a token's block-major index
+    uint32_t* t1_s = bm_s + cap;                                 // [cap] the first word-proposal's topic
+    uint16_t* doc_s = reinterpret_cast<uint16_t*>(t1_s + cap);   // [cap] a token's document, relative to the tile
     const int tid = threadIdx.x;
     const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
     const int32_t nseg = s1 - s0;
@@ -93,28 +97,33 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = v.doc_off[s0 + j] - base;
     for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
     __syncthreads();
+    // which document each token belongs to: one warp per document writes its index
     const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-    for (int d = warp; d < nseg; d += nwarps) {
-        const int32_t first = soff[d], len = soff[d + 1] - first;
-        if (len == 0) continue;
-        uint32_t* tab = slots + DK_SLOTS_PER_TOKEN * first;
-        const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)len;
-        for (int j = first + lane; j < first + len; j += 32) {
-            const uint32_t k = topic[j];
-            uint32_t at = 0xFFFFFFFFu;
-            if (k < (uint32_t)v.K) at = dk_insert(tab, cap, k, v.count_bits);
-            if (at == 0xFFFFFFFFu) {
-                atomicOr(v.err, k < (uint32_t)v.K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
-                at = 0;
-            }
-            topic[j] = at;
+    for (int d = warp; d < nseg; d += nwarps)
+        for (int j = soff[d] + lane; j < soff[d + 1]; j += 32) doc_s[j] = (uint16_t)d;
+    __syncthreads();
+    // every token adds itself to its document's table and notes the slot
+    for (int j = tid; j < cnt; j += blockDim.x) {
+        const int32_t first = soff[doc_s[j]], len = soff[doc_s[j] + 1] - first;
+        const uint32_t k = topic[j];
+        uint32_t at = 0xFFFFFFFFu;
+        if (k < (uint32_t)v.K)
+            at = dk_insert(slots + DK_SLOTS_PER_TOKEN * first, DK_SLOTS_PER_TOKEN * (uint32_t)len, k, v.count_bits);
+        if (at == 0xFFFFFFFFu) {
+            atomicOr(v.err, k < (uint32_t)v.K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
+            at = 0;
         }
-        __syncwarp();  // the document's table is complete: only this warp touches it
+        topic[j] = at;
+    }
+    __syncthreads();
+    // the tables are complete: every token gathers its share
+    for (int j = tid; j < cnt; j += blockDim.x) {
+        const int32_t first = soff[doc_s[j]], len = soff[doc_s[j] + 1] - first;
+        const uint32_t* tab = slots + DK_SLOTS_PER_TOKEN * first;
         const uint32_t* slot_of = topic + first;
-        auto slot_at = [slot_of](uint32_t j) { return slot_of[j]; };
-        for (int j = first + lane; j < first + len; j += 32)
-            doc_side_token<T>(v, tab, (uint32_t)(base + j), (uint32_t)len, tab[topic[j]], t1_s[j], bm_s[j], slot_at,
-                              key, sweep, mh_steps);
+        auto slot_at = [slot_of](uint32_t jj) { return slot_of[jj]; };
+        doc_side_token<T>(v, tab, (uint32_t)(base + j), (uint32_t)len, tab[topic[j]], t1_s[j], bm_s[j], slot_at, key,
+                          sweep, mh_steps);
     }
 }
 
@@ -153,13 +162,23 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
     }
 }
 
+size_t doc_tile_smem_bytes(int tile_tokens) { return (size_t)tile_tokens * DOC_TILE_SMEM_PER_TOKEN + 16; }
+
+void set_doc_smem_limits()
+{
+    const int bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
+    cudaFuncSetAttribute(k_doc_tile<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
 template <typename T>
 static int doc_side_t(Ctx& c, int mh_steps)
 {
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     int launches = 0;
     if (c.n_doc_tiles) {
-        k_doc_tile<T><<<c.n_doc_tiles, 256, 0, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps);
+        k_doc_tile<T><<<c.n_doc_tiles, c.doc_threads, doc_tile_smem_bytes(c.doc_tile), c.stream>>>(
+            c.v, c.doc_tiles, c.doc_tile, key, c.sweep, mh_steps);
         ++launches;
     }
     if (c.n_long_docs) {

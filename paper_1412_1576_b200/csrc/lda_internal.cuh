@@ -21,11 +21,23 @@ enum : int {
 };
 
 constexpr uint32_t DK_EMPTY = 0xFFFFFFFFu;  // == DK_EMPTY_SLOT of the device helpers
+constexpr int DK_SLOTS_PER_TOKEN_HOST = 4;   // == DK_SLOTS_PER_TOKEN of the device helpers
 constexpr int SORT_TILE = 2048;      // tokens per segmented-sort tile (one CTA)
-constexpr int DOC_TILE = 1024;       // tokens per tile of whole documents in the n_kd rebuild (one CTA)
+// Tiles of whole documents (one CTA each) of the document-side kernels: tokens per tile and
+// threads per CTA, chosen per corpus from these shapes; longer documents get a CTA of their own.
+constexpr int DOC_TILE_SHAPES = 4;
+constexpr int DOC_TILE_TOKENS[DOC_TILE_SHAPES] = {384, 768, 1536, 3072};
+constexpr int DOC_TILE_THREADS[DOC_TILE_SHAPES] = {128, 256, 512, 1024};
+constexpr int DOC_TILE_MAX = 3072;
+// shared memory per token of a tile: 4 table slots, document offset, topic/slot, block-major
+// index, first proposal (4 bytes each), document index (2 bytes)
+constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DK_SLOTS_PER_TOKEN_HOST + 4 + 4 + 4 + 4 + 2;
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (bins)
 constexpr int HIST_CHUNK = 16384;    // tokens per CTA in the histogram path
-constexpr int HOT_TILE = 8192;       // MH kernel: tokens of one hot word per CTA
+#ifndef LDA_HOT_TILE
+#define LDA_HOT_TILE 8192
+#endif
+constexpr int HOT_TILE = LDA_HOT_TILE;  // MH kernels: tokens of one hot word per CTA
 constexpr int COLD_TILE = 2048;      // MH kernel: tokens of a tile of whole tail words
 constexpr int COLD_WORDS = 512;      // MH kernel: words per tail tile
 constexpr int HOT_STAGE_MAX_K = 16384;  // dense rows up to this many topics are staged in shared memory
@@ -89,6 +101,7 @@ struct Ctx {
     cudaStream_t stream = nullptr;
     bool wide_topics = false;  // false: 16-bit topic storage, true: 32-bit
     int block_shift = 21;  // log2 of the tokens per block of the block-major order
+    int doc_tile = DOC_TILE_TOKENS[0], doc_threads = DOC_TILE_THREADS[0];  // shape of the document tiles
     int side_steps = 0;    // number of steps the exchange buffers are allocated for
     double dense_frac = 0.05;
     double dense_min_tf = 64;
@@ -136,6 +149,7 @@ int launch_alias_dense(Ctx& c);
 int launch_alias_sparse(Ctx& c);
 int launch_sample(Ctx& c, int mh_steps);   // all passes of the MH step; needs ensure_exchange()
 int launch_doc_side(Ctx& c, int mh_steps);  // pass 2 of the MH step
+size_t doc_tile_smem_bytes(int tile_tokens);  // dynamic shared memory of the document-tile kernels
 int ensure_exchange(Ctx& c, int mh_steps);  // (re)allocates View::prop / View::dside; LDA_* status
 int launch_loglik(Ctx& c, double* out3_host);
 int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host);

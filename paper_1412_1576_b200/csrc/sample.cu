@@ -23,10 +23,21 @@
 namespace lda {
 
 constexpr double INV_2_32 = 1.0 / 4294967296.0;
-#ifndef LDA_HOT_THREADS
-#define LDA_HOT_THREADS 512
+// launch shapes of the hot-word kernel: threads per CTA and CTAs per SM the compiler must allow
+#ifndef LDA_PROPOSE_THREADS
+#define LDA_PROPOSE_THREADS 512
 #endif
-constexpr int HOT_THREADS = LDA_HOT_THREADS;
+#ifndef LDA_PROPOSE_MIN_CTAS
+#define LDA_PROPOSE_MIN_CTAS 2
+#endif
+#ifndef LDA_ACCEPT_THREADS
+#define LDA_ACCEPT_THREADS 768
+#endif
+#ifndef LDA_ACCEPT_MIN_CTAS
+#define LDA_ACCEPT_MIN_CTAS 2
+#endif
+constexpr int PROPOSE_THREADS = LDA_PROPOSE_THREADS;
+constexpr int ACCEPT_THREADS = LDA_ACCEPT_THREADS;
 constexpr int COLD_THREADS = 256;
 constexpr int STAGE_WAIT_LIMIT = 1 << 20;
 
@@ -312,7 +323,8 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
 
 // Hot words: tile = (word, first token, count).  ACCEPT = false: pass 1, true: pass 3.
 template <typename T, int CH, bool STAGED, bool ACCEPT>
-__global__ void __launch_bounds__(HOT_THREADS)
+__global__ void __launch_bounds__(ACCEPT ? ACCEPT_THREADS : PROPOSE_THREADS,
+                                  ACCEPT ? LDA_ACCEPT_MIN_CTAS : LDA_PROPOSE_MIN_CTAS)
 k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
 {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
@@ -345,8 +357,8 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     tile.mix = __ldg(v.mix32 + w);
     tile.bar = &bar;
     tile.ready = !(STAGED && ACCEPT);
-    if (ACCEPT) accept_tokens<T, CH>(v, tile, p0, p0 + cnt, HOT_THREADS, key, sweep, mh_steps);
-    else propose_tokens<T>(v, tile, p0, p0 + cnt, HOT_THREADS, key, sweep, mh_steps);
+    if (ACCEPT) accept_tokens<T, CH>(v, tile, p0, p0 + cnt, ACCEPT_THREADS, key, sweep, mh_steps);
+    else propose_tokens<T>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
     // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one
 }
 
@@ -447,7 +459,7 @@ static int sample_tc(Ctx& c, int mh_steps)
     int launches = 0;
     // pass 1: word-proposals
     if (c.n_hot_tiles) {
-        k_word_hot<T, CH, false, false><<<c.n_hot_tiles, HOT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key, c.sweep,
+        k_word_hot<T, CH, false, false><<<c.n_hot_tiles, PROPOSE_THREADS, 0, c.stream>>>(v, c.hot_tiles, key, c.sweep,
                                                                                     mh_steps);
         ++launches;
     }
@@ -463,10 +475,10 @@ static int sample_tc(Ctx& c, int mh_steps)
     cudaEventRecord(c.ev[9], c.stream);
     if (c.n_hot_tiles) {
         if (staged)
-            k_word_hot<T, CH, true, true><<<c.n_hot_tiles, HOT_THREADS, (size_t)v.dense_stride * 8, c.stream>>>(
+            k_word_hot<T, CH, true, true><<<c.n_hot_tiles, ACCEPT_THREADS, (size_t)v.dense_stride * 8, c.stream>>>(
                 v, c.hot_tiles, key, c.sweep, mh_steps);
         else
-            k_word_hot<T, CH, false, true><<<c.n_hot_tiles, HOT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
+            k_word_hot<T, CH, false, true><<<c.n_hot_tiles, ACCEPT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
                                                                                        c.sweep, mh_steps);
         ++launches;
     }
