@@ -31,7 +31,7 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 #define LDA_PROPOSE_MIN_CTAS 2
 #endif
 #ifndef LDA_ACCEPT_THREADS
-#define LDA_ACCEPT_THREADS 768
+#define LDA_ACCEPT_THREADS 512
 #endif
 #ifndef LDA_ACCEPT_MIN_CTAS
 #define LDA_ACCEPT_MIN_CTAS 2
@@ -245,11 +245,37 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
     const size_t N = (size_t)v.N;
     T* zw = reinterpret_cast<T*>(v.zw);
     bool bad = false;
-    for (int32_t p = p_begin + (int32_t)threadIdx.x; p < p_end; p += nthreads) {
-        const uint32_t tok = __ldcs(v.tok_orig + p);
-        const uint32_t at = __ldcs(v.inv + p);
-        const uint32_t* side = v.dside + (size_t)at * v.side_stride;  // what pass 2 gathered for this token
-        const uint32_t own = __ldcs(side);
+    // The reads of a token are issued ahead of its turn: (token id, block-major index) two
+    // iterations early, the gathered record (which needs that index) one iteration early.
+    const uint4* side4 = reinterpret_cast<const uint4*>(v.dside);
+    const int32_t quads = v.side_stride >> 2;
+    int32_t p = p_begin + (int32_t)threadIdx.x;
+    uint32_t tok_c = 0, at_c = 0, tok_n = 0, at_n = 0;
+    uint4 rec_c = make_uint4(0u, 0u, 0u, 0u);
+    if (p < p_end) {
+        tok_c = __ldcs(v.tok_orig + p);
+        at_c = __ldcs(v.inv + p);
+    }
+    if (p + nthreads < p_end) {
+        tok_n = __ldcs(v.tok_orig + p + nthreads);
+        at_n = __ldcs(v.inv + p + nthreads);
+    }
+    if (p < p_end) rec_c = __ldcs(side4 + (size_t)at_c * quads);
+    for (; p < p_end; p += nthreads) {
+        const uint32_t tok = tok_c, at = at_c;
+        const uint4 rec = rec_c;  // own record, then the first three words pass 2 gathered
+        tok_c = tok_n;
+        at_c = at_n;
+        if (p + nthreads < p_end) rec_c = __ldcs(side4 + (size_t)at_c * quads);
+        if (p + 2 * nthreads < p_end) {
+            tok_n = __ldcs(v.tok_orig + p + 2 * nthreads);
+            at_n = __ldcs(v.inv + p + 2 * nthreads);
+        }
+        const uint32_t* side = v.dside + (size_t)at * v.side_stride;
+        auto side_word = [&](int32_t i) {
+            return i == 1 ? rec.y : i == 2 ? rec.z : i == 3 ? rec.w : __ldcs(side + i);
+        };
+        const uint32_t own = rec.x;
         const typename Tile::Ref w = tile.ref(p - p_begin);
         uint32_t z0 = 0, s = 0;
         int32_t n_sd = 0, n_sw = 0, n_s = 0;
@@ -260,10 +286,10 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 e[i] = 0;
                 ua[i] = 0;
                 if (m0 + i < mh_steps) {
-                    e[i] = __ldcs(side + 1 + m0 + i);
+                    e[i] = side_word(1 + m0 + i);
                     // acceptance uniform: word 3 of the step's Philox block; pass 2 already drew the
                     // doc steps' blocks and left that word beside the gathered counts
-                    ua[i] = (i & 1) ? __ldcs(side + 1 + mh_steps + ((m0 + i) >> 1))
+                    ua[i] = (i & 1) ? side_word(1 + mh_steps + ((m0 + i) >> 1))
                                     : philox4x32_10(make_uint4(tok, sweep, (uint32_t)(m0 + i), 0u), key).w;
                 }
             }
