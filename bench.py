@@ -122,13 +122,14 @@ def algorithmic_bytes_per_token(mh_steps: int, topic_bytes: int, rho_wk: float) 
     T, M = topic_bytes, mh_steps
     W = (M + 1) // 2
     return {
-        # token id, block-major index, one alias bin per draw, proposed topics out
-        "propose": 4 + 4 + 8 * W + T * W,
+        # token id, block-major index, one alias bin per draw, proposed topics and acceptance uniforms out
+        "propose": 4 + 4 + 8 * W + T * W + 4 * W,
         # block-major index, z in, proposed topics in, gathered words out (own record, one word per
         # step, one acceptance uniform per doc step, padded to 16 bytes)
         "doc_side": 4 + T + T * W + 4 * ((1 + M + M // 2 + 3) // 4 * 4),
-        # token id, block-major index, gathered words in, z out in both orders, n_kw row once per nonzero
-        "accept": 4 + 4 + 4 * (1 + M) + 2 * T + 8.0 * rho_wk,
+        # block-major index, gathered words and the word steps' uniforms in, z out in both orders,
+        # n_kw row once per nonzero
+        "accept": 4 + 4 * ((1 + M + M // 2 + 3) // 4 * 4) + 4 * W + 2 * T + 8.0 * rho_wk,
         "count_wk": T + 8.0 * rho_wk,
         "count_k": T,
         # row in, table out (split point, alias, packed bin), construction scratch out and in

@@ -104,28 +104,32 @@ int lda::ensure_exchange(Ctx& c, int mh_steps)
             if (c.allocs[i] == p) { c.allocs.erase(c.allocs.begin() + i); break; }
         cudaFree(p);
     };
-    auto bytes_for = [&](int steps, size_t& prop_b, size_t& side_b, int& stride) {
+    auto bytes_for = [&](int steps, size_t& prop_b, size_t& side_b, size_t& ua_b, int& stride) {
         const size_t zt = c.wide_topics ? 4 : 2, n = (size_t)c.N;
         stride = (1 + steps + steps / 2 + 3) & ~3;  // own, one word per step, one uniform per doc step
         prop_b = zt * (((size_t)steps + 1) / 2) * n;
         side_b = 4 * (size_t)stride * n;
+        ua_b = 4 * (((size_t)steps + 1) / 2) * n;
     };
     cudaStreamSynchronize(c.stream);
-    size_t pb = 0, sb = 0;
+    size_t pb = 0, sb = 0, ub = 0;
     int stride = 0;
     if (c.side_steps) {
-        bytes_for(c.side_steps, pb, sb, stride);
-        c.device_bytes -= (int64_t)(pb + sb);
+        bytes_for(c.side_steps, pb, sb, ub, stride);
+        c.device_bytes -= (int64_t)(pb + sb + ub);
     }
     drop(c.v.prop);
     drop(c.v.dside);
+    drop(c.v.ua_w);
     c.v.prop = nullptr;
     c.v.dside = nullptr;
+    c.v.ua_w = nullptr;
     c.side_steps = 0;
-    bytes_for(mh_steps, pb, sb, stride);
+    bytes_for(mh_steps, pb, sb, ub, stride);
     c.v.prop = dev_alloc(c, pb);
     c.v.dside = (uint32_t*)dev_alloc(c, sb);
-    if (!c.v.prop || !c.v.dside) {
+    c.v.ua_w = (uint32_t*)dev_alloc(c, ub);
+    if (!c.v.prop || !c.v.dside || !c.v.ua_w) {
         c.err = "device allocation failed";
         return LDA_ENOMEM;
     }

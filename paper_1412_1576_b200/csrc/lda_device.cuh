@@ -38,17 +38,18 @@ constexpr int DK_SLOTS_PER_TOKEN = 4;
 
 __device__ __forceinline__ uint32_t dk_home(uint32_t k, uint32_t cap) { return __umulhi(k * DK_HASH_MULT, cap); }
 
-// Adds one occurrence of topic k to the table `tab[0..cap)`: claims an empty slot with
-// compare-and-swap (or finds the topic's slot), then adds one to its count bits.  Safe against
-// concurrent insertions into the same table.  Returns the slot, or DK_EMPTY_SLOT if the table had
-// no room (which the load factor rules out).
+// Adds one occurrence of topic k to the table `tab[0..cap)`: claims an empty slot with one
+// compare-and-swap that also sets the count to 1, or finds the topic's slot and adds one to its
+// count bits.  Safe against concurrent insertions into the same table.  Returns the slot, or
+// DK_EMPTY_SLOT if the table had no room (which the load factor rules out).
 __device__ __forceinline__ uint32_t dk_insert(uint32_t* tab, uint32_t cap, uint32_t k, int count_bits)
 {
-    const uint32_t fresh = k << count_bits;
+    const uint32_t first = (k << count_bits) | 1u;
     uint32_t h = dk_home(k, cap);
     for (uint32_t n = 0; n < cap; ++n) {
-        const uint32_t prev = atomicCAS(&tab[h], DK_EMPTY_SLOT, fresh);
-        if (prev == DK_EMPTY_SLOT || (prev >> count_bits) == k) {
+        const uint32_t prev = atomicCAS(&tab[h], DK_EMPTY_SLOT, first);
+        if (prev == DK_EMPTY_SLOT) return h;
+        if ((prev >> count_bits) == k) {
             atomicAdd(&tab[h], 1u);
             return h;
         }

@@ -58,6 +58,7 @@ struct View {
     const uint32_t* bm_of_tok;  // [N] block-major index of the token with document-order index i
     // per-sweep exchange buffers between the word-order and the document-order passes
     void* prop;        // [word steps][N] block-major: topics proposed by the word-proposals (topic type)
+    uint32_t* ua_w;    // [word steps][N] word order: acceptance uniforms of the word-proposal steps
     uint32_t* dside;   // [N][side_stride] block-major: own record, per step (topic << count_bits) | n_kd,
                        // per doc step its acceptance uniform
     int32_t side_stride;  // words per token in dside, a multiple of 4

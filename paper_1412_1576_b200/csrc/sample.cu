@@ -226,6 +226,7 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
             int32_t n_tw;
             tile.draw_finish(w, d, t, n_tw);
             __stcs(prop + (size_t)(m >> 1) * v.N + at, (T)t);
+            __stcs(v.ua_w + (size_t)(m >> 1) * v.N + p, r.w);  // the step's acceptance uniform, for pass 3
         }
     }
 }
@@ -245,32 +246,22 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
     const size_t N = (size_t)v.N;
     T* zw = reinterpret_cast<T*>(v.zw);
     bool bad = false;
-    // The reads of a token are issued ahead of its turn: (token id, block-major index) two
-    // iterations early, the gathered record (which needs that index) one iteration early.
+    // The reads of a token are issued ahead of its turn: its block-major index two iterations
+    // early, the gathered record (which needs that index) one iteration early.
     const uint4* side4 = reinterpret_cast<const uint4*>(v.dside);
     const int32_t quads = v.side_stride >> 2;
     int32_t p = p_begin + (int32_t)threadIdx.x;
-    uint32_t tok_c = 0, at_c = 0, tok_n = 0, at_n = 0;
+    uint32_t at_c = 0, at_n = 0;
     uint4 rec_c = make_uint4(0u, 0u, 0u, 0u);
-    if (p < p_end) {
-        tok_c = __ldcs(v.tok_orig + p);
-        at_c = __ldcs(v.inv + p);
-    }
-    if (p + nthreads < p_end) {
-        tok_n = __ldcs(v.tok_orig + p + nthreads);
-        at_n = __ldcs(v.inv + p + nthreads);
-    }
+    if (p < p_end) at_c = __ldcs(v.inv + p);
+    if (p + nthreads < p_end) at_n = __ldcs(v.inv + p + nthreads);
     if (p < p_end) rec_c = __ldcs(side4 + (size_t)at_c * quads);
     for (; p < p_end; p += nthreads) {
-        const uint32_t tok = tok_c, at = at_c;
+        const uint32_t at = at_c;
         const uint4 rec = rec_c;  // own record, then the first three words pass 2 gathered
-        tok_c = tok_n;
         at_c = at_n;
         if (p + nthreads < p_end) rec_c = __ldcs(side4 + (size_t)at_c * quads);
-        if (p + 2 * nthreads < p_end) {
-            tok_n = __ldcs(v.tok_orig + p + 2 * nthreads);
-            at_n = __ldcs(v.inv + p + 2 * nthreads);
-        }
+        if (p + 2 * nthreads < p_end) at_n = __ldcs(v.inv + p + 2 * nthreads);
         const uint32_t* side = v.dside + (size_t)at * v.side_stride;
         auto side_word = [&](int32_t i) {
             return i == 1 ? rec.y : i == 2 ? rec.z : i == 3 ? rec.w : __ldcs(side + i);
@@ -287,10 +278,10 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 ua[i] = 0;
                 if (m0 + i < mh_steps) {
                     e[i] = side_word(1 + m0 + i);
-                    // acceptance uniform: word 3 of the step's Philox block; pass 2 already drew the
-                    // doc steps' blocks and left that word beside the gathered counts
+                    // acceptance uniform: word 3 of the step's Philox block, drawn by the pass that made
+                    // the proposal (pass 1: word steps, pass 2: doc steps) and left for this one
                     ua[i] = (i & 1) ? side_word(1 + mh_steps + ((m0 + i) >> 1))
-                                    : philox4x32_10(make_uint4(tok, sweep, (uint32_t)(m0 + i), 0u), key).w;
+                                    : __ldcs(v.ua_w + (size_t)((m0 + i) >> 1) * N + p);
                 }
             }
             if (m0 == 0) {
