@@ -12,6 +12,8 @@
 // (topic, its n_kd) per token.
 // No per-token global atomics: a CTA touches global counters once per bin it
 // actually filled (documents longer than a tile are the one exception).
+#include <algorithm>
+
 #include "lda_device.cuh"
 #include "lda_internal.cuh"
 
@@ -259,29 +261,48 @@ k_long_doc_hash(const int32_t* __restrict__ long_docs, const int32_t* __restrict
     }
 }
 
-// n_k: histogram of all assignments, CTA-private shared-memory bins.
-template <typename T>
+// n_k = sum over words of n_kw (Section 3), taken from the rows the n_kw rebuild has just written
+// instead of from another pass over the assignments:
+//   - dense rows: column sums, one thread per topic and group of rows;
+//   - sorted rows of the words without a dense row: CTA-private shared-memory bins over a chunk
+//     of words, flushed with one global add per nonzero bin.
+__global__ void __launch_bounds__(256)
+k_nk_from_dense(const int32_t* __restrict__ dense_rows, int32_t n_dense, int32_t K, int32_t stride,
+                int32_t* __restrict__ nk)
+{
+    const int32_t k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    int32_t s = 0;
+    for (int32_t r = blockIdx.y; r < n_dense; r += gridDim.y) s += __ldcs(dense_rows + (size_t)r * stride + k);
+    if (s) atomicAdd(&nk[k], s);
+}
+
 __global__ void __launch_bounds__(512)
-k_count_k(const T* __restrict__ z, int32_t n, int32_t* __restrict__ nk, int32_t K, int32_t window,
-          int* err)
+k_nk_from_sparse(const int32_t* __restrict__ row_start, const int32_t* __restrict__ wk_nnz,
+                 const uint32_t* __restrict__ wk_topic, const uint32_t* __restrict__ wk_count,
+                 const int32_t* __restrict__ dense_slot, int32_t V, int32_t* __restrict__ nk, int32_t K,
+                 int32_t window)
 {
     extern __shared__ int32_t bins[];
-    const int64_t per = ((int64_t)n + gridDim.x - 1) / gridDim.x;
-    const int64_t lo = per * blockIdx.x, hi = min((int64_t)n, lo + per);
+    const int32_t per = (V + gridDim.x - 1) / gridDim.x;
+    const int32_t w_lo = per * blockIdx.x, w_hi = min(V, w_lo + per);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     for (int32_t k0 = 0; k0 < K; k0 += window) {
         const int32_t nb = min(window, K - k0);
         for (int b = threadIdx.x; b < nb; b += blockDim.x) bins[b] = 0;
         __syncthreads();
-        for (int64_t j = lo + threadIdx.x; j < hi; j += blockDim.x) {
-            const uint32_t k = (uint32_t)z[j];
-            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
-            const uint32_t b = k - (uint32_t)k0;
-            if (b < (uint32_t)nb) atomicAdd(&bins[b], 1);
+        for (int32_t w = w_lo + warp; w < w_hi; w += nwarps) {
+            if (dense_slot[w] >= 0) continue;
+            const int32_t r0 = row_start[w], n = wk_nnz[w];
+            for (int32_t j = lane; j < n; j += 32) {
+                const uint32_t b = wk_topic[r0 + j] - (uint32_t)k0;
+                if (b < (uint32_t)nb) atomicAdd(&bins[b], (int32_t)wk_count[r0 + j]);
+            }
         }
         __syncthreads();
         for (int b = threadIdx.x; b < nb; b += blockDim.x) {
-            const int32_t v = bins[b];
-            if (v) atomicAdd(&nk[k0 + b], v);
+            const int32_t n = bins[b];
+            if (n) atomicAdd(&nk[k0 + b], n);
         }
         __syncthreads();
     }
@@ -336,19 +357,26 @@ static int count_wk_t(Ctx& c)
     return launches;
 }
 
-template <typename T>
-static int count_k_t(Ctx& c)
+// Must follow launch_count_wk(): reads the rows it wrote.
+static int count_k(Ctx& c)
 {
     View& v = c.v;
     cudaMemsetAsync(v.nk, 0, (size_t)c.K * 4, c.stream);
     if (c.N == 0) return 0;
-    const int win = hist_window(c);
-    int grid = (int)((c.N + 65535) / 65536);
-    if (grid > 148 * 4) grid = 148 * 4;
-    if (grid < 1) grid = 1;
-    k_count_k<T><<<grid, 512, (size_t)win * 4, c.stream>>>((const T*)v.zw, (int32_t)c.N, v.nk,
-                                                          c.K, win, v.err);
-    return 1;
+    int launches = 0;
+    if (c.n_dense) {
+        const dim3 grid((unsigned)((c.K + 255) / 256), (unsigned)std::min(c.n_dense, 64));
+        k_nk_from_dense<<<grid, 256, 0, c.stream>>>(v.dense_rows, c.n_dense, c.K, v.dense_stride, v.nk);
+        ++launches;
+    }
+    if (c.n_dense < c.V) {
+        const int win = hist_window(c);
+        const int grid = std::min(148 * 2, (int)((c.V + 511) / 512));
+        k_nk_from_sparse<<<grid, 512, (size_t)win * 4, c.stream>>>(v.row_start, v.wk_nnz, v.wk_topic, v.wk_count,
+                                                                  v.dense_slot, c.V, v.nk, c.K, win);
+        ++launches;
+    }
+    return launches;
 }
 
 template <typename T>
@@ -371,7 +399,7 @@ static int count_dk_t(Ctx& c)
 }
 
 int launch_count_wk(Ctx& c) { return c.wide_topics ? count_wk_t<int32_t>(c) : count_wk_t<uint16_t>(c); }
-int launch_count_k(Ctx& c) { return c.wide_topics ? count_k_t<int32_t>(c) : count_k_t<uint16_t>(c); }
+int launch_count_k(Ctx& c) { return count_k(c); }
 int launch_count_dk(Ctx& c) { return c.wide_topics ? count_dk_t<int32_t>(c) : count_dk_t<uint16_t>(c); }
 
 int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host)
@@ -395,8 +423,7 @@ void set_hist_smem_limits()
     cudaFuncSetAttribute(k_doc_hash<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
     cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
     cudaFuncSetAttribute(k_hist_chunks<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
-    cudaFuncSetAttribute(k_count_k<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
-    cudaFuncSetAttribute(k_count_k<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
+    cudaFuncSetAttribute(k_nk_from_sparse, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
 }
 
 }  // namespace lda
