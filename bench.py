@@ -131,7 +131,7 @@ def algorithmic_bytes_per_token(mh_steps: int, topic_bytes: int, rho_wk: float) 
         # n_kw row once per nonzero
         "accept": 4 + 4 * ((1 + M + M // 2 + 3) // 4 * 4) + 4 * W + 2 * T + 8.0 * rho_wk,
         "count_wk": T + 8.0 * rho_wk,
-        "count_k": T,
+        "count_k": 8.0 * rho_wk,   # the rebuilt rows read again
         # row in, table out (split point, alias, packed bin), construction scratch out and in
         "alias_sparse": (8 + 8 + 8 + 40) * rho_wk,
     }
@@ -260,7 +260,7 @@ def run_ours(args):
     per_ms = {k: phases["ms_" + k] / args.steps for k in b_alg}
     kernels = {"propose": "k_word_hot/k_word_cold (pass 1)", "doc_side": "k_doc_tile",
                "accept": "k_word_hot/k_word_cold (pass 3)", "count_wk": "n_kw rebuild kernels",
-               "count_k": "k_count_k", "alias_sparse": "k_alias_sparse_*"}
+               "count_k": "k_nk_from_dense/k_nk_from_sparse", "alias_sparse": "k_alias_sparse_*"}
     top = max(per_ms, key=per_ms.get)          # the dominant kernel of the sweep, by measured time
     top_ms = per_ms[top]
     achieved = b_alg[top] * N / (top_ms * 1e-3) / 1e9 if top_ms > 0 else 0.0
