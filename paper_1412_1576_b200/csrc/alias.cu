@@ -224,7 +224,10 @@ __global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, ul
 }
 
 // One CTA per word whose row can be longer than ALIAS_WARP_MAX.
-__global__ void __launch_bounds__(256)
+#ifndef LDA_ALIAS_BLOCK_THREADS
+#define LDA_ALIAS_BLOCK_THREADS 256
+#endif
+__global__ void __launch_bounds__(LDA_ALIAS_BLOCK_THREADS)
 k_alias_sparse_block(View v, const int32_t* __restrict__ words, ull* sc_w, ull* sc_de, uint32_t* sc_item)
 {
     __shared__ ull smem[33];
@@ -254,7 +257,7 @@ int launch_alias_sparse(Ctx& c)
     k_alias_sparse_warp<<<grid, 256, 0, c.stream>>>(c.v, c.sc_w, c.sc_de, c.sc_item);
     ++launches;
     if (c.n_alias_big) {
-        k_alias_sparse_block<<<c.n_alias_big, 256, 0, c.stream>>>(c.v, c.alias_big, c.sc_w, c.sc_de,
+        k_alias_sparse_block<<<c.n_alias_big, LDA_ALIAS_BLOCK_THREADS, 0, c.stream>>>(c.v, c.alias_big, c.sc_w, c.sc_de,
                                                                  c.sc_item);
         ++launches;
     }

@@ -20,6 +20,13 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k)
     return c;
 }
 
+// (double)x for an unsigned 32-bit x, exactly, without the (slow) integer-to-double conversion
+// instruction: x placed in the low mantissa bits of 2^52, then 2^52 subtracted.
+__device__ __forceinline__ double u32_to_double(uint32_t x)
+{
+    return __dsub_rn(__hiloint2double(0x43300000, (int)x), 4503599627370496.0);
+}
+
 // floor(r * n / 2^32): a 32-bit random word mapped to {0..n-1}.
 __device__ __forceinline__ uint32_t scale_to_range(uint32_t r, uint32_t n) { return __umulhi(r, n); }
 

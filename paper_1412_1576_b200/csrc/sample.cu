@@ -308,22 +308,22 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 const bool live = m0 + i < mh_steps && t[i] != s;
                 const int32_t n_td = (int32_t)(e[i] & cmask);
                 const int32_t e_s = (s == z0), e_t = (t[i] == z0);
-                double num = __dadd_rn((double)(n_td - e_t), alpha);
-                num = __dmul_rn(num, __dadd_rn((double)(n_tw[i] - e_t), beta));
-                num = __dmul_rn(num, __dadd_rn((double)(n_s - e_s), Vb));
-                double den = __dadd_rn((double)(n_sd - e_s), alpha);
-                den = __dmul_rn(den, __dadd_rn((double)(n_sw - e_s), beta));
-                den = __dmul_rn(den, __dadd_rn((double)(n_t[i] - e_t), Vb));
+                double num = __dadd_rn(u32_to_double((uint32_t)(n_td - e_t)), alpha);
+                num = __dmul_rn(num, __dadd_rn(u32_to_double((uint32_t)(n_tw[i] - e_t)), beta));
+                num = __dmul_rn(num, __dadd_rn(u32_to_double((uint32_t)(n_s - e_s)), Vb));
+                double den = __dadd_rn(u32_to_double((uint32_t)(n_sd - e_s)), alpha);
+                den = __dmul_rn(den, __dadd_rn(u32_to_double((uint32_t)(n_sw - e_s)), beta));
+                den = __dmul_rn(den, __dadd_rn(u32_to_double((uint32_t)(n_t[i] - e_t)), Vb));
                 if ((i & 1) == 0) {
-                    num = __dmul_rn(num, __dadd_rn((double)n_sw, beta));
-                    num = __dmul_rn(num, __dadd_rn((double)n_t[i], Vb));
-                    den = __dmul_rn(den, __dadd_rn((double)n_tw[i], beta));
-                    den = __dmul_rn(den, __dadd_rn((double)n_s, Vb));
+                    num = __dmul_rn(num, __dadd_rn(u32_to_double((uint32_t)n_sw), beta));
+                    num = __dmul_rn(num, __dadd_rn(u32_to_double((uint32_t)n_t[i]), Vb));
+                    den = __dmul_rn(den, __dadd_rn(u32_to_double((uint32_t)n_tw[i]), beta));
+                    den = __dmul_rn(den, __dadd_rn(u32_to_double((uint32_t)n_s), Vb));
                 } else {
-                    num = __dmul_rn(num, __dadd_rn((double)n_sd, alpha));
-                    den = __dmul_rn(den, __dadd_rn((double)n_td, alpha));
+                    num = __dmul_rn(num, __dadd_rn(u32_to_double((uint32_t)n_sd), alpha));
+                    den = __dmul_rn(den, __dadd_rn(u32_to_double((uint32_t)n_td), alpha));
                 }
-                const double u = __dmul_rn((double)ua[i], INV_2_32);
+                const double u = __dmul_rn(u32_to_double((uint32_t)ua[i]), INV_2_32);
                 if (live && __dmul_rn(u, den) < num) {
                     s = t[i];
                     n_sd = n_td;
