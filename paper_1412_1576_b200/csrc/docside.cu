@@ -67,19 +67,18 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
     __stcs(reinterpret_cast<uint4*>(out), make_uint4(own, w1, w2, w3));
 }
 
-// `cap` = tokens a tile can hold (the shared-memory carve-up); small tiles keep many CTAs per SM,
-// which is what hides the gathers of the first phase.
-template <typename T>
-__global__ void __launch_bounds__(1024)
-k_doc_tile(View v, const int32_t* __restrict__ tiles, int32_t cap, uint2 key, uint32_t sweep, int32_t mh_steps)
+// `cap` = tokens a tile can hold (the shared-memory carve-up) = DOC_TILE_ROUNDS x blockDim.x: a
+// thread owns at most DOC_TILE_ROUNDS tokens and keeps what it read about them in registers across
+// the phases.  Small tiles keep many CTAs per SM, which is what hides the gathers of the first phase.
+template <typename T, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1536 / THREADS)
+k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
 {
+    constexpr int cap = DOC_TILE_ROUNDS * THREADS;
     extern __shared__ __align__(16) uint32_t doc_smem[];
     uint32_t* slots = doc_smem;                                  // [4 * cap] the tile's tables
     int32_t* soff = reinterpret_cast<int32_t*>(slots + DK_SLOTS_PER_TOKEN * cap);  // [cap + 1] document offsets
-    uint32_t* topic = reinterpret_cast<uint32_t*>(soff + cap + 1);  // [cap] a token's topic, later its slot
-    uint32_t* bm_s = topic + cap;                                // [cap] a token's block-major index
-    uint32_t* t1_s = bm_s + cap;                                 // [cap] the first word-proposal's topic
-    uint16_t* doc_s = reinterpret_cast<uint16_t*>(t1_s + cap);   // [cap] a token's document, relative to the tile
+    uint32_t* slot_s = reinterpret_cast<uint32_t*>(soff + cap + 1);  // [cap] slot (inside its table) of a token's topic
     const int tid = threadIdx.x;
     const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
     const int32_t nseg = s1 - s0;
@@ -88,42 +87,60 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, int32_t cap, uint2 key, ui
     if (cnt == 0) return;
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
     const T* prop = reinterpret_cast<const T*>(v.prop);
-    for (int j = tid; j < cnt; j += blockDim.x) {
-        const uint32_t bm = __ldcs(v.bm_of_tok + base + j);
-        bm_s[j] = bm;
-        topic[j] = (uint32_t)__ldcg(zbm + bm);
-        t1_s[j] = (uint32_t)__ldcg(prop + bm);
+    uint32_t bm[DOC_TILE_ROUNDS], z[DOC_TILE_ROUNDS], t1[DOC_TILE_ROUNDS];
+    int32_t first[DOC_TILE_ROUNDS], len[DOC_TILE_ROUNDS];
+#pragma unroll
+    for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
+        const int j = tid + r * THREADS;
+        bm[r] = z[r] = t1[r] = 0;
+        if (j < cnt) {
+            bm[r] = __ldcs(v.bm_of_tok + base + j);
+            z[r] = (uint32_t)__ldcg(zbm + bm[r]);
+            t1[r] = (uint32_t)__ldcg(prop + bm[r]);
+        }
     }
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = v.doc_off[s0 + j] - base;
-    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
+    const uint4 empty4 = make_uint4(DK_EMPTY, DK_EMPTY, DK_EMPTY, DK_EMPTY);
+    for (int j = tid; j < cnt; j += blockDim.x) reinterpret_cast<uint4*>(slots)[j] = empty4;
     __syncthreads();
-    // which document each token belongs to: one warp per document writes its index
-    const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-    for (int d = warp; d < nseg; d += nwarps)
-        for (int j = soff[d] + lane; j < soff[d + 1]; j += 32) doc_s[j] = (uint16_t)d;
-    __syncthreads();
-    // every token adds itself to its document's table and notes the slot
-    for (int j = tid; j < cnt; j += blockDim.x) {
-        const int32_t first = soff[doc_s[j]], len = soff[doc_s[j] + 1] - first;
-        const uint32_t k = topic[j];
-        uint32_t at = 0xFFFFFFFFu;
-        if (k < (uint32_t)v.K)
-            at = dk_insert(slots + DK_SLOTS_PER_TOKEN * first, DK_SLOTS_PER_TOKEN * (uint32_t)len, k, v.count_bits);
-        if (at == 0xFFFFFFFFu) {
-            atomicOr(v.err, k < (uint32_t)v.K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
-            at = 0;
+    // every token finds its document, adds itself to the document's table and notes the slot
+#pragma unroll
+    for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
+        const int j = tid + r * THREADS;
+        first[r] = 0;
+        len[r] = 1;
+        if (j < cnt) {
+            int lo = 0, hi = nseg;  // last document with soff[doc] <= j
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (soff[mid] <= j) lo = mid; else hi = mid;
+            }
+            first[r] = soff[lo];
+            len[r] = soff[lo + 1] - first[r];
+            uint32_t at = 0xFFFFFFFFu;
+            if (z[r] < (uint32_t)v.K)
+                at = dk_insert(slots + DK_SLOTS_PER_TOKEN * first[r], DK_SLOTS_PER_TOKEN * (uint32_t)len[r], z[r],
+                               v.count_bits);
+            if (at == 0xFFFFFFFFu) {
+                atomicOr(v.err, z[r] < (uint32_t)v.K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
+                at = 0;
+            }
+            slot_s[j] = at;
+            z[r] = at;  // from here on: the slot
         }
-        topic[j] = at;
     }
     __syncthreads();
     // the tables are complete: every token gathers its share
-    for (int j = tid; j < cnt; j += blockDim.x) {
-        const int32_t first = soff[doc_s[j]], len = soff[doc_s[j] + 1] - first;
-        const uint32_t* tab = slots + DK_SLOTS_PER_TOKEN * first;
-        const uint32_t* slot_of = topic + first;
-        auto slot_at = [slot_of](uint32_t jj) { return slot_of[jj]; };
-        doc_side_token<T>(v, tab, (uint32_t)(base + j), (uint32_t)len, tab[topic[j]], t1_s[j], bm_s[j], slot_at, key,
-                          sweep, mh_steps);
+#pragma unroll
+    for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
+        const int j = tid + r * THREADS;
+        if (j < cnt) {
+            const uint32_t* tab = slots + DK_SLOTS_PER_TOKEN * first[r];
+            const uint32_t* slot_of = slot_s + first[r];
+            auto slot_at = [slot_of](uint32_t jj) { return slot_of[jj]; };
+            doc_side_token<T>(v, tab, (uint32_t)(base + j), (uint32_t)len[r], tab[z[r]], t1[r], bm[r], slot_at, key,
+                              sweep, mh_steps);
+        }
     }
 }
 
@@ -167,8 +184,10 @@ size_t doc_tile_smem_bytes(int tile_tokens) { return (size_t)tile_tokens * DOC_T
 void set_doc_smem_limits()
 {
     const int bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
-    cudaFuncSetAttribute(k_doc_tile<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    cudaFuncSetAttribute(k_doc_tile<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<int32_t, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<uint16_t, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes / 2);
+    cudaFuncSetAttribute(k_doc_tile<int32_t, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes / 2);
 }
 
 template <typename T>
@@ -177,8 +196,13 @@ static int doc_side_t(Ctx& c, int mh_steps)
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     int launches = 0;
     if (c.n_doc_tiles) {
-        k_doc_tile<T><<<c.n_doc_tiles, c.doc_threads, doc_tile_smem_bytes(c.doc_tile), c.stream>>>(
-            c.v, c.doc_tiles, c.doc_tile, key, c.sweep, mh_steps);
+        const size_t smem = doc_tile_smem_bytes(c.doc_tile);
+        switch (c.doc_threads) {
+            case 128: k_doc_tile<T, 128><<<c.n_doc_tiles, 128, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            case 256: k_doc_tile<T, 256><<<c.n_doc_tiles, 256, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            case 512: k_doc_tile<T, 512><<<c.n_doc_tiles, 512, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            default: k_doc_tile<T, 1024><<<c.n_doc_tiles, 1024, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+        }
         ++launches;
     }
     if (c.n_long_docs) {

@@ -29,9 +29,10 @@ constexpr int DOC_TILE_SHAPES = 4;
 constexpr int DOC_TILE_TOKENS[DOC_TILE_SHAPES] = {384, 768, 1536, 3072};
 constexpr int DOC_TILE_THREADS[DOC_TILE_SHAPES] = {128, 256, 512, 1024};
 constexpr int DOC_TILE_MAX = 3072;
-// shared memory per token of a tile: 4 table slots, document offset, topic/slot, block-major
-// index, first proposal (4 bytes each), document index (2 bytes)
-constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DK_SLOTS_PER_TOKEN_HOST + 4 + 4 + 4 + 4 + 2;
+constexpr int DOC_TILE_ROUNDS = 3;  // tokens per thread: every shape holds 3 x its thread count
+static_assert(DOC_TILE_TOKENS[0] == 3 * DOC_TILE_THREADS[0] && DOC_TILE_TOKENS[3] == 3 * DOC_TILE_THREADS[3], "tile shapes");
+// shared memory per token of a tile: 4 table slots, document offset, topic/slot (4 bytes each)
+constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DK_SLOTS_PER_TOKEN_HOST + 4 + 4;
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (bins)
 constexpr int HIST_CHUNK = 16384;    // tokens per CTA in the histogram path
 #ifndef LDA_HOT_TILE
