@@ -51,7 +51,11 @@ static int read_err(Ctx& c, int* bits)
         cudaStreamSynchronize(c.stream) != cudaSuccess)
         return cuda_fail(&c, "reading the device error word");
     if (*bits) cudaMemsetAsync(c.v.err, 0, sizeof(int), c.stream);
-    if (cudaGetLastError() != cudaSuccess) return cuda_fail(&c, "kernel launch");
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        c.err = std::string("kernel launch: ") + cudaGetErrorString(e);
+        return LDA_ECUDA;
+    }
     return LDA_OK;
 }
 

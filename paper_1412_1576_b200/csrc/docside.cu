@@ -186,8 +186,6 @@ void set_doc_smem_limits()
     const int bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
     cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     cudaFuncSetAttribute(k_doc_tile<int32_t, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    cudaFuncSetAttribute(k_doc_tile<uint16_t, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes / 2);
-    cudaFuncSetAttribute(k_doc_tile<int32_t, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes / 2);
 }
 
 template <typename T>

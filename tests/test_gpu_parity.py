@@ -189,6 +189,29 @@ def test_block_size_is_invisible(small_corpus, block_log2):
         assert a == pytest.approx(b, rel=1e-10)
 
 
+def test_mid_shape_documents_and_lognormal_lengths():
+    """Documents of ~330 tokens (a larger document-tile shape than the 90-token configs pick) and a
+    heavy-tailed length law whose longest documents get a CTA of their own."""
+    c = synth.make("mid", seed=1, scale=0.01)
+    g, o = _pair(c, seed=21)
+    _assert_same_counts(g, o)
+    for sweep in range(2):
+        g.sweep(1, 2)
+        o.sweep(1, 2)
+        assert np.array_equal(g.get_assignments(), o.get_assignments()), sweep
+    _assert_same_counts(g, o)
+    _assert_same_tables(g, o)
+    c = synth.generate(V=2000, K=300, D=1500, length=("lognormal", 100, 1.2), zipf_s=1.0, alpha=0.05, beta=0.01,
+                       seed=12)
+    g, o = _pair(c, seed=22)
+    g.sweep(2, 4)
+    o.sweep(2, 4)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_counts(g, o)
+    for a, b in zip(g.loglik(), o.loglik()):
+        assert a == pytest.approx(b, rel=1e-10)
+
+
 def test_edge_cases():
     # empty documents, a single token, one topic, absent words
     w = np.array([3, 3, 0, 7, 7, 7], np.int32)
