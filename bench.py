@@ -137,6 +137,19 @@ def algorithmic_bytes_per_token(mh_steps: int, topic_bytes: int, rho_wk: float) 
     }
 
 
+def over_ranks(dist, device, ms: float, n_tokens: float):
+    """Replicas only: the job's time is the slowest rank's, its work the sum over ranks.
+    Returns (max over ranks of ms, sum over ranks of n_tokens); identity without a process group."""
+    if dist is None:
+        return float(ms), float(n_tokens)
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([float(n_tokens)], device=device, dtype=torch.float64)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(n.item())
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -203,15 +216,7 @@ def run_ours(args):
         phases[k] = getattr(s, k)
     launches = s.kernel_launches
     rho_sum = args.steps * s.nnz_wk / max(N, 1)
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        tot = torch.tensor([float(N)], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
-        total_tokens = float(tot.item())
-    else:
-        total_tokens = float(N)
+    ms, total_tokens = over_ranks(dist, "cuda", ms, N)
     ms_per_step = ms / args.steps
     value = total_tokens / (ms_per_step * 1e-3)
     st1 = lda.stats()
@@ -238,10 +243,7 @@ def run_ours(args):
         e_ms = ev0.elapsed_time(ev1)
         wall_ms = (time.perf_counter() - t0) * 1e3
         e_ms = max(e_ms, wall_ms)   # host-side work between calls counts too
-        if dist is not None:
-            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms, _ = over_ranks(dist, "cuda", e_ms, N)
         e2e = {"value": total_tokens / (e_ms / args.e2e_steps * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": 4 * N, "d2h_bytes_per_step": 4 * N + 24,
                "steps": args.e2e_steps, "loglik": ll[0] if ll else None,
