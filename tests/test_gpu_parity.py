@@ -212,6 +212,68 @@ def test_mid_shape_documents_and_lognormal_lengths():
         assert a == pytest.approx(b, rel=1e-10)
 
 
+def test_large_shape_sample_against_oracle():
+    """The benchmark's workload shape (V = 141 000, K = 10 000, Poisson(90) documents, Zipf 1.1) at 1 % of its
+    documents: same kernels, tile shapes and hot/tail split as the full run, small enough for the oracle."""
+    c = synth.make("large", seed=0, scale=0.01)
+    g, o = _pair(c, seed=1234)
+    g.sweep(1, 2)
+    o.sweep(1, 2)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    assert np.array_equal(g.get_nk(), o.get_nk())
+    g.sweep(1, 4)
+    o.sweep(1, 4)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    # equal counts, so only the order of summation differs: the oracle adds ~1.5e7 lgamma terms one after
+    # the other (error up to n * 2^-53 relative to the sum of magnitudes), the library in 592 partial sums
+    for a, b in zip(g.loglik(), o.loglik()):
+        assert a == pytest.approx(b, rel=1e-9)
+
+
+def test_full_size_invariants():
+    """The benchmark's full workload (738 M tokens) in the configuration bench.py times: the count tables
+    must be exactly those of the library's own assignments (properties that hold at any size), and
+    a sample of documents is recounted by brute force."""
+    import torch
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * 2 ** 30:
+        pytest.skip("needs about 60 GB of free device memory")
+    c = synth.make("large", seed=0, device="cuda")
+    N, D = c.n_tokens, c.n_docs
+    g = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
+    g.load_corpus(c.word_ids, c.doc_offsets)
+    off = c.doc_offsets.cpu().numpy()
+    words = c.word_ids
+    g.init(1234)
+    g.sweep(2, 2)
+    z = torch.from_numpy(g.get_assignments()).cuda()
+    assert z.numel() == N and int(z.min()) >= 0 and int(z.max()) < c.K
+    nk = torch.bincount(z, minlength=c.K).cpu().numpy()
+    assert np.array_equal(g.get_nk(), nk)                       # sum_w n_kw = n_k = histogram of z
+    assert int(nk.sum()) == N
+    st = g.stats()
+    # nonzeros of n_kw and n_kd = distinct (word, topic) and (document, topic) pairs of z
+    key_w = words.long() * c.K + z.long()
+    assert st["nnz_wk"] == int(torch.unique(key_w).numel())
+    del key_w
+    doc = torch.repeat_interleave(torch.arange(D, device="cuda"), torch.diff(c.doc_offsets.cuda()))
+    key_d = doc * c.K + z.long()
+    del doc
+    assert st["nnz_dk"] == int(torch.unique(key_d).numel())
+    del key_d
+    # the log-likelihood is a function of the tables: recompute its document part for a sample of
+    # documents is not possible without the tables, so recount n_kw for a sample of words instead
+    ro, top, cnt = g.get_csr(binding.LDA_NWK)
+    rng = np.random.default_rng(0)
+    wcpu = None
+    for w in rng.integers(0, c.V, size=20):
+        sel = (words == int(w))
+        zz = z[sel].cpu().numpy()
+        uk, uc = np.unique(zz, return_counts=True)
+        assert np.array_equal(top[ro[w]:ro[w + 1]], uk)
+        assert np.array_equal(cnt[ro[w]:ro[w + 1]], uc)
+
+
 def test_edge_cases():
     # empty documents, a single token, one topic, absent words
     w = np.array([3, 3, 0, 7, 7, 7], np.int32)
