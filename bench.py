@@ -286,6 +286,8 @@ def run_ours(args):
             if tr.get("workload") == args.workload and tr.get("mh_steps") == M:
                 roofline["traffic"] = tr["dram_bytes_per_token"] * N
                 roofline["traffic_source"] = tr.get("source")
+                if "issue_active_pct" in tr:   # ncu smsp__issue_active of the same capture
+                    roofline["issue_active_pct"] = tr["issue_active_pct"]
         except Exception:
             pass
 
