@@ -328,7 +328,7 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     bool ok = true;
     auto A = [&](size_t bytes) { void* p = dev_alloc(c, bytes); ok = ok && p; return p; };
     v.zw = A(n1 * zt);
-    v.zbm = A(n1 * zt);
+    v.zbm = A(2 * n1 * zt);  // (topic, first word-proposal) pairs
     v.rec = (uint32_t*)A(n1 * 4 + 16);  // + one aligned group of four words past the last record
     v.row_start = upload(c, row_start);
     v.dense_slot = upload(c, dense_slot);

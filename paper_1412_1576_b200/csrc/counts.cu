@@ -206,7 +206,7 @@ k_doc_hash(const int32_t* __restrict__ tiles, int32_t cap, const int32_t* __rest
     const int32_t cnt = doc_off[s1] - base;
     if (cnt == 0) return;
     // the tile's documents lie in one or two blocks of the block-major order: these reads hit L2
-    for (int j = tid; j < cnt; j += blockDim.x) topic[j] = (uint32_t)__ldcg(zbm + __ldcs(bm_of_tok + base + j));
+    for (int j = tid; j < cnt; j += blockDim.x) topic[j] = (uint32_t)__ldcg(zbm + 2 * (size_t)__ldcs(bm_of_tok + base + j));
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = doc_off[s0 + j] - base;
     for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
     __syncthreads();
@@ -248,7 +248,7 @@ k_long_doc_hash(const int32_t* __restrict__ long_docs, const int32_t* __restrict
     for (uint32_t j = threadIdx.x; j < cap; j += blockDim.x) tab[j] = DK_EMPTY;
     __syncthreads();
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-        const uint32_t k = (uint32_t)zbm[bm_of_tok[first + j]];
+        const uint32_t k = (uint32_t)zbm[2 * (size_t)bm_of_tok[first + j]];
         uint32_t at = 0xFFFFFFFFu;
         if (k < (uint32_t)K) at = dk_insert(tab, cap, k, count_bits);
         if (at == 0xFFFFFFFFu) atomicOr(err, k < (uint32_t)K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);

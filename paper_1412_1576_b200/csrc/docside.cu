@@ -20,6 +20,21 @@ namespace lda {
 
 constexpr double INV_2_32 = 1.0 / 4294967296.0;
 
+// A token's current topic and its first word-proposal sit side by side at its block-major index:
+// one read brings both.
+__device__ __forceinline__ void load_topic_pair(const uint16_t* zbm, uint32_t bm, uint32_t& z, uint32_t& t1)
+{
+    const uint32_t w = __ldcg(reinterpret_cast<const uint32_t*>(zbm) + bm);
+    z = w & 0xFFFFu;
+    t1 = w >> 16;
+}
+__device__ __forceinline__ void load_topic_pair(const int32_t* zbm, uint32_t bm, uint32_t& z, uint32_t& t1)
+{
+    const uint2 w = __ldcg(reinterpret_cast<const uint2*>(zbm) + bm);
+    z = w.x;
+    t1 = w.y;
+}
+
 // Everything pass 3 needs from the document side for one token, written at the token's
 // block-major index `bm`.
 //   tab     : the document's table, 4 * doc_len slots
@@ -86,7 +101,6 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     const int32_t cnt = v.doc_off[s1] - base;
     if (cnt == 0) return;
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
-    const T* prop = reinterpret_cast<const T*>(v.prop);
     uint32_t bm[DOC_TILE_ROUNDS], z[DOC_TILE_ROUNDS], t1[DOC_TILE_ROUNDS];
     int32_t first[DOC_TILE_ROUNDS], len[DOC_TILE_ROUNDS];
 #pragma unroll
@@ -95,8 +109,7 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
         bm[r] = z[r] = t1[r] = 0;
         if (j < cnt) {
             bm[r] = __ldcs(v.bm_of_tok + base + j);
-            z[r] = (uint32_t)__ldcg(zbm + bm[r]);
-            t1[r] = (uint32_t)__ldcg(prop + bm[r]);
+            load_topic_pair(zbm, bm[r], z[r], t1[r]);
         }
     }
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = v.doc_off[s0 + j] - base;
@@ -155,13 +168,12 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
     const int32_t first = v.doc_off[d], cnt = v.doc_off[d + 1] - first;
     const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)cnt;
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
-    const T* prop = reinterpret_cast<const T*>(v.prop);
     uint32_t* tab = v.dk_slots + DK_SLOTS_PER_TOKEN * (size_t)first;
     uint32_t* slot_of = v.rec + first;
     for (uint32_t j = threadIdx.x; j < cap; j += blockDim.x) tab[j] = DK_EMPTY;
     __syncthreads();
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-        const uint32_t k = (uint32_t)zbm[v.bm_of_tok[first + j]];
+        const uint32_t k = (uint32_t)zbm[2 * (size_t)v.bm_of_tok[first + j]];
         uint32_t at = 0xFFFFFFFFu;
         if (k < (uint32_t)v.K) at = dk_insert(tab, cap, k, v.count_bits);
         if (at == 0xFFFFFFFFu) {
@@ -174,7 +186,7 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
     auto slot_at = [slot_of](uint32_t j) { return slot_of[j]; };
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
         const uint32_t bm = v.bm_of_tok[first + j];
-        doc_side_token<T>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)prop[bm], bm,
+        doc_side_token<T>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)zbm[2 * (size_t)bm + 1], bm,
                           slot_at, key, sweep, mh_steps);
     }
 }

@@ -58,14 +58,15 @@ struct View {
     const uint32_t* inv;        // [N] block-major index of the token at word-sorted position p
     const uint32_t* bm_of_tok;  // [N] block-major index of the token with document-order index i
     // per-sweep exchange buffers between the word-order and the document-order passes
-    void* prop;        // [word steps][N] block-major: topics proposed by the word-proposals (topic type)
+    void* prop;        // [word steps][N] block-major: topics proposed by the word-proposals after the first
     uint32_t* ua_w;    // [word steps][N] word order: acceptance uniforms of the word-proposal steps
     uint32_t* dside;   // [N][side_stride] block-major: own record, per step (topic << count_bits) | n_kd,
                        // per doc step its acceptance uniform
     int32_t side_stride;  // words per token in dside, a multiple of 4
     // assignments (topic type: u16 or i32) after the last MH step or initialisation
     void* zw;   // word-sorted order: read by the n_kw / n_k rebuild
-    void* zbm;  // block-major order: read (through bm_of_tok) by everything that works per document
+    void* zbm;  // block-major order, two entries per token: its topic, read (through bm_of_tok) by everything
+                // that works per document, and beside it the first word-proposal of the running MH step
     // Document order, valid after launch_count_dk() only (the exported form of n_kd):
     // rec[i] = (z_i << count_bits) | n_kd[d][z_i].
     uint32_t* rec;

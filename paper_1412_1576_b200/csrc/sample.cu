@@ -225,7 +225,9 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
             uint32_t t;
             int32_t n_tw;
             tile.draw_finish(w, d, t, n_tw);
-            __stcs(prop + (size_t)(m >> 1) * v.N + at, (T)t);
+            // the first proposal goes beside the token's topic, the later ones to arrays of their own
+            if (m == 0) __stcs(reinterpret_cast<T*>(v.zbm) + 2 * (size_t)at + 1, (T)t);
+            else __stcs(prop + (size_t)(m >> 1) * v.N + at, (T)t);
             __stcs(v.ua_w + (size_t)(m >> 1) * v.N + p, r.w);  // the step's acceptance uniform, for pass 3
         }
     }
@@ -333,7 +335,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
             }
         }
         __stcs(zw + p, (T)s);
-        __stcs(reinterpret_cast<T*>(v.zbm) + at, (T)s);
+        __stcs(reinterpret_cast<T*>(v.zbm) + 2 * (size_t)at, (T)s);
     }
     if (bad) atomicOr(v.err, ERR_COUNT_ZERO);
 }
@@ -430,7 +432,7 @@ __global__ void k_init(View v, uint2 key)
         const uint4 r = philox4x32_10(make_uint4(tok, 0u, 0u, 1u), key);
         const T z = (T)scale_to_range(r.x, (uint32_t)v.K);
         zw[p] = z;
-        zbm[v.inv[p]] = z;
+        zbm[2 * (size_t)v.inv[p]] = z;
     }
 }
 
@@ -447,7 +449,7 @@ __global__ void k_spread(View v, const int32_t* __restrict__ z_in)
             a = 0;
         }
         zw[p] = (T)a;
-        zbm[v.inv[p]] = (T)a;
+        zbm[2 * (size_t)v.inv[p]] = (T)a;
     }
 }
 
@@ -457,7 +459,7 @@ __global__ void k_export(View v, int32_t* __restrict__ out)
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < v.N;
          i += (int64_t)gridDim.x * blockDim.x)
-        out[i] = (int32_t)zbm[v.bm_of_tok[i]];
+        out[i] = (int32_t)zbm[2 * (size_t)v.bm_of_tok[i]];
 }
 
 static int grid_for(int64_t n, int block)
