@@ -78,8 +78,8 @@ int lda_set_stream(lda_ctx* ctx, void* cuda_stream);
  *   "dense_frac"   fraction of the vocabulary (by term frequency) whose n_kw rows are dense (Section 5)
  *   "dense_min_tf" words rarer than this stay sparse even inside dense_frac
  *   "block_log2"   log2 of the tokens per block of documents in the block-major token order that the
- *                  document-side pass of the MH step walks (default 21: the records and n_kd tables
- *                  of one block, 12 bytes per token, stay in L2 while the pass is on it)             */
+ *                  document-side pass of the MH step walks (default 22: the exchange buffers
+ *                  of one block, 20 bytes per token, stay in L2 while the document pass is on it)             */
 int lda_set_option(lda_ctx* ctx, const char* key, double value);
 
 /* Corpus in document order: token i has word word_ids[i]; document d owns tokens

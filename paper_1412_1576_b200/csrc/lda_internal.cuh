@@ -103,7 +103,7 @@ struct Ctx {
     int device = 0;
     cudaStream_t stream = nullptr;
     bool wide_topics = false;  // false: 16-bit topic storage, true: 32-bit
-    int block_shift = 21;  // log2 of the tokens per block of the block-major order
+    int block_shift = 22;  // log2 of the tokens per block of the block-major order
     int doc_tile = DOC_TILE_TOKENS[0], doc_threads = DOC_TILE_THREADS[0];  // shape of the document tiles
     int side_steps = 0;    // number of steps the exchange buffers are allocated for
     double dense_frac = 0.05;
