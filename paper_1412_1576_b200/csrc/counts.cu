@@ -7,9 +7,11 @@
 //     encodes them;
 //   - hot words: shared-memory histogram over a window of topics, merged into
 //     the word's dense row, then compacted into the sorted row.
-// n_kd (segments = documents over the document-order z): per document an
-// open-addressing table built by insertion in shared memory, plus one record
-// (topic, its n_kd) per token.
+// n_k: column sums of the rows just written.
+// n_kd (segments = documents): the MH step builds every document's table itself, per tile, in
+// shared memory (docside.cu); the kernels here write the same tables to device memory -- plus one
+// record (topic, its n_kd) per token -- when a caller asks for them (lda_get_counts, lda_loglik,
+// lda_get_stats).
 // No per-token global atomics: a CTA touches global counters once per bin it
 // actually filled (documents longer than a tile are the one exception).
 #include <algorithm>
@@ -183,11 +185,10 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
     if (threadIdx.x == 0) wk_nnz[w] = done;
 }
 
-// n_kd as per-document open-addressing tables (layout and probe order: dk_insert in lda_device.cuh).  One CTA per
-// tile of whole documents holding <= SORT_TILE tokens: the tile's tables are built in shared
-// memory by insertion (claim a slot with compare-and-swap, then add one to its count bits) and
-// written out in one coalesced pass.  Every token's record (topic, n_kd of its topic in its
-// document) is written next to it, so that the MH step gets both in one read.
+// n_kd as per-document open-addressing tables in device memory, for export (layout and probe
+// order: dk_insert in lda_device.cuh).  One CTA per tile of whole documents (`cap` tokens at
+// most): the tile's tables are built in shared memory by insertion and written out in one
+// coalesced pass, together with every token's record (topic, n_kd of its topic in its document).
 //
 template <typename T>
 __global__ void __launch_bounds__(1024)
