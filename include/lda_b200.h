@@ -76,7 +76,7 @@ int lda_set_stream(lda_ctx* ctx, void* cuda_stream);
 
 /* Tunables that never change results.  Must be set before lda_load_corpus().
  *   "dense_frac"   fraction of the vocabulary (by term frequency) whose n_kw rows are dense (Section 5)
- *   "dense_min_tf" words rarer than this stay sparse even inside dense_frac
+ *   "dense_min_tf" words rarer than this (or than K/8) stay sparse even inside dense_frac
  *   "block_log2"   log2 of the tokens per block of documents in the block-major token order that the
  *                  document-side pass of the MH step walks (default 22: the exchange buffers
  *                  of one block, 20 bytes per token, stay in L2 while the document pass is on it)             */

@@ -227,7 +227,8 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         std::vector<int32_t> tmp(tf);
         const size_t nth = (size_t)std::min<int64_t>(n_top, V) - 1;
         std::nth_element(tmp.begin(), tmp.begin() + nth, tmp.end(), std::greater<int32_t>());
-        tf_cut = std::max<int32_t>(tmp[nth], (int32_t)std::max(1.0, c.dense_min_tf));
+        // a dense row of K counters only pays for a word with a fair share of K tokens
+        tf_cut = std::max<int32_t>({tmp[nth], (int32_t)std::max(1.0, c.dense_min_tf), K / 8});
     }
     std::vector<int32_t> dense_slot((size_t)V, -1), dense_words, row_start((size_t)V + 1), alias_big;
     std::vector<int32_t> hist_chunks, word_tiles;

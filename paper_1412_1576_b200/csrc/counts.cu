@@ -166,19 +166,27 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
     const int32_t w = dense_words[blockIdx.x];
     const int32_t* row = dense_rows + (size_t)dense_slot[w] * stride;
     const int32_t out0 = row_start[w], cap = row_start[w + 1] - out0;
+    // four consecutive topics per thread and step (rows are padded to a multiple of four and start
+    // 16-byte aligned; the padding is never written, so it reads as zero)
     int32_t done = 0;
-    for (int32_t k0 = 0; k0 < K; k0 += blockDim.x) {
-        const int32_t k = k0 + threadIdx.x;
-        const int32_t n = (k < K) ? row[k] : 0;
+    for (int32_t k0 = 0; k0 < stride; k0 += 4 * blockDim.x) {
+        const int32_t k = k0 + 4 * (int32_t)threadIdx.x;
+        int4 n = make_int4(0, 0, 0, 0);
+        if (k < stride) n = __ldcs(reinterpret_cast<const int4*>(row + k));
+        const int32_t mine = (n.x > 0) + (n.y > 0) + (n.z > 0) + (n.w > 0);
         int32_t total;
-        const int32_t pos = block_scan_excl<int32_t>(n > 0 ? 1 : 0, scan_tmp, total);
-        if (n > 0) {
-            if (done + pos < cap) {
-                wk_topic[out0 + done + pos] = (uint32_t)k;
-                wk_count[out0 + done + pos] = (uint32_t)n;
-            } else {
-                atomicOr(err, ERR_ROW_OVERFLOW);
-            }
+        int32_t pos = done + block_scan_excl<int32_t>(mine, scan_tmp, total);
+        if (pos + mine > cap) {
+            atomicOr(err, ERR_ROW_OVERFLOW);
+        } else {
+            const int32_t nv[4] = {n.x, n.y, n.z, n.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (nv[q] > 0) {
+                    wk_topic[out0 + pos] = (uint32_t)(k + q);
+                    wk_count[out0 + pos] = (uint32_t)nv[q];
+                    ++pos;
+                }
         }
         done += total;
     }
