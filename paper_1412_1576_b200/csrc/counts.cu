@@ -132,24 +132,26 @@ k_hist_chunks(const int32_t* __restrict__ chunks, const T* __restrict__ z,
               const int32_t* __restrict__ dense_slot, int32_t* __restrict__ dense_rows, int32_t K,
               int32_t stride, int32_t window, int* err)
 {
-    extern __shared__ int32_t bins[];
+    // two 16-bit counters per word of shared memory: a chunk holds at most HIST_CHUNK < 65536 tokens
+    extern __shared__ uint32_t bins2[];
     const int32_t w = chunks[3 * blockIdx.x], first = chunks[3 * blockIdx.x + 1],
                   cnt = chunks[3 * blockIdx.x + 2];
     int32_t* row = dense_rows + (size_t)dense_slot[w] * stride;
     for (int32_t k0 = 0; k0 < K; k0 += window) {
-        const int32_t nb = min(window, K - k0);
-        for (int b = threadIdx.x; b < nb; b += blockDim.x) bins[b] = 0;
+        const int32_t nb = min(window, K - k0), nw = (nb + 1) >> 1;
+        for (int b = threadIdx.x; b < nw; b += blockDim.x) bins2[b] = 0;
         __syncthreads();
         for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
             const uint32_t k = (uint32_t)z[first + j];
             if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
             const uint32_t b = k - (uint32_t)k0;
-            if (b < (uint32_t)nb) atomicAdd(&bins[b], 1);
+            if (b < (uint32_t)nb) atomicAdd(&bins2[b >> 1], (b & 1u) ? 0x10000u : 1u);
         }
         __syncthreads();
-        for (int b = threadIdx.x; b < nb; b += blockDim.x) {
-            const int32_t n = bins[b];
-            if (n) atomicAdd(&row[k0 + b], n);
+        for (int b = threadIdx.x; b < nw; b += blockDim.x) {
+            const uint32_t n2 = bins2[b];
+            if (n2 & 0xFFFFu) atomicAdd(&row[k0 + 2 * b], (int32_t)(n2 & 0xFFFFu));
+            if (n2 >> 16) atomicAdd(&row[k0 + 2 * b + 1], (int32_t)(n2 >> 16));
         }
         __syncthreads();
     }
@@ -355,8 +357,8 @@ static int count_wk_t(Ctx& c)
     }
     if (c.n_dense) {
         cudaMemsetAsync(v.dense_rows, 0, (size_t)c.n_dense * v.dense_stride * 4, c.stream);
-        const int win = hist_window(c);
-        k_hist_chunks<T><<<c.n_hist_chunks, 512, (size_t)win * 4, c.stream>>>(
+        const int win = c.K < HIST16_BINS ? c.K : HIST16_BINS;
+        k_hist_chunks<T><<<c.n_hist_chunks, 512, (size_t)((win + 1) / 2) * 4, c.stream>>>(
             c.hist_chunks, z, v.dense_slot, v.dense_rows, c.K, v.dense_stride, win, v.err);
         k_compact_dense<<<c.n_dense, 256, 0, c.stream>>>(c.dense_words, v.dense_slot, v.dense_rows,
                                                          v.row_start, v.wk_topic, v.wk_count,
@@ -430,8 +432,8 @@ void set_hist_smem_limits()
     const int doc_bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
     cudaFuncSetAttribute(k_doc_hash<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
     cudaFuncSetAttribute(k_doc_hash<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
-    cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
-    cudaFuncSetAttribute(k_hist_chunks<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
+    cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST16_BINS * 2);
+    cudaFuncSetAttribute(k_hist_chunks<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST16_BINS * 2);
     cudaFuncSetAttribute(k_nk_from_sparse, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
 }
 
