@@ -3,8 +3,9 @@
 // n_kw (segments = words over the word-sorted z): per word, the sorted list of
 // (topic, count).  Two paths, chosen per word at load time:
 //   - tail words: whole words are packed into tiles of <= SORT_TILE tokens; one
-//     CTA sorts the tile's (word, topic) keys in shared memory and run-length
-//     encodes them;
+//     CTA counts each word's topics in a shared-memory hash table and reads them
+//     back in topic order through a bitmap over the topics (K <= 16384), or sorts
+//     the tile's (word, topic) keys (larger K);
 //   - hot words: shared-memory histogram over a window of topics, merged into
 //     the word's dense row, then compacted into the sorted row.
 // n_k: column sums of the rows just written.
@@ -35,8 +36,9 @@ struct EmitWord {
     __device__ __forceinline__ void rows(int32_t seg, int32_t n) const { nnz[seg] = n; }
 };
 
-// One CTA per tile of whole segments [s0, s1) holding <= SORT_TILE tokens and
-// <= SORT_TILE segments.
+// Tail words when K is large (the bitmap of k_word_rows would cost more than the sort): one CTA per
+// tile of whole words [s0, s1) holding <= SORT_TILE tokens and <= SORT_TILE words sorts the tile's
+// (word, topic) keys in shared memory (bitonic) and run-length encodes them.
 template <typename T, class Emit>
 __global__ void __launch_bounds__(256)
 k_seg_count_sorted(const int32_t* __restrict__ tiles, const int32_t* __restrict__ seg_off,
@@ -121,6 +123,70 @@ k_seg_count_sorted(const int32_t* __restrict__ tiles, const int32_t* __restrict_
         emit.entry(s0 + seg, rank, key & kmask, (uint32_t)(headpos[h + 1] - j));
     }
     for (int j = tid; j < nseg; j += blockDim.x) emit.rows(s0 + j, hidx[soff[j + 1]] - hidx[soff[j]]);
+}
+
+// Tail words: one CTA per tile of whole words [s0, s1) holding <= SORT_TILE tokens; the words are
+// taken one after the other.  A word's tokens are counted in a shared-memory hash table (same
+// tables as n_kd: 4 slots per token) and marked in a bitmap over the K topics; the bitmap, read in
+// order, gives the sorted row: the rank of a topic is the number of set bits before it.
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_word_rows(const int32_t* __restrict__ tiles, const int32_t* __restrict__ word_off, const T* __restrict__ z,
+            const int32_t* __restrict__ row_start, uint32_t* __restrict__ wk_topic, uint32_t* __restrict__ wk_count,
+            int32_t* __restrict__ wk_nnz, int32_t K, int* err)
+{
+    constexpr int CB = 12;  // count bits of a table entry: a tail word has at most SORT_TILE = 2048 tokens
+    static_assert(SORT_TILE < (1 << CB), "count bits");
+    extern __shared__ uint32_t word_smem[];
+    __shared__ uint32_t table[DK_SLOTS_PER_TOKEN * SORT_TILE];
+    __shared__ int32_t scan_tmp[33];
+    const int32_t bw = (K + 31) >> 5;
+    uint32_t* bitmap = word_smem;  // [bw] topics present in the word
+    uint32_t* before = word_smem + bw;  // [bw] set bits before each bitmap word
+    const int tid = threadIdx.x;
+    const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
+    for (int32_t w = s0; w < s1; ++w) {
+        const int32_t first = word_off[w], n = word_off[w + 1] - first;
+        if (n == 0) {
+            if (tid == 0) wk_nnz[w] = 0;
+            continue;
+        }
+        const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)n;
+        for (int32_t i = tid; i < bw; i += blockDim.x) bitmap[i] = 0;
+        for (uint32_t i = tid; i < cap; i += blockDim.x) table[i] = DK_EMPTY;
+        __syncthreads();
+        for (int32_t j = tid; j < n; j += blockDim.x) {
+            const uint32_t k = (uint32_t)__ldcs(z + first + j);
+            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+            atomicOr(&bitmap[k >> 5], 1u << (k & 31u));
+            if (dk_insert(table, cap, k, CB) == DK_EMPTY) atomicOr(err, ERR_ROW_OVERFLOW);
+        }
+        __syncthreads();
+        int32_t running = 0;
+        for (int32_t i0 = 0; i0 < bw; i0 += blockDim.x) {
+            const int32_t i = i0 + tid;
+            const int32_t c = i < bw ? __popc(bitmap[i]) : 0;
+            int32_t total;
+            const int32_t pos = block_scan_excl<int32_t>(c, scan_tmp, total);
+            if (i < bw) before[i] = (uint32_t)(running + pos);
+            running += total;
+        }
+        __syncthreads();
+        const int32_t out0 = row_start[w];
+        for (int32_t i = tid; i < bw; i += blockDim.x) {
+            uint32_t m = bitmap[i];
+            int32_t r = out0 + (int32_t)before[i];
+            while (m) {
+                const uint32_t k = 32u * (uint32_t)i + (uint32_t)(__ffs((int)m) - 1);
+                m &= m - 1u;
+                wk_topic[r] = k;
+                wk_count[r] = dk_lookup(table, cap, k, CB) & ((1u << CB) - 1u);
+                ++r;
+            }
+        }
+        if (tid == 0) wk_nnz[w] = running;
+        __syncthreads();
+    }
 }
 
 // Hot words: one CTA per chunk of a word's tokens; histogram of a window of
@@ -350,9 +416,15 @@ static int count_wk_t(Ctx& c)
     int launches = 0;
     const T* z = (const T*)v.zw;
     if (c.n_word_tiles) {
-        EmitWord e{v.row_start, v.wk_topic, v.wk_count, v.wk_nnz};
-        k_seg_count_sorted<T, EmitWord><<<c.n_word_tiles, 256, 0, c.stream>>>(
-            c.word_tiles, v.word_off, z, v.topic_bits, c.K, e, v.err);
+        if (c.K <= WORD_ROWS_BITMAP_MAX_K) {
+            const size_t smem = 2 * (size_t)((c.K + 31) / 32) * 4;
+            k_word_rows<T><<<c.n_word_tiles, 256, smem, c.stream>>>(c.word_tiles, v.word_off, z, v.row_start,
+                                                                   v.wk_topic, v.wk_count, v.wk_nnz, c.K, v.err);
+        } else {
+            EmitWord e{v.row_start, v.wk_topic, v.wk_count, v.wk_nnz};
+            k_seg_count_sorted<T, EmitWord><<<c.n_word_tiles, 256, 0, c.stream>>>(
+                c.word_tiles, v.word_off, z, v.topic_bits, c.K, e, v.err);
+        }
         ++launches;
     }
     if (c.n_dense) {

@@ -34,6 +34,7 @@ static_assert(DOC_TILE_TOKENS[0] == 3 * DOC_TILE_THREADS[0] && DOC_TILE_TOKENS[3
 // shared memory per token of a tile: 4 table slots, document offset, topic/slot (4 bytes each)
 constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DK_SLOTS_PER_TOKEN_HOST + 4 + 4;
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (32-bit bins)
+constexpr int WORD_ROWS_BITMAP_MAX_K = 16384;  // tail rows: topic bitmap up to this K, key sort above
 constexpr int HIST16_BINS = 106496;  // window of the per-chunk n_kw histogram (16-bit bins, 208 KB)
 constexpr int HIST_CHUNK = 16384;    // tokens per CTA in the histogram path
 static_assert(HIST_CHUNK < 65536, "the per-chunk histogram counts in 16 bits");
