@@ -23,7 +23,7 @@ typedef unsigned long long ull;
 
 template <bool BLOCK>
 struct Group {
-    ull* smem;  // CTA groups only: >= 33 entries
+    ull* smem;  // CTA groups only: >= 99 entries
     __device__ __forceinline__ int rank() const { return BLOCK ? (int)threadIdx.x : (int)(threadIdx.x & 31); }
     __device__ __forceinline__ int size() const { return BLOCK ? (int)blockDim.x : 32; }
     __device__ __forceinline__ void sync() const
@@ -35,12 +35,43 @@ struct Group {
         if (BLOCK) return block_reduce_sum<ull>(v, smem);
         return warp_reduce_sum<ull>(v);
     }
-    __device__ __forceinline__ ull scan_excl(ull v, ull& total) const
+    // Exclusive scans of three values at once (one pass, one set of barriers); v[] in, prefixes
+    // out in v[], totals in tot[].  CTA groups need 99 entries of `smem`.
+    __device__ __forceinline__ void scan_excl3(ull (&v)[3], ull (&tot)[3]) const
     {
-        if (BLOCK) return block_scan_excl<ull>(v, smem, total);
-        const ull incl = warp_scan_incl<ull>(v);
-        total = __shfl_sync(0xffffffffu, incl, 31);
-        return incl - v;
+        ull incl[3];
+#pragma unroll
+        for (int q = 0; q < 3; ++q) incl[q] = warp_scan_incl<ull>(v[q]);
+        if (!BLOCK) {
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                tot[q] = __shfl_sync(0xffffffffu, incl[q], 31);
+                v[q] = incl[q] - v[q];
+            }
+            return;
+        }
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+        __syncthreads();
+        if (lane == 31) {
+#pragma unroll
+            for (int q = 0; q < 3; ++q) smem[33 * q + warp] = incl[q];
+        }
+        __syncthreads();
+        if (warp == 0) {
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                const ull w = (lane < nw) ? smem[33 * q + lane] : 0ull;
+                const ull wi = warp_scan_incl<ull>(w);
+                smem[33 * q + lane] = wi - w;
+                if (lane == 31) smem[33 * q + 32] = wi;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            tot[q] = smem[33 * q + 32];
+            v[q] = smem[33 * q + warp] + incl[q] - v[q];
+        }
     }
 };
 
@@ -96,10 +127,10 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
         const ull a = valid ? (ull)n * (sc_w[i] >> sh) : 0;
         const bool light = valid && a <= W, heavy = valid && a > W;
         const ull def = light ? W - a : 0, sur = heavy ? a - W : 0;
-        ull c_tot, d_tot, e_tot;
-        const ull c_pre = g.scan_excl((light ? 1ull : 0ull) | (heavy ? (1ull << 32) : 0ull), c_tot);
-        const ull d_pre = g.scan_excl(def, d_tot);
-        const ull e_pre = g.scan_excl(sur, e_tot);
+        ull pre[3] = {(light ? 1ull : 0ull) | (heavy ? (1ull << 32) : 0ull), def, sur}, tot[3];
+        g.scan_excl3(pre, tot);
+        const ull c_pre = pre[0], d_pre = pre[1], e_pre = pre[2];
+        const ull c_tot = tot[0], d_tot = tot[1], e_tot = tot[2];
         if (valid) sc_w[i] = a;
         if (light) {
             const uint32_t l = L + (uint32_t)c_pre;
@@ -185,7 +216,7 @@ struct SparseWeight {
 
 __global__ void __launch_bounds__(1024) k_alias_dense(View v, ull* sc)
 {
-    __shared__ ull smem[33];
+    __shared__ ull smem[99];
     Group<true> g{smem};
     const int32_t K = v.K;
     DenseWeight wf{v.nk, v.beta, v.Vbeta};
@@ -230,7 +261,7 @@ __global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, ul
 __global__ void __launch_bounds__(LDA_ALIAS_BLOCK_THREADS)
 k_alias_sparse_block(View v, const int32_t* __restrict__ words, ull* sc_w, ull* sc_de, uint32_t* sc_item)
 {
-    __shared__ ull smem[33];
+    __shared__ ull smem[99];
     Group<true> g{smem};
     const int32_t w = words[blockIdx.x];
     const int32_t n = v.wk_nnz[w];
