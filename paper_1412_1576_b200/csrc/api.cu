@@ -552,19 +552,15 @@ int lda_set_assignments(lda_ctx* h, const int32_t* z, uint64_t seed, uint32_t sw
     if (c.N > 0 && !z) return fail(&c, LDA_EINVAL, "null assignments");
     int rc = check_device(c);
     if (rc) return rc;
-    int32_t* zdev = nullptr;
-    if (cudaMalloc(&zdev, (size_t)std::max<int64_t>(c.N, 1) * 4) != cudaSuccess) {
-        cudaGetLastError();
-        return fail(&c, LDA_ENOMEM, "device allocation failed");
-    }
-    if (c.N > 0 && cudaMemcpyAsync(zdev, z, (size_t)c.N * 4, cudaMemcpyHostToDevice, c.stream) != cudaSuccess) {
-        cudaFree(zdev);
+    // the record array (one word per token, only meaningful while the exported n_kd is valid)
+    // doubles as the staging buffer: no allocation here
+    int32_t* zdev = reinterpret_cast<int32_t*>(c.v.rec);
+    c.dk_valid = false;
+    if (c.N > 0 && cudaMemcpyAsync(zdev, z, (size_t)c.N * 4, cudaMemcpyHostToDevice, c.stream) != cudaSuccess)
         return cuda_fail(&c, "copying assignments");
-    }
     launch_spread_assignments(c, zdev);
     int bits = 0;
     rc = read_err(c, &bits);
-    cudaFree(zdev);
     if (rc) return rc;
     if (bits & ERR_TOPIC_RANGE) { c.inited = false; return fail(&c, LDA_ERANGE, "assignment outside [0,K)"); }
     c.seed = seed;
@@ -737,15 +733,11 @@ int lda_get_assignments(lda_ctx* h, int32_t* z_out)
     if (c.N == 0) return LDA_OK;
     int rc = check_device(c);
     if (rc) return rc;
-    int32_t* zdev = nullptr;
-    if (cudaMalloc(&zdev, (size_t)c.N * 4) != cudaSuccess) {
-        cudaGetLastError();
-        return fail(&c, LDA_ENOMEM, "device allocation failed");
-    }
+    int32_t* zdev = reinterpret_cast<int32_t*>(c.v.rec);  // staging, see lda_set_assignments
+    c.dk_valid = false;
     launch_export_assignments(c, zdev);
     cudaError_t e = cudaMemcpyAsync(z_out, zdev, (size_t)c.N * 4, cudaMemcpyDeviceToHost, c.stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
-    cudaFree(zdev);
     if (e != cudaSuccess) return cuda_fail(&c, "copying assignments");
     return LDA_OK;
 }
