@@ -217,6 +217,7 @@ typedef struct ldaref_ctx {
     int tables_valid;
     uint64_t seed;
     uint32_t sweep;      /* number of sweeps done since init */
+    int proposals;       /* 0 cycle (word, doc, word, ...), 1 word-proposal only, 2 doc-proposal only */
     int loaded, inited;
 } ldaref_ctx;
 
@@ -527,7 +528,9 @@ static int32_t run_chain(const ldaref_ctx *c, int64_t i, uint32_t sweep, int32_t
     for (int32_t m = 0; m < steps; ++m) {
         uint32_t ctr[4] = {(uint32_t)i, sweep, (uint32_t)m, 0u}, r[4];
         ldaref_philox4x32_10(ctr, key, r);
-        int kind = m & 1;
+        /* Section 4.3: the cycle alternates the two proposals; each alone is a valid MH kernel
+         * for the same target (the variants compared in Figure 11) */
+        int kind = c->proposals == 0 ? (m & 1) : c->proposals - 1;
         int32_t t = kind == 0 ? draw_word_proposal(c, c->word[i], r[0], r[1], r[2])
                               : draw_doc_proposal(c, c->doc_of[i], r[0], r[1]);
         if (t == s) continue;
@@ -537,6 +540,15 @@ static int32_t run_chain(const ldaref_ctx *c, int64_t i, uint32_t sweep, int32_t
         if (u * den < num) s = t;
     }
     return s;
+}
+
+/* Which proposals a chain uses (Section 4.3, Figure 11): 0 = cycle (default), 1 = word-proposal
+ * on every step, 2 = doc-proposal on every step. */
+int ldaref_set_proposals(ldaref_ctx *c, int mode)
+{
+    if (!c || mode < 0 || mode > 2) return LDAREF_EINVAL;
+    c->proposals = mode;
+    return LDAREF_OK;
 }
 
 /* `iters` sweeps.  During a sweep every count and every z that is read is the

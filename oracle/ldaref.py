@@ -61,6 +61,7 @@ def lib():
             L.ldaref_set_assignments.argtypes = [vp, _p(np.int32), C.c_uint64, C.c_uint32]
             L.ldaref_build_tables.argtypes = [vp]
             L.ldaref_sweep.argtypes = [vp, C.c_int32, C.c_int32]
+            L.ldaref_set_proposals.argtypes = [vp, C.c_int]
             L.ldaref_sample_tokens.argtypes = [vp, _p(np.int64), C.c_int64, C.c_int32,
                                                _p(np.int32)]
             L.ldaref_sweep_prefix.argtypes = [vp, C.c_int64, C.c_int32, _p(np.int32)]
@@ -152,6 +153,10 @@ class Oracle:
     def set_assignments(self, z, seed: int, sweep: int = 0):
         _check(lib().ldaref_set_assignments(self._h, np.ascontiguousarray(z, np.int32), seed,
                                             sweep), "set_assignments")
+
+    def set_proposals(self, mode: int):
+        """0 = cycle (word, doc, word, ...), 1 = word-proposal only, 2 = doc-proposal only."""
+        _check(lib().ldaref_set_proposals(self._h, mode), "set_proposals")
 
     def sweep(self, iters: int, mh_steps: int):
         _check(lib().ldaref_sweep(self._h, iters, mh_steps), "sweep")

@@ -269,6 +269,64 @@ def test_chain_with_zero_steps_keeps_state_and_one_step_is_word_proposal(tiny):
             assert got == (t if accept else z[i])
 
 
+def test_single_proposal_chains_still_land_on_eq4():
+    """Section 4.3: either proposal alone is a valid MH kernel for Eq. 4 (alpha, beta > 0 give
+    both full support); the word-only and doc-only chains of Fig. 11 have the same target."""
+    c, o, z, (n_wk, n_dk, n_k, doc) = _toy(V=10, K=5, D=5, L=10, seed=8)
+    wid = c.word_ids.numpy()
+    n_rep = 20_000
+    i = 28
+    p = _target(c, n_wk, n_dk, n_k, wid[i], doc[i], z[i])
+    pi = p / p.sum()
+    hists = {}
+    for mode in (1, 2):
+        o.set_proposals(mode)
+        h = np.zeros(c.K)
+        for rep in range(n_rep):
+            h[o.chain(i, 5000 + rep, 32)] += 1
+        hists[mode] = h
+        assert stats.chisquare(h, pi * n_rep).pvalue > 1e-4
+    assert not np.array_equal(hists[1], hists[2])     # different kernels, same target
+    with pytest.raises(Exception):
+        o.set_proposals(3)
+
+
+def _by_hand(o, i, z0, wid, doc, key, sweep, kinds):
+    s = int(z0)
+    for m, kind in enumerate(kinds):
+        r = ldaref.philox([i, sweep, m, 0], key)
+        if kind == 0:
+            t = o.word_proposal(int(wid[i]), int(r[0]), int(r[1]), int(r[2]))
+        else:
+            t = o.doc_proposal(int(doc[i]), int(r[0]), int(r[1]))
+        if t == s:
+            continue
+        num, den = o.accept_ratio(i, s, t, kind)
+        if (int(r[3]) / 2.0 ** 32) * den < num:
+            s = t
+    return s
+
+
+def test_proposal_modes_pick_the_proposal_of_each_step(tiny):
+    """Step m of a chain draws the word-proposal (Eq. 6-8) or the doc-proposal (Eq. 9-11):
+    cycle = word on even m, doc on odd m; the two single-proposal modes use one kind on every m."""
+    c, o, z, (_, _, _, doc) = tiny
+    wid = c.word_ids.numpy()
+    key = [SEED & 0xFFFFFFFF, SEED >> 32]
+    differ = 0
+    try:
+        for i in (1, 17, 333, 4242, 5000, 6001):
+            want = {}
+            for mode, kinds in ((0, (0, 1, 0)), (1, (0, 0, 0)), (2, (1, 1, 1))):
+                o.set_proposals(mode)
+                want[mode] = _by_hand(o, i, z[i], wid, doc, key, 9, kinds)
+                assert o.chain(i, 9, 3) == want[mode]
+            differ += len(set(want.values())) > 1
+    finally:
+        o.set_proposals(0)
+    assert differ > 0
+
+
 def test_sweep_is_frozen_and_order_independent(tiny_corpus):
     """Sampling tokens one by one from the sweep-start state equals the sweep."""
     c = tiny_corpus
