@@ -82,6 +82,19 @@ int lda_set_stream(lda_ctx* ctx, void* cuda_stream);
  *                  of one block, 20 bytes per token, stay in L2 while the document pass is on it)             */
 int lda_set_option(lda_ctx* ctx, const char* key, double value);
 
+/* Which proposal the steps of a token's chain draw (Section 4.3; the variants compared in
+ * Figure 11).  Either proposal alone is a valid MH kernel for Eq. 4; the cycle mixes best.
+ *   LDA_PROPOSALS_CYCLE  step m draws the word-proposal (Eq. 6-8) when m is even and the
+ *                        doc-proposal (Eq. 9-11) when m is odd (default)
+ *   LDA_PROPOSALS_WORD   every step draws the word-proposal
+ *   LDA_PROPOSALS_DOC    every step draws the doc-proposal
+ * May be called at any time between sweeps; it changes results (not only speed) from the next
+ * lda_sweep() on and keeps the Philox counter layout.  Other values: LDA_EINVAL. */
+#define LDA_PROPOSALS_CYCLE 0
+#define LDA_PROPOSALS_WORD 1
+#define LDA_PROPOSALS_DOC 2
+int lda_set_proposals(lda_ctx* ctx, int mode);
+
 /* Corpus in document order: token i has word word_ids[i]; document d owns tokens
  * [doc_offsets[d], doc_offsets[d+1]); doc_offsets has n_docs+1 entries, [0] = 0,
  * [n_docs] = n_tokens; empty documents are legal.  Builds the word-sorted token
@@ -103,8 +116,9 @@ int lda_init(lda_ctx* ctx, uint64_t seed);
 int lda_set_assignments(lda_ctx* ctx, const int32_t* z, uint64_t seed, uint32_t sweep);
 
 /* `iters` frozen-counts sweeps of `mh_steps` proposals per token (Section 4.2-4.3,
- * Eq. 6-13; Section 6 "immutable model").  Randomness: one Philox block per
- * (token, sweep, step), counter (token, sweep, step, 0). */
+ * Eq. 6-13; Section 6 "immutable model"), the proposal of each step chosen by
+ * lda_set_proposals().  Randomness: one Philox block per (token, sweep, step), counter
+ * (token, sweep, step, 0). */
 int lda_sweep(lda_ctx* ctx, int32_t iters, int32_t mh_steps);
 
 /* Collapsed joint log p(w,z): word part + document part (Section 7.2, Figure 11).

@@ -20,7 +20,7 @@ LDA_OK, LDA_EINVAL, LDA_ERANGE, LDA_ESTATE, LDA_ENOMEM, LDA_ECUDA, LDA_EINTERNAL
 LDA_NK, LDA_NWK, LDA_NDK = 0, 1, 2
 
 EXPORTS = [
-    "lda_create", "lda_set_stream", "lda_set_option", "lda_load_corpus", "lda_load_corpus_device",
+    "lda_create", "lda_set_stream", "lda_set_option", "lda_set_proposals", "lda_load_corpus", "lda_load_corpus_device",
     "lda_init", "lda_set_assignments", "lda_sweep", "lda_loglik", "lda_get_counts",
     "lda_get_assignments", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
     "lda_dense_table_noalloc",
@@ -70,6 +70,7 @@ def load_library(path: str | None = None):
     L.lda_create.argtypes = [i32, i32, dbl, dbl, C.POINTER(vp)]
     L.lda_set_stream.argtypes = [vp, vp]
     L.lda_set_option.argtypes = [vp, C.c_char_p, dbl]
+    L.lda_set_proposals.argtypes = [vp, C.c_int]
     L.lda_load_corpus.argtypes = [vp, vp, i64, vp, i64]
     L.lda_load_corpus_device.argtypes = [vp, vp, i64, vp, i64]
     L.lda_init.argtypes = [vp, u64]
@@ -107,6 +108,13 @@ def lda_set_stream(h, cuda_stream):
 
 def lda_set_option(h, key, value):
     return load_library().lda_set_option(h, key.encode(), float(value))
+
+
+PROPOSALS_CYCLE, PROPOSALS_WORD, PROPOSALS_DOC = 0, 1, 2
+
+
+def lda_set_proposals(h, mode):
+    return load_library().lda_set_proposals(h, int(mode))
 
 
 def lda_load_corpus(h, word_ids, doc_offsets):
@@ -254,6 +262,10 @@ class LightLDA:
 
     def set_assignments(self, z, seed: int, sweep: int = 0):
         self._ck(lda_set_assignments(self._h, z, seed, sweep), "lda_set_assignments")
+
+    def set_proposals(self, mode: int):
+        """PROPOSALS_CYCLE (word, doc, word, ...), PROPOSALS_WORD or PROPOSALS_DOC (Section 4.3)."""
+        self._ck(lda_set_proposals(self._h, mode), "lda_set_proposals")
 
     def sweep(self, iters: int, mh_steps: int):
         self._ck(lda_sweep(self._h, iters, mh_steps), "lda_sweep")

@@ -101,25 +101,28 @@ static void free_corpus(Ctx& c)
 // Buffers the passes of the MH step hand results to each other in; sized by the number of steps.
 int lda::ensure_exchange(Ctx& c, int mh_steps)
 {
-    if (c.N == 0 || (mh_steps <= c.side_steps && c.v.dside)) return LDA_OK;
+    if (c.N == 0 || (mh_steps <= c.side_steps && c.side_mode == c.proposals && c.v.dside)) return LDA_OK;
     auto drop = [&](void* p) {
         if (!p) return;
         for (size_t i = 0; i < c.allocs.size(); ++i)
             if (c.allocs[i] == p) { c.allocs.erase(c.allocs.begin() + i); break; }
         cudaFree(p);
     };
-    auto bytes_for = [&](int steps, size_t& prop_b, size_t& side_b, size_t& ua_b, int& stride) {
+    auto bytes_for = [&](int mode, int steps, size_t& prop_b, size_t& side_b, size_t& ua_b, int& stride) {
         const size_t zt = c.wide_topics ? 4 : 2, n = (size_t)c.N;
-        stride = (1 + steps + steps / 2 + 3) & ~3;  // own, one word per step, one uniform per doc step
-        prop_b = zt * (((size_t)steps + 1) / 2) * n;
+        const int n_word = mode == LDA_PROPOSALS_CYCLE ? (steps + 1) / 2 : mode == LDA_PROPOSALS_WORD ? steps : 0;
+        const int n_doc = steps - n_word;
+        const size_t planes = (size_t)(n_word > 0 ? n_word : 1);
+        stride = (1 + steps + n_doc + 3) & ~3;  // own, one word per step, one uniform per doc step
+        prop_b = zt * planes * n;
         side_b = 4 * (size_t)stride * n;
-        ua_b = 4 * (((size_t)steps + 1) / 2) * n;
+        ua_b = 4 * planes * n;
     };
     cudaStreamSynchronize(c.stream);
     size_t pb = 0, sb = 0, ub = 0;
     int stride = 0;
     if (c.side_steps) {
-        bytes_for(c.side_steps, pb, sb, ub, stride);
+        bytes_for(c.side_mode, c.side_steps, pb, sb, ub, stride);
         c.device_bytes -= (int64_t)(pb + sb + ub);
     }
     drop(c.v.prop);
@@ -129,7 +132,7 @@ int lda::ensure_exchange(Ctx& c, int mh_steps)
     c.v.dside = nullptr;
     c.v.ua_w = nullptr;
     c.side_steps = 0;
-    bytes_for(mh_steps, pb, sb, ub, stride);
+    bytes_for(c.proposals, mh_steps, pb, sb, ub, stride);
     c.v.prop = dev_alloc(c, pb);
     c.v.dside = (uint32_t*)dev_alloc(c, sb);
     c.v.ua_w = (uint32_t*)dev_alloc(c, ub);
@@ -139,6 +142,7 @@ int lda::ensure_exchange(Ctx& c, int mh_steps)
     }
     c.v.side_stride = stride;
     c.side_steps = mh_steps;
+    c.side_mode = c.proposals;
     return LDA_OK;
 }
 
@@ -481,6 +485,16 @@ int lda_set_option(lda_ctx* h, const char* key, double value)
         return LDA_OK;
     }
     return fail(&c, LDA_EINVAL, "unknown option");
+}
+
+int lda_set_proposals(lda_ctx* h, int mode)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (mode != LDA_PROPOSALS_CYCLE && mode != LDA_PROPOSALS_WORD && mode != LDA_PROPOSALS_DOC)
+        return fail(&c, LDA_EINVAL, "unknown proposal mode");
+    c.proposals = mode;  // the exchange buffers are laid out again by the next sweep
+    return LDA_OK;
 }
 
 int lda_load_corpus(lda_ctx* h, const int32_t* word_ids, int64_t n_tokens, const int64_t* doc_offsets,

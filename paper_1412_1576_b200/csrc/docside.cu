@@ -39,7 +39,7 @@ __device__ __forceinline__ void load_topic_pair(const int32_t* zbm, uint32_t bm,
 // block-major index `bm`.
 //   tab     : the document's table, 4 * doc_len slots
 //   slot_at : slot holding the topic of the document's j-th token
-template <typename T, class SlotAt>
+template <typename T, int MODE, class SlotAt>
 __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* tab, uint32_t tok, uint32_t doc_len,
                                                uint32_t own, uint32_t t_first, uint32_t bm, const SlotAt& slot_at,
                                                uint2 key, uint32_t sweep, int32_t mh_steps)
@@ -58,26 +58,36 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
         else if (at == 3) w3 = val;
         else __stcs(out + at, val);
     };
-    for (int32_t st = 0; st < mh_steps; st += 2) {
-        // word-proposal of step st: n_kd at the topic pass 1 drew
-        const uint32_t t1 = st == 0 ? t_first : (uint32_t)__ldcg(prop + (size_t)(st >> 1) * N + bm);
+    // word-proposal of step st, the wi-th of its kind: n_kd at the topic pass 1 drew
+    auto word_step = [&](int32_t st, int32_t wi) {
+        const uint32_t t1 = wi == 0 ? t_first : (uint32_t)__ldcg(prop + (size_t)wi * N + bm);
         const uint32_t e1 = dk_lookup(tab, cap, t1, cb);
         put(1 + st, e1 ? e1 : t1 << cb);
-        if (st + 1 < mh_steps) {
-            // doc-proposal of step st+1
-            const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)(st + 1), 0u), key);
-            const double uu = __dmul_rn((double)r.x, INV_2_32);
-            uint32_t o2;
-            if (__dmul_rn(uu, __dadd_rn(n_d, v.Kalpha)) < n_d) {
-                o2 = tab[slot_at(scale_to_range(r.y, doc_len))];
-            } else {
-                const uint32_t t2 = scale_to_range(r.y, (uint32_t)v.K);
-                const uint32_t e2 = dk_lookup(tab, cap, t2, cb);
-                o2 = e2 ? e2 : t2 << cb;
-            }
-            put(2 + st, o2);
-            put(1 + mh_steps + (st >> 1), r.w);  // the step's acceptance uniform
+    };
+    // doc-proposal of step st, the di-th of its kind
+    auto doc_step = [&](int32_t st, int32_t di) {
+        const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)st, 0u), key);
+        const double uu = __dmul_rn((double)r.x, INV_2_32);
+        uint32_t o2;
+        if (__dmul_rn(uu, __dadd_rn(n_d, v.Kalpha)) < n_d) {
+            o2 = tab[slot_at(scale_to_range(r.y, doc_len))];
+        } else {
+            const uint32_t t2 = scale_to_range(r.y, (uint32_t)v.K);
+            const uint32_t e2 = dk_lookup(tab, cap, t2, cb);
+            o2 = e2 ? e2 : t2 << cb;
         }
+        put(1 + st, o2);
+        put(1 + mh_steps + di, r.w);  // the step's acceptance uniform
+    };
+    if (MODE == LDA_PROPOSALS_CYCLE) {
+        for (int32_t st = 0; st < mh_steps; st += 2) {
+            word_step(st, st >> 1);
+            if (st + 1 < mh_steps) doc_step(st + 1, st >> 1);
+        }
+    } else if (MODE == LDA_PROPOSALS_WORD) {
+        for (int32_t st = 0; st < mh_steps; ++st) word_step(st, st);
+    } else {
+        for (int32_t st = 0; st < mh_steps; ++st) doc_step(st, st);
     }
     __stcs(reinterpret_cast<uint4*>(out), make_uint4(own, w1, w2, w3));
 }
@@ -85,7 +95,7 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
 // `cap` = tokens a tile can hold (the shared-memory carve-up) = DOC_TILE_ROUNDS x blockDim.x: a
 // thread owns at most DOC_TILE_ROUNDS tokens and keeps what it read about them in registers across
 // the phases.  Small tiles keep many CTAs per SM, which is what hides the gathers of the first phase.
-template <typename T, int THREADS>
+template <typename T, int THREADS, int MODE>
 __global__ void __launch_bounds__(THREADS, 1536 / THREADS)
 k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
 {
@@ -151,7 +161,7 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
             const uint32_t* tab = slots + DK_SLOTS_PER_TOKEN * first[r];
             const uint32_t* slot_of = slot_s + first[r];
             auto slot_at = [slot_of](uint32_t jj) { return slot_of[jj]; };
-            doc_side_token<T>(v, tab, (uint32_t)(base + j), (uint32_t)len[r], tab[z[r]], t1[r], bm[r], slot_at, key,
+            doc_side_token<T, MODE>(v, tab, (uint32_t)(base + j), (uint32_t)len[r], tab[z[r]], t1[r], bm[r], slot_at, key,
                               sweep, mh_steps);
         }
     }
@@ -160,7 +170,7 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
 // Documents longer than a tile: one CTA per document; the table lives in the document's range of
 // the global slot array and the slot indices in its range of the record array (both are scratch
 // here: the exported n_kd tables are rebuilt on demand).
-template <typename T>
+template <typename T, int MODE>
 __global__ void __launch_bounds__(512)
 k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32_t sweep, int32_t mh_steps)
 {
@@ -186,7 +196,7 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
     auto slot_at = [slot_of](uint32_t j) { return slot_of[j]; };
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
         const uint32_t bm = v.bm_of_tok[first + j];
-        doc_side_token<T>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)zbm[2 * (size_t)bm + 1], bm,
+        doc_side_token<T, MODE>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)zbm[2 * (size_t)bm + 1], bm,
                           slot_at, key, sweep, mh_steps);
     }
 }
@@ -196,30 +206,44 @@ size_t doc_tile_smem_bytes(int tile_tokens) { return (size_t)tile_tokens * DOC_T
 void set_doc_smem_limits()
 {
     const int bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
-    cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    cudaFuncSetAttribute(k_doc_tile<int32_t, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024, LDA_PROPOSALS_CYCLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<int32_t, 1024, LDA_PROPOSALS_CYCLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024, LDA_PROPOSALS_WORD>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<int32_t, 1024, LDA_PROPOSALS_WORD>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024, LDA_PROPOSALS_DOC>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<int32_t, 1024, LDA_PROPOSALS_DOC>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
-template <typename T>
-static int doc_side_t(Ctx& c, int mh_steps)
+template <typename T, int MODE>
+static int doc_side_tm(Ctx& c, int mh_steps)
 {
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     int launches = 0;
     if (c.n_doc_tiles) {
         const size_t smem = doc_tile_smem_bytes(c.doc_tile);
         switch (c.doc_threads) {
-            case 128: k_doc_tile<T, 128><<<c.n_doc_tiles, 128, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
-            case 256: k_doc_tile<T, 256><<<c.n_doc_tiles, 256, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
-            case 512: k_doc_tile<T, 512><<<c.n_doc_tiles, 512, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
-            default: k_doc_tile<T, 1024><<<c.n_doc_tiles, 1024, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            case 128: k_doc_tile<T, 128, MODE><<<c.n_doc_tiles, 128, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            case 256: k_doc_tile<T, 256, MODE><<<c.n_doc_tiles, 256, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            case 512: k_doc_tile<T, 512, MODE><<<c.n_doc_tiles, 512, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            default: k_doc_tile<T, 1024, MODE><<<c.n_doc_tiles, 1024, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
         }
         ++launches;
     }
     if (c.n_long_docs) {
-        k_long_doc_tile<T><<<c.n_long_docs, 512, 0, c.stream>>>(c.v, c.long_docs, key, c.sweep, mh_steps);
+        k_long_doc_tile<T, MODE><<<c.n_long_docs, 512, 0, c.stream>>>(c.v, c.long_docs, key, c.sweep, mh_steps);
         ++launches;
     }
     return launches;
+}
+
+template <typename T>
+static int doc_side_t(Ctx& c, int mh_steps)
+{
+    switch (c.proposals) {
+        case LDA_PROPOSALS_WORD: return doc_side_tm<T, LDA_PROPOSALS_WORD>(c, mh_steps);
+        case LDA_PROPOSALS_DOC: return doc_side_tm<T, LDA_PROPOSALS_DOC>(c, mh_steps);
+        default: return doc_side_tm<T, LDA_PROPOSALS_CYCLE>(c, mh_steps);
+    }
 }
 
 int launch_doc_side(Ctx& c, int mh_steps)

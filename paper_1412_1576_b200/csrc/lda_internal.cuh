@@ -10,6 +10,19 @@
 
 namespace lda {
 
+// The proposal schedule of a chain (Section 4.3): whether step m draws the doc-proposal, and the
+// running index of step m among the steps of its own kind.
+template <int MODE>
+__host__ __device__ constexpr bool step_is_doc(int m)
+{
+    return MODE == LDA_PROPOSALS_CYCLE ? (m & 1) != 0 : MODE == LDA_PROPOSALS_DOC;
+}
+template <int MODE>
+__host__ __device__ constexpr int step_kind_index(int m)
+{
+    return MODE == LDA_PROPOSALS_CYCLE ? m >> 1 : m;
+}
+
 // Device error word bits (set by kernels, read by the host after a sweep).
 enum : int {
     ERR_WORD_RANGE = 1,   // a word id outside [0,V) at load
@@ -109,6 +122,8 @@ struct Ctx {
     int block_shift = 22;  // log2 of the tokens per block of the block-major order
     int doc_tile = DOC_TILE_TOKENS[0], doc_threads = DOC_TILE_THREADS[0];  // shape of the document tiles
     int side_steps = 0;    // number of steps the exchange buffers are allocated for
+    int side_mode = 0;     // ... and the proposal schedule they are laid out for
+    int proposals = 0;     // LDA_PROPOSALS_*: which proposal each step of a chain draws
     double dense_frac = 0.05;
     double dense_min_tf = 64;
     bool loaded = false, inited = false, tables_valid = false;

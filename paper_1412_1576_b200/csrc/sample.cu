@@ -206,10 +206,11 @@ struct ColdTile {
 };
 
 // --- pass 1: word-proposals (word order) ---------------------------------------------------------
-// Draws the topic proposed by every word-proposal step (even steps, Eq. 6) of the tile's tokens.
+// Draws the topic proposed by every word-proposal step (Eq. 6; the even steps of the cycle) of the
+// tile's tokens.
 // A proposal depends on (token, sweep, step) and the frozen tables only, never on the chain's
 // state, so all of them can be drawn before anything is accepted.
-template <typename T, class Tile>
+template <typename T, int MODE, class Tile>
 __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, const int32_t p_begin,
                                                const int32_t p_end, const int32_t nthreads, const uint2 key,
                                                const uint32_t sweep, const int32_t mh_steps)
@@ -219,16 +220,17 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
         const uint32_t tok = __ldcs(v.tok_orig + p);
         const uint32_t at = __ldcs(v.inv + p);  // the document-side pass reads block-major
         const typename Tile::Ref w = tile.ref(p - p_begin);
-        for (int32_t m = 0; m < mh_steps; m += 2) {
+        for (int32_t m = 0; m < mh_steps; m += (MODE == LDA_PROPOSALS_CYCLE ? 2 : 1)) {
+            const int32_t wi = step_kind_index<MODE>(m);
             const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)m, 0u), key);
             const Draw d = tile.draw_issue(w, v, r);
             uint32_t t;
             int32_t n_tw;
             tile.draw_finish(w, d, t, n_tw);
             // the first proposal goes beside the token's topic, the later ones to arrays of their own
-            if (m == 0) __stcs(reinterpret_cast<T*>(v.zbm) + 2 * (size_t)at + 1, (T)t);
-            else __stcs(prop + (size_t)(m >> 1) * v.N + at, (T)t);
-            __stcs(v.ua_w + (size_t)(m >> 1) * v.N + p, r.w);  // the step's acceptance uniform, for pass 3
+            if (wi == 0) __stcs(reinterpret_cast<T*>(v.zbm) + 2 * (size_t)at + 1, (T)t);
+            else __stcs(prop + (size_t)wi * v.N + at, (T)t);
+            __stcs(v.ua_w + (size_t)wi * v.N + p, r.w);  // the step's acceptance uniform, for pass 3
         }
     }
 }
@@ -236,7 +238,7 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
 // --- pass 3: accept / reject (word order) -----------------------------------------------------------
 // Runs the chain of every token of the tile: everything the document side contributes was
 // gathered by pass 2, the word side comes from the tile's staged rows.
-template <typename T, int CH, class Tile>
+template <typename T, int CH, int MODE, class Tile>
 __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const int32_t p_begin, const int32_t p_end,
                                               const int32_t nthreads, const uint2 key, const uint32_t sweep,
                                               const int32_t mh_steps)
@@ -244,7 +246,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
     const int cb = v.count_bits;
     const uint32_t cmask = (1u << cb) - 1u;
     const double alpha = v.alpha, beta = v.beta, Vb = v.Vbeta;
-    static_assert(CH % 2 == 0, "a group of steps starts on a word-proposal");
+    static_assert(CH % 2 == 0, "in the cycle a group of steps starts on a word-proposal");
     const size_t N = (size_t)v.N;
     T* zw = reinterpret_cast<T*>(v.zw);
     bool bad = false;
@@ -282,8 +284,8 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                     e[i] = side_word(1 + m0 + i);
                     // acceptance uniform: word 3 of the step's Philox block, drawn by the pass that made
                     // the proposal (pass 1: word steps, pass 2: doc steps) and left for this one
-                    ua[i] = (i & 1) ? side_word(1 + mh_steps + ((m0 + i) >> 1))
-                                    : __ldcs(v.ua_w + (size_t)((m0 + i) >> 1) * N + p);
+                    ua[i] = step_is_doc<MODE>(i) ? side_word(1 + mh_steps + step_kind_index<MODE>(m0 + i))
+                                                 : __ldcs(v.ua_w + (size_t)step_kind_index<MODE>(m0 + i) * N + p);
                 }
             }
             if (m0 == 0) {
@@ -316,7 +318,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 double den = __dadd_rn(u32_to_double((uint32_t)(n_sd - e_s)), alpha);
                 den = __dmul_rn(den, __dadd_rn(u32_to_double((uint32_t)(n_sw - e_s)), beta));
                 den = __dmul_rn(den, __dadd_rn(u32_to_double((uint32_t)(n_t[i] - e_t)), Vb));
-                if ((i & 1) == 0) {
+                if (!step_is_doc<MODE>(i)) {
                     num = __dmul_rn(num, __dadd_rn(u32_to_double((uint32_t)n_sw), beta));
                     num = __dmul_rn(num, __dadd_rn(u32_to_double((uint32_t)n_t[i]), Vb));
                     den = __dmul_rn(den, __dadd_rn(u32_to_double((uint32_t)n_tw[i]), beta));
@@ -341,7 +343,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
 }
 
 // Hot words: tile = (word, first token, count).  ACCEPT = false: pass 1, true: pass 3.
-template <typename T, int CH, bool STAGED, bool ACCEPT>
+template <typename T, int CH, bool STAGED, bool ACCEPT, int MODE>
 __global__ void __launch_bounds__(ACCEPT ? ACCEPT_THREADS : PROPOSE_THREADS,
                                   ACCEPT ? LDA_ACCEPT_MIN_CTAS : LDA_PROPOSE_MIN_CTAS)
 k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
@@ -376,13 +378,13 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     tile.mix = __ldg(v.mix32 + w);
     tile.bar = &bar;
     tile.ready = !(STAGED && ACCEPT);
-    if (ACCEPT) accept_tokens<T, CH>(v, tile, p0, p0 + cnt, ACCEPT_THREADS, key, sweep, mh_steps);
-    else propose_tokens<T>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
+    if (ACCEPT) accept_tokens<T, CH, MODE>(v, tile, p0, p0 + cnt, ACCEPT_THREADS, key, sweep, mh_steps);
+    else propose_tokens<T, MODE>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
     // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one
 }
 
 // Tail words: tile = range of whole words [w0, w1) with at most COLD_TILE tokens.
-template <typename T, int CH, bool ACCEPT>
+template <typename T, int CH, bool ACCEPT, int MODE>
 __global__ void __launch_bounds__(COLD_THREADS)
 k_word_cold(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
 {
@@ -416,8 +418,8 @@ k_word_cold(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep
     }
     __syncthreads();
     ColdTile tile{woff_s, rs_s, nnz_s, mix_s, topic_s, count_s, thr_s, idx_s, nw, v.nk};
-    if (ACCEPT) accept_tokens<T, CH>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
-    else propose_tokens<T>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
+    if (ACCEPT) accept_tokens<T, CH, MODE>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
+    else propose_tokens<T, MODE>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
 }
 
 // z_i uniform on {0..K-1}: Philox counter (token, 0, 0, 1), word 0.
@@ -469,21 +471,21 @@ static int grid_for(int64_t n, int block)
     return g < 1 ? 1 : (int)g;
 }
 
-template <typename T, int CH>
+template <typename T, int CH, int MODE>
 static int sample_tc(Ctx& c, int mh_steps)
 {
     const View& v = c.v;
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     const bool staged = c.K <= HOT_STAGE_MAX_K;
     int launches = 0;
-    // pass 1: word-proposals
-    if (c.n_hot_tiles) {
-        k_word_hot<T, CH, false, false><<<c.n_hot_tiles, PROPOSE_THREADS, 0, c.stream>>>(v, c.hot_tiles, key, c.sweep,
+    // pass 1: word-proposals (none in a doc-proposal-only chain)
+    if (MODE != LDA_PROPOSALS_DOC && c.n_hot_tiles) {
+        k_word_hot<T, CH, false, false, MODE><<<c.n_hot_tiles, PROPOSE_THREADS, 0, c.stream>>>(v, c.hot_tiles, key, c.sweep,
                                                                                     mh_steps);
         ++launches;
     }
-    if (c.n_cold_tiles) {
-        k_word_cold<T, CH, false><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
+    if (MODE != LDA_PROPOSALS_DOC && c.n_cold_tiles) {
+        k_word_cold<T, CH, false, MODE><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
                                                                                 mh_steps);
         ++launches;
     }
@@ -494,15 +496,15 @@ static int sample_tc(Ctx& c, int mh_steps)
     cudaEventRecord(c.ev[9], c.stream);
     if (c.n_hot_tiles) {
         if (staged)
-            k_word_hot<T, CH, true, true><<<c.n_hot_tiles, ACCEPT_THREADS, (size_t)v.dense_stride * 8, c.stream>>>(
+            k_word_hot<T, CH, true, true, MODE><<<c.n_hot_tiles, ACCEPT_THREADS, (size_t)v.dense_stride * 8, c.stream>>>(
                 v, c.hot_tiles, key, c.sweep, mh_steps);
         else
-            k_word_hot<T, CH, false, true><<<c.n_hot_tiles, ACCEPT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
+            k_word_hot<T, CH, false, true, MODE><<<c.n_hot_tiles, ACCEPT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
                                                                                        c.sweep, mh_steps);
         ++launches;
     }
     if (c.n_cold_tiles) {
-        k_word_cold<T, CH, true><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
+        k_word_cold<T, CH, true, MODE><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
                                                                                mh_steps);
         ++launches;
     }
@@ -513,7 +515,17 @@ static int sample_tc(Ctx& c, int mh_steps)
 template <typename T>
 static int sample_t(Ctx& c, int mh_steps)
 {
-    return mh_steps <= 2 ? sample_tc<T, 2>(c, mh_steps) : sample_tc<T, 4>(c, mh_steps);
+    switch (c.proposals) {
+        case LDA_PROPOSALS_WORD:
+            return mh_steps <= 2 ? sample_tc<T, 2, LDA_PROPOSALS_WORD>(c, mh_steps)
+                                 : sample_tc<T, 4, LDA_PROPOSALS_WORD>(c, mh_steps);
+        case LDA_PROPOSALS_DOC:
+            return mh_steps <= 2 ? sample_tc<T, 2, LDA_PROPOSALS_DOC>(c, mh_steps)
+                                 : sample_tc<T, 4, LDA_PROPOSALS_DOC>(c, mh_steps);
+        default:
+            return mh_steps <= 2 ? sample_tc<T, 2, LDA_PROPOSALS_CYCLE>(c, mh_steps)
+                                 : sample_tc<T, 4, LDA_PROPOSALS_CYCLE>(c, mh_steps);
+    }
 }
 
 // Reads the records and tables of the sweep-start state; writes zw and zbm.
@@ -526,8 +538,12 @@ int launch_sample(Ctx& c, int mh_steps)
 template <typename T, int CH>
 static void set_hot_limit()
 {
-    cudaFuncSetAttribute(k_word_hot<T, CH, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         HOT_STAGE_MAX_K * 8);
+    cudaFuncSetAttribute(k_word_hot<T, CH, true, true, LDA_PROPOSALS_CYCLE>,
+                         cudaFuncAttributeMaxDynamicSharedMemorySize, HOT_STAGE_MAX_K * 8);
+    cudaFuncSetAttribute(k_word_hot<T, CH, true, true, LDA_PROPOSALS_WORD>,
+                         cudaFuncAttributeMaxDynamicSharedMemorySize, HOT_STAGE_MAX_K * 8);
+    cudaFuncSetAttribute(k_word_hot<T, CH, true, true, LDA_PROPOSALS_DOC>,
+                         cudaFuncAttributeMaxDynamicSharedMemorySize, HOT_STAGE_MAX_K * 8);
 }
 
 void set_sample_smem_limits()

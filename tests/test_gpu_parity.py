@@ -176,6 +176,45 @@ def test_hot_words_with_unstaged_rows_and_odd_step_counts():
     _assert_same_counts(g, o)
 
 
+@pytest.mark.parametrize("mode", [binding.PROPOSALS_WORD, binding.PROPOSALS_DOC])
+def test_single_proposal_chains(tiny_corpus, small_corpus, mode):
+    """Word-proposal-only and doc-proposal-only chains (Section 4.3, Fig. 11): every token agrees
+    with the oracle's chain of the same schedule, at several step counts, on hot and tail words."""
+    for c, sweeps in ((tiny_corpus, 3), (small_corpus, 2)):
+        g, o = _pair(c, seed=11)
+        g.set_proposals(mode)
+        o.set_proposals(mode)
+        for mh_steps in (2, 1, 5, 4):
+            g.sweep(sweeps, mh_steps)
+            o.sweep(sweeps, mh_steps)
+            assert np.array_equal(g.get_assignments(), o.get_assignments()), mh_steps
+        _assert_same_counts(g, o)
+        # back to the cycle on the same context: the exchange buffers are laid out again
+        g.set_proposals(binding.PROPOSALS_CYCLE)
+        o.set_proposals(0)
+        g.sweep(1, 2)
+        o.sweep(1, 2)
+        assert np.array_equal(g.get_assignments(), o.get_assignments())
+        for a, b in zip(g.loglik(), o.loglik()):
+            assert a == pytest.approx(b, rel=1e-10)
+
+
+def test_single_proposal_chains_wide_topics_long_documents_unstaged_rows():
+    c = synth.generate(V=300, K=70_000, D=40, length=("fixed", 100), zipf_s=1.0, alpha=0.01, beta=0.01,
+                       seed=4)
+    c2 = synth.generate(V=50, K=40, D=6, length=("fixed", 5000), zipf_s=1.0, alpha=0.1, beta=0.01, seed=5)
+    c3 = synth.generate(V=40, K=20_000, D=300, length=("fixed", 400), zipf_s=1.0, alpha=0.05, beta=0.01, seed=8)
+    for c in (c, c2, c3):
+        for mode in (binding.PROPOSALS_WORD, binding.PROPOSALS_DOC):
+            g, o = _pair(c, seed=3)
+            g.set_proposals(mode)
+            o.set_proposals(mode)
+            g.sweep(2, 3)
+            o.sweep(2, 3)
+            assert np.array_equal(g.get_assignments(), o.get_assignments()), mode
+            _assert_same_counts(g, o)
+
+
 @pytest.mark.parametrize("block_log2", [10, 14])
 def test_block_size_is_invisible(small_corpus, block_log2):
     """The block-major exchange order is a layout choice: any block size gives the same sweep."""
@@ -317,6 +356,9 @@ def test_error_paths():
     g.init(0)
     with pytest.raises(binding.LdaError) as e:
         g.sweep(1, 0)
+    assert e.value.status == binding.LDA_EINVAL
+    with pytest.raises(binding.LdaError) as e:
+        g.set_proposals(3)
     assert e.value.status == binding.LDA_EINVAL
     g.sweep(1, 2)   # the context is still usable after the refused calls
 
