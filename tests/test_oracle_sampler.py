@@ -416,3 +416,24 @@ def test_loglik_rises_towards_sequential_gibbs_level(tiny_corpus):
     z.set_assignments(zz, 3)
     ll_gibbs = z.loglik()[0]
     assert abs(ll_mh - ll_gibbs) < 0.05 * abs(ll_gibbs)
+
+
+def test_each_single_proposal_neglects_one_part_of_the_likelihood():
+    """Section 4.3 / Fig. 11, qualitative (the paper prints no number): with few MH steps the
+    word-proposal alone leaves the document part of the likelihood behind and the doc-proposal
+    alone the word part; the cycle is between the two on both parts."""
+    cfg = dict(synth.CONFIGS["small"])
+    cfg["D"] = 500
+    c = synth.generate(seed=0, **cfg)
+    parts = {}
+    for mode in (0, 1, 2):
+        o = ldaref.Oracle(c.V, c.K, c.alpha, c.beta)
+        o.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+        o.init(5)
+        o.set_proposals(mode)
+        o.sweep(40, 2)
+        _, parts[mode, "word"], parts[mode, "doc"] = o.loglik()
+    assert parts[1, "word"] > parts[0, "word"] > parts[2, "word"]
+    assert parts[2, "doc"] > parts[0, "doc"] > parts[1, "doc"]
+    # the neglected part is far behind, the other one only a little ahead
+    assert parts[0, "word"] - parts[2, "word"] > 5 * (parts[2, "doc"] - parts[0, "doc"])
