@@ -95,10 +95,12 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
 // `cap` = tokens a tile can hold (the shared-memory carve-up) = DOC_TILE_ROUNDS x blockDim.x: a
 // thread owns at most DOC_TILE_ROUNDS tokens and keeps what it read about them in registers across
 // the phases.  Small tiles keep many CTAs per SM, which is what hides the gathers of the first phase.
-template <typename T, int THREADS, int MODE>
+// FIXED > 0: the number of steps is this compile-time constant (the argument is ignored).
+template <typename T, int THREADS, int MODE, int FIXED>
 __global__ void __launch_bounds__(THREADS, 1536 / THREADS)
-k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
+k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps_arg)
 {
+    const int32_t mh_steps = FIXED > 0 ? FIXED : mh_steps_arg;
     constexpr int cap = DOC_TILE_ROUNDS * THREADS;
     extern __shared__ __align__(16) uint32_t doc_smem[];
     uint32_t* slots = doc_smem;                                  // [4 * cap] the tile's tables
@@ -170,10 +172,11 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
 // Documents longer than a tile: one CTA per document; the table lives in the document's range of
 // the global slot array and the slot indices in its range of the record array (both are scratch
 // here: the exported n_kd tables are rebuilt on demand).
-template <typename T, int MODE>
+template <typename T, int MODE, int FIXED>
 __global__ void __launch_bounds__(512)
-k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32_t sweep, int32_t mh_steps)
+k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32_t sweep, int32_t mh_steps_arg)
 {
+    const int32_t mh_steps = FIXED > 0 ? FIXED : mh_steps_arg;
     const int32_t d = long_docs[blockIdx.x];
     const int32_t first = v.doc_off[d], cnt = v.doc_off[d + 1] - first;
     const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)cnt;
@@ -203,18 +206,26 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
 
 size_t doc_tile_smem_bytes(int tile_tokens) { return (size_t)tile_tokens * DOC_TILE_SMEM_PER_TOKEN + 16; }
 
-void set_doc_smem_limits()
+template <typename T, int MODE, int FIXED>
+static void set_doc_limit()
 {
-    const int bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
-    cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024, LDA_PROPOSALS_CYCLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    cudaFuncSetAttribute(k_doc_tile<int32_t, 1024, LDA_PROPOSALS_CYCLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024, LDA_PROPOSALS_WORD>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    cudaFuncSetAttribute(k_doc_tile<int32_t, 1024, LDA_PROPOSALS_WORD>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    cudaFuncSetAttribute(k_doc_tile<uint16_t, 1024, LDA_PROPOSALS_DOC>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    cudaFuncSetAttribute(k_doc_tile<int32_t, 1024, LDA_PROPOSALS_DOC>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaFuncSetAttribute(k_doc_tile<T, 1024, MODE, FIXED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)doc_tile_smem_bytes(DOC_TILE_MAX));
 }
 
-template <typename T, int MODE>
+void set_doc_smem_limits()
+{
+    set_doc_limit<uint16_t, LDA_PROPOSALS_CYCLE, 0>();
+    set_doc_limit<uint16_t, LDA_PROPOSALS_CYCLE, 2>();
+    set_doc_limit<uint16_t, LDA_PROPOSALS_WORD, 0>();
+    set_doc_limit<uint16_t, LDA_PROPOSALS_DOC, 0>();
+    set_doc_limit<int32_t, LDA_PROPOSALS_CYCLE, 0>();
+    set_doc_limit<int32_t, LDA_PROPOSALS_CYCLE, 2>();
+    set_doc_limit<int32_t, LDA_PROPOSALS_WORD, 0>();
+    set_doc_limit<int32_t, LDA_PROPOSALS_DOC, 0>();
+}
+
+template <typename T, int MODE, int FIXED>
 static int doc_side_tm(Ctx& c, int mh_steps)
 {
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
@@ -222,15 +233,15 @@ static int doc_side_tm(Ctx& c, int mh_steps)
     if (c.n_doc_tiles) {
         const size_t smem = doc_tile_smem_bytes(c.doc_tile);
         switch (c.doc_threads) {
-            case 128: k_doc_tile<T, 128, MODE><<<c.n_doc_tiles, 128, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
-            case 256: k_doc_tile<T, 256, MODE><<<c.n_doc_tiles, 256, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
-            case 512: k_doc_tile<T, 512, MODE><<<c.n_doc_tiles, 512, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
-            default: k_doc_tile<T, 1024, MODE><<<c.n_doc_tiles, 1024, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            case 128: k_doc_tile<T, 128, MODE, FIXED><<<c.n_doc_tiles, 128, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            case 256: k_doc_tile<T, 256, MODE, FIXED><<<c.n_doc_tiles, 256, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            case 512: k_doc_tile<T, 512, MODE, FIXED><<<c.n_doc_tiles, 512, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
+            default: k_doc_tile<T, 1024, MODE, FIXED><<<c.n_doc_tiles, 1024, smem, c.stream>>>(c.v, c.doc_tiles, key, c.sweep, mh_steps); break;
         }
         ++launches;
     }
     if (c.n_long_docs) {
-        k_long_doc_tile<T, MODE><<<c.n_long_docs, 512, 0, c.stream>>>(c.v, c.long_docs, key, c.sweep, mh_steps);
+        k_long_doc_tile<T, MODE, FIXED><<<c.n_long_docs, 512, 0, c.stream>>>(c.v, c.long_docs, key, c.sweep, mh_steps);
         ++launches;
     }
     return launches;
@@ -240,9 +251,11 @@ template <typename T>
 static int doc_side_t(Ctx& c, int mh_steps)
 {
     switch (c.proposals) {
-        case LDA_PROPOSALS_WORD: return doc_side_tm<T, LDA_PROPOSALS_WORD>(c, mh_steps);
-        case LDA_PROPOSALS_DOC: return doc_side_tm<T, LDA_PROPOSALS_DOC>(c, mh_steps);
-        default: return doc_side_tm<T, LDA_PROPOSALS_CYCLE>(c, mh_steps);
+        case LDA_PROPOSALS_WORD: return doc_side_tm<T, LDA_PROPOSALS_WORD, 0>(c, mh_steps);
+        case LDA_PROPOSALS_DOC: return doc_side_tm<T, LDA_PROPOSALS_DOC, 0>(c, mh_steps);
+        default:  // the cycle with two steps has kernels of its own
+            return mh_steps == 2 ? doc_side_tm<T, LDA_PROPOSALS_CYCLE, 2>(c, mh_steps)
+                                 : doc_side_tm<T, LDA_PROPOSALS_CYCLE, 0>(c, mh_steps);
     }
 }
 

@@ -343,11 +343,14 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
 }
 
 // Hot words: tile = (word, first token, count).  ACCEPT = false: pass 1, true: pass 3.
-template <typename T, int CH, bool STAGED, bool ACCEPT, int MODE>
+// FIXED > 0: the number of steps is this compile-time constant (the argument is ignored), which
+// removes the step loops and their predicates from the accept/reject chain.
+template <typename T, int CH, bool STAGED, bool ACCEPT, int MODE, int FIXED>
 __global__ void __launch_bounds__(ACCEPT ? ACCEPT_THREADS : PROPOSE_THREADS,
                                   ACCEPT ? LDA_ACCEPT_MIN_CTAS : LDA_PROPOSE_MIN_CTAS)
-k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
+k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps_arg)
 {
+    const int32_t mh_steps = FIXED > 0 ? FIXED : mh_steps_arg;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ __align__(8) unsigned long long bar;
     constexpr bool PACKED = sizeof(T) == 2;
@@ -384,10 +387,11 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
 }
 
 // Tail words: tile = range of whole words [w0, w1) with at most COLD_TILE tokens.
-template <typename T, int CH, bool ACCEPT, int MODE>
+template <typename T, int CH, bool ACCEPT, int MODE, int FIXED>
 __global__ void __launch_bounds__(COLD_THREADS)
-k_word_cold(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps)
+k_word_cold(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps_arg)
 {
+    const int32_t mh_steps = FIXED > 0 ? FIXED : mh_steps_arg;
     __shared__ int32_t woff_s[COLD_WORDS + 1];  // first token of each word, relative to the tile
     __shared__ int32_t rs_s[COLD_WORDS + 1];    // first row slot of each word, relative to the tile
     __shared__ int32_t nnz_s[COLD_WORDS];
@@ -471,43 +475,55 @@ static int grid_for(int64_t n, int block)
     return g < 1 ? 1 : (int)g;
 }
 
+template <typename T, int CH, int MODE, int FIXED>
+static int launch_accept(Ctx& c, uint2 key, int mh_steps)
+{
+    const View& v = c.v;
+    int launches = 0;
+    if (c.n_hot_tiles) {
+        if (c.K <= HOT_STAGE_MAX_K)
+            k_word_hot<T, CH, true, true, MODE, FIXED>
+                <<<c.n_hot_tiles, ACCEPT_THREADS, (size_t)v.dense_stride * 8, c.stream>>>(v, c.hot_tiles, key, c.sweep,
+                                                                                          mh_steps);
+        else
+            k_word_hot<T, CH, false, true, MODE, FIXED>
+                <<<c.n_hot_tiles, ACCEPT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key, c.sweep, mh_steps);
+        ++launches;
+    }
+    if (c.n_cold_tiles) {
+        k_word_cold<T, CH, true, MODE, FIXED><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key,
+                                                                                           c.sweep, mh_steps);
+        ++launches;
+    }
+    return launches;
+}
+
 template <typename T, int CH, int MODE>
 static int sample_tc(Ctx& c, int mh_steps)
 {
     const View& v = c.v;
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
-    const bool staged = c.K <= HOT_STAGE_MAX_K;
     int launches = 0;
     // pass 1: word-proposals (none in a doc-proposal-only chain)
     if (MODE != LDA_PROPOSALS_DOC && c.n_hot_tiles) {
-        k_word_hot<T, CH, false, false, MODE><<<c.n_hot_tiles, PROPOSE_THREADS, 0, c.stream>>>(v, c.hot_tiles, key, c.sweep,
-                                                                                    mh_steps);
+        k_word_hot<T, CH, false, false, MODE, 0><<<c.n_hot_tiles, PROPOSE_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
+                                                                                                c.sweep, mh_steps);
         ++launches;
     }
     if (MODE != LDA_PROPOSALS_DOC && c.n_cold_tiles) {
-        k_word_cold<T, CH, false, MODE><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
-                                                                                mh_steps);
+        k_word_cold<T, CH, false, MODE, 0><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
+                                                                                        mh_steps);
         ++launches;
     }
     // pass 2: document side
     cudaEventRecord(c.ev[8], c.stream);
     launches += launch_doc_side(c, mh_steps);
-    // pass 3: accept / reject
+    // pass 3: accept / reject; the cycle with two steps has kernels of its own
     cudaEventRecord(c.ev[9], c.stream);
-    if (c.n_hot_tiles) {
-        if (staged)
-            k_word_hot<T, CH, true, true, MODE><<<c.n_hot_tiles, ACCEPT_THREADS, (size_t)v.dense_stride * 8, c.stream>>>(
-                v, c.hot_tiles, key, c.sweep, mh_steps);
-        else
-            k_word_hot<T, CH, false, true, MODE><<<c.n_hot_tiles, ACCEPT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
-                                                                                       c.sweep, mh_steps);
-        ++launches;
-    }
-    if (c.n_cold_tiles) {
-        k_word_cold<T, CH, true, MODE><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
-                                                                               mh_steps);
-        ++launches;
-    }
+    if (CH == 2 && MODE == LDA_PROPOSALS_CYCLE && mh_steps == 2)
+        launches += launch_accept<T, 2, LDA_PROPOSALS_CYCLE, 2>(c, key, mh_steps);
+    else
+        launches += launch_accept<T, CH, MODE, 0>(c, key, mh_steps);
     return launches;
 }
 
@@ -535,15 +551,20 @@ int launch_sample(Ctx& c, int mh_steps)
     return c.wide_topics ? sample_t<int32_t>(c, mh_steps) : sample_t<uint16_t>(c, mh_steps);
 }
 
+template <typename T, int CH, int MODE, int FIXED>
+static void set_hot_limit_one()
+{
+    cudaFuncSetAttribute(k_word_hot<T, CH, true, true, MODE, FIXED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         HOT_STAGE_MAX_K * 8);
+}
+
 template <typename T, int CH>
 static void set_hot_limit()
 {
-    cudaFuncSetAttribute(k_word_hot<T, CH, true, true, LDA_PROPOSALS_CYCLE>,
-                         cudaFuncAttributeMaxDynamicSharedMemorySize, HOT_STAGE_MAX_K * 8);
-    cudaFuncSetAttribute(k_word_hot<T, CH, true, true, LDA_PROPOSALS_WORD>,
-                         cudaFuncAttributeMaxDynamicSharedMemorySize, HOT_STAGE_MAX_K * 8);
-    cudaFuncSetAttribute(k_word_hot<T, CH, true, true, LDA_PROPOSALS_DOC>,
-                         cudaFuncAttributeMaxDynamicSharedMemorySize, HOT_STAGE_MAX_K * 8);
+    set_hot_limit_one<T, CH, LDA_PROPOSALS_CYCLE, 0>();
+    set_hot_limit_one<T, CH, LDA_PROPOSALS_WORD, 0>();
+    set_hot_limit_one<T, CH, LDA_PROPOSALS_DOC, 0>();
+    if (CH == 2) set_hot_limit_one<T, 2, LDA_PROPOSALS_CYCLE, 2>();
 }
 
 void set_sample_smem_limits()
