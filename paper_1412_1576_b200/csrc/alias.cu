@@ -254,13 +254,17 @@ __global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, ul
     }
 }
 
-// One CTA per word whose row can be longer than ALIAS_WARP_MAX.
-#ifndef LDA_ALIAS_BLOCK_THREADS
-#define LDA_ALIAS_BLOCK_THREADS 256
-#endif
-__global__ void __launch_bounds__(LDA_ALIAS_BLOCK_THREADS)
-k_alias_sparse_block(View v, const int32_t* __restrict__ words, ull* sc_w, ull* sc_de, uint32_t* sc_item)
+// One CTA per word whose row can be longer than ALIAS_WARP_MAX.  The construction's scratch
+// (20 bytes per item) lives in shared memory when the row has at most `smem_items` items; a longer
+// row keeps the array its binary searches run over (8 bytes per item) there as long as that fits,
+// and the rest -- or, beyond that, everything -- in the row's range of the scratch arrays in
+// device memory.
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
+k_alias_sparse_block(View v, const int32_t* __restrict__ words, ull* sc_w, ull* sc_de, uint32_t* sc_item,
+                     int32_t smem_items)
 {
+    extern __shared__ __align__(16) unsigned char alias_scratch[];
     __shared__ ull smem[99];
     Group<true> g{smem};
     const int32_t w = words[blockIdx.x];
@@ -268,9 +272,20 @@ k_alias_sparse_block(View v, const int32_t* __restrict__ words, ull* sc_w, ull* 
     if (n <= ALIAS_WARP_MAX) return;
     const int32_t r0 = v.row_start[w];
     SparseWeight wf{v.wk_topic + r0, v.wk_count + r0, v.nk, v.Vbeta};
-    const ull S = build_alias_row<true>(g, n, wf, sc_w + r0, sc_de + r0, sc_item + r0, v.al_thr + r0,
-                                        v.al_idx + r0, v.al_pk ? v.al_pk + r0 : nullptr, v.wk_topic + r0,
-                                        v.err);
+    uint2* pk = v.al_pk ? v.al_pk + r0 : nullptr;
+    ull S;
+    if (n <= smem_items) {
+        ull* w_s = reinterpret_cast<ull*>(alias_scratch);
+        ull* de_s = w_s + smem_items;
+        uint32_t* item_s = reinterpret_cast<uint32_t*>(de_s + smem_items);
+        S = build_alias_row<true>(g, n, wf, w_s, de_s, item_s, v.al_thr + r0, v.al_idx + r0, pk, v.wk_topic + r0, v.err);
+    } else if ((int64_t)n * 8 <= (int64_t)smem_items * ALIAS_SCRATCH_PER_ITEM) {
+        S = build_alias_row<true>(g, n, wf, sc_w + r0, reinterpret_cast<ull*>(alias_scratch), sc_item + r0,
+                                  v.al_thr + r0, v.al_idx + r0, pk, v.wk_topic + r0, v.err);
+    } else {
+        S = build_alias_row<true>(g, n, wf, sc_w + r0, sc_de + r0, sc_item + r0, v.al_thr + r0, v.al_idx + r0, pk,
+                                  v.wk_topic + r0, v.err);
+    }
     if (threadIdx.x == 0) v.mix32[w] = mixture_threshold(S, *v.dense_mass);
 }
 
@@ -287,12 +302,27 @@ int launch_alias_sparse(Ctx& c)
     if (grid > 148 * 16) grid = 148 * 16;
     k_alias_sparse_warp<<<grid, 256, 0, c.stream>>>(c.v, c.sc_w, c.sc_de, c.sc_item);
     ++launches;
-    if (c.n_alias_big) {
-        k_alias_sparse_block<<<c.n_alias_big, LDA_ALIAS_BLOCK_THREADS, 0, c.stream>>>(c.v, c.alias_big, c.sc_w, c.sc_de,
-                                                                 c.sc_item);
+    // words whose row cannot exceed ALIAS_SMEM_ITEMS_MID come first in the list
+    if (c.n_alias_mid) {
+        k_alias_sparse_block<256><<<c.n_alias_mid, 256, ALIAS_SMEM_ITEMS_MID * ALIAS_SCRATCH_PER_ITEM, c.stream>>>(
+            c.v, c.alias_big, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_MID);
+        ++launches;
+    }
+    if (c.n_alias_big > c.n_alias_mid) {
+        k_alias_sparse_block<512>
+            <<<c.n_alias_big - c.n_alias_mid, 512, ALIAS_SMEM_ITEMS_BIG * ALIAS_SCRATCH_PER_ITEM, c.stream>>>(
+                c.v, c.alias_big + c.n_alias_mid, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_BIG);
         ++launches;
     }
     return launches;
+}
+
+void set_alias_smem_limits()
+{
+    cudaFuncSetAttribute(k_alias_sparse_block<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         ALIAS_SMEM_ITEMS_MID * ALIAS_SCRATCH_PER_ITEM);
+    cudaFuncSetAttribute(k_alias_sparse_block<512>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         ALIAS_SMEM_ITEMS_BIG * ALIAS_SCRATCH_PER_ITEM);
 }
 
 }  // namespace lda

@@ -10,6 +10,7 @@ namespace lda {
 void set_hist_smem_limits();
 void set_sample_smem_limits();
 void set_doc_smem_limits();
+void set_alias_smem_limits();
 
 void* dev_alloc(Ctx& c, size_t bytes)
 {
@@ -234,14 +235,15 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         // a dense row of K counters only pays for a word with a fair share of K tokens
         tf_cut = std::max<int32_t>({tmp[nth], (int32_t)std::max(1.0, c.dense_min_tf), K / 8});
     }
-    std::vector<int32_t> dense_slot((size_t)V, -1), dense_words, row_start((size_t)V + 1), alias_big;
+    std::vector<int32_t> dense_slot((size_t)V, -1), dense_words, row_start((size_t)V + 1), alias_big, alias_mid;
     std::vector<int32_t> hist_chunks, word_tiles;
     int64_t cap_total = 0;
     for (int32_t w = 0; w < V; ++w) {
         row_start[w] = (int32_t)cap_total;
         const int32_t cap = std::min(tf[w], K);
         cap_total += cap;
-        if (cap > ALIAS_WARP_MAX) alias_big.push_back(w);
+        if (cap > ALIAS_SMEM_ITEMS_MID) alias_big.push_back(w);
+        else if (cap > ALIAS_WARP_MAX) alias_mid.push_back(w);
         if (tf[w] > SORT_TILE || (tf[w] > 0 && tf[w] >= tf_cut)) {
             dense_slot[w] = (int32_t)dense_words.size();
             dense_words.push_back(w);
@@ -324,6 +326,8 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.n_dense = (int32_t)dense_words.size();
     c.n_hist_chunks = (int32_t)(hist_chunks.size() / 3);
     c.n_long_docs = (int32_t)long_docs.size();
+    c.n_alias_mid = (int32_t)alias_mid.size();
+    alias_big.insert(alias_big.begin(), alias_mid.begin(), alias_mid.end());
     c.n_alias_big = (int32_t)alias_big.size();
     c.n_hot_tiles = (int32_t)(hot_tiles.size() / 3);
     c.n_cold_tiles = (int32_t)(cold_tiles.size() / 2);
@@ -437,6 +441,7 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
     set_hist_smem_limits();
     set_sample_smem_limits();
     set_doc_smem_limits();
+    set_alias_smem_limits();
     *out = h;
     return LDA_OK;
 }

@@ -39,7 +39,7 @@ __device__ __forceinline__ void load_topic_pair(const int32_t* zbm, uint32_t bm,
 // block-major index `bm`.
 //   tab     : the document's table, 4 * doc_len slots
 //   slot_at : slot holding the topic of the document's j-th token
-template <typename T, int MODE, class SlotAt>
+template <typename T, int MODE, int FIXED, class SlotAt>
 __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* tab, uint32_t tok, uint32_t doc_len,
                                                uint32_t own, uint32_t t_first, uint32_t bm, const SlotAt& slot_at,
                                                uint2 key, uint32_t sweep, int32_t mh_steps)
@@ -50,13 +50,22 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
     const size_t N = (size_t)v.N;
     uint32_t* out = v.dside + (size_t)bm * v.side_stride;
     const double n_d = (double)doc_len;
-    // words 0..3 go out as one 16-byte store at the end, the rest one by one
-    uint32_t w1 = 0u, w2 = 0u, w3 = 0u;
+    // words 0..3 (the whole record when the step count is fixed at compile time) are collected in
+    // registers and go out as 16-byte stores at the end, the rest one by one
+    constexpr int REGW = (FIXED > 0 && step_record_words<MODE>(FIXED) > 4) ? 8 : 4;
+    static_assert(FIXED == 0 || step_record_words<MODE>(FIXED) <= 8, "the record is kept in eight registers");
+    uint32_t wr[REGW];
+#pragma unroll
+    for (int q = 0; q < REGW; ++q) wr[q] = 0u;
     auto put = [&](int at, uint32_t val) {
-        if (at == 1) w1 = val;
-        else if (at == 2) w2 = val;
-        else if (at == 3) w3 = val;
-        else __stcs(out + at, val);
+        if (FIXED > 0) {
+            wr[at] = val;  // the step loops are unrolled: `at` is a constant
+        } else {
+            if (at == 1) wr[1] = val;
+            else if (at == 2) wr[2] = val;
+            else if (at == 3) wr[3] = val;
+            else __stcs(out + at, val);
+        }
     };
     // word-proposal of step st, the wi-th of its kind: n_kd at the topic pass 1 drew
     auto word_step = [&](int32_t st, int32_t wi) {
@@ -80,16 +89,20 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
         put(1 + mh_steps + di, r.w);  // the step's acceptance uniform
     };
     if (MODE == LDA_PROPOSALS_CYCLE) {
+#pragma unroll
         for (int32_t st = 0; st < mh_steps; st += 2) {
             word_step(st, st >> 1);
             if (st + 1 < mh_steps) doc_step(st + 1, st >> 1);
         }
     } else if (MODE == LDA_PROPOSALS_WORD) {
+#pragma unroll
         for (int32_t st = 0; st < mh_steps; ++st) word_step(st, st);
     } else {
+#pragma unroll
         for (int32_t st = 0; st < mh_steps; ++st) doc_step(st, st);
     }
-    __stcs(reinterpret_cast<uint4*>(out), make_uint4(own, w1, w2, w3));
+    __stcs(reinterpret_cast<uint4*>(out), make_uint4(own, wr[1], wr[2], wr[3]));
+    if (REGW == 8) __stcs(reinterpret_cast<uint4*>(out) + 1, make_uint4(wr[4], wr[5], wr[6], wr[7]));
 }
 
 // `cap` = tokens a tile can hold (the shared-memory carve-up) = DOC_TILE_ROUNDS x blockDim.x: a
@@ -163,7 +176,7 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
             const uint32_t* tab = slots + DK_SLOTS_PER_TOKEN * first[r];
             const uint32_t* slot_of = slot_s + first[r];
             auto slot_at = [slot_of](uint32_t jj) { return slot_of[jj]; };
-            doc_side_token<T, MODE>(v, tab, (uint32_t)(base + j), (uint32_t)len[r], tab[z[r]], t1[r], bm[r], slot_at, key,
+            doc_side_token<T, MODE, FIXED>(v, tab, (uint32_t)(base + j), (uint32_t)len[r], tab[z[r]], t1[r], bm[r], slot_at, key,
                               sweep, mh_steps);
         }
     }
@@ -199,7 +212,7 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
     auto slot_at = [slot_of](uint32_t j) { return slot_of[j]; };
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
         const uint32_t bm = v.bm_of_tok[first + j];
-        doc_side_token<T, MODE>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)zbm[2 * (size_t)bm + 1], bm,
+        doc_side_token<T, MODE, FIXED>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)zbm[2 * (size_t)bm + 1], bm,
                           slot_at, key, sweep, mh_steps);
     }
 }
@@ -217,12 +230,18 @@ void set_doc_smem_limits()
 {
     set_doc_limit<uint16_t, LDA_PROPOSALS_CYCLE, 0>();
     set_doc_limit<uint16_t, LDA_PROPOSALS_CYCLE, 2>();
+    set_doc_limit<uint16_t, LDA_PROPOSALS_CYCLE, 4>();
     set_doc_limit<uint16_t, LDA_PROPOSALS_WORD, 0>();
+    set_doc_limit<uint16_t, LDA_PROPOSALS_WORD, 2>();
     set_doc_limit<uint16_t, LDA_PROPOSALS_DOC, 0>();
+    set_doc_limit<uint16_t, LDA_PROPOSALS_DOC, 2>();
     set_doc_limit<int32_t, LDA_PROPOSALS_CYCLE, 0>();
     set_doc_limit<int32_t, LDA_PROPOSALS_CYCLE, 2>();
+    set_doc_limit<int32_t, LDA_PROPOSALS_CYCLE, 4>();
     set_doc_limit<int32_t, LDA_PROPOSALS_WORD, 0>();
+    set_doc_limit<int32_t, LDA_PROPOSALS_WORD, 2>();
     set_doc_limit<int32_t, LDA_PROPOSALS_DOC, 0>();
+    set_doc_limit<int32_t, LDA_PROPOSALS_DOC, 2>();
 }
 
 template <typename T, int MODE, int FIXED>
@@ -251,11 +270,17 @@ template <typename T>
 static int doc_side_t(Ctx& c, int mh_steps)
 {
     switch (c.proposals) {
-        case LDA_PROPOSALS_WORD: return doc_side_tm<T, LDA_PROPOSALS_WORD, 0>(c, mh_steps);
-        case LDA_PROPOSALS_DOC: return doc_side_tm<T, LDA_PROPOSALS_DOC, 0>(c, mh_steps);
-        default:  // the cycle with two steps has kernels of its own
-            return mh_steps == 2 ? doc_side_tm<T, LDA_PROPOSALS_CYCLE, 2>(c, mh_steps)
-                                 : doc_side_tm<T, LDA_PROPOSALS_CYCLE, 0>(c, mh_steps);
+        // chains of two steps (and the cycle with four) have kernels of their own
+        case LDA_PROPOSALS_WORD:
+            return mh_steps == 2 ? doc_side_tm<T, LDA_PROPOSALS_WORD, 2>(c, mh_steps)
+                                 : doc_side_tm<T, LDA_PROPOSALS_WORD, 0>(c, mh_steps);
+        case LDA_PROPOSALS_DOC:
+            return mh_steps == 2 ? doc_side_tm<T, LDA_PROPOSALS_DOC, 2>(c, mh_steps)
+                                 : doc_side_tm<T, LDA_PROPOSALS_DOC, 0>(c, mh_steps);
+        default:
+            return mh_steps == 2   ? doc_side_tm<T, LDA_PROPOSALS_CYCLE, 2>(c, mh_steps)
+                   : mh_steps == 4 ? doc_side_tm<T, LDA_PROPOSALS_CYCLE, 4>(c, mh_steps)
+                                   : doc_side_tm<T, LDA_PROPOSALS_CYCLE, 0>(c, mh_steps);
     }
 }
 

@@ -23,6 +23,14 @@ __host__ __device__ constexpr int step_kind_index(int m)
     return MODE == LDA_PROPOSALS_CYCLE ? m >> 1 : m;
 }
 
+// Words of the record the document side leaves per token for a chain of m steps: the token's own
+// (topic, n_kd) word, one (topic, n_kd) word per step, one acceptance uniform per doc step.
+template <int MODE>
+__host__ __device__ constexpr int step_record_words(int m)
+{
+    return 1 + m + (MODE == LDA_PROPOSALS_CYCLE ? m / 2 : MODE == LDA_PROPOSALS_DOC ? m : 0);
+}
+
 // Device error word bits (set by kernels, read by the host after a sweep).
 enum : int {
     ERR_WORD_RANGE = 1,   // a word id outside [0,V) at load
@@ -49,7 +57,10 @@ constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DK_SLOTS_PER_TOKEN_HOST + 4 + 4;
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (32-bit bins)
 constexpr int WORD_ROWS_BITMAP_MAX_K = 16384;  // tail rows: topic bitmap up to this K, key sort above
 constexpr int HIST16_BINS = 106496;  // window of the per-chunk n_kw histogram (16-bit bins, 208 KB)
-constexpr int HIST_CHUNK = 16384;    // tokens per CTA in the histogram path
+#ifndef LDA_HIST_CHUNK
+#define LDA_HIST_CHUNK 32768
+#endif
+constexpr int HIST_CHUNK = LDA_HIST_CHUNK;    // tokens per CTA in the histogram path
 static_assert(HIST_CHUNK < 65536, "the per-chunk histogram counts in 16 bits");
 #ifndef LDA_HOT_TILE
 #define LDA_HOT_TILE 8192
@@ -59,6 +70,9 @@ constexpr int COLD_TILE = 2048;      // MH kernel: tokens of a tile of whole tai
 constexpr int COLD_WORDS = 512;      // MH kernel: words per tail tile
 constexpr int HOT_STAGE_MAX_K = 16384;  // dense rows up to this many topics are staged in shared memory
 constexpr int ALIAS_WARP_MAX = 256;  // rows up to this many items are built by one warp
+constexpr int ALIAS_SCRATCH_PER_ITEM = 20;   // bytes of construction scratch per item
+constexpr int ALIAS_SMEM_ITEMS_MID = 2048;   // rows a 256-thread CTA builds entirely in shared memory
+constexpr int ALIAS_SMEM_ITEMS_BIG = 4096;   // ... and a 512-thread CTA
 
 // Everything a kernel needs, passed by value.
 struct View {
@@ -134,13 +148,14 @@ struct Ctx {
     View v{};
     // host-side work lists (device copies below)
     int32_t n_word_tiles = 0, n_doc_tiles = 0, n_dense = 0, n_hist_chunks = 0, n_long_docs = 0,
-            n_alias_big = 0, n_hot_tiles = 0, n_cold_tiles = 0;
+            n_alias_big = 0, n_alias_mid = 0, n_hot_tiles = 0, n_cold_tiles = 0;
     int32_t* word_tiles = nullptr;   // [n_word_tiles*2] word ranges sorted per CTA
     int32_t* doc_tiles = nullptr;    // [n_doc_tiles*2]
     int32_t* dense_words = nullptr;  // [n_dense]
     int32_t* hist_chunks = nullptr;  // [n_hist_chunks*3] (word, first token, count)
     int32_t* long_docs = nullptr;    // [n_long_docs]
-    int32_t* alias_big = nullptr;    // [n_alias_big] words whose row can exceed ALIAS_WARP_MAX
+    int32_t* alias_big = nullptr;    // [n_alias_big] words whose row can exceed ALIAS_WARP_MAX; the first
+                                     // n_alias_mid of them cannot exceed ALIAS_SMEM_ITEMS_MID
     int32_t* hot_tiles = nullptr;    // [n_hot_tiles*3] (word, first token, count): MH kernel, hot words
     int32_t* cold_tiles = nullptr;   // [n_cold_tiles*2] word ranges of whole tail words: MH kernel
     // alias-construction scratch

@@ -30,6 +30,9 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 #ifndef LDA_PROPOSE_MIN_CTAS
 #define LDA_PROPOSE_MIN_CTAS 2
 #endif
+#ifndef LDA_PROPOSE_FIXED_MIN_CTAS
+#define LDA_PROPOSE_FIXED_MIN_CTAS 3
+#endif
 #ifndef LDA_ACCEPT_THREADS
 #define LDA_ACCEPT_THREADS 512
 #endif
@@ -238,7 +241,7 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
 // --- pass 3: accept / reject (word order) -----------------------------------------------------------
 // Runs the chain of every token of the tile: everything the document side contributes was
 // gathered by pass 2, the word side comes from the tile's staged rows.
-template <typename T, int CH, int MODE, class Tile>
+template <typename T, int CH, int MODE, int FIXED, class Tile>
 __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const int32_t p_begin, const int32_t p_end,
                                               const int32_t nthreads, const uint2 key, const uint32_t sweep,
                                               const int32_t mh_steps)
@@ -254,20 +257,30 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
     // early, the gathered record (which needs that index) one iteration early.
     const uint4* side4 = reinterpret_cast<const uint4*>(v.dside);
     const int32_t quads = v.side_stride >> 2;
+    // with the step count fixed at compile time a record of more than four words is read ahead whole
+    constexpr bool TWO = FIXED > 0 && step_record_words<MODE>(FIXED) > 4;
+    static_assert(FIXED == 0 || step_record_words<MODE>(FIXED) <= 8, "the record is read as two 16-byte words");
     int32_t p = p_begin + (int32_t)threadIdx.x;
     uint32_t at_c = 0, at_n = 0;
-    uint4 rec_c = make_uint4(0u, 0u, 0u, 0u);
+    uint4 rec_c = make_uint4(0u, 0u, 0u, 0u), rec2_c = make_uint4(0u, 0u, 0u, 0u);
     if (p < p_end) at_c = __ldcs(v.inv + p);
     if (p + nthreads < p_end) at_n = __ldcs(v.inv + p + nthreads);
-    if (p < p_end) rec_c = __ldcs(side4 + (size_t)at_c * quads);
+    if (p < p_end) {
+        rec_c = __ldcs(side4 + (size_t)at_c * quads);
+        if (TWO) rec2_c = __ldcs(side4 + (size_t)at_c * quads + 1);
+    }
     for (; p < p_end; p += nthreads) {
         const uint32_t at = at_c;
-        const uint4 rec = rec_c;  // own record, then the first three words pass 2 gathered
+        const uint4 rec = rec_c, rec2 = rec2_c;  // own record, then the words pass 2 gathered
         at_c = at_n;
-        if (p + nthreads < p_end) rec_c = __ldcs(side4 + (size_t)at_c * quads);
+        if (p + nthreads < p_end) {
+            rec_c = __ldcs(side4 + (size_t)at_c * quads);
+            if (TWO) rec2_c = __ldcs(side4 + (size_t)at_c * quads + 1);
+        }
         if (p + 2 * nthreads < p_end) at_n = __ldcs(v.inv + p + 2 * nthreads);
         const uint32_t* side = v.dside + (size_t)at * v.side_stride;
         auto side_word = [&](int32_t i) {
+            if (TWO && i >= 4) return i == 4 ? rec2.x : i == 5 ? rec2.y : i == 6 ? rec2.z : rec2.w;
             return i == 1 ? rec.y : i == 2 ? rec.z : i == 3 ? rec.w : __ldcs(side + i);
         };
         const uint32_t own = rec.x;
@@ -344,10 +357,12 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
 
 // Hot words: tile = (word, first token, count).  ACCEPT = false: pass 1, true: pass 3.
 // FIXED > 0: the number of steps is this compile-time constant (the argument is ignored), which
-// removes the step loops and their predicates from the accept/reject chain.
+// removes the step loops and their predicates (and, in pass 1, enough registers for a third CTA per SM).
 template <typename T, int CH, bool STAGED, bool ACCEPT, int MODE, int FIXED>
 __global__ void __launch_bounds__(ACCEPT ? ACCEPT_THREADS : PROPOSE_THREADS,
-                                  ACCEPT ? LDA_ACCEPT_MIN_CTAS : LDA_PROPOSE_MIN_CTAS)
+                                  ACCEPT      ? LDA_ACCEPT_MIN_CTAS
+                                  : FIXED > 0 ? LDA_PROPOSE_FIXED_MIN_CTAS
+                                              : LDA_PROPOSE_MIN_CTAS)
 k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps_arg)
 {
     const int32_t mh_steps = FIXED > 0 ? FIXED : mh_steps_arg;
@@ -381,7 +396,7 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     tile.mix = __ldg(v.mix32 + w);
     tile.bar = &bar;
     tile.ready = !(STAGED && ACCEPT);
-    if (ACCEPT) accept_tokens<T, CH, MODE>(v, tile, p0, p0 + cnt, ACCEPT_THREADS, key, sweep, mh_steps);
+    if (ACCEPT) accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, ACCEPT_THREADS, key, sweep, mh_steps);
     else propose_tokens<T, MODE>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
     // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one
 }
@@ -422,7 +437,7 @@ k_word_cold(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep
     }
     __syncthreads();
     ColdTile tile{woff_s, rs_s, nnz_s, mix_s, topic_s, count_s, thr_s, idx_s, nw, v.nk};
-    if (ACCEPT) accept_tokens<T, CH, MODE>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
+    if (ACCEPT) accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
     else propose_tokens<T, MODE>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
 }
 
@@ -498,30 +513,45 @@ static int launch_accept(Ctx& c, uint2 key, int mh_steps)
     return launches;
 }
 
+template <typename T, int CH, int MODE, int FIXED>
+static int launch_propose(Ctx& c, uint2 key, int mh_steps)
+{
+    const View& v = c.v;
+    int launches = 0;
+    if (c.n_hot_tiles) {
+        k_word_hot<T, CH, false, false, MODE, FIXED><<<c.n_hot_tiles, PROPOSE_THREADS, 0, c.stream>>>(
+            v, c.hot_tiles, key, c.sweep, mh_steps);
+        ++launches;
+    }
+    if (c.n_cold_tiles) {
+        k_word_cold<T, CH, false, MODE, FIXED><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key,
+                                                                                            c.sweep, mh_steps);
+        ++launches;
+    }
+    return launches;
+}
+
 template <typename T, int CH, int MODE>
 static int sample_tc(Ctx& c, int mh_steps)
 {
-    const View& v = c.v;
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     int launches = 0;
     // pass 1: word-proposals (none in a doc-proposal-only chain)
-    if (MODE != LDA_PROPOSALS_DOC && c.n_hot_tiles) {
-        k_word_hot<T, CH, false, false, MODE, 0><<<c.n_hot_tiles, PROPOSE_THREADS, 0, c.stream>>>(v, c.hot_tiles, key,
-                                                                                                c.sweep, mh_steps);
-        ++launches;
-    }
-    if (MODE != LDA_PROPOSALS_DOC && c.n_cold_tiles) {
-        k_word_cold<T, CH, false, MODE, 0><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key, c.sweep,
-                                                                                        mh_steps);
-        ++launches;
+    if (MODE != LDA_PROPOSALS_DOC) {
+        if (CH == 2 && mh_steps == 2)
+            launches += launch_propose<T, 2, MODE, 2>(c, key, mh_steps);
+        else
+            launches += launch_propose<T, CH, MODE, 0>(c, key, mh_steps);
     }
     // pass 2: document side
     cudaEventRecord(c.ev[8], c.stream);
     launches += launch_doc_side(c, mh_steps);
-    // pass 3: accept / reject; the cycle with two steps has kernels of its own
+    // pass 3: accept / reject; chains of two steps (and the cycle with four) have kernels of their own
     cudaEventRecord(c.ev[9], c.stream);
-    if (CH == 2 && MODE == LDA_PROPOSALS_CYCLE && mh_steps == 2)
-        launches += launch_accept<T, 2, LDA_PROPOSALS_CYCLE, 2>(c, key, mh_steps);
+    if (CH == 2 && mh_steps == 2)
+        launches += launch_accept<T, 2, MODE, 2>(c, key, mh_steps);
+    else if (CH == 4 && MODE == LDA_PROPOSALS_CYCLE && mh_steps == 4)
+        launches += launch_accept<T, 4, LDA_PROPOSALS_CYCLE, 4>(c, key, mh_steps);
     else
         launches += launch_accept<T, CH, MODE, 0>(c, key, mh_steps);
     return launches;
@@ -564,7 +594,12 @@ static void set_hot_limit()
     set_hot_limit_one<T, CH, LDA_PROPOSALS_CYCLE, 0>();
     set_hot_limit_one<T, CH, LDA_PROPOSALS_WORD, 0>();
     set_hot_limit_one<T, CH, LDA_PROPOSALS_DOC, 0>();
-    if (CH == 2) set_hot_limit_one<T, 2, LDA_PROPOSALS_CYCLE, 2>();
+    if (CH == 2) {
+        set_hot_limit_one<T, 2, LDA_PROPOSALS_CYCLE, 2>();
+        set_hot_limit_one<T, 2, LDA_PROPOSALS_WORD, 2>();
+        set_hot_limit_one<T, 2, LDA_PROPOSALS_DOC, 2>();
+    }
+    if (CH == 4) set_hot_limit_one<T, 4, LDA_PROPOSALS_CYCLE, 4>();
 }
 
 void set_sample_smem_limits()

@@ -169,11 +169,16 @@ def test_hot_words_with_unstaged_rows_and_odd_step_counts():
     step counts that end on a word-proposal or exceed one group of four."""
     c = synth.generate(V=40, K=20_000, D=300, length=("fixed", 400), zipf_s=1.0, alpha=0.05, beta=0.01, seed=8)
     g, o = _pair(c, seed=5)
+    # rows of a few hundred to more than ten thousand items: every scratch placement of the alias build
+    nnz = np.diff(o.get_csr(ldaref.NWK)[0])
+    assert nnz.min() < 2048 < 4096 < np.sort(nnz)[-3] and nnz.max() > 10240
+    _assert_same_tables(g, o)
     for mh_steps in (2, 5, 3):
         g.sweep(1, mh_steps)
         o.sweep(1, mh_steps)
         assert np.array_equal(g.get_assignments(), o.get_assignments()), mh_steps
     _assert_same_counts(g, o)
+    _assert_same_tables(g, o)
 
 
 @pytest.mark.parametrize("mode", [binding.PROPOSALS_WORD, binding.PROPOSALS_DOC])
