@@ -259,8 +259,11 @@ __global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, ul
 // row keeps the array its binary searches run over (8 bytes per item) there as long as that fits,
 // and the rest -- or, beyond that, everything -- in the row's range of the scratch arrays in
 // device memory.
+#ifndef LDA_ALIAS_MID_MIN_CTAS
+#define LDA_ALIAS_MID_MIN_CTAS 1
+#endif
 template <int THREADS>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? LDA_ALIAS_MID_MIN_CTAS : 1)
 k_alias_sparse_block(View v, const int32_t* __restrict__ words, ull* sc_w, ull* sc_de, uint32_t* sc_item,
                      int32_t smem_items)
 {

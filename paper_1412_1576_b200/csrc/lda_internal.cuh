@@ -69,9 +69,15 @@ constexpr int HOT_TILE = LDA_HOT_TILE;  // MH kernels: tokens of one hot word pe
 constexpr int COLD_TILE = 2048;      // MH kernel: tokens of a tile of whole tail words
 constexpr int COLD_WORDS = 512;      // MH kernel: words per tail tile
 constexpr int HOT_STAGE_MAX_K = 16384;  // dense rows up to this many topics are staged in shared memory
-constexpr int ALIAS_WARP_MAX = 256;  // rows up to this many items are built by one warp
+#ifndef LDA_ALIAS_WARP_MAX
+#define LDA_ALIAS_WARP_MAX 512
+#endif
+constexpr int ALIAS_WARP_MAX = LDA_ALIAS_WARP_MAX;  // rows up to this many items are built by one warp
 constexpr int ALIAS_SCRATCH_PER_ITEM = 20;   // bytes of construction scratch per item
-constexpr int ALIAS_SMEM_ITEMS_MID = 2048;   // rows a 256-thread CTA builds entirely in shared memory
+#ifndef LDA_ALIAS_SMEM_ITEMS_MID
+#define LDA_ALIAS_SMEM_ITEMS_MID 2048
+#endif
+constexpr int ALIAS_SMEM_ITEMS_MID = LDA_ALIAS_SMEM_ITEMS_MID;   // rows a 256-thread CTA builds entirely in shared memory
 constexpr int ALIAS_SMEM_ITEMS_BIG = 4096;   // ... and a 512-thread CTA
 
 // Everything a kernel needs, passed by value.

@@ -33,6 +33,9 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 #ifndef LDA_PROPOSE_FIXED_MIN_CTAS
 #define LDA_PROPOSE_FIXED_MIN_CTAS 3
 #endif
+#ifndef LDA_ACCEPT_FIXED2_THREADS
+#define LDA_ACCEPT_FIXED2_THREADS 768
+#endif
 #ifndef LDA_ACCEPT_THREADS
 #define LDA_ACCEPT_THREADS 512
 #endif
@@ -40,7 +43,11 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 #define LDA_ACCEPT_MIN_CTAS 2
 #endif
 constexpr int PROPOSE_THREADS = LDA_PROPOSE_THREADS;
-constexpr int ACCEPT_THREADS = LDA_ACCEPT_THREADS;
+// the two-step chain needs few enough registers for two CTAs of 768 threads per SM
+__host__ __device__ constexpr int accept_threads(int fixed)
+{
+    return fixed == 2 ? LDA_ACCEPT_FIXED2_THREADS : LDA_ACCEPT_THREADS;
+}
 constexpr int COLD_THREADS = 256;
 constexpr int STAGE_WAIT_LIMIT = 1 << 20;
 
@@ -359,7 +366,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
 // FIXED > 0: the number of steps is this compile-time constant (the argument is ignored), which
 // removes the step loops and their predicates (and, in pass 1, enough registers for a third CTA per SM).
 template <typename T, int CH, bool STAGED, bool ACCEPT, int MODE, int FIXED>
-__global__ void __launch_bounds__(ACCEPT ? ACCEPT_THREADS : PROPOSE_THREADS,
+__global__ void __launch_bounds__(ACCEPT ? accept_threads(FIXED) : PROPOSE_THREADS,
                                   ACCEPT      ? LDA_ACCEPT_MIN_CTAS
                                   : FIXED > 0 ? LDA_PROPOSE_FIXED_MIN_CTAS
                                               : LDA_PROPOSE_MIN_CTAS)
@@ -396,7 +403,7 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     tile.mix = __ldg(v.mix32 + w);
     tile.bar = &bar;
     tile.ready = !(STAGED && ACCEPT);
-    if (ACCEPT) accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, ACCEPT_THREADS, key, sweep, mh_steps);
+    if (ACCEPT) accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, accept_threads(FIXED), key, sweep, mh_steps);
     else propose_tokens<T, MODE>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
     // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one
 }
@@ -498,11 +505,11 @@ static int launch_accept(Ctx& c, uint2 key, int mh_steps)
     if (c.n_hot_tiles) {
         if (c.K <= HOT_STAGE_MAX_K)
             k_word_hot<T, CH, true, true, MODE, FIXED>
-                <<<c.n_hot_tiles, ACCEPT_THREADS, (size_t)v.dense_stride * 8, c.stream>>>(v, c.hot_tiles, key, c.sweep,
+                <<<c.n_hot_tiles, accept_threads(FIXED), (size_t)v.dense_stride * 8, c.stream>>>(v, c.hot_tiles, key, c.sweep,
                                                                                           mh_steps);
         else
             k_word_hot<T, CH, false, true, MODE, FIXED>
-                <<<c.n_hot_tiles, ACCEPT_THREADS, 0, c.stream>>>(v, c.hot_tiles, key, c.sweep, mh_steps);
+                <<<c.n_hot_tiles, accept_threads(FIXED), 0, c.stream>>>(v, c.hot_tiles, key, c.sweep, mh_steps);
         ++launches;
     }
     if (c.n_cold_tiles) {
