@@ -19,6 +19,8 @@
 namespace lda {
 
 constexpr double INV_2_32 = 1.0 / 4294967296.0;
+// slots per token of the tables a tile builds in shared memory (DOC_TILE_SLOTS, a multiple of 4)
+constexpr int TILE_SLOTS = DOC_TILE_SLOTS;
 
 // A token's current topic and its first word-proposal sit side by side at its block-major index:
 // one read brings both.
@@ -39,12 +41,12 @@ __device__ __forceinline__ void load_topic_pair(const int32_t* zbm, uint32_t bm,
 // block-major index `bm`.
 //   tab     : the document's table, 4 * doc_len slots
 //   slot_at : slot holding the topic of the document's j-th token
-template <typename T, int MODE, int FIXED, class SlotAt>
+template <typename T, int MODE, int FIXED, int SLOTS, class SlotAt>
 __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* tab, uint32_t tok, uint32_t doc_len,
                                                uint32_t own, uint32_t t_first, uint32_t bm, const SlotAt& slot_at,
                                                uint2 key, uint32_t sweep, int32_t mh_steps)
 {
-    const uint32_t cap = DK_SLOTS_PER_TOKEN * doc_len;
+    const uint32_t cap = SLOTS * doc_len;
     const int cb = v.count_bits;
     const T* prop = reinterpret_cast<const T*>(v.prop);
     const size_t N = (size_t)v.N;
@@ -116,8 +118,8 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     const int32_t mh_steps = FIXED > 0 ? FIXED : mh_steps_arg;
     constexpr int cap = DOC_TILE_ROUNDS * THREADS;
     extern __shared__ __align__(16) uint32_t doc_smem[];
-    uint32_t* slots = doc_smem;                                  // [4 * cap] the tile's tables
-    int32_t* soff = reinterpret_cast<int32_t*>(slots + DK_SLOTS_PER_TOKEN * cap);  // [cap + 1] document offsets
+    uint32_t* slots = doc_smem;                                  // [TILE_SLOTS * cap] the tile's tables
+    int32_t* soff = reinterpret_cast<int32_t*>(slots + TILE_SLOTS * cap);  // [cap + 1] document offsets
     uint32_t* slot_s = reinterpret_cast<uint32_t*>(soff + cap + 1);  // [cap] slot (inside its table) of a token's topic
     const int tid = threadIdx.x;
     const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
@@ -139,7 +141,7 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     }
     for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = v.doc_off[s0 + j] - base;
     const uint4 empty4 = make_uint4(DK_EMPTY, DK_EMPTY, DK_EMPTY, DK_EMPTY);
-    for (int j = tid; j < cnt; j += blockDim.x) reinterpret_cast<uint4*>(slots)[j] = empty4;
+    for (int j = tid; j < cnt * (TILE_SLOTS / 4); j += blockDim.x) reinterpret_cast<uint4*>(slots)[j] = empty4;
     __syncthreads();
     // every token finds its document, adds itself to the document's table and notes the slot
 #pragma unroll
@@ -157,7 +159,7 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
             len[r] = soff[lo + 1] - first[r];
             uint32_t at = 0xFFFFFFFFu;
             if (z[r] < (uint32_t)v.K)
-                at = dk_insert(slots + DK_SLOTS_PER_TOKEN * first[r], DK_SLOTS_PER_TOKEN * (uint32_t)len[r], z[r],
+                at = dk_insert(slots + TILE_SLOTS * first[r], TILE_SLOTS * (uint32_t)len[r], z[r],
                                v.count_bits);
             if (at == 0xFFFFFFFFu) {
                 atomicOr(v.err, z[r] < (uint32_t)v.K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
@@ -173,10 +175,10 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
         const int j = tid + r * THREADS;
         if (j < cnt) {
-            const uint32_t* tab = slots + DK_SLOTS_PER_TOKEN * first[r];
+            const uint32_t* tab = slots + TILE_SLOTS * first[r];
             const uint32_t* slot_of = slot_s + first[r];
             auto slot_at = [slot_of](uint32_t jj) { return slot_of[jj]; };
-            doc_side_token<T, MODE, FIXED>(v, tab, (uint32_t)(base + j), (uint32_t)len[r], tab[z[r]], t1[r], bm[r], slot_at, key,
+            doc_side_token<T, MODE, FIXED, TILE_SLOTS>(v, tab, (uint32_t)(base + j), (uint32_t)len[r], tab[z[r]], t1[r], bm[r], slot_at, key,
                               sweep, mh_steps);
         }
     }
@@ -212,7 +214,7 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
     auto slot_at = [slot_of](uint32_t j) { return slot_of[j]; };
     for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
         const uint32_t bm = v.bm_of_tok[first + j];
-        doc_side_token<T, MODE, FIXED>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)zbm[2 * (size_t)bm + 1], bm,
+        doc_side_token<T, MODE, FIXED, DK_SLOTS_PER_TOKEN>(v, tab, (uint32_t)(first + j), (uint32_t)cnt, tab[slot_of[j]], (uint32_t)zbm[2 * (size_t)bm + 1], bm,
                           slot_at, key, sweep, mh_steps);
     }
 }

@@ -53,7 +53,12 @@ constexpr int DOC_TILE_MAX = 3072;
 constexpr int DOC_TILE_ROUNDS = 3;  // tokens per thread: every shape holds 3 x its thread count
 static_assert(DOC_TILE_TOKENS[0] == 3 * DOC_TILE_THREADS[0] && DOC_TILE_TOKENS[3] == 3 * DOC_TILE_THREADS[3], "tile shapes");
 // shared memory per token of a tile: 4 table slots, document offset, topic/slot (4 bytes each)
-constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DK_SLOTS_PER_TOKEN_HOST + 4 + 4;
+#ifndef LDA_DOC_TILE_SLOTS
+#define LDA_DOC_TILE_SLOTS 4
+#endif
+constexpr int DOC_TILE_SLOTS = LDA_DOC_TILE_SLOTS;  // slots per token of a tile's tables in shared memory
+static_assert(DOC_TILE_SLOTS % 4 == 0, "a tile's tables are cleared 16 bytes at a time");
+constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DOC_TILE_SLOTS + 4 + 4;
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (32-bit bins)
 constexpr int WORD_ROWS_BITMAP_MAX_K = 16384;  // tail rows: topic bitmap up to this K, key sort above
 constexpr int HIST16_BINS = 106496;  // window of the per-chunk n_kw histogram (16-bit bins, 208 KB)

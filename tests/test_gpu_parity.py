@@ -77,6 +77,16 @@ def test_other_step_counts_tiny(tiny_corpus, mh_steps):
     assert np.array_equal(g.get_assignments(), o.get_assignments())
 
 
+def test_four_step_cycle_small_config(small_corpus):
+    """The cycle with four steps (the step count of the "large" configuration) has kernels of its own:
+    tiles of whole documents, hot and tail words."""
+    g, o = _pair(small_corpus, seed=9)
+    g.sweep(2, 4)
+    o.sweep(2, 4)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_counts(g, o)
+
+
 def test_small_config_sweeps_counts_tables_loglik(small_corpus):
     """~2M tokens: many tiles, ragged tails, dense and sparse words, hot-word histogram path."""
     c = small_corpus
