@@ -298,25 +298,29 @@ int launch_alias_dense(Ctx& c)
     return 1;
 }
 
+// The three kernels build the tables of different words: they run side by side, the one with the
+// longest rows (and the longest tail) first.
 int launch_alias_sparse(Ctx& c)
 {
     int launches = 0;
-    int grid = (int)(((int64_t)c.V * 32 + 255) / 256);
-    if (grid > 148 * 16) grid = 148 * 16;
-    k_alias_sparse_warp<<<grid, 256, 0, c.stream>>>(c.v, c.sc_w, c.sc_de, c.sc_item);
-    ++launches;
+    fork_streams(c);
     // words whose row cannot exceed ALIAS_SMEM_ITEMS_MID come first in the list
-    if (c.n_alias_mid) {
-        k_alias_sparse_block<256><<<c.n_alias_mid, 256, ALIAS_SMEM_ITEMS_MID * ALIAS_SCRATCH_PER_ITEM, c.stream>>>(
-            c.v, c.alias_big, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_MID);
-        ++launches;
-    }
     if (c.n_alias_big > c.n_alias_mid) {
         k_alias_sparse_block<512>
             <<<c.n_alias_big - c.n_alias_mid, 512, ALIAS_SMEM_ITEMS_BIG * ALIAS_SCRATCH_PER_ITEM, c.stream>>>(
                 c.v, c.alias_big + c.n_alias_mid, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_BIG);
         ++launches;
     }
+    if (c.n_alias_mid) {
+        k_alias_sparse_block<256><<<c.n_alias_mid, 256, ALIAS_SMEM_ITEMS_MID * ALIAS_SCRATCH_PER_ITEM, c.side[0]>>>(
+            c.v, c.alias_big, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_MID);
+        ++launches;
+    }
+    int grid = (int)(((int64_t)c.V * 32 + 255) / 256);
+    if (grid > 148 * 16) grid = 148 * 16;
+    k_alias_sparse_warp<<<grid, 256, 0, c.side[1]>>>(c.v, c.sc_w, c.sc_de, c.sc_item);
+    ++launches;
+    join_streams(c);
     return launches;
 }
 

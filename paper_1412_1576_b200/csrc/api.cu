@@ -438,6 +438,17 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
             return LDA_ECUDA;
         }
     c.have_events = true;
+    {
+        bool ok = cudaEventCreateWithFlags(&c.ev_fork, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < 2 && ok; ++i)
+            ok = cudaEventCreateWithFlags(&c.ev_join[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaStreamCreateWithFlags(&c.side[i], cudaStreamNonBlocking) == cudaSuccess;
+        c.have_side = true;  // lda_destroy() releases whatever was created
+        if (!ok) {
+            lda_destroy(h);
+            return LDA_ECUDA;
+        }
+    }
     set_hist_smem_limits();
     set_sample_smem_limits();
     set_doc_smem_limits();
@@ -452,6 +463,16 @@ void lda_destroy(lda_ctx* h)
     Ctx& c = h->c;
     cudaSetDevice(c.device);
     cudaStreamSynchronize(c.stream);
+    if (c.have_side) {
+        for (int i = 0; i < 2; ++i) {
+            if (c.side[i]) {
+                cudaStreamSynchronize(c.side[i]);
+                cudaStreamDestroy(c.side[i]);
+            }
+            if (c.ev_join[i]) cudaEventDestroy(c.ev_join[i]);
+        }
+        if (c.ev_fork) cudaEventDestroy(c.ev_fork);
+    }
     if (c.have_events)
         for (int i = 0; i < 10; ++i) cudaEventDestroy(c.ev[i]);
     dev_free_all(c);

@@ -415,14 +415,16 @@ static int count_wk_t(Ctx& c)
     View& v = c.v;
     int launches = 0;
     const T* z = (const T*)v.zw;
+    // the tail words' rows and the hot words' rows are built side by side
+    fork_streams(c);
     if (c.n_word_tiles) {
         if (c.K <= WORD_ROWS_BITMAP_MAX_K) {
             const size_t smem = 2 * (size_t)((c.K + 31) / 32) * 4;
-            k_word_rows<T><<<c.n_word_tiles, 256, smem, c.stream>>>(c.word_tiles, v.word_off, z, v.row_start,
-                                                                   v.wk_topic, v.wk_count, v.wk_nnz, c.K, v.err);
+            k_word_rows<T><<<c.n_word_tiles, 256, smem, c.side[0]>>>(c.word_tiles, v.word_off, z, v.row_start,
+                                                                    v.wk_topic, v.wk_count, v.wk_nnz, c.K, v.err);
         } else {
             EmitWord e{v.row_start, v.wk_topic, v.wk_count, v.wk_nnz};
-            k_seg_count_sorted<T, EmitWord><<<c.n_word_tiles, 256, 0, c.stream>>>(
+            k_seg_count_sorted<T, EmitWord><<<c.n_word_tiles, 256, 0, c.side[0]>>>(
                 c.word_tiles, v.word_off, z, v.topic_bits, c.K, e, v.err);
         }
         ++launches;
@@ -437,6 +439,7 @@ static int count_wk_t(Ctx& c)
                                                          v.wk_nnz, c.K, v.dense_stride, v.err);
         launches += 2;
     }
+    join_streams(c);
     return launches;
 }
 
@@ -447,6 +450,8 @@ static int count_k(Ctx& c)
     cudaMemsetAsync(v.nk, 0, (size_t)c.K * 4, c.stream);
     if (c.N == 0) return 0;
     int launches = 0;
+    // both kernels add into n_k (integer adds: any order gives the same sums)
+    fork_streams(c);
     if (c.n_dense) {
         const dim3 grid((unsigned)((c.K + 255) / 256), (unsigned)std::min(c.n_dense, 64));
         k_nk_from_dense<<<grid, 256, 0, c.stream>>>(v.dense_rows, c.n_dense, c.K, v.dense_stride, v.nk);
@@ -455,10 +460,11 @@ static int count_k(Ctx& c)
     if (c.n_dense < c.V) {
         const int win = hist_window(c);
         const int grid = std::min(148 * 2, (int)((c.V + 511) / 512));
-        k_nk_from_sparse<<<grid, 512, (size_t)win * 4, c.stream>>>(v.row_start, v.wk_nnz, v.wk_topic, v.wk_count,
-                                                                  v.dense_slot, c.V, v.nk, c.K, win);
+        k_nk_from_sparse<<<grid, 512, (size_t)win * 4, c.side[0]>>>(v.row_start, v.wk_nnz, v.wk_topic, v.wk_count,
+                                                                   v.dense_slot, c.V, v.nk, c.K, win);
         ++launches;
     }
+    join_streams(c);
     return launches;
 }
 

@@ -182,8 +182,27 @@ struct Ctx {
     int64_t launches = 0;
     cudaEvent_t ev[10] = {};  // 0..6 bracket the phases of a sweep, 8 and 9 the passes of the MH step
     bool have_events = false;
+    // Two more streams for kernels of one phase that touch different words: fork_streams() makes them
+    // wait for the work queued on `stream` so far, join_streams() makes `stream` wait for theirs.
+    cudaStream_t side[2] = {};
+    cudaEvent_t ev_fork = nullptr, ev_join[2] = {};
+    bool have_side = false;
     std::string err;
 };
+
+inline void fork_streams(Ctx& c)
+{
+    cudaEventRecord(c.ev_fork, c.stream);
+    for (int i = 0; i < 2; ++i) cudaStreamWaitEvent(c.side[i], c.ev_fork, 0);
+}
+
+inline void join_streams(Ctx& c)
+{
+    for (int i = 0; i < 2; ++i) {
+        cudaEventRecord(c.ev_join[i], c.side[i]);
+        cudaStreamWaitEvent(c.stream, c.ev_join[i], 0);
+    }
+}
 
 // --- launchers (each returns the number of kernels it launched) -----------------
 int launch_init(Ctx& c);
