@@ -245,6 +245,18 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
     }
 }
 
+// The new topic goes out together with the other half of its pair (the word-proposal of this step,
+// which nobody reads any more; pass 1 of the next step overwrites it): a whole word per token, so
+// that the runs the tile writes fill their sectors and L2 has nothing to merge them with.
+__device__ __forceinline__ void store_topic_pair(uint16_t* zbm, uint32_t at, uint32_t s)
+{
+    __stcs(reinterpret_cast<uint32_t*>(zbm) + at, s);
+}
+__device__ __forceinline__ void store_topic_pair(int32_t* zbm, uint32_t at, uint32_t s)
+{
+    __stcs(reinterpret_cast<uint2*>(zbm) + at, make_uint2(s, 0u));
+}
+
 // --- pass 3: accept / reject (word order) -----------------------------------------------------------
 // Runs the chain of every token of the tile: everything the document side contributes was
 // gathered by pass 2, the word side comes from the tile's staged rows.
@@ -357,7 +369,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
             }
         }
         __stcs(zw + p, (T)s);
-        __stcs(reinterpret_cast<T*>(v.zbm) + 2 * (size_t)at, (T)s);
+        store_topic_pair(reinterpret_cast<T*>(v.zbm), at, s);
     }
     if (bad) atomicOr(v.err, ERR_COUNT_ZERO);
 }

@@ -142,6 +142,25 @@ def test_counts_consistent_with_own_assignments(small_corpus):
         assert np.array_equal(ro, np.searchsorted(uk // c.K, np.arange(rows + 1)))
 
 
+def test_checkpoint_and_warm_start_continue_bit_exactly(small_corpus):
+    """Section 6 (fault tolerance by warm start): the assignments are the whole checkpoint.  A fresh
+    context given z, the seed and the sweep counter continues exactly like the one that never stopped."""
+    c = small_corpus
+    a = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
+    a.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    a.init(SEED)
+    a.sweep(2, 2)
+    z_ckpt = a.get_assignments().copy()
+    a.sweep(2, 2)
+    b = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
+    b.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    b.set_assignments(z_ckpt, SEED, 2)
+    b.sweep(2, 2)
+    assert np.array_equal(a.get_assignments(), b.get_assignments())
+    assert np.array_equal(a.get_nk(), b.get_nk())
+    assert a.loglik() == b.loglik()
+
+
 @pytest.mark.parametrize("dense_frac", [0.0, 1.0])
 def test_dense_sparse_split_is_invisible(tiny_corpus, dense_frac):
     """Section 5: the hybrid row storage must not change any result."""
