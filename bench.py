@@ -224,21 +224,25 @@ def run_ours(args):
     # --- end to end through the host-buffer entry points -----------------------------------
     e2e = None
     if not args.no_e2e and args.e2e_steps > 0:
-        z_host = torch.empty(N, dtype=torch.int32).pin_memory()
-        binding.lda_get_assignments_ptr(lda._h, z_host.data_ptr())
+        # topics cross the host link in 16 bits when the library stores them so (K <= 65536)
+        narrow = cfg["K"] <= 65536
+        zb = 2 if narrow else 4
+        z_host = torch.empty(N, dtype=torch.int16 if narrow else torch.int32).pin_memory()
+        set_z = binding.lda_set_assignments_u16_ptr if narrow else binding.lda_set_assignments_ptr
+        get_z = binding.lda_get_assignments_u16_ptr if narrow else binding.lda_get_assignments_ptr
+        get_z(lda._h, z_host.data_ptr())
         # one untimed round trip first (first touch of the pinned buffer, lazy initialisations)
-        rc = binding.lda_set_assignments_ptr(lda._h, z_host.data_ptr(), 1234 + rank, st1["sweeps_done"])
+        rc = set_z(lda._h, z_host.data_ptr(), 1234 + rank, st1["sweeps_done"])
         assert rc == 0, binding.lda_last_error(lda._h)
         barrier()
         t0 = time.perf_counter()
         ev0.record(stream)
         ll = None
         for i in range(args.e2e_steps):
-            rc = binding.lda_set_assignments_ptr(lda._h, z_host.data_ptr(), 1234 + rank,
-                                                 st1["sweeps_done"] + i)
+            rc = set_z(lda._h, z_host.data_ptr(), 1234 + rank, st1["sweeps_done"] + i)
             assert rc == 0, binding.lda_last_error(lda._h)
             lda.sweep(1, M)
-            rc = binding.lda_get_assignments_ptr(lda._h, z_host.data_ptr())
+            rc = get_z(lda._h, z_host.data_ptr())
             assert rc == 0
             ll = lda.loglik()
         ev1.record(stream)
@@ -247,10 +251,11 @@ def run_ours(args):
         wall_ms = (time.perf_counter() - t0) * 1e3
         e_ms = max(e_ms, wall_ms)   # host-side work between calls counts too
         e_ms, _ = over_ranks(dist, "cuda", e_ms, N)
+        sfx = "_u16" if narrow else ""
         e2e = {"value": total_tokens / (e_ms / args.e2e_steps * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": 4 * N, "d2h_bytes_per_step": 4 * N + 24,
+               "h2d_bytes_per_step": zb * N, "d2h_bytes_per_step": zb * N + 24,
                "steps": args.e2e_steps, "loglik": ll[0] if ll else None,
-               "what": "lda_set_assignments(host z) + lda_sweep(1) + lda_get_assignments(host z) + lda_loglik"}
+               "what": f"lda_set_assignments{sfx}(host z) + lda_sweep(1) + lda_get_assignments{sfx}(host z) + lda_loglik"}
         del z_host
 
     if rank != 0:

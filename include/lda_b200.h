@@ -115,6 +115,10 @@ int lda_init(lda_ctx* ctx, uint64_t seed);
  * entries in the caller's document order, each in [0,K). */
 int lda_set_assignments(lda_ctx* ctx, const int32_t* z, uint64_t seed, uint32_t sweep);
 
+/* The same with 16-bit topics: half the bytes over the host link.  Needs K <= 65536 (the library
+ * then stores topics in 16 bits itself); LDA_ERANGE otherwise. */
+int lda_set_assignments_u16(lda_ctx* ctx, const uint16_t* z, uint64_t seed, uint32_t sweep);
+
 /* `iters` frozen-counts sweeps of `mh_steps` proposals per token (Section 4.2-4.3,
  * Eq. 6-13; Section 6 "immutable model"), the proposal of each step chosen by
  * lda_set_proposals().  Randomness: one Philox block per (token, sweep, step), counter
@@ -134,6 +138,9 @@ int lda_get_counts(lda_ctx* ctx, int which, int64_t* row_offsets, int32_t* topic
 
 /* Current assignments, n_tokens entries in the caller's document order. */
 int lda_get_assignments(lda_ctx* ctx, int32_t* z_out);
+
+/* The same as 16-bit topics; needs K <= 65536, LDA_ERANGE otherwise. */
+int lda_get_assignments_u16(lda_ctx* ctx, uint16_t* z_out);
 
 /* Word-proposal tables built from the current counts (Section 4.2): per-word sparse
  * alias tables indexed like the LDA_NWK rows (split point as a 32-bit fraction,

@@ -21,8 +21,8 @@ LDA_NK, LDA_NWK, LDA_NDK = 0, 1, 2
 
 EXPORTS = [
     "lda_create", "lda_set_stream", "lda_set_option", "lda_set_proposals", "lda_load_corpus", "lda_load_corpus_device",
-    "lda_init", "lda_set_assignments", "lda_sweep", "lda_loglik", "lda_get_counts",
-    "lda_get_assignments", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
+    "lda_init", "lda_set_assignments", "lda_set_assignments_u16", "lda_sweep", "lda_loglik", "lda_get_counts",
+    "lda_get_assignments", "lda_get_assignments_u16", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
     "lda_dense_table_noalloc",
 ]
 
@@ -75,10 +75,12 @@ def load_library(path: str | None = None):
     L.lda_load_corpus_device.argtypes = [vp, vp, i64, vp, i64]
     L.lda_init.argtypes = [vp, u64]
     L.lda_set_assignments.argtypes = [vp, vp, u64, u32]
+    L.lda_set_assignments_u16.argtypes = [vp, vp, u64, u32]
     L.lda_sweep.argtypes = [vp, i32, i32]
     L.lda_loglik.argtypes = [vp, C.POINTER(dbl), C.POINTER(dbl), C.POINTER(dbl)]
     L.lda_get_counts.argtypes = [vp, C.c_int, vp, vp, vp, i64, C.POINTER(i64)]
     L.lda_get_assignments.argtypes = [vp, vp]
+    L.lda_get_assignments_u16.argtypes = [vp, vp]
     L.lda_get_tables.argtypes = [vp, vp, vp, i64, vp, vp, vp, C.POINTER(u64)]
     L.lda_get_stats.argtypes = [vp, C.POINTER(lda_stats)]
     L.lda_dense_table_noalloc.argtypes = [vp, i32, i32, dbl, vp, vp, vp, vp, vp]
@@ -143,6 +145,15 @@ def lda_set_assignments_ptr(h, z_host_ptr, seed, sweep=0):
     return load_library().lda_set_assignments(h, C.c_void_p(z_host_ptr), seed, sweep)
 
 
+def lda_set_assignments_u16(h, z, seed, sweep=0):
+    z = np.ascontiguousarray(z, np.uint16)
+    return load_library().lda_set_assignments_u16(h, z.ctypes.data, seed, sweep)
+
+
+def lda_set_assignments_u16_ptr(h, z_host_ptr, seed, sweep=0):
+    return load_library().lda_set_assignments_u16(h, C.c_void_p(z_host_ptr), seed, sweep)
+
+
 def lda_sweep(h, iters, mh_steps):
     return load_library().lda_sweep(h, iters, mh_steps)
 
@@ -171,6 +182,14 @@ def lda_get_assignments(h, z_out):
 
 def lda_get_assignments_ptr(h, z_host_ptr):
     return load_library().lda_get_assignments(h, C.c_void_p(z_host_ptr))
+
+
+def lda_get_assignments_u16(h, z_out):
+    return load_library().lda_get_assignments_u16(h, z_out.ctypes.data)
+
+
+def lda_get_assignments_u16_ptr(h, z_host_ptr):
+    return load_library().lda_get_assignments_u16(h, C.c_void_p(z_host_ptr))
 
 
 def lda_get_tables(h, sp_thr32, sp_alias, mix32, dn_thr32, dn_alias):
@@ -263,6 +282,9 @@ class LightLDA:
     def set_assignments(self, z, seed: int, sweep: int = 0):
         self._ck(lda_set_assignments(self._h, z, seed, sweep), "lda_set_assignments")
 
+    def set_assignments_u16(self, z, seed: int, sweep: int = 0):
+        self._ck(lda_set_assignments_u16(self._h, z, seed, sweep), "lda_set_assignments_u16")
+
     def set_proposals(self, mode: int):
         """PROPOSALS_CYCLE (word, doc, word, ...), PROPOSALS_WORD or PROPOSALS_DOC (Section 4.3)."""
         self._ck(lda_set_proposals(self._h, mode), "lda_set_proposals")
@@ -295,6 +317,11 @@ class LightLDA:
     def get_assignments(self) -> np.ndarray:
         out = np.zeros(max(self.N, 1), np.int32)
         self._ck(lda_get_assignments(self._h, out), "lda_get_assignments")
+        return out[:self.N]
+
+    def get_assignments_u16(self) -> np.ndarray:
+        out = np.zeros(max(self.N, 1), np.uint16)
+        self._ck(lda_get_assignments_u16(self._h, out), "lda_get_assignments_u16")
         return out[:self.N]
 
     def get_tables(self):

@@ -584,21 +584,23 @@ int lda_init(lda_ctx* h, uint64_t seed)
     return LDA_OK;
 }
 
-int lda_set_assignments(lda_ctx* h, const int32_t* z, uint64_t seed, uint32_t sweep)
+static int set_assignments(lda_ctx* h, const void* z, bool narrow, uint64_t seed, uint32_t sweep)
 {
     if (!h) return LDA_EINVAL;
     Ctx& c = h->c;
     if (!c.loaded) return fail(&c, LDA_ESTATE, "lda_set_assignments before lda_load_corpus");
+    if (narrow && c.wide_topics) return fail(&c, LDA_ERANGE, "16-bit assignments need K <= 65536");
     if (c.N > 0 && !z) return fail(&c, LDA_EINVAL, "null assignments");
     int rc = check_device(c);
     if (rc) return rc;
     // the record array (one word per token, only meaningful while the exported n_kd is valid)
     // doubles as the staging buffer: no allocation here
-    int32_t* zdev = reinterpret_cast<int32_t*>(c.v.rec);
+    void* zdev = c.v.rec;
     c.dk_valid = false;
-    if (c.N > 0 && cudaMemcpyAsync(zdev, z, (size_t)c.N * 4, cudaMemcpyHostToDevice, c.stream) != cudaSuccess)
+    if (c.N > 0 &&
+        cudaMemcpyAsync(zdev, z, (size_t)c.N * (narrow ? 2 : 4), cudaMemcpyHostToDevice, c.stream) != cudaSuccess)
         return cuda_fail(&c, "copying assignments");
-    launch_spread_assignments(c, zdev);
+    launch_spread_assignments(c, zdev, narrow);
     int bits = 0;
     rc = read_err(c, &bits);
     if (rc) return rc;
@@ -610,6 +612,16 @@ int lda_set_assignments(lda_ctx* h, const int32_t* z, uint64_t seed, uint32_t sw
     if (bits) return fail(&c, LDA_EINTERNAL, "count rebuild raised the device error word");
     c.inited = true;
     return LDA_OK;
+}
+
+int lda_set_assignments(lda_ctx* h, const int32_t* z, uint64_t seed, uint32_t sweep)
+{
+    return set_assignments(h, z, false, seed, sweep);
+}
+
+int lda_set_assignments_u16(lda_ctx* h, const uint16_t* z, uint64_t seed, uint32_t sweep)
+{
+    return set_assignments(h, z, true, seed, sweep);
 }
 
 int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
@@ -764,23 +776,29 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
     return LDA_OK;
 }
 
-int lda_get_assignments(lda_ctx* h, int32_t* z_out)
+static int get_assignments(lda_ctx* h, void* z_out, bool narrow)
 {
     if (!h) return LDA_EINVAL;
     Ctx& c = h->c;
     if (!c.inited) return fail(&c, LDA_ESTATE, "lda_get_assignments before lda_init");
+    if (narrow && c.wide_topics) return fail(&c, LDA_ERANGE, "16-bit assignments need K <= 65536");
     if (c.N > 0 && !z_out) return fail(&c, LDA_EINVAL, "null output");
     if (c.N == 0) return LDA_OK;
     int rc = check_device(c);
     if (rc) return rc;
-    int32_t* zdev = reinterpret_cast<int32_t*>(c.v.rec);  // staging, see lda_set_assignments
+    void* zdev = c.v.rec;  // staging, see set_assignments()
     c.dk_valid = false;
-    launch_export_assignments(c, zdev);
-    cudaError_t e = cudaMemcpyAsync(z_out, zdev, (size_t)c.N * 4, cudaMemcpyDeviceToHost, c.stream);
+    launch_export_assignments(c, zdev, narrow);
+    cudaError_t e =
+        cudaMemcpyAsync(z_out, zdev, (size_t)c.N * (narrow ? 2 : 4), cudaMemcpyDeviceToHost, c.stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
     if (e != cudaSuccess) return cuda_fail(&c, "copying assignments");
     return LDA_OK;
 }
+
+int lda_get_assignments(lda_ctx* h, int32_t* z_out) { return get_assignments(h, z_out, false); }
+
+int lda_get_assignments_u16(lda_ctx* h, uint16_t* z_out) { return get_assignments(h, z_out, true); }
 
 int lda_get_tables(lda_ctx* h, uint32_t* sp_thr32, int32_t* sp_alias, int64_t capacity, uint32_t* mix32,
                    uint32_t* dn_thr32, int32_t* dn_alias, uint64_t* dense_mass)

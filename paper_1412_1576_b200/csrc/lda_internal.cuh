@@ -206,8 +206,8 @@ inline void join_streams(Ctx& c)
 
 // --- launchers (each returns the number of kernels it launched) -----------------
 int launch_init(Ctx& c);
-int launch_spread_assignments(Ctx& c, const int32_t* z_dev);  // z (doc order, i32) -> both layouts
-int launch_export_assignments(Ctx& c, int32_t* z_dev);
+int launch_spread_assignments(Ctx& c, const void* z_dev, bool narrow);  // z (doc order; u16 if narrow, else i32) -> both layouts
+int launch_export_assignments(Ctx& c, void* z_dev, bool narrow);
 int launch_count_wk(Ctx& c);
 int launch_count_k(Ctx& c);
 int launch_count_dk(Ctx& c);

@@ -476,30 +476,41 @@ __global__ void k_init(View v, uint2 key)
     }
 }
 
-template <typename T>
-__global__ void k_spread(View v, const int32_t* __restrict__ z_in)
+// Import of assignments given in the caller's document order (IN = int32_t or uint16_t), in two
+// steps that each stay coalesced on one side: document order -> block-major order (the scattered
+// writes stay inside one block of that order at a time), then block-major -> word order.
+template <typename T, typename IN>
+__global__ void k_spread(View v, const IN* __restrict__ z_in)
 {
-    T* zw = reinterpret_cast<T*>(v.zw);
     T* zbm = reinterpret_cast<T*>(v.zbm);
-    for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < v.N;
-         p += (int64_t)gridDim.x * blockDim.x) {
-        int32_t a = z_in[v.tok_orig[p]];
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < v.N;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t a = (int64_t)z_in[i];
         if (a < 0 || a >= v.K) {
             atomicOr(v.err, ERR_TOPIC_RANGE);
             a = 0;
         }
-        zw[p] = (T)a;
-        zbm[2 * (size_t)v.inv[p]] = (T)a;
+        zbm[2 * (size_t)__ldcs(v.bm_of_tok + i)] = (T)a;
     }
 }
 
 template <typename T>
-__global__ void k_export(View v, int32_t* __restrict__ out)
+__global__ void k_word_order_topics(View v)
+{
+    T* zw = reinterpret_cast<T*>(v.zw);
+    const T* zbm = reinterpret_cast<const T*>(v.zbm);
+    for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < v.N;
+         p += (int64_t)gridDim.x * blockDim.x)
+        zw[p] = zbm[2 * (size_t)__ldcs(v.inv + p)];
+}
+
+template <typename T, typename OUT>
+__global__ void k_export(View v, OUT* __restrict__ out)
 {
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < v.N;
          i += (int64_t)gridDim.x * blockDim.x)
-        out[i] = (int32_t)zbm[2 * (size_t)v.bm_of_tok[i]];
+        out[i] = (OUT)zbm[2 * (size_t)v.bm_of_tok[i]];
 }
 
 static int grid_for(int64_t n, int block)
@@ -639,20 +650,29 @@ int launch_init(Ctx& c)
     return 1;
 }
 
-int launch_spread_assignments(Ctx& c, const int32_t* z_dev)
+// `narrow`: the caller's array holds 16-bit topics (only with 16-bit topic storage), else int32.
+int launch_spread_assignments(Ctx& c, const void* z_dev, bool narrow)
 {
     if (c.N == 0) return 0;
     const int g = grid_for(c.N, 256);
-    if (c.wide_topics) k_spread<int32_t><<<g, 256, 0, c.stream>>>(c.v, z_dev);
-    else k_spread<uint16_t><<<g, 256, 0, c.stream>>>(c.v, z_dev);
-    return 1;
+    if (c.wide_topics) {
+        k_spread<int32_t, int32_t><<<g, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev);
+        k_word_order_topics<int32_t><<<g, 256, 0, c.stream>>>(c.v);
+    } else {
+        if (narrow) k_spread<uint16_t, uint16_t><<<g, 256, 0, c.stream>>>(c.v, (const uint16_t*)z_dev);
+        else k_spread<uint16_t, int32_t><<<g, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev);
+        k_word_order_topics<uint16_t><<<g, 256, 0, c.stream>>>(c.v);
+    }
+    return 2;
 }
 
-int launch_export_assignments(Ctx& c, int32_t* z_dev)
+int launch_export_assignments(Ctx& c, void* z_dev, bool narrow)
 {
     if (c.N == 0) return 0;
-    if (c.wide_topics) k_export<int32_t><<<grid_for(c.N, 256), 256, 0, c.stream>>>(c.v, z_dev);
-    else k_export<uint16_t><<<grid_for(c.N, 256), 256, 0, c.stream>>>(c.v, z_dev);
+    const int g = grid_for(c.N, 256);
+    if (c.wide_topics) k_export<int32_t, int32_t><<<g, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev);
+    else if (narrow) k_export<uint16_t, uint16_t><<<g, 256, 0, c.stream>>>(c.v, (uint16_t*)z_dev);
+    else k_export<uint16_t, int32_t><<<g, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev);
     return 1;
 }
 

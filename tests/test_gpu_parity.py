@@ -161,6 +161,37 @@ def test_checkpoint_and_warm_start_continue_bit_exactly(small_corpus):
     assert a.loglik() == b.loglik()
 
 
+def test_sixteen_bit_import_and_export(small_corpus):
+    c = small_corpus
+    g, o = _pair(c, seed=4)
+    g.sweep(1, 2)
+    o.sweep(1, 2)
+    z16 = g.get_assignments_u16()
+    assert z16.dtype == np.uint16 and np.array_equal(z16.astype(np.int32), o.get_assignments())
+    h = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
+    h.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    h.set_assignments_u16(z16, 4, 1)
+    _assert_same_counts(h, o)
+    h.sweep(1, 2)
+    o.sweep(1, 2)
+    assert np.array_equal(h.get_assignments(), o.get_assignments())
+    bad = z16.copy()
+    bad[5] = c.K
+    with pytest.raises(binding.LdaError) as e:
+        h.set_assignments_u16(bad, 4, 1)
+    assert e.value.status == binding.LDA_ERANGE
+    # 32-bit topic storage has no 16-bit form
+    w = binding.LightLDA(8, 70_000, 0.1, 0.1)
+    w.load_corpus(np.array([0, 1, 2], np.int32), np.array([0, 3], np.int64))
+    w.init(1)
+    with pytest.raises(binding.LdaError) as e:
+        w.get_assignments_u16()
+    assert e.value.status == binding.LDA_ERANGE
+    with pytest.raises(binding.LdaError) as e:
+        w.set_assignments_u16(np.zeros(3, np.uint16), 1)
+    assert e.value.status == binding.LDA_ERANGE
+
+
 @pytest.mark.parametrize("dense_frac", [0.0, 1.0])
 def test_dense_sparse_split_is_invisible(tiny_corpus, dense_frac):
     """Section 5: the hybrid row storage must not change any result."""
