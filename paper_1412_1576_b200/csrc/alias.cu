@@ -119,34 +119,40 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
         if (r == 0) atomicOr(err, ERR_ALIAS);
         return W44;
     }
-    uint32_t L = 0, H = 0;
-    ull d_sum = 0, e_sum = 0;
-    for (int32_t i0 = 0; i0 < n; i0 += gs) {
-        const int32_t i = i0 + r;
-        const bool valid = i < n;
-        const ull a = valid ? (ull)n * (sc_w[i] >> sh) : 0;
-        const bool light = valid && a <= W, heavy = valid && a > W;
-        const ull def = light ? W - a : 0, sur = heavy ? a - W : 0;
-        ull pre[3] = {(light ? 1ull : 0ull) | (heavy ? (1ull << 32) : 0ull), def, sur}, tot[3];
-        g.scan_excl3(pre, tot);
-        const ull c_pre = pre[0], d_pre = pre[1], e_pre = pre[2];
-        const ull c_tot = tot[0], d_tot = tot[1], e_tot = tot[2];
-        if (valid) sc_w[i] = a;
-        if (light) {
-            const uint32_t l = L + (uint32_t)c_pre;
-            sc_de[l] = d_sum + d_pre;
-            sc_item[l] = (uint32_t)i;
-        }
-        if (heavy) {
-            const uint32_t m = H + (uint32_t)(c_pre >> 32);
-            sc_de[n - 1 - m] = e_sum + e_pre + sur;
-            sc_item[n - 1 - m] = (uint32_t)i;
-        }
-        L += (uint32_t)c_tot;
-        H += (uint32_t)(c_tot >> 32);
-        d_sum += d_tot;
-        e_sum += e_tot;
+    // Every thread takes a run of consecutive items (lights and heavies are numbered in ascending
+    // item order): one pass to count them and add up their deficits and surpluses, one scan of the
+    // threads' totals, one pass to write the prefix of every item.
+    g.sync();  // the weights were written item by item across the group
+    const int32_t seg = (n + gs - 1) / gs;
+    const int32_t i_first = min(n, r * seg), i_last = min(n, i_first + seg);
+    ull cnt = 0, d_mine = 0, e_mine = 0;
+    for (int32_t i = i_first; i < i_last; ++i) {
+        const ull a = (ull)n * (sc_w[i] >> sh);
+        if (a <= W) { cnt += 1ull; d_mine += W - a; } else { cnt += 1ull << 32; e_mine += a - W; }
     }
+    ull pre[3] = {cnt, d_mine, e_mine}, tot[3];
+    g.scan_excl3(pre, tot);
+    {
+        uint32_t l = (uint32_t)pre[0], m = (uint32_t)(pre[0] >> 32);
+        ull d_at = pre[1], e_at = pre[2];
+        for (int32_t i = i_first; i < i_last; ++i) {
+            const ull a = (ull)n * (sc_w[i] >> sh);
+            sc_w[i] = a;
+            if (a <= W) {
+                sc_de[l] = d_at;  // deficits of the lights before this one
+                sc_item[l] = (uint32_t)i;
+                ++l;
+                d_at += W - a;
+            } else {
+                e_at += a - W;
+                sc_de[n - 1 - m] = e_at;  // surpluses of the heavies up to and including this one
+                sc_item[n - 1 - m] = (uint32_t)i;
+                ++m;
+            }
+        }
+    }
+    const uint32_t L = (uint32_t)tot[0], H = (uint32_t)(tot[0] >> 32);
+    const ull d_sum = tot[1];
     g.sync();
     for (uint32_t l = r; l < L; l += gs) {
         const uint32_t i = sc_item[l];
