@@ -31,8 +31,12 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 #define LDA_PROPOSE_MIN_CTAS 2
 #endif
 #ifndef LDA_PROPOSE_FIXED_MIN_CTAS
-#define LDA_PROPOSE_FIXED_MIN_CTAS 3
+#define LDA_PROPOSE_FIXED_MIN_CTAS 4
 #endif
+#ifndef LDA_PROPOSE_TOKENS
+#define LDA_PROPOSE_TOKENS 2
+#endif
+constexpr int PROPOSE_TOKENS = LDA_PROPOSE_TOKENS;  // tokens a thread of the two-step propose kernel takes per turn
 #ifndef LDA_ACCEPT_FIXED2_THREADS
 #define LDA_ACCEPT_FIXED2_THREADS 768
 #endif
@@ -220,27 +224,62 @@ struct ColdTile {
 // tile's tokens.
 // A proposal depends on (token, sweep, step) and the frozen tables only, never on the chain's
 // state, so all of them can be drawn before anything is accepted.
-template <typename T, int MODE, class Tile>
+template <typename T, int MODE, int FIXED, class Tile>
 __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, const int32_t p_begin,
                                                const int32_t p_end, const int32_t nthreads, const uint2 key,
                                                const uint32_t sweep, const int32_t mh_steps)
 {
     T* prop = reinterpret_cast<T*>(v.prop);
-    for (int32_t p = p_begin + (int32_t)threadIdx.x; p < p_end; p += nthreads) {
-        const uint32_t tok = __ldcs(v.tok_orig + p);
-        const uint32_t at = __ldcs(v.inv + p);  // the document-side pass reads block-major
-        const typename Tile::Ref w = tile.ref(p - p_begin);
-        for (int32_t m = 0; m < mh_steps; m += (MODE == LDA_PROPOSALS_CYCLE ? 2 : 1)) {
-            const int32_t wi = step_kind_index<MODE>(m);
-            const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)m, 0u), key);
-            const Draw d = tile.draw_issue(w, v, r);
-            uint32_t t;
-            int32_t n_tw;
-            tile.draw_finish(w, d, t, n_tw);
-            // the first proposal goes beside the token's topic, the later ones to arrays of their own
-            if (wi == 0) __stcs(reinterpret_cast<T*>(v.zbm) + 2 * (size_t)at + 1, (T)t);
-            else __stcs(prop + (size_t)wi * v.N + at, (T)t);
-            __stcs(v.ua_w + (size_t)wi * v.N + p, r.w);  // the step's acceptance uniform, for pass 3
+    if (FIXED == 2 && MODE == LDA_PROPOSALS_CYCLE) {
+        // One word step per token: a thread takes PROPOSE_TOKENS tokens per turn, so that their
+        // table reads (the pass waits for little else) are in flight together.
+        constexpr int U = PROPOSE_TOKENS;
+        for (int32_t p0 = p_begin + (int32_t)threadIdx.x; p0 < p_end; p0 += U * nthreads) {
+            uint32_t tok[U], at[U], ua[U];
+            Draw d[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int32_t p = p0 + u * nthreads;
+                const bool live = p < p_end;
+                tok[u] = live ? __ldcs(v.tok_orig + p) : 0u;
+                at[u] = live ? __ldcs(v.inv + p) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int32_t p = p0 + u * nthreads;
+                const uint4 r = philox4x32_10(make_uint4(tok[u], sweep, 0u, 0u), key);
+                ua[u] = r.w;
+                d[u] = tile.draw_issue(tile.ref((p < p_end ? p : p0) - p_begin), v, r);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int32_t p = p0 + u * nthreads;
+                uint32_t t;
+                int32_t n_tw;
+                tile.draw_finish(tile.ref((p < p_end ? p : p0) - p_begin), d[u], t, n_tw);
+                if (p < p_end) {
+                    __stcs(reinterpret_cast<T*>(v.zbm) + 2 * (size_t)at[u] + 1, (T)t);
+                    __stcs(v.ua_w + p, ua[u]);
+                }
+            }
+        }
+    } else {
+        for (int32_t p = p_begin + (int32_t)threadIdx.x; p < p_end; p += nthreads) {
+            const uint32_t tok = __ldcs(v.tok_orig + p);
+            const uint32_t at = __ldcs(v.inv + p);  // the document-side pass reads block-major
+            const typename Tile::Ref w = tile.ref(p - p_begin);
+            for (int32_t m = 0; m < mh_steps; m += (MODE == LDA_PROPOSALS_CYCLE ? 2 : 1)) {
+                const int32_t wi = step_kind_index<MODE>(m);
+                const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)m, 0u), key);
+                const Draw d = tile.draw_issue(w, v, r);
+                uint32_t t;
+                int32_t n_tw;
+                tile.draw_finish(w, d, t, n_tw);
+                // the first proposal goes beside the token's topic, the later ones to arrays of their own
+                if (wi == 0) __stcs(reinterpret_cast<T*>(v.zbm) + 2 * (size_t)at + 1, (T)t);
+                else __stcs(prop + (size_t)wi * v.N + at, (T)t);
+                __stcs(v.ua_w + (size_t)wi * v.N + p, r.w);  // the step's acceptance uniform, for pass 3
+            }
         }
     }
 }
@@ -416,7 +455,7 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     tile.bar = &bar;
     tile.ready = !(STAGED && ACCEPT);
     if (ACCEPT) accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, accept_threads(FIXED), key, sweep, mh_steps);
-    else propose_tokens<T, MODE>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
+    else propose_tokens<T, MODE, FIXED>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
     // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one
 }
 
@@ -457,7 +496,7 @@ k_word_cold(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep
     __syncthreads();
     ColdTile tile{woff_s, rs_s, nnz_s, mix_s, topic_s, count_s, thr_s, idx_s, nw, v.nk};
     if (ACCEPT) accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
-    else propose_tokens<T, MODE>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
+    else propose_tokens<T, MODE, FIXED>(v, tile, p0, p0 + cnt, COLD_THREADS, key, sweep, mh_steps);
 }
 
 // z_i uniform on {0..K-1}: Philox counter (token, 0, 0, 1), word 0.
