@@ -207,12 +207,32 @@ k_hist_chunks(const int32_t* __restrict__ chunks, const T* __restrict__ z,
         const int32_t nb = min(window, K - k0), nw = (nb + 1) >> 1;
         for (int b = threadIdx.x; b < nw; b += blockDim.x) bins2[b] = 0;
         __syncthreads();
-        for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-            const uint32_t k = (uint32_t)z[first + j];
-            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+        auto add = [&](uint32_t k) {
+            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); return; }
             const uint32_t b = k - (uint32_t)k0;
             if (b < (uint32_t)nb) atomicAdd(&bins2[b >> 1], (b & 1u) ? 0x10000u : 1u);
+        };
+        // the chunk's topics are read 16 bytes at a time; what lies before the first and after the
+        // last 16-byte boundary one by one
+        constexpr int E = 16 / (int)sizeof(T);
+        const int32_t head = min(cnt, (int32_t)((E - (first & (E - 1))) & (E - 1)));
+        const int32_t nvec = (cnt - head) / E;
+        const uint4* zv = reinterpret_cast<const uint4*>(z + first + head);
+        for (int q = threadIdx.x; q < nvec; q += blockDim.x) {
+            const uint4 x = __ldcs(zv + q);
+            const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (sizeof(T) == 2) {
+                    add(xs[u] & 0xFFFFu);
+                    add(xs[u] >> 16);
+                } else {
+                    add(xs[u]);
+                }
+            }
         }
+        for (int j = threadIdx.x; j < cnt - nvec * E; j += blockDim.x)
+            add((uint32_t)z[first + (j < head ? j : nvec * E + j)]);
         __syncthreads();
         for (int b = threadIdx.x; b < nw; b += blockDim.x) {
             const uint32_t n2 = bins2[b];
