@@ -367,11 +367,20 @@ __global__ void __launch_bounds__(256)
 k_nk_from_dense(const int32_t* __restrict__ dense_rows, int32_t n_dense, int32_t K, int32_t stride,
                 int32_t* __restrict__ nk)
 {
-    const int32_t k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= K) return;
-    int32_t s = 0;
-    for (int32_t r = blockIdx.y; r < n_dense; r += gridDim.y) s += __ldcs(dense_rows + (size_t)r * stride + k);
-    if (s) atomicAdd(&nk[k], s);
+    // four consecutive topics per thread (rows are padded to a multiple of four and 16-byte aligned;
+    // the padding is never written, so it reads as zero), a slice of the rows per blockIdx.y
+    const int32_t k = 4 * (blockIdx.x * blockDim.x + threadIdx.x);
+    if (k >= stride) return;
+    int4 s = make_int4(0, 0, 0, 0);
+#pragma unroll 4
+    for (int32_t r = blockIdx.y; r < n_dense; r += gridDim.y) {
+        const int4 x = __ldcs(reinterpret_cast<const int4*>(dense_rows + (size_t)r * stride + k));
+        s.x += x.x; s.y += x.y; s.z += x.z; s.w += x.w;
+    }
+    if (s.x) atomicAdd(&nk[k], s.x);
+    if (s.y && k + 1 < K) atomicAdd(&nk[k + 1], s.y);
+    if (s.z && k + 2 < K) atomicAdd(&nk[k + 2], s.z);
+    if (s.w && k + 3 < K) atomicAdd(&nk[k + 3], s.w);
 }
 
 __global__ void __launch_bounds__(512)
@@ -473,13 +482,13 @@ static int count_k(Ctx& c)
     // both kernels add into n_k (integer adds: any order gives the same sums)
     fork_streams(c);
     if (c.n_dense) {
-        const dim3 grid((unsigned)((c.K + 255) / 256), (unsigned)std::min(c.n_dense, 64));
+        const dim3 grid((unsigned)((v.dense_stride / 4 + 255) / 256), (unsigned)std::min(c.n_dense, 256));
         k_nk_from_dense<<<grid, 256, 0, c.stream>>>(v.dense_rows, c.n_dense, c.K, v.dense_stride, v.nk);
         ++launches;
     }
     if (c.n_dense < c.V) {
         const int win = hist_window(c);
-        const int grid = std::min(148 * 2, (int)((c.V + 511) / 512));
+        const int grid = std::min(148 * 4, (int)((c.V + 511) / 512));
         k_nk_from_sparse<<<grid, 512, (size_t)win * 4, c.side[0]>>>(v.row_start, v.wk_nnz, v.wk_topic, v.wk_count,
                                                                    v.dense_slot, c.V, v.nk, c.K, win);
         ++launches;
