@@ -83,6 +83,33 @@ __device__ __forceinline__ uint32_t to_frac32(ull part, ull whole)
     return q > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)q;
 }
 
+// to_frac32(part, whole) for many parts <= whole of one whole: the quotient from a double
+// reciprocal of the (shifted) whole, then set right with the exact integer remainder.  The
+// estimate is within 2^-20 of the true quotient (two roundings of 2^-53 on a value <= 2^32), so
+// its integer part is off by one at most.
+struct Frac32 {
+    int sh;
+    uint32_t w;  // whole >> sh, < 2^32
+    double inv;  // 1 / w
+    __device__ __forceinline__ explicit Frac32(ull whole)
+    {
+        sh = bit_length(whole) - 32;
+        if (sh < 0) sh = 0;
+        w = (uint32_t)(whole >> sh);
+        inv = __ddiv_rn(1.0, u32_to_double(w));
+    }
+    __device__ __forceinline__ uint32_t operator()(ull part) const
+    {
+        const uint32_t p = (uint32_t)(part >> sh);  // part <= whole
+        const ull x = (ull)p << 32;
+        ull q = __double2ull_rz(__dmul_rn(__dmul_rn(u32_to_double(p), 4294967296.0), inv));
+        const long long r = (long long)(x - q * (ull)w);
+        if (r < 0) --q;
+        else if (r >= (long long)w) ++q;
+        return q > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)q;
+    }
+};
+
 // One bin in the form the MH kernel reads with a single load.  With `topic` (a word's sorted
 // row) the second word holds the topics of the bin's own item and of its alias item, 16 bits
 // each; without it (the dense table, whose items are the topics) it holds the alias.
@@ -98,9 +125,10 @@ __device__ __forceinline__ void store_packed_bin(uint2* out_pk, const uint32_t* 
 // out_pk (may be null) receives the packed form of every bin, see store_packed_bin().
 // Returns W44 (the sum of the fixed-point weights) to every thread of the group.
 template <bool BLOCK, class Weight>
-__device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, ull* sc_w, ull* sc_de,
-                               uint32_t* sc_item, uint32_t* out_thr, uint32_t* out_idx, uint2* out_pk,
-                               const uint32_t* pk_topic, int* err)
+__device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, ull* __restrict__ sc_w,
+                               ull* __restrict__ sc_de, uint32_t* __restrict__ sc_item,
+                               uint32_t* __restrict__ out_thr, uint32_t* __restrict__ out_idx,
+                               uint2* __restrict__ out_pk, const uint32_t* __restrict__ pk_topic, int* err)
 {
     const int r = g.rank(), gs = g.size();
     ull s = 0;
@@ -154,6 +182,7 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
     const uint32_t L = (uint32_t)tot[0], H = (uint32_t)(tot[0] >> 32);
     const ull d_sum = tot[1];
     g.sync();
+    const Frac32 frac(W);
     for (uint32_t l = r; l < L; l += gs) {
         const uint32_t i = sc_item[l];
         const ull a = sc_w[i];
@@ -168,7 +197,7 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
             if (lo >= H) { atomicOr(err, ERR_ALIAS); lo = H ? H - 1 : 0; }
             al = H ? sc_item[n - 1 - lo] : i;
         }
-        const uint32_t thr32 = to_frac32(a, W);
+        const uint32_t thr32 = frac(a);
         out_thr[i] = thr32;
         out_idx[i] = al;
         store_packed_bin(out_pk, pk_topic, i, thr32, al);
@@ -188,7 +217,7 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
             if (m + 1 >= H) atomicOr(err, ERR_ALIAS);
             else al = sc_item[n - 1 - (m + 1)];
         }
-        const uint32_t thr32 = to_frac32(thr, W);
+        const uint32_t thr32 = frac(thr);
         out_thr[i] = thr32;
         out_idx[i] = al;
         store_packed_bin(out_pk, pk_topic, i, thr32, al);
