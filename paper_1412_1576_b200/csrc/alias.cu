@@ -266,11 +266,18 @@ __device__ __forceinline__ uint32_t mixture_threshold(ull S, ull B)
     return to_frac32(S, S + B);
 }
 
-// One warp per word, rows of at most ALIAS_WARP_MAX items.
-__global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, ull* sc_de, uint32_t* sc_item)
+// One warp per word, rows of at most ALIAS_WARP_MAX items.  The two scratch arrays the binary
+// searches run over live in shared memory (12 bytes per item and warp), the third in the row's
+// range of the scratch array in device memory.
+__global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w)
 {
+    extern __shared__ __align__(16) unsigned char alias_scratch[];
     Group<false> g{nullptr};
     const int warps = (gridDim.x * blockDim.x) >> 5;
+    const int wic = threadIdx.x >> 5;
+    ull* de_s = reinterpret_cast<ull*>(alias_scratch) + (size_t)wic * ALIAS_WARP_MAX;
+    uint32_t* item_s = reinterpret_cast<uint32_t*>(reinterpret_cast<ull*>(alias_scratch) + 8 * ALIAS_WARP_MAX) +
+                       (size_t)wic * ALIAS_WARP_MAX;
     const ull B = *v.dense_mass;
     for (int32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < v.V; w += warps) {
         const int32_t n = v.wk_nnz[w];
@@ -281,9 +288,8 @@ __global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, ul
         }
         const int32_t r0 = v.row_start[w];
         SparseWeight wf{v.wk_topic + r0, v.wk_count + r0, v.nk, v.Vbeta};
-        const ull S = build_alias_row<false>(g, n, wf, sc_w + r0, sc_de + r0, sc_item + r0, v.al_thr + r0,
-                                             v.al_idx + r0, v.al_pk ? v.al_pk + r0 : nullptr,
-                                             v.wk_topic + r0, v.err);
+        const ull S = build_alias_row<false>(g, n, wf, sc_w + r0, de_s, item_s, v.al_thr + r0, v.al_idx + r0,
+                                             v.al_pk ? v.al_pk + r0 : nullptr, v.wk_topic + r0, v.err);
         if ((threadIdx.x & 31) == 0) v.mix32[w] = mixture_threshold(S, B);
         __syncwarp();
     }
@@ -353,7 +359,7 @@ int launch_alias_sparse(Ctx& c)
     }
     int grid = (int)(((int64_t)c.V * 32 + 255) / 256);
     if (grid > 148 * 16) grid = 148 * 16;
-    k_alias_sparse_warp<<<grid, 256, 0, c.side[1]>>>(c.v, c.sc_w, c.sc_de, c.sc_item);
+    k_alias_sparse_warp<<<grid, 256, ALIAS_WARP_SMEM, c.side[1]>>>(c.v, c.sc_w);
     ++launches;
     join_streams(c);
     return launches;
@@ -361,6 +367,7 @@ int launch_alias_sparse(Ctx& c)
 
 void set_alias_smem_limits()
 {
+    cudaFuncSetAttribute(k_alias_sparse_warp, cudaFuncAttributeMaxDynamicSharedMemorySize, ALIAS_WARP_SMEM);
     cudaFuncSetAttribute(k_alias_sparse_block<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          ALIAS_SMEM_ITEMS_MID * ALIAS_SCRATCH_PER_ITEM);
     cudaFuncSetAttribute(k_alias_sparse_block<512>, cudaFuncAttributeMaxDynamicSharedMemorySize,

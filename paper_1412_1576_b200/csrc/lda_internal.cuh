@@ -78,6 +78,7 @@ constexpr int HOT_STAGE_MAX_K = 16384;  // dense rows up to this many topics are
 #define LDA_ALIAS_WARP_MAX 512
 #endif
 constexpr int ALIAS_WARP_MAX = LDA_ALIAS_WARP_MAX;  // rows up to this many items are built by one warp
+constexpr int ALIAS_WARP_SMEM = 8 * ALIAS_WARP_MAX * 12;  // eight warps per CTA, 12 bytes of scratch per item
 constexpr int ALIAS_SCRATCH_PER_ITEM = 20;   // bytes of construction scratch per item
 #ifndef LDA_ALIAS_SMEM_ITEMS_MID
 #define LDA_ALIAS_SMEM_ITEMS_MID 2048
