@@ -47,11 +47,14 @@ constexpr int SORT_TILE = 2048;      // tokens per segmented-sort tile (one CTA)
 // Tiles of whole documents (one CTA each) of the document-side kernels: tokens per tile and
 // threads per CTA, chosen per corpus from these shapes; longer documents get a CTA of their own.
 constexpr int DOC_TILE_SHAPES = 4;
-constexpr int DOC_TILE_TOKENS[DOC_TILE_SHAPES] = {384, 768, 1536, 3072};
+#ifndef LDA_DOC_TILE_ROUNDS
+#define LDA_DOC_TILE_ROUNDS 3
+#endif
+constexpr int DOC_TILE_ROUNDS = LDA_DOC_TILE_ROUNDS;  // tokens per thread: every shape holds this many times its thread count
 constexpr int DOC_TILE_THREADS[DOC_TILE_SHAPES] = {128, 256, 512, 1024};
-constexpr int DOC_TILE_MAX = 3072;
-constexpr int DOC_TILE_ROUNDS = 3;  // tokens per thread: every shape holds 3 x its thread count
-static_assert(DOC_TILE_TOKENS[0] == 3 * DOC_TILE_THREADS[0] && DOC_TILE_TOKENS[3] == 3 * DOC_TILE_THREADS[3], "tile shapes");
+constexpr int DOC_TILE_TOKENS[DOC_TILE_SHAPES] = {DOC_TILE_ROUNDS * 128, DOC_TILE_ROUNDS * 256, DOC_TILE_ROUNDS * 512,
+                                                  DOC_TILE_ROUNDS * 1024};
+constexpr int DOC_TILE_MAX = DOC_TILE_ROUNDS * 1024;
 // shared memory per token of a tile: 4 table slots, document offset, topic/slot (4 bytes each)
 #ifndef LDA_DOC_TILE_SLOTS
 #define LDA_DOC_TILE_SLOTS 4
