@@ -111,8 +111,14 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
 // thread owns at most DOC_TILE_ROUNDS tokens and keeps what it read about them in registers across
 // the phases.  Small tiles keep many CTAs per SM, which is what hides the gathers of the first phase.
 // FIXED > 0: the number of steps is this compile-time constant (the argument is ignored).
+// Threads the compiler must leave room for per SM: the two-step kernels with a word step need few
+// enough registers to fill the SM (16 CTAs of 128 threads), the others three quarters of it.
+__host__ __device__ constexpr int doc_resident_threads(int mode, int fixed)
+{
+    return (fixed == 2 && mode != LDA_PROPOSALS_DOC) ? 2048 : 1536;
+}
 template <typename T, int THREADS, int MODE, int FIXED>
-__global__ void __launch_bounds__(THREADS, 1536 / THREADS)
+__global__ void __launch_bounds__(THREADS, doc_resident_threads(MODE, FIXED) / THREADS)
 k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps_arg)
 {
     const int32_t mh_steps = FIXED > 0 ? FIXED : mh_steps_arg;
