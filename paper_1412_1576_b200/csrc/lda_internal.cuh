@@ -71,7 +71,7 @@ constexpr int HIST16_BINS = 106496;  // window of the per-chunk n_kw histogram (
 constexpr int HIST_CHUNK = LDA_HIST_CHUNK;    // tokens per CTA in the histogram path
 static_assert(HIST_CHUNK < 65536, "the per-chunk histogram counts in 16 bits");
 #ifndef LDA_HOT_TILE
-#define LDA_HOT_TILE 8192
+#define LDA_HOT_TILE 16384
 #endif
 constexpr int HOT_TILE = LDA_HOT_TILE;  // MH kernels: tokens of one hot word per CTA
 constexpr int COLD_TILE = 2048;      // MH kernel: tokens of a tile of whole tail words
