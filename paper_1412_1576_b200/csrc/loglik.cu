@@ -11,15 +11,29 @@
 namespace lda {
 
 constexpr int LL_BLOCKS = 592;
+// Counts below this take lgamma(count + prior) - lgamma(prior) from a table in shared memory that
+// every CTA fills with the same expression: same values as calling lgamma() per entry.
+constexpr int LL_TABLE = 512;
+
+__device__ __forceinline__ void fill_ll_table(double* tab, double prior, double lg_prior)
+{
+    for (int c = threadIdx.x; c < LL_TABLE; c += blockDim.x) tab[c] = lgamma((double)c + prior) - lg_prior;
+    __syncthreads();
+}
 
 __global__ void __launch_bounds__(256) k_ll_word(View v, double lg_beta, double* __restrict__ out)
 {
     __shared__ double tmp[32];
+    __shared__ double small[LL_TABLE];
+    fill_ll_table(small, v.beta, lg_beta);
     const int warps = (gridDim.x * blockDim.x) >> 5, lane = threadIdx.x & 31;
     double s = 0.0;
     for (int32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < v.V; w += warps) {
         const int32_t r0 = v.row_start[w], n = v.wk_nnz[w];
-        for (int32_t j = lane; j < n; j += 32) s += lgamma((double)v.wk_count[r0 + j] + v.beta) - lg_beta;
+        for (int32_t j = lane; j < n; j += 32) {
+            const uint32_t c = v.wk_count[r0 + j];
+            s += c < (uint32_t)LL_TABLE ? small[c] : lgamma((double)c + v.beta) - lg_beta;
+        }
     }
     for (int32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < v.K; k += gridDim.x * blockDim.x)
         s -= lgamma((double)v.nk[k] + v.Vbeta);
@@ -30,6 +44,8 @@ __global__ void __launch_bounds__(256) k_ll_word(View v, double lg_beta, double*
 __global__ void __launch_bounds__(256) k_ll_doc(View v, double lg_alpha, double* __restrict__ out)
 {
     __shared__ double tmp[32];
+    __shared__ double small[LL_TABLE];
+    fill_ll_table(small, v.alpha, lg_alpha);
     const int warps = (gridDim.x * blockDim.x) >> 5, lane = threadIdx.x & 31;
     const uint32_t cmask = (1u << v.count_bits) - 1u;
     double s = 0.0;
@@ -38,7 +54,10 @@ __global__ void __launch_bounds__(256) k_ll_doc(View v, double lg_alpha, double*
         const uint32_t* tab = v.dk_slots + DK_SLOTS_PER_TOKEN * (size_t)d0;
         for (int32_t j = lane; j < n; j += 32) {
             const uint32_t e = tab[j];
-            if (e != DK_EMPTY) s += lgamma((double)(e & cmask) + v.alpha) - lg_alpha;
+            if (e != DK_EMPTY) {
+                const uint32_t c = e & cmask;
+                s += c < (uint32_t)LL_TABLE ? small[c] : lgamma((double)c + v.alpha) - lg_alpha;
+            }
         }
         if (lane == 0) s -= lgamma((double)(v.doc_off[d + 1] - d0) + v.Kalpha);
     }
