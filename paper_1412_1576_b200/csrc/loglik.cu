@@ -50,13 +50,19 @@ __global__ void __launch_bounds__(256) k_ll_doc(View v, double lg_alpha, double*
     const uint32_t cmask = (1u << v.count_bits) - 1u;
     double s = 0.0;
     for (int32_t d = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; d < v.D; d += warps) {
-        const int32_t d0 = v.doc_off[d], n = DK_SLOTS_PER_TOKEN * (v.doc_off[d + 1] - d0);
-        const uint32_t* tab = v.dk_slots + DK_SLOTS_PER_TOKEN * (size_t)d0;
-        for (int32_t j = lane; j < n; j += 32) {
-            const uint32_t e = tab[j];
-            if (e != DK_EMPTY) {
-                const uint32_t c = e & cmask;
-                s += c < (uint32_t)LL_TABLE ? small[c] : lgamma((double)c + v.alpha) - lg_alpha;
+        // a document's table: four slots per token, read 16 bytes at a time
+        static_assert(DK_SLOTS_PER_TOKEN == 4, "one 16-byte read per token of the document");
+        const int32_t d0 = v.doc_off[d], len = v.doc_off[d + 1] - d0;
+        const uint4* tab = reinterpret_cast<const uint4*>(v.dk_slots) + (size_t)d0;
+        for (int32_t j = lane; j < len; j += 32) {
+            const uint4 q = __ldcs(tab + j);
+            const uint32_t es[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (es[u] != DK_EMPTY) {
+                    const uint32_t c = es[u] & cmask;
+                    s += c < (uint32_t)LL_TABLE ? small[c] : lgamma((double)c + v.alpha) - lg_alpha;
+                }
             }
         }
         if (lane == 0) s -= lgamma((double)(v.doc_off[d + 1] - d0) + v.Kalpha);
