@@ -521,16 +521,17 @@ __global__ void k_init(View v, uint2 key)
 template <typename T, typename IN>
 __global__ void k_spread(View v, const IN* __restrict__ z_in)
 {
+    // one token per thread, CTAs in document order: the scattered writes of the CTAs in flight stay
+    // inside one block of the block-major order (a grid-stride loop would let them drift apart)
     T* zbm = reinterpret_cast<T*>(v.zbm);
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < v.N;
-         i += (int64_t)gridDim.x * blockDim.x) {
-        int64_t a = (int64_t)z_in[i];
-        if (a < 0 || a >= v.K) {
-            atomicOr(v.err, ERR_TOPIC_RANGE);
-            a = 0;
-        }
-        zbm[2 * (size_t)__ldcs(v.bm_of_tok + i)] = (T)a;
+    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i >= v.N) return;
+    int64_t a = (int64_t)z_in[i];
+    if (a < 0 || a >= v.K) {
+        atomicOr(v.err, ERR_TOPIC_RANGE);
+        a = 0;
     }
+    store_topic_pair(zbm, __ldcs(v.bm_of_tok + i), (uint32_t)a);  // the proposal half means nothing between sweeps
 }
 
 template <typename T>
@@ -546,10 +547,10 @@ __global__ void k_word_order_topics(View v)
 template <typename T, typename OUT>
 __global__ void k_export(View v, OUT* __restrict__ out)
 {
+    // one token per thread, CTAs in document order (see k_spread)
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < v.N;
-         i += (int64_t)gridDim.x * blockDim.x)
-        out[i] = (OUT)zbm[2 * (size_t)v.bm_of_tok[i]];
+    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i < v.N) out[i] = (OUT)zbm[2 * (size_t)__ldcs(v.bm_of_tok + i)];
 }
 
 static int grid_for(int64_t n, int block)
@@ -694,12 +695,13 @@ int launch_spread_assignments(Ctx& c, const void* z_dev, bool narrow)
 {
     if (c.N == 0) return 0;
     const int g = grid_for(c.N, 256);
+    const unsigned full = (unsigned)((c.N + 255) / 256);  // one token per thread
     if (c.wide_topics) {
-        k_spread<int32_t, int32_t><<<g, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev);
+        k_spread<int32_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev);
         k_word_order_topics<int32_t><<<g, 256, 0, c.stream>>>(c.v);
     } else {
-        if (narrow) k_spread<uint16_t, uint16_t><<<g, 256, 0, c.stream>>>(c.v, (const uint16_t*)z_dev);
-        else k_spread<uint16_t, int32_t><<<g, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev);
+        if (narrow) k_spread<uint16_t, uint16_t><<<full, 256, 0, c.stream>>>(c.v, (const uint16_t*)z_dev);
+        else k_spread<uint16_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev);
         k_word_order_topics<uint16_t><<<g, 256, 0, c.stream>>>(c.v);
     }
     return 2;
@@ -708,10 +710,10 @@ int launch_spread_assignments(Ctx& c, const void* z_dev, bool narrow)
 int launch_export_assignments(Ctx& c, void* z_dev, bool narrow)
 {
     if (c.N == 0) return 0;
-    const int g = grid_for(c.N, 256);
-    if (c.wide_topics) k_export<int32_t, int32_t><<<g, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev);
-    else if (narrow) k_export<uint16_t, uint16_t><<<g, 256, 0, c.stream>>>(c.v, (uint16_t*)z_dev);
-    else k_export<uint16_t, int32_t><<<g, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev);
+    const unsigned full = (unsigned)((c.N + 255) / 256);  // one token per thread
+    if (c.wide_topics) k_export<int32_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev);
+    else if (narrow) k_export<uint16_t, uint16_t><<<full, 256, 0, c.stream>>>(c.v, (uint16_t*)z_dev);
+    else k_export<uint16_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev);
     return 1;
 }
 
