@@ -270,7 +270,7 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     }
     // MH kernel work lists: a hot word (more tokens than a tail tile holds; it has a dense row by
     // the rule above) is cut into runs of HOT_TILE tokens, tail words are packed whole into tiles
-    std::vector<int32_t> hot_tiles, cold_tiles;
+    std::vector<int32_t> hot_tiles, hot_tiles_propose, cold_tiles;
     {
         static_assert(COLD_TILE >= SORT_TILE, "every word longer than a tail tile must have a dense row");
         int32_t s0 = 0, tok = 0;
@@ -284,6 +284,11 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
                     hot_tiles.push_back(w);
                     hot_tiles.push_back(word_off[w] + o);
                     hot_tiles.push_back(std::min(HOT_TILE, tf[w] - o));
+                }
+                for (int32_t o = 0; o < tf[w]; o += HOT_TILE_PROPOSE) {
+                    hot_tiles_propose.push_back(w);
+                    hot_tiles_propose.push_back(word_off[w] + o);
+                    hot_tiles_propose.push_back(std::min(HOT_TILE_PROPOSE, tf[w] - o));
                 }
                 continue;
             }
@@ -330,6 +335,7 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     alias_big.insert(alias_big.begin(), alias_mid.begin(), alias_mid.end());
     c.n_alias_big = (int32_t)alias_big.size();
     c.n_hot_tiles = (int32_t)(hot_tiles.size() / 3);
+    c.n_hot_tiles_propose = (int32_t)(hot_tiles_propose.size() / 3);
     c.n_cold_tiles = (int32_t)(cold_tiles.size() / 2);
 
     const size_t n1 = (size_t)std::max<int64_t>(N, 1), cap1 = (size_t)std::max<int64_t>(cap_total, 1);
@@ -348,9 +354,10 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.long_docs = upload(c, long_docs);
     c.alias_big = upload(c, alias_big);
     c.hot_tiles = upload(c, hot_tiles);
+    c.hot_tiles_propose = upload(c, hot_tiles_propose);
     c.cold_tiles = upload(c, cold_tiles);
     ok = ok && v.row_start && v.dense_slot && c.word_tiles && c.doc_tiles && c.dense_words &&
-         c.hist_chunks && c.long_docs && c.alias_big && c.hot_tiles && c.cold_tiles;
+         c.hist_chunks && c.long_docs && c.alias_big && c.hot_tiles && c.hot_tiles_propose && c.cold_tiles;
     v.wk_nnz = (int32_t*)A((size_t)V * 4);
     v.wk_topic = (uint32_t*)A(cap1 * 4);
     v.wk_count = (uint32_t*)A(cap1 * 4);

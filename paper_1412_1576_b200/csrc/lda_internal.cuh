@@ -71,9 +71,13 @@ constexpr int HIST16_BINS = 106496;  // window of the per-chunk n_kw histogram (
 constexpr int HIST_CHUNK = LDA_HIST_CHUNK;    // tokens per CTA in the histogram path
 static_assert(HIST_CHUNK < 65536, "the per-chunk histogram counts in 16 bits");
 #ifndef LDA_HOT_TILE
-#define LDA_HOT_TILE 16384
+#define LDA_HOT_TILE 32768
 #endif
-constexpr int HOT_TILE = LDA_HOT_TILE;  // MH kernels: tokens of one hot word per CTA
+#ifndef LDA_HOT_TILE_PROPOSE
+#define LDA_HOT_TILE_PROPOSE 8192
+#endif
+constexpr int HOT_TILE = LDA_HOT_TILE;  // accept pass: tokens of one hot word per CTA (the word's row is staged once per CTA)
+constexpr int HOT_TILE_PROPOSE = LDA_HOT_TILE_PROPOSE;  // propose pass: nothing is staged, shorter runs balance better
 constexpr int COLD_TILE = 2048;      // MH kernel: tokens of a tile of whole tail words
 constexpr int COLD_WORDS = 512;      // MH kernel: words per tail tile
 constexpr int HOT_STAGE_MAX_K = 16384;  // dense rows up to this many topics are staged in shared memory
@@ -163,7 +167,7 @@ struct Ctx {
     View v{};
     // host-side work lists (device copies below)
     int32_t n_word_tiles = 0, n_doc_tiles = 0, n_dense = 0, n_hist_chunks = 0, n_long_docs = 0,
-            n_alias_big = 0, n_alias_mid = 0, n_hot_tiles = 0, n_cold_tiles = 0;
+            n_alias_big = 0, n_alias_mid = 0, n_hot_tiles = 0, n_hot_tiles_propose = 0, n_cold_tiles = 0;
     int32_t* word_tiles = nullptr;   // [n_word_tiles*2] word ranges sorted per CTA
     int32_t* doc_tiles = nullptr;    // [n_doc_tiles*2]
     int32_t* dense_words = nullptr;  // [n_dense]
@@ -171,7 +175,8 @@ struct Ctx {
     int32_t* long_docs = nullptr;    // [n_long_docs]
     int32_t* alias_big = nullptr;    // [n_alias_big] words whose row can exceed ALIAS_WARP_MAX; the first
                                      // n_alias_mid of them cannot exceed ALIAS_SMEM_ITEMS_MID
-    int32_t* hot_tiles = nullptr;    // [n_hot_tiles*3] (word, first token, count): MH kernel, hot words
+    int32_t* hot_tiles = nullptr;    // [n_hot_tiles*3] (word, first token, count): MH kernel, hot word (accept pass)
+    int32_t* hot_tiles_propose = nullptr;  // the same cut into the shorter runs of the propose passs
     int32_t* cold_tiles = nullptr;   // [n_cold_tiles*2] word ranges of whole tail words: MH kernel
     // alias-construction scratch
     unsigned long long* sc_w = nullptr;   // [row capacity total] scaled masses

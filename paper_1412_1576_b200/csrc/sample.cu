@@ -588,9 +588,9 @@ static int launch_propose(Ctx& c, uint2 key, int mh_steps)
 {
     const View& v = c.v;
     int launches = 0;
-    if (c.n_hot_tiles) {
-        k_word_hot<T, CH, false, false, MODE, FIXED><<<c.n_hot_tiles, PROPOSE_THREADS, 0, c.stream>>>(
-            v, c.hot_tiles, key, c.sweep, mh_steps);
+    if (c.n_hot_tiles_propose) {
+        k_word_hot<T, CH, false, false, MODE, FIXED><<<c.n_hot_tiles_propose, PROPOSE_THREADS, 0, c.stream>>>(
+            v, c.hot_tiles_propose, key, c.sweep, mh_steps);
         ++launches;
     }
     if (c.n_cold_tiles) {
