@@ -488,7 +488,7 @@ static int count_k(Ctx& c)
     }
     if (c.n_dense < c.V) {
         const int win = hist_window(c);
-        const int grid = std::min(148 * 4, (int)((c.V + 511) / 512));
+        const int grid = std::min(148 * 4, (int)((c.V + 255) / 256));
         k_nk_from_sparse<<<grid, 512, (size_t)win * 4, c.side[0]>>>(v.row_start, v.wk_nnz, v.wk_topic, v.wk_count,
                                                                    v.dense_slot, c.V, v.nk, c.K, win);
         ++launches;
