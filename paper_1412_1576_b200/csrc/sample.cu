@@ -34,7 +34,7 @@ constexpr double INV_2_32 = 1.0 / 4294967296.0;
 #define LDA_PROPOSE_FIXED_MIN_CTAS 4
 #endif
 #ifndef LDA_PROPOSE_TOKENS
-#define LDA_PROPOSE_TOKENS 2
+#define LDA_PROPOSE_TOKENS 3
 #endif
 constexpr int PROPOSE_TOKENS = LDA_PROPOSE_TOKENS;  // tokens a thread of the two-step propose kernel takes per turn
 #ifndef LDA_ACCEPT_FIXED2_THREADS
