@@ -42,22 +42,44 @@ def _stale() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
+def build_library(force: bool = False, verbose: bool = False, extra_flags=(), out: str | None = None) -> str:
+    """Compiles every source to an object file (in parallel) and links them.  ``extra_flags`` and
+    ``out`` build a variant of the library somewhere else (objects then go to a folder of their own)."""
+    out = out or LIB_PATH
+    if not force and not extra_flags and out == LIB_PATH and not _stale():
         return LIB_PATH
-    os.makedirs(LIB_DIR, exist_ok=True)
-    tmp = LIB_PATH + f".{os.getpid()}.tmp"
-    cmd = [_nvcc()] + NVCC_FLAGS + sources() + ["-o", tmp]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    log = res.stdout + res.stderr
-    with open(os.path.join(LIB_DIR, "build.log"), "w") as f:
-        f.write(" ".join(cmd) + "\n" + log)
-    if res.returncode != 0:
+    os.makedirs(os.path.dirname(out), exist_ok=True)
+    obj_dir = os.path.join(os.path.dirname(out), "_build" if out == LIB_PATH and not extra_flags
+                           else "_build_" + os.path.basename(out))
+    os.makedirs(obj_dir, exist_ok=True)
+    compile_flags = [f for f in NVCC_FLAGS if f != "-shared"] + list(extra_flags)
+    procs = []
+    for src in sources():
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
+        cmd = [_nvcc()] + compile_flags + ["-c", src, "-o", obj]
+        procs.append((cmd, obj, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+    log, failed, objs = "", False, []
+    for cmd, obj, pr in procs:
+        text = pr.communicate()[0]
+        log += " ".join(cmd) + "\n" + text
+        failed = failed or pr.returncode != 0
+        objs.append(obj)
+    if not failed:
+        tmp = out + f".{os.getpid()}.tmp"
+        cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared"] + objs + ["-o", tmp]
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        log += " ".join(cmd) + "\n" + res.stdout + res.stderr
+        failed = res.returncode != 0
+        if not failed:
+            os.replace(tmp, out)
+    with open(os.path.join(os.path.dirname(out), "build.log" if out == LIB_PATH else os.path.basename(out) + ".log"),
+              "w") as f:
+        f.write(log)
+    if failed:
         raise RuntimeError("nvcc failed:\n" + log[-8000:])
-    os.replace(tmp, LIB_PATH)
     if verbose:
         print(log)
-    return LIB_PATH
+    return out
 
 
 if __name__ == "__main__":
