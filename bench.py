@@ -22,6 +22,8 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+PHASES = ("ms_alias_dense", "ms_alias_sparse", "ms_sample", "ms_count_wk", "ms_count_k", "ms_count_dk", "ms_total",
+          "ms_propose", "ms_doc_side", "ms_accept")
 METRIC = "sampled tokens/sec per sweep"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
@@ -41,6 +43,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-windows", action="store_true", help="skip the late-sweep and own-step-count windows")
+    ap.add_argument("--late-sweep", type=int, default=50, help="first sweep of the late window")
     return ap.parse_args()
 
 
@@ -116,9 +120,10 @@ def workload_config(args):
 
 
 def algorithmic_bytes_per_token(mh_steps: int, topic_bytes: int, rho_wk: float) -> dict:
-    """Bytes each kernel of a sweep must move per token (useful bytes: what it reads and writes
-    once, no sector or line overfetch).  T = topic bytes, M = steps, W = word-proposal steps,
-    rho = nnz(n_kw) / N.  The unit is one token; one launch processes all N tokens."""
+    """Traffic of THIS DESIGN per token and kernel: what each kernel reads and writes once (no
+    sector or line overfetch), exchange buffers between the three passes of the MH step included.
+    T = topic bytes, M = steps, W = word-proposal steps, rho = nnz(n_kw) / N.  The unit is one
+    token; one launch processes all N tokens.  The method's own bytes: method_bytes_per_token()."""
     T, M = topic_bytes, mh_steps
     W = (M + 1) // 2
     return {
@@ -135,6 +140,16 @@ def algorithmic_bytes_per_token(mh_steps: int, topic_bytes: int, rho_wk: float) 
         # row in, table out (split point, alias, packed bin), construction scratch out and in
         "alias_sparse": (8 + 8 + 8 + 40) * rho_wk,
     }
+
+
+def method_bytes_per_token(mh_steps: int, topic_bytes: int, rho_wk: float, rho_dk: float) -> float:
+    """Bytes the METHOD has to move per token and sweep, whatever the kernel design: the token's
+    ids and its topic streamed in and out in both orders (8 + 3T), the document-side gathers of the
+    chain (T per doc-proposal, 4 per n_kd lookup at the start topic and at every proposed one), the
+    rebuild re-reading z in both orders and writing n_kd (2T + 4 rho_d), and per nonzero of n_kw
+    its row entry plus the alias bin written and read (T + 20).  M = 2, T = 2: 32 + 4 rho_d + 22 rho."""
+    T, M = topic_bytes, mh_steps
+    return (8 + 3 * T) + (M // 2) * T + 4 * (M + 1) + 2 * T + 4.0 * rho_dk + (T + 20.0) * rho_wk
 
 
 def over_ranks(dist, device, ms: float, n_tokens: float):
@@ -184,10 +199,8 @@ def run_ours(args):
     del corpus
     torch.cuda.empty_cache()
     lda.init(1234 + rank)
-
-    for _ in range(args.warmup):
-        lda.sweep(1, M)
-    st0 = lda.stats()
+    lda.sweep(1, M)            # first launches of every kernel (module load), on a state that is thrown away
+    lda.init(1234 + rank)
 
     def barrier():
         torch.cuda.synchronize()
@@ -195,13 +208,34 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_sweeps(n, steps):
+        """n sweeps in one call between two events on the launch stream; returns (ms, stats of the call)."""
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        lda.sweep(n, steps)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1), binding.lda_get_stats(lda._h)[1]
+
+    def window(first, n, ms, st):
+        return {"sweeps": [first, first + n], "ms_per_step": ms / n, "value": N / (ms / n * 1e-3),
+                "nnz_wk": st.nnz_wk, "nnz_dk": st.nnz_dk,
+                "phases_ms_per_step": {k: getattr(st, k) / n for k in PHASES}}
+
+    # the first two sweeps from the uniform random start (dense model), reported beside the main window
+    windows = {}
+    ms_a, st_a = timed_sweeps(2, M)
+    windows["first"] = window(0, 2, ms_a, st_a)
+    for _ in range(max(0, args.warmup - 2)):
+        lda.sweep(1, M)
+    st0 = lda.stats()
+
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    phases = dict(ms_alias_dense=0.0, ms_alias_sparse=0.0, ms_sample=0.0, ms_count_wk=0.0,
-                  ms_count_k=0.0, ms_count_dk=0.0, ms_total=0.0, ms_propose=0.0, ms_doc_side=0.0,
-                  ms_accept=0.0)
+    phases = {k: 0.0 for k in PHASES}
     launches = 0
     rho_sum = 0.0
     barrier()
@@ -209,17 +243,37 @@ def run_ours(args):
     lda.sweep(args.steps, M)          # K sweeps in one call: nothing but the sweeps is inside the timed region
     ev1.record(stream)
     barrier()
-    ms = ev0.elapsed_time(ev1)
+    ms = own_ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop() if rank == 0 else None
     s = binding.lda_get_stats(lda._h)[1]   # phase times and launches summed over the K sweeps
     for k in phases:
         phases[k] = getattr(s, k)
     launches = s.kernel_launches
+    accept_stats = {k: getattr(s, k) for k in ("word_proposed", "word_accepted", "doc_proposed", "doc_accepted")
+                    if hasattr(s, k)}
     rho_sum = args.steps * s.nnz_wk / max(N, 1)
+    rho_dk = s.nnz_dk / max(N, 1)
     ms, total_tokens = over_ranks(dist, "cuda", ms, N)
     ms_per_step = ms / args.steps
     value = total_tokens / (ms_per_step * 1e-3)
     st1 = lda.stats()
+    windows["main"] = window(st0["sweeps_done"], args.steps, own_ms, s)
+
+    # later sweeps (sparser model) and the configuration's own step count, outside the main window
+    if not args.no_windows:
+        done = st1["sweeps_done"]
+        if done < args.late_sweep:
+            lda.sweep(args.late_sweep - done, M)
+            done = args.late_sweep
+        ms_c, st_c = timed_sweeps(10, M)
+        windows["late"] = window(done, 10, ms_c, st_c)
+        own_steps = cfg.get("mh_steps", M)
+        if own_steps != M:
+            lda.sweep(1, own_steps)      # lays the exchange buffers out for the other step count
+            ms_d, st_d = timed_sweeps(5, own_steps)
+            windows[f"mh{own_steps}"] = dict(window(done + 11, 5, ms_d, st_d), mh_steps=own_steps)
+            lda.sweep(1, M)
+        st1 = dict(st1, sweeps_done=lda.stats()["sweeps_done"])
 
     # --- end to end through the host-buffer entry points -----------------------------------
     e2e = None
@@ -280,22 +334,44 @@ def run_ours(args):
                 "share_of_step": top_ms / ms_per_step if ms_per_step else None}
     sweep_bytes = sum(b_alg.values())
     sweep_ms = phases["ms_total"] / args.steps
+    # the method's own bytes (whatever the kernel design) and what they say about the whole sweep
+    b_method = method_bytes_per_token(M, topic_bytes, rho, rho_dk)
+    tokens_per_s_1gpu = N / (sweep_ms * 1e-3) if sweep_ms > 0 else 0.0
+    roofline["survey_b_alg_bytes_per_token"] = b_method
+    roofline["useful_frac"] = tokens_per_s_1gpu * b_method / 1e9 / peak
+    roofline["useful_frac_what"] = ("tokens/s x the method's bytes per token (8 + 3T + floor(M/2) T + 4 (M+1) + 2T + "
+                                    "4 rho_d + (T+20) rho, with this run's rho = nnz(n_kw)/N and rho_d = nnz(n_kd)/N) "
+                                    "over the measured copy bandwidth")
+    roofline["rho_wk"], roofline["rho_dk"] = rho, rho_dk
     roofline["whole_sweep"] = {
-        "algorithmic_bytes_per_token": sweep_bytes,
+        "what": "traffic of this design (exchange buffers between the three passes included), not the method's bytes",
+        "design_bytes_per_token": sweep_bytes,
         "achieved": sweep_bytes * N / (sweep_ms * 1e-3) / 1e9 if sweep_ms > 0 else 0.0,
         "frac": (sweep_bytes * N / (sweep_ms * 1e-3) / 1e9) / peak if sweep_ms > 0 else 0.0,
-        "per_kernel": {k: {"ms": per_ms[k], "bytes_per_token": b_alg[k],
+        "per_kernel": {k: {"ms": per_ms[k], "design_bytes_per_token": b_alg[k],
                            "frac": (b_alg[k] * N / (per_ms[k] * 1e-3) / 1e9 / peak) if per_ms[k] > 0 else None}
                        for k in b_alg}}
     prof = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(prof):
         try:
-            tr = json.load(open(prof)).get(top, {})
+            table = json.load(open(prof))
+            tr = table.get(top, {})
             if tr.get("workload") == args.workload and tr.get("mh_steps") == M:
                 roofline["traffic"] = tr["dram_bytes_per_token"] * N
                 roofline["traffic_source"] = tr.get("source")
                 if "issue_active_pct" in tr:   # ncu smsp__issue_active of the same capture
                     roofline["issue_active_pct"] = tr["issue_active_pct"]
+            # bytes moved by the whole sweep: measured DRAM bytes per token of every per-sweep kernel
+            need = ("alias_dense", "alias_sparse", "propose", "doc_side", "accept", "count_wk", "count_k")
+            have = {k: table[k] for k in need if k in table and table[k].get("workload") == args.workload
+                    and table[k].get("mh_steps") == M}
+            if len(have) == len(need) and sweep_ms > 0:
+                moved = sum(v["dram_bytes_per_token"] for v in have.values())
+                roofline["bytes_moved_per_token"] = moved
+                roofline["bytes_moved_frac"] = moved * N / (sweep_ms * 1e-3) / 1e9 / peak
+                roofline["bytes_moved_what"] = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of every per-sweep "
+                                                "kernel (profiles/traffic.json, per token) x N over the sweep time, "
+                                                "over the measured copy bandwidth")
         except Exception:
             pass
 
@@ -316,7 +392,7 @@ def run_ours(args):
                    "sweeps_timed": [st0["sweeps_done"], st0["sweeps_done"] + args.steps],
                    "top10pct_vocab_token_share": gen_stats["top10pct_vocab_token_share"]},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-        "cpu_baseline": cpu,
+        "cpu_baseline": cpu, "windows": windows, "accept_counts": accept_stats,
         "phases_ms_per_step": {k: v / args.steps for k, v in phases.items()},
         "state": {"nnz_wk": st1["nnz_wk"], "nnz_dk": st1["nnz_dk"], "dense_words": st1["n_dense_words"],
                   "device_bytes": st1["device_bytes"], "generate_s": gen_s, "load_s": load_s},
@@ -326,56 +402,72 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def _oracle_setup(args, scale_cap_tokens=40e6):
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except Exception:
+        return max(1, os.cpu_count() or 1)
+
+
+def _oracle_setup(args, tokens_cap):
     """The oracle on a bounded sample of the workload: the same generator with
     fewer documents (same V, K, length law, priors)."""
     from oracle import ldaref
     from paper_1412_1576_b200 import synth
     cfg = workload_config(args)
-    avg_len = {"fixed": lambda l: l[1], "poisson": lambda l: l[1], "lognormal": lambda l: l[1]}[cfg["length"][0]](cfg["length"])
-    d_cap = max(1, int(scale_cap_tokens / max(avg_len, 1)))
-    sample_scale = 1.0
-    if cfg["D"] > d_cap:
-        sample_scale = d_cap / cfg["D"]
-        cfg["D"] = d_cap
+    avg_len = cfg["length"][1]
+    cfg["D"] = max(1, min(cfg["D"], int(tokens_cap / max(avg_len, 1))))
     c = synth.generate(seed=args.seed, device="cpu", **cfg)
     o = ldaref.Oracle(c.V, c.K, c.alpha, c.beta)
     o.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
     o.init(1234)
-    return o, c, sample_scale
+    return o, c
 
 
 def cpu_baseline(args, seconds):
-    o, c, sample_scale = _oracle_setup(args)
+    """The oracle as it stands on the host cores: one WHOLE sweep (table build, token loop, count
+    rebuild) over a bounded corpus of the workload's generator with the token loop on all cores,
+    and the token loop alone on one core beside it."""
+    cores = host_cores()
     M = args.mh_steps
-    n = min(c.n_tokens, 200_000)
-    t0 = time.perf_counter(); o.sweep_prefix(n, M); dt = time.perf_counter() - t0
-    n2 = int(min(c.n_tokens, max(n, n / max(dt, 1e-6) * seconds)))
-    t0 = time.perf_counter(); o.sweep_prefix(n2, M); dt = time.perf_counter() - t0
-    return {"value": n2 / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"first {n2} tokens of one sweep (tables already built) on the same generator "
-                      f"with {c.n_docs} documents ({c.n_tokens} tokens), mh_steps={M}"}
+    o, c = _oracle_setup(args, 2e6)                       # probe: how fast is this host?
+    sec = o.sweep_threads(1, M, cores)
+    rate = c.n_tokens / max(float(sec.sum()), 1e-6)
+    o.close()
+    o, c = _oracle_setup(args, min(40e6, max(2e6, rate * seconds * 0.5)))
+    sec = o.sweep_threads(1, M, cores)                    # the timed sample
+    whole = float(sec.sum())
+    n1 = int(min(c.n_tokens, max(100_000, 1.0e6 * seconds * 0.4)))
+    t0 = time.perf_counter(); o.sweep_prefix(n1, M); dt1 = time.perf_counter() - t0
+    return {"value": c.n_tokens / whole, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"one whole oracle sweep (alias tables + token loop on {cores} threads + count rebuild) over "
+                      f"{c.n_docs} documents ({c.n_tokens} tokens) of the same generator, mh_steps={M}",
+            "phases_s": {"tables": float(sec[0]), "token_loop": float(sec[1]), "count_rebuild": float(sec[2])},
+            "token_loop_only": {"value": c.n_tokens / max(float(sec[1]), 1e-9), "cores": cores},
+            "one_core": {"value": n1 / dt1, "cores": 1,
+                         "sample": f"token loop over the first {n1} tokens of the next sweep, tables prebuilt"}}
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    o, c, sample_scale = _oracle_setup(args, scale_cap_tokens=20e6)
+    cores = host_cores()
     M = args.mh_steps
-    n = min(c.n_tokens, 100_000)
-    t0 = time.perf_counter(); o.sweep_prefix(n, M); dt = time.perf_counter() - t0
-    budget = 60.0 / max(1, args.steps + args.warmup)
-    n_step = int(min(c.n_tokens, max(1000, n / max(dt, 1e-6) * budget)))
+    o, c = _oracle_setup(args, 2e6)                       # probe
+    sec = o.sweep_threads(1, M, cores)
+    rate = c.n_tokens / max(float(sec.sum()), 1e-6)
+    o.close()
+    budget = 90.0 / max(1, args.steps + args.warmup)      # seconds per step
+    o, c = _oracle_setup(args, min(40e6, max(2e5, rate * budget)))
     for _ in range(args.warmup):
-        o.sweep_prefix(n_step, M)
+        o.sweep_threads(1, M, cores)
     t0 = time.perf_counter()
-    for _ in range(args.steps):
-        o.sweep_prefix(n_step, M)
+    o.sweep_threads(args.steps, M, cores)
     dt = time.perf_counter() - t0
-    value = n_step * args.steps / dt
-    sample = (f"each step = first {n_step} tokens of one oracle sweep on the same generator with "
-              f"{c.n_docs} documents ({c.n_tokens} tokens), mh_steps={M}")
+    value = c.n_tokens * args.steps / dt
+    sample = (f"each step = one whole oracle sweep (alias tables + token loop on {cores} threads + count rebuild) over "
+              f"{c.n_docs} documents ({c.n_tokens} tokens) of the same generator, mh_steps={M}")
     cfg = workload_config(args)
     line = {
         "impl": "reference", "metric": f"{METRIC} (mh_steps={M})", "value": value, "unit": UNIT,
@@ -384,7 +476,7 @@ def run_reference(args):
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"{args.workload} LDA" + (f" x{args.scale}" if args.scale != 1.0 else ""),
                    "V": cfg["V"], "K": cfg["K"], "mh_steps": M, "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }

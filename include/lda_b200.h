@@ -60,11 +60,17 @@ typedef struct lda_stats {
     float ms_sample;          /* token MH step, all passes        (Eq. 6-13)    */
     float ms_count_wk;        /* n_kw rebuild                     (Section 3)   */
     float ms_count_k;         /* n_k rebuild                                    */
-    float ms_count_dk;        /* n_kd rebuild                     (Eq. 12)      */
+    float ms_count_dk;        /* always 0: n_kd is rebuilt inside the MH step's document pass (Eq. 12), tile by
+                                 tile in shared memory; its time is part of ms_doc_side */
     float ms_total;           /* first launch to last kernel end                */
     float ms_propose;         /* MH step, pass 1: word-proposals   (part of ms_sample) */
     float ms_doc_side;        /* MH step, pass 2: document side    (part of ms_sample) */
     float ms_accept;          /* MH step, pass 3: accept / reject  (part of ms_sample) */
+    /* Proposals of the last lda_sweep() by kind (Section 4.2: Eq. 7 / Eq. 10 acceptance): how many
+     * steps drew the word-proposal / the doc-proposal (every token takes every step), and how many of
+     * them moved the chain (proposed topic differs from the current one and was accepted). */
+    int64_t word_proposed, word_accepted;
+    int64_t doc_proposed, doc_accepted;
 } lda_stats;
 
 /* Model dimensions and symmetric priors of the collapsed LDA model (Section 3,

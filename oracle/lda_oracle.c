@@ -1,7 +1,8 @@
 /*
  * CPU ORACLE -- TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.
  *
- * A plain, slow, single-threaded C restatement of one frozen-counts sweep of
+ * A plain, slow C restatement (single-threaded; one entry point shares the token loop of a
+ * sweep among host threads, unchanged, for the benchmark's all-cores figure) of one frozen-counts sweep of
  * the LightLDA Metropolis-Hastings token sampler, written from the paper's
  * equations.  It exists so that the CUDA path can be compared with something
  * that can be checked against the paper by eye.  Only the tests, the smoke
@@ -33,10 +34,12 @@
  * Readings taken where the paper is silent are stated at the function that
  * takes them.
  */
+#define _POSIX_C_SOURCE 199309L
 #include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+#include <time.h>
 
 #define LDAREF_OK 0
 #define LDAREF_EINVAL (-1)
@@ -47,6 +50,13 @@
 #define LDAREF_NK 0
 #define LDAREF_NWK 1
 #define LDAREF_NDK 2
+
+static double wall_seconds(void)
+{
+    struct timespec ts;
+    clock_gettime(CLOCK_MONOTONIC, &ts);
+    return (double)ts.tv_sec + 1e-9 * (double)ts.tv_nsec;
+}
 
 /* ------------------------------------------------------------------------- */
 /* Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as    */
@@ -218,6 +228,7 @@ typedef struct ldaref_ctx {
     uint64_t seed;
     uint32_t sweep;      /* number of sweeps done since init */
     int proposals;       /* 0 cycle (word, doc, word, ...), 1 word-proposal only, 2 doc-proposal only */
+    int64_t moves[2];    /* steps of the last sweep call that moved a chain: word-, doc-proposals */
     int loaded, inited;
 } ldaref_ctx;
 
@@ -521,7 +532,7 @@ static void accept_ratio(const ldaref_ctx *c, int64_t i, int32_t s, int32_t t, i
  * to the current state changes nothing; otherwise accept iff u*den < num
  * with u = r3 / 2^32, which accepts with probability min{1, num/den}
  * (Eq. 7, Eq. 10). */
-static int32_t run_chain(const ldaref_ctx *c, int64_t i, uint32_t sweep, int32_t steps)
+static int32_t run_chain(const ldaref_ctx *c, int64_t i, uint32_t sweep, int32_t steps, int64_t *moves)
 {
     uint32_t key[2] = {(uint32_t)c->seed, (uint32_t)(c->seed >> 32)};
     int32_t s = c->z[i];
@@ -537,7 +548,10 @@ static int32_t run_chain(const ldaref_ctx *c, int64_t i, uint32_t sweep, int32_t
         double num, den;
         accept_ratio(c, i, s, t, kind, &num, &den);
         double u = (double)r[3] * (1.0 / 4294967296.0);
-        if (u * den < num) s = t;
+        if (u * den < num) {
+            s = t;
+            if (moves) moves[kind] += 1; /* accepted, and the state changed (t != s) */
+        }
     }
     return s;
 }
@@ -559,10 +573,11 @@ int ldaref_sweep(ldaref_ctx *c, int32_t iters, int32_t mh_steps)
 {
     if (!c || iters < 0 || mh_steps < 1) return LDAREF_EINVAL;
     if (!c->inited) return LDAREF_ESTATE;
+    c->moves[0] = c->moves[1] = 0;
     for (int32_t it = 0; it < iters; ++it) {
         int rc = ldaref_build_tables(c);
         if (rc) return rc;
-        for (int64_t i = 0; i < c->N; ++i) c->z_new[i] = run_chain(c, i, c->sweep, mh_steps);
+        for (int64_t i = 0; i < c->N; ++i) c->z_new[i] = run_chain(c, i, c->sweep, mh_steps, c->moves);
         int32_t *tmp = c->z; c->z = c->z_new; c->z_new = tmp;
         rc = rebuild_counts(c);
         if (rc) return rc;
@@ -581,7 +596,7 @@ int ldaref_sample_tokens(ldaref_ctx *c, const int64_t *tokens, int64_t n, int32_
     if (!c->tables_valid) { int rc = ldaref_build_tables(c); if (rc) return rc; }
     for (int64_t j = 0; j < n; ++j) {
         if (tokens[j] < 0 || tokens[j] >= c->N) return LDAREF_ERANGE;
-        z_out[j] = run_chain(c, tokens[j], c->sweep, mh_steps);
+        z_out[j] = run_chain(c, tokens[j], c->sweep, mh_steps, NULL);
     }
     return LDAREF_OK;
 }
@@ -592,7 +607,47 @@ int ldaref_sweep_prefix(ldaref_ctx *c, int64_t n, int32_t mh_steps, int32_t *z_o
     if (!c || !z_out || n < 0 || n > (c ? c->N : 0) || mh_steps < 1) return LDAREF_EINVAL;
     if (!c->inited) return LDAREF_ESTATE;
     if (!c->tables_valid) { int rc = ldaref_build_tables(c); if (rc) return rc; }
-    for (int64_t i = 0; i < n; ++i) z_out[i] = run_chain(c, i, c->sweep, mh_steps);
+    for (int64_t i = 0; i < n; ++i) z_out[i] = run_chain(c, i, c->sweep, mh_steps, NULL);
+    return LDAREF_OK;
+}
+
+/* The same sweep with the token loop shared among `threads` host threads (OpenMP).  Every chain
+ * reads only the sweep-start state and writes only its own z_new[i] (Section 6: the model is
+ * immutable while sampled), so the result is the serial sweep's, token for token; the table build
+ * and the count rebuild stay serial.  seconds[0..2], when given, receive the wall time of the
+ * table build, the token loop and the count rebuild, summed over the iterations. */
+int ldaref_sweep_threads(ldaref_ctx *c, int32_t iters, int32_t mh_steps, int32_t threads,
+                         double *seconds)
+{
+    if (!c || iters < 0 || mh_steps < 1 || threads < 1) return LDAREF_EINVAL;
+    if (!c->inited) return LDAREF_ESTATE;
+    if (seconds) seconds[0] = seconds[1] = seconds[2] = 0.0;
+    int64_t moves_w = 0, moves_d = 0;
+    for (int32_t it = 0; it < iters; ++it) {
+        double t0 = wall_seconds();
+        int rc = ldaref_build_tables(c);
+        if (rc) return rc;
+        double t1 = wall_seconds();
+        const int64_t N = c->N;
+        const uint32_t sweep = c->sweep;
+        int32_t *z_new = c->z_new;
+#pragma omp parallel for num_threads(threads) schedule(static) reduction(+ : moves_w, moves_d)
+        for (int64_t i = 0; i < N; ++i) {
+            int64_t mv[2] = {0, 0};
+            z_new[i] = run_chain(c, i, sweep, mh_steps, mv);
+            moves_w += mv[0];
+            moves_d += mv[1];
+        }
+        double t2 = wall_seconds();
+        int32_t *tmp = c->z; c->z = c->z_new; c->z_new = tmp;
+        rc = rebuild_counts(c);
+        if (rc) return rc;
+        c->sweep += 1;
+        double t3 = wall_seconds();
+        if (seconds) { seconds[0] += t1 - t0; seconds[1] += t2 - t1; seconds[2] += t3 - t2; }
+    }
+    c->moves[0] = moves_w;
+    c->moves[1] = moves_d;
     return LDAREF_OK;
 }
 
@@ -604,7 +659,7 @@ int ldaref_chain(ldaref_ctx *c, int64_t token, uint32_t sweep, int32_t steps, in
     if (!c->inited) return LDAREF_ESTATE;
     if (token < 0 || token >= c->N) return LDAREF_ERANGE;
     if (!c->tables_valid) { int rc = ldaref_build_tables(c); if (rc) return rc; }
-    *z_out = run_chain(c, token, sweep, steps);
+    *z_out = run_chain(c, token, sweep, steps, NULL);
     return LDAREF_OK;
 }
 
@@ -646,16 +701,32 @@ int ldaref_accept_ratio(ldaref_ctx *c, int64_t token, int32_t s, int32_t t, int3
  *          - sum_k lgamma(n_k + V*beta)
  *   doc  = D*lgamma(K*alpha) + sum_{n_kd>0} [lgamma(n_kd+alpha) - lgamma(alpha)]
  *          - sum_d lgamma(n_d + K*alpha)                                       */
+/* Compensated sum (Neumaier's form of Kahan summation): `sum` plus the rounding errors collected in `err`. */
+typedef struct { double sum, err; } ksum;
+static void ksum_add(ksum *a, double x)
+{
+    double t = a->sum + x;
+    if (fabs(a->sum) >= fabs(x)) a->err += (a->sum - t) + x;
+    else a->err += (x - t) + a->sum;
+    a->sum = t;
+}
+static double ksum_value(const ksum *a) { return a->sum + a->err; }
+
 int ldaref_loglik(ldaref_ctx *c, double *total, double *word_ll, double *doc_ll)
 {
     if (!c) return LDAREF_EINVAL;
     if (!c->inited) return LDAREF_ESTATE;
-    double lw = (double)c->K * lgamma(c->Vbeta);
+    /* Each of the formula's sums is taken with compensated (Kahan-Neumaier) addition and the groups
+     * are combined at the end.  Plain one-by-one addition is not good enough here: K*lgamma(V*beta)
+     * and sum_k lgamma(n_k + V*beta) are ~1e10 each at V = 1e6, K = 1e5 and nearly cancel, and the
+     * millions of equal terms lgamma(1 + prior) - lgamma(prior) round the same way every time, so
+     * the error grows with their number (measured: 0.3 absolute on -2.4e8). */
     double lg_beta = lgamma(c->beta), lg_alpha = lgamma(c->alpha);
+    ksum w_nonzero = {0.0, 0.0}, w_topics = {0.0, 0.0}, d_nonzero = {0.0, 0.0}, d_lengths = {0.0, 0.0};
     for (int64_t p = 0; p < c->row_off[c->V]; ++p)
-        lw += lgamma((double)c->row_count[p] + c->beta) - lg_beta;
-    for (int32_t k = 0; k < c->K; ++k) lw -= lgamma((double)c->nk[k] + c->Vbeta);
-    double ld = (double)c->D * lgamma(c->Kalpha);
+        ksum_add(&w_nonzero, lgamma((double)c->row_count[p] + c->beta) - lg_beta);
+    for (int32_t k = 0; k < c->K; ++k) ksum_add(&w_topics, lgamma((double)c->nk[k] + c->Vbeta));
+    double lw = ((double)c->K * lgamma(c->Vbeta) - ksum_value(&w_topics)) + ksum_value(&w_nonzero);
     int32_t *tally = (int32_t *)calloc((size_t)c->K, sizeof(int32_t));
     if (!tally) return LDAREF_ENOMEM;
     for (int64_t d = 0; d < c->D; ++d) {
@@ -663,11 +734,12 @@ int ldaref_loglik(ldaref_ctx *c, double *total, double *word_ll, double *doc_ll)
         for (int64_t j = lo; j < hi; ++j) tally[c->z[j]] += 1;
         for (int64_t j = lo; j < hi; ++j) {
             int32_t n = tally[c->z[j]];
-            if (n) { ld += lgamma((double)n + c->alpha) - lg_alpha; tally[c->z[j]] = 0; }
+            if (n) { ksum_add(&d_nonzero, lgamma((double)n + c->alpha) - lg_alpha); tally[c->z[j]] = 0; }
         }
-        ld -= lgamma((double)(hi - lo) + c->Kalpha);
+        ksum_add(&d_lengths, lgamma((double)(hi - lo) + c->Kalpha));
     }
     free(tally);
+    double ld = ((double)c->D * lgamma(c->Kalpha) - ksum_value(&d_lengths)) + ksum_value(&d_nonzero);
     if (word_ll) *word_ll = lw;
     if (doc_ll) *doc_ll = ld;
     if (total) *total = lw + ld;
@@ -760,3 +832,13 @@ int ldaref_get_tables(ldaref_ctx *c, uint32_t *sp_thr32, int32_t *sp_alias, int6
 }
 
 uint32_t ldaref_sweeps_done(const ldaref_ctx *c) { return c ? c->sweep : 0; }
+
+/* Steps of the last ldaref_sweep / ldaref_sweep_threads call that moved a chain (the proposed topic
+ * differed from the current one and passed the test of Eq. 7 / Eq. 10): [0] word-, [1] doc-proposals. */
+int ldaref_get_moves(const ldaref_ctx *c, int64_t *out2)
+{
+    if (!c || !out2) return LDAREF_EINVAL;
+    out2[0] = c->moves[0];
+    out2[1] = c->moves[1];
+    return LDAREF_OK;
+}

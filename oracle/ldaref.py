@@ -28,7 +28,7 @@ def build(force: bool = False) -> str:
     os.makedirs(os.path.dirname(_OUT), exist_ok=True)
     if force or not os.path.exists(_OUT) or os.path.getmtime(_OUT) < os.path.getmtime(_SRC):
         tmp = _OUT + f".{os.getpid()}.tmp"
-        subprocess.check_call(["gcc", "-std=c11", "-O2", "-ffp-contract=off", "-fno-fast-math",
+        subprocess.check_call(["gcc", "-std=c11", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
                                "-Wall", "-Wextra", "-shared", "-fPIC", _SRC, "-o", tmp, "-lm"])
         os.replace(tmp, _OUT)
     return _OUT
@@ -61,6 +61,7 @@ def lib():
             L.ldaref_set_assignments.argtypes = [vp, _p(np.int32), C.c_uint64, C.c_uint32]
             L.ldaref_build_tables.argtypes = [vp]
             L.ldaref_sweep.argtypes = [vp, C.c_int32, C.c_int32]
+            L.ldaref_sweep_threads.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, _p(np.float64)]
             L.ldaref_set_proposals.argtypes = [vp, C.c_int]
             L.ldaref_sample_tokens.argtypes = [vp, _p(np.int64), C.c_int64, C.c_int32,
                                                _p(np.int32)]
@@ -80,6 +81,7 @@ def lib():
             L.ldaref_get_assignments.argtypes = [vp, _p(np.int32)]
             L.ldaref_get_tables.argtypes = [vp, vp, vp, C.c_int64, vp, vp, vp,
                                             C.POINTER(C.c_uint64)]
+            L.ldaref_get_moves.argtypes = [vp, _p(np.int64)]
             L.ldaref_sweeps_done.argtypes = [vp]
             L.ldaref_sweeps_done.restype = C.c_uint32
             _lib = L
@@ -161,6 +163,13 @@ class Oracle:
     def sweep(self, iters: int, mh_steps: int):
         _check(lib().ldaref_sweep(self._h, iters, mh_steps), "sweep")
 
+    def sweep_threads(self, iters: int, mh_steps: int, threads: int) -> np.ndarray:
+        """The same sweeps with the token loop on `threads` host threads; returns the seconds spent
+        in (table build, token loop, count rebuild)."""
+        sec = np.zeros(3, np.float64)
+        _check(lib().ldaref_sweep_threads(self._h, iters, mh_steps, threads, sec), "sweep_threads")
+        return sec
+
     def sample_tokens(self, tokens, mh_steps: int) -> np.ndarray:
         t = np.ascontiguousarray(tokens, np.int64)
         out = np.zeros(t.size, np.int32)
@@ -236,6 +245,12 @@ class Oracle:
                                        C.byref(B)), "get_tables")
         return dict(row_off=off, sp_thr32=sp_thr[:nnz], sp_alias=sp_al[:nnz], mix32=mix,
                     dn_thr32=dthr, dn_alias=dal, dense_mass=B.value)
+
+    def moves(self):
+        """(word-proposal steps, doc-proposal steps) of the last sweep call that moved a chain."""
+        out = np.zeros(2, np.int64)
+        _check(lib().ldaref_get_moves(self._h, out), "get_moves")
+        return int(out[0]), int(out[1])
 
     @property
     def sweeps_done(self) -> int:

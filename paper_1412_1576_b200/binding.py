@@ -36,6 +36,8 @@ class lda_stats(C.Structure):
         ("ms_count_wk", C.c_float), ("ms_count_k", C.c_float), ("ms_count_dk", C.c_float),
         ("ms_total", C.c_float), ("ms_propose", C.c_float), ("ms_doc_side", C.c_float),
         ("ms_accept", C.c_float),
+        ("word_proposed", C.c_int64), ("word_accepted", C.c_int64),
+        ("doc_proposed", C.c_int64), ("doc_accepted", C.c_int64),
     ]
 
     def as_dict(self):

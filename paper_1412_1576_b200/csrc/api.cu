@@ -84,13 +84,14 @@ static void free_corpus(Ctx& c)
     for (void* p : c.allocs)
         if (p == (void*)err) keep.push_back(p); else cudaFree(p);
     c.allocs = keep;
-    c.device_bytes = keep.empty() ? 0 : 16;
+    c.device_bytes = keep.empty() ? 0 : 32;
     View nv{};
     nv.V = c.V; nv.K = c.K; nv.alpha = c.alpha; nv.beta = c.beta;
     nv.Vbeta = (double)c.V * c.beta;
     nv.Kalpha = (double)c.K * c.alpha;
     nv.dense_stride = (c.K + 3) & ~3;
     nv.err = err;
+    nv.moves = c.v.moves;
     c.v = nv;
     c.loaded = c.inited = c.tables_valid = c.dk_valid = false;
     c.N = c.D = 0;
@@ -429,16 +430,17 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
     c.v.Vbeta = (double)V * beta;
     c.v.Kalpha = (double)K * alpha;
     c.v.dense_stride = (K + 3) & ~3;
-    c.v.err = (int*)dev_alloc(c, 16);
-    if (!c.v.err || cudaMemset(c.v.err, 0, 16) != cudaSuccess) {
+    c.v.err = (int*)dev_alloc(c, 32);  // the error word and, 16 bytes on, the two move counters
+    c.v.moves = c.v.err ? reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(c.v.err) + 16) : nullptr;
+    if (!c.v.err || cudaMemset(c.v.err, 0, 32) != cudaSuccess) {
         dev_free_all(c);
         delete h;
         cudaGetLastError();
         return LDA_ECUDA;
     }
-    for (int i = 0; i < 10; ++i)
-        if (cudaEventCreate(&c.ev[i]) != cudaSuccess) {
-            for (int j = 0; j < i; ++j) cudaEventDestroy(c.ev[j]);
+    for (int i = 0; i < Ctx::EV_RING * 10; ++i)
+        if (cudaEventCreate(&c.ev_ring[i / 10][i % 10]) != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(c.ev_ring[j / 10][j % 10]);
             dev_free_all(c);
             delete h;
             cudaGetLastError();
@@ -481,7 +483,7 @@ void lda_destroy(lda_ctx* h)
         if (c.ev_fork) cudaEventDestroy(c.ev_fork);
     }
     if (c.have_events)
-        for (int i = 0; i < 10; ++i) cudaEventDestroy(c.ev[i]);
+        for (int i = 0; i < Ctx::EV_RING * 10; ++i) cudaEventDestroy(c.ev_ring[i / 10][i % 10]);
     dev_free_all(c);
     cudaGetLastError();
     delete h;
@@ -645,42 +647,70 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
         s.ms_total = s.ms_propose = s.ms_doc_side = s.ms_accept = 0.f;
     s.kernel_launches = 0;
     s.iters = iters;
-    for (int32_t it = 0; it < iters; ++it) {
-        int64_t n = 0;
-        cudaEventRecord(c.ev[0], c.stream);
-        n += launch_alias_dense(c);
-        cudaEventRecord(c.ev[1], c.stream);
-        n += launch_alias_sparse(c);
-        cudaEventRecord(c.ev[2], c.stream);
-        n += launch_sample(c, mh_steps);
-        cudaEventRecord(c.ev[3], c.stream);
-        n += launch_count_wk(c);
-        cudaEventRecord(c.ev[4], c.stream);
-        n += launch_count_k(c);
-        cudaEventRecord(c.ev[5], c.stream);
-        cudaEventRecord(c.ev[6], c.stream);  // n_kd is rebuilt inside the next MH step, per tile
-        c.tables_valid = false;
-        c.dk_valid = false;
-        c.sweep += 1;
+    s.word_proposed = s.word_accepted = s.doc_proposed = s.doc_accepted = 0;
+    if (cudaMemsetAsync(c.v.moves, 0, 16, c.stream) != cudaSuccess) return cuda_fail(&c, "clearing the move counters");
+    // Iterations are queued without waiting for each other; the host waits once per EV_RING of them
+    // (and after the last) to read the error word, the move counters and the phase timings.
+    for (int32_t it0 = 0; it0 < iters; it0 += Ctx::EV_RING) {
+        const int32_t batch = std::min<int32_t>(Ctx::EV_RING, iters - it0);
+        for (int32_t b = 0; b < batch; ++b) {
+            c.ev = c.ev_ring[b];
+            int64_t n = 0;
+            cudaEventRecord(c.ev[0], c.stream);
+            n += launch_alias_dense(c);
+            cudaEventRecord(c.ev[1], c.stream);
+            n += launch_alias_sparse(c);
+            cudaEventRecord(c.ev[2], c.stream);
+            n += launch_sample(c, mh_steps);
+            cudaEventRecord(c.ev[3], c.stream);
+            n += launch_count_wk(c);
+            cudaEventRecord(c.ev[4], c.stream);
+            n += launch_count_k(c);
+            cudaEventRecord(c.ev[5], c.stream);
+            cudaEventRecord(c.ev[6], c.stream);  // n_kd is rebuilt inside the next MH step, per tile
+            c.tables_valid = false;
+            c.dk_valid = false;
+            c.sweep += 1;
+            s.kernel_launches += n;
+        }
+        c.ev = c.ev_ring[0];
         int bits = 0;
-        if ((rc = read_err(c, &bits))) return rc;
+        if ((rc = read_err(c, &bits))) { c.inited = false; return rc; }
         if (bits) {
-            c.err = "a kernel raised the device error word: " + std::to_string(bits);
+            // some iteration of this batch met inconsistent tables: the state is not to be trusted
+            c.inited = false;
+            c.err = "a kernel raised the device error word: " + std::to_string(bits) +
+                    " (call lda_init or lda_set_assignments again)";
             return LDA_EINTERNAL;
         }
-        float ms[7] = {0};
-        for (int i = 0; i < 6; ++i) cudaEventElapsedTime(&ms[i], c.ev[i], c.ev[i + 1]);
-        cudaEventElapsedTime(&ms[6], c.ev[0], c.ev[6]);
-        if (c.N > 0) {
-            float a = 0.f, b = 0.f, d = 0.f;
-            cudaEventElapsedTime(&a, c.ev[2], c.ev[8]);
-            cudaEventElapsedTime(&b, c.ev[8], c.ev[9]);
-            cudaEventElapsedTime(&d, c.ev[9], c.ev[3]);
-            s.ms_propose += a; s.ms_doc_side += b; s.ms_accept += d;
+        for (int32_t b = 0; b < batch; ++b) {
+            cudaEvent_t* ev = c.ev_ring[b];
+            float ms[7] = {0};
+            for (int i = 0; i < 6; ++i) cudaEventElapsedTime(&ms[i], ev[i], ev[i + 1]);
+            cudaEventElapsedTime(&ms[6], ev[0], ev[6]);
+            if (c.N > 0) {
+                float a = 0.f, bb = 0.f, d = 0.f;
+                cudaEventElapsedTime(&a, ev[2], ev[8]);
+                cudaEventElapsedTime(&bb, ev[8], ev[9]);
+                cudaEventElapsedTime(&d, ev[9], ev[3]);
+                s.ms_propose += a; s.ms_doc_side += bb; s.ms_accept += d;
+            }
+            s.ms_alias_dense += ms[0]; s.ms_alias_sparse += ms[1]; s.ms_sample += ms[2];
+            s.ms_count_wk += ms[3]; s.ms_count_k += ms[4]; s.ms_count_dk += ms[5]; s.ms_total += ms[6];
         }
-        s.ms_alias_dense += ms[0]; s.ms_alias_sparse += ms[1]; s.ms_sample += ms[2];
-        s.ms_count_wk += ms[3]; s.ms_count_k += ms[4]; s.ms_count_dk += ms[5]; s.ms_total += ms[6];
-        s.kernel_launches += n;
+    }
+    {
+        unsigned long long moves[2] = {0, 0};
+        if (cudaMemcpyAsync(moves, c.v.moves, 16, cudaMemcpyDeviceToHost, c.stream) != cudaSuccess ||
+            cudaStreamSynchronize(c.stream) != cudaSuccess)
+            return cuda_fail(&c, "reading the move counters");
+        const int64_t n_word = c.proposals == LDA_PROPOSALS_CYCLE  ? (mh_steps + 1) / 2
+                               : c.proposals == LDA_PROPOSALS_WORD ? mh_steps
+                                                                   : 0;
+        s.word_proposed = (int64_t)iters * c.N * n_word;
+        s.doc_proposed = (int64_t)iters * c.N * (mh_steps - n_word);
+        s.word_accepted = (int64_t)moves[0];
+        s.doc_accepted = (int64_t)moves[1];
     }
     return LDA_OK;
 }

@@ -144,6 +144,7 @@ struct View {
     // (four slots per token, load <= 0.25); layout and probe order: dk_insert in lda_device.cuh.
     uint32_t* dk_slots;
     int* err;
+    unsigned long long* moves;  // [2] steps of the running lda_sweep() that moved a chain: word-, doc-proposals
 };
 
 struct Ctx {
@@ -189,7 +190,11 @@ struct Ctx {
     int64_t device_bytes = 0;
     lda_stats stats{};
     int64_t launches = 0;
-    cudaEvent_t ev[10] = {};  // 0..6 bracket the phases of a sweep, 8 and 9 the passes of the MH step
+    // Events of up to EV_RING iterations of a sweep call (per iteration: 0..6 bracket the phases, 8 and
+    // 9 the passes of the MH step); the host waits and reads them once per EV_RING iterations.
+    static constexpr int EV_RING = 8;
+    cudaEvent_t ev_ring[EV_RING][10] = {};
+    cudaEvent_t* ev = ev_ring[0];  // the running iteration's
     bool have_events = false;
     // Two more streams for kernels of one phase that touch different words: fork_streams() makes them
     // wait for the work queued on `stream` so far, join_streams() makes `stream` wait for theirs.

@@ -116,12 +116,22 @@ struct HotTile {
     uint32_t mix;
     void* bar;   // STAGED: barrier the bulk copy of the row completes on
     bool ready;  // the row has landed
+    bool gave_up;  // STAGED: the wait for the copy ran out; the rows are read from global memory instead
+    const int32_t* row_global;  // where the staged copies came from
+    const int32_t* nk_global;
     __device__ __forceinline__ Ref ref(int32_t) const { return Ref{}; }
-    // Called before the first lookup: the row must have landed by then.
+    // Called before the first lookup: the row must have landed by then.  If the bounded wait runs
+    // out, the error word is raised and this thread reads the (identical) rows in global memory, so
+    // nothing is ever read from shared memory the copy has not filled.
     __device__ __forceinline__ void prepare(const View& v)
     {
         if (STAGED && !ready) {
-            if (!mbar_wait_bounded(bar, 0, STAGE_WAIT_LIMIT)) atomicOr(v.err, ERR_STAGE);
+            if (!mbar_wait_bounded(bar, 0, STAGE_WAIT_LIMIT)) {
+                atomicOr(v.err, ERR_STAGE);
+                gave_up = true;
+                row = row_global;
+                nk_tab = nk_global;
+            }
             ready = true;
         }
     }
@@ -175,6 +185,7 @@ struct ColdTile {
     const uint32_t* idx;
     int32_t nw;
     const int32_t* nk_tab;  // n_k in global memory
+    static constexpr bool gave_up = false;
     __device__ __forceinline__ int32_t nk(uint32_t k) const { return __ldg(nk_tab + k); }
     __device__ __forceinline__ Ref ref(int32_t q) const
     {
@@ -311,6 +322,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
     const size_t N = (size_t)v.N;
     T* zw = reinterpret_cast<T*>(v.zw);
     bool bad = false;
+    uint32_t moved_w = 0, moved_d = 0;  // steps of this thread's tokens that moved the chain, by proposal
     // The reads of a token are issued ahead of its turn: its block-major index two iterations
     // early, the gathered record (which needs that index) one iteration early.
     const uint4* side4 = reinterpret_cast<const uint4*>(v.dside);
@@ -400,6 +412,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 }
                 const double u = __dmul_rn(u32_to_double((uint32_t)ua[i]), INV_2_32);
                 if (live && __dmul_rn(u, den) < num) {
+                    if (step_is_doc<MODE>(i)) ++moved_d; else ++moved_w;
                     s = t[i];
                     n_sd = n_td;
                     n_sw = n_tw[i];
@@ -411,6 +424,21 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
         store_topic_pair(reinterpret_cast<T*>(v.zbm), at, s);
     }
     if (bad) atomicOr(v.err, ERR_COUNT_ZERO);
+    // one add per CTA and kind to the sweep's counters
+    __shared__ uint32_t moved_s[2];
+    if (threadIdx.x == 0) moved_s[0] = moved_s[1] = 0u;
+    __syncthreads();
+    moved_w = warp_reduce_sum<uint32_t>(moved_w);
+    moved_d = warp_reduce_sum<uint32_t>(moved_d);
+    if ((threadIdx.x & 31) == 0) {
+        if (moved_w) atomicAdd(&moved_s[0], moved_w);
+        if (moved_d) atomicAdd(&moved_s[1], moved_d);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (moved_s[0]) atomicAdd(v.moves + 0, (unsigned long long)moved_s[0]);
+        if (moved_s[1]) atomicAdd(v.moves + 1, (unsigned long long)moved_s[1]);
+    }
 }
 
 // Hot words: tile = (word, first token, count).  ACCEPT = false: pass 1, true: pass 3.
@@ -454,9 +482,15 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     tile.mix = __ldg(v.mix32 + w);
     tile.bar = &bar;
     tile.ready = !(STAGED && ACCEPT);
+    tile.gave_up = false;
+    tile.row_global = row_g;
+    tile.nk_global = v.nk;
     if (ACCEPT) accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, accept_threads(FIXED), key, sweep, mh_steps);
     else propose_tokens<T, MODE, FIXED>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
-    // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one
+    // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one.  A thread
+    // whose wait ran out waits once more (bounded again) before the CTA may retire: a bulk copy still
+    // in flight must not land in shared memory that belongs to the next CTA.
+    if (STAGED && ACCEPT && tile.gave_up) mbar_wait_bounded(&bar, 0, STAGE_WAIT_LIMIT);
 }
 
 // Tail words: tile = range of whole words [w0, w1) with at most COLD_TILE tokens.

@@ -29,6 +29,13 @@ def _assert_same_counts(g, o):
         assert np.array_equal(a[2], b[2])
 
 
+def _assert_same_moves(g, o, n_tokens, word_steps, doc_steps, iters=1):
+    """lda_stats' proposal counters of the last sweep call against the oracle's."""
+    st = g.stats()
+    assert (st["word_proposed"], st["doc_proposed"]) == (iters * n_tokens * word_steps, iters * n_tokens * doc_steps)
+    assert (st["word_accepted"], st["doc_accepted"]) == o.moves()
+
+
 def _assert_same_tables(g, o):
     a, b = g.get_tables(), o.get_tables()
     assert a["dense_mass"] == b["dense_mass"]
@@ -58,11 +65,13 @@ def test_tables_bit_equal_tiny(tiny_corpus):
 
 def test_sweeps_bit_equal_tiny(tiny_corpus):
     """fp64 acceptance in the same operation order: every token agrees, every sweep."""
+    c = tiny_corpus
     g, o = _pair(tiny_corpus)
     for sweep in range(20):
         g.sweep(1, 2)
         o.sweep(1, 2)
         assert np.array_equal(g.get_assignments(), o.get_assignments()), sweep
+        _assert_same_moves(g, o, c.n_tokens, 1, 1)
     _assert_same_counts(g, o)
     lg, lo = g.loglik(), o.loglik()
     for a, b in zip(lg, lo):
@@ -84,6 +93,7 @@ def test_four_step_cycle_small_config(small_corpus):
     g.sweep(2, 4)
     o.sweep(2, 4)
     assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_moves(g, o, small_corpus.n_tokens, 2, 2, iters=2)
     _assert_same_counts(g, o)
 
 
@@ -253,6 +263,8 @@ def test_single_proposal_chains(tiny_corpus, small_corpus, mode):
             g.sweep(sweeps, mh_steps)
             o.sweep(sweeps, mh_steps)
             assert np.array_equal(g.get_assignments(), o.get_assignments()), mh_steps
+            _assert_same_moves(g, o, c.n_tokens, mh_steps if mode == binding.PROPOSALS_WORD else 0,
+                               mh_steps if mode == binding.PROPOSALS_DOC else 0, iters=sweeps)
         _assert_same_counts(g, o)
         # back to the cycle on the same context: the exchange buffers are laid out again
         g.set_proposals(binding.PROPOSALS_CYCLE)
@@ -332,50 +344,6 @@ def test_large_shape_sample_against_oracle():
     # the other (error up to n * 2^-53 relative to the sum of magnitudes), the library in 592 partial sums
     for a, b in zip(g.loglik(), o.loglik()):
         assert a == pytest.approx(b, rel=1e-9)
-
-
-def test_full_size_invariants():
-    """The benchmark's full workload (738 M tokens) in the configuration bench.py times: the count tables
-    must be exactly those of the library's own assignments (properties that hold at any size), and
-    a sample of documents is recounted by brute force."""
-    import torch
-    free, _ = torch.cuda.mem_get_info()
-    if free < 70 * 2 ** 30:
-        pytest.skip("needs about 60 GB of free device memory")
-    c = synth.make("large", seed=0, device="cuda")
-    N, D = c.n_tokens, c.n_docs
-    g = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
-    g.load_corpus(c.word_ids, c.doc_offsets)
-    off = c.doc_offsets.cpu().numpy()
-    words = c.word_ids
-    g.init(1234)
-    g.sweep(2, 2)
-    z = torch.from_numpy(g.get_assignments()).cuda()
-    assert z.numel() == N and int(z.min()) >= 0 and int(z.max()) < c.K
-    nk = torch.bincount(z, minlength=c.K).cpu().numpy()
-    assert np.array_equal(g.get_nk(), nk)                       # sum_w n_kw = n_k = histogram of z
-    assert int(nk.sum()) == N
-    st = g.stats()
-    # nonzeros of n_kw and n_kd = distinct (word, topic) and (document, topic) pairs of z
-    key_w = words.long() * c.K + z.long()
-    assert st["nnz_wk"] == int(torch.unique(key_w).numel())
-    del key_w
-    doc = torch.repeat_interleave(torch.arange(D, device="cuda"), torch.diff(c.doc_offsets.cuda()))
-    key_d = doc * c.K + z.long()
-    del doc
-    assert st["nnz_dk"] == int(torch.unique(key_d).numel())
-    del key_d
-    # the log-likelihood is a function of the tables: recompute its document part for a sample of
-    # documents is not possible without the tables, so recount n_kw for a sample of words instead
-    ro, top, cnt = g.get_csr(binding.LDA_NWK)
-    rng = np.random.default_rng(0)
-    wcpu = None
-    for w in rng.integers(0, c.V, size=20):
-        sel = (words == int(w))
-        zz = z[sel].cpu().numpy()
-        uk, uc = np.unique(zz, return_counts=True)
-        assert np.array_equal(top[ro[w]:ro[w + 1]], uk)
-        assert np.array_equal(cnt[ro[w]:ro[w + 1]], uc)
 
 
 def test_edge_cases():

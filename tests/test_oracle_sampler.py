@@ -341,6 +341,45 @@ def test_sweep_is_frozen_and_order_independent(tiny_corpus):
     assert a.sweeps_done == 2
 
 
+def test_threaded_sweep_is_the_serial_sweep(tiny_corpus, small_corpus):
+    """The entry point that shares the token loop among host threads (the benchmark's all-cores leg)
+    gives the serial sweep's assignments, counts and move counters, token for token."""
+    for c, sweeps in ((tiny_corpus, 3), (small_corpus, 1)):
+        a, b = _oracle(c, 5), _oracle(c, 5)
+        a.sweep(sweeps, 2)
+        sec = b.sweep_threads(sweeps, 2, 4)
+        assert sec.shape == (3,) and (sec >= 0).all()
+        assert np.array_equal(a.get_assignments(), b.get_assignments())
+        assert np.array_equal(a.get_nk(), b.get_nk())
+        assert a.moves() == b.moves()
+        assert a.loglik() == b.loglik()
+        assert a.sweeps_done == b.sweeps_done == sweeps
+
+
+def test_move_counters_count_the_steps_that_changed_the_state(tiny_corpus):
+    """With one step per token a chain moved iff the token's topic changed; with doc-proposals
+    only, nothing is booked as a word-proposal move (and the other way round)."""
+    c = tiny_corpus
+    o = _oracle(c, 8)
+    o.sweep(2, 2)
+    z0 = o.get_assignments().copy()
+    o.sweep(1, 1)                       # the cycle's first step is the word-proposal
+    changed = int((o.get_assignments() != z0).sum())
+    assert o.moves() == (changed, 0) and changed > 0
+    o.set_proposals(2)
+    z0 = o.get_assignments().copy()
+    o.sweep(1, 1)
+    changed = int((o.get_assignments() != z0).sum())
+    assert o.moves() == (0, changed) and changed > 0
+    # two steps: at least as many moves as changed tokens, at most two per token
+    o.set_proposals(0)
+    z0 = o.get_assignments().copy()
+    o.sweep(1, 2)
+    w, d = o.moves()
+    changed = int((o.get_assignments() != z0).sum())
+    assert changed <= w + d <= 2 * c.n_tokens and w > 0 and d > 0
+
+
 # ---- log-likelihood -----------------------------------------------------------------
 
 def _sequential_joint(c, z):
@@ -370,6 +409,28 @@ def test_loglik_equals_sequential_urn_probability(tiny):
     assert lw == pytest.approx(sw, rel=1e-10)
     assert ld == pytest.approx(sd, rel=1e-10)
     assert total == pytest.approx(sw + sd, rel=1e-10)
+
+
+def test_loglik_is_accurate_where_its_large_sums_nearly_cancel():
+    """The big-model shape (V = 1e6, K = 1e5): K*lgamma(V*beta) and sum_k lgamma(n_k + V*beta) are
+    ~8e9 each and cancel to ~1e7.  The closed form, evaluated with exactly rounded sums (math.fsum
+    over scipy's gammaln), pins the oracle's value to 1e-13 of the sum of magnitudes (adding the
+    terms one by one onto the large ones misses that by two orders of magnitude)."""
+    from scipy.special import gammaln
+    c = synth.make("big", seed=3, scale=0.002)
+    o = _oracle(c, seed=2)
+    o.sweep_threads(1, 2, 4)
+    total, lw, ld = o.loglik()
+    nk = o.get_nk().astype(np.float64)
+    _, _, cw = o.get_csr(ldaref.NWK)
+    _, _, cd = o.get_csr(ldaref.NDK)
+    nd = np.diff(c.doc_offsets.numpy()).astype(np.float64)
+    V, K, D, al, be = c.V, c.K, nd.size, c.alpha, c.beta
+    w_terms = [K * math.lgamma(V * be)] + list(gammaln(cw + be) - math.lgamma(be)) + list(-gammaln(nk + V * be))
+    d_terms = [D * math.lgamma(K * al)] + list(gammaln(cd + al) - math.lgamma(al)) + list(-gammaln(nd + K * al))
+    for got, terms in ((lw, w_terms), (ld, d_terms)):
+        assert abs(got - math.fsum(terms)) <= 1e-13 * math.fsum(abs(t) for t in terms)
+    assert total == lw + ld
 
 
 def test_loglik_single_topic_closed_form():
