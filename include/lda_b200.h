@@ -131,6 +131,18 @@ int lda_set_assignments_u16(lda_ctx* ctx, const uint16_t* z, uint64_t seed, uint
  * (token, sweep, step, 0). */
 int lda_sweep(lda_ctx* ctx, int32_t iters, int32_t mh_steps);
 
+/* Yardstick, not a fast path: `iters` frozen sweeps in which every token draws its new topic from the
+ * collapsed conditional itself (Section 3, Eq. 1) under the sweep-start counts with the token's own
+ * contribution removed -- the law the MH chain of lda_sweep() converges to as mh_steps grows
+ * (Section 4.1).  The conditional is split as in Section 4, Eq. 3 (a term over the document's topics
+ * + a smoothing term over all topics); every term is floored to a multiple of 2^-44 and the draw is
+ * the inverse CDF over these integer masses (document term first, topics ascending), so results do
+ * not depend on summation order.  Randomness: Philox counter (token, sweep, 0, 2), word 0.
+ * Cost per token O(K_d log K_w + log K); keeps V*K running sums of 8 bytes while it runs.
+ * Limits (LDA_ERANGE): K <= 16384, V*K*8 bytes <= 24 GiB, K*alpha < 2^17, documents < 2^19 tokens.
+ * Counts, sweep counter and lda_loglik() behave as after lda_sweep(); lda_stats is left alone. */
+int lda_gibbs_sweep(lda_ctx* ctx, int32_t iters);
+
 /* Collapsed joint log p(w,z): word part + document part (Section 7.2, Figure 11).
  * Any output pointer may be NULL. */
 int lda_loglik(lda_ctx* ctx, double* total, double* word_ll, double* doc_ll);

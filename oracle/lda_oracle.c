@@ -701,6 +701,190 @@ int ldaref_accept_ratio(ldaref_ctx *c, int64_t token, int32_t s, int32_t t, int3
  *          - sum_k lgamma(n_k + V*beta)
  *   doc  = D*lgamma(K*alpha) + sum_{n_kd>0} [lgamma(n_kd+alpha) - lgamma(alpha)]
  *          - sum_d lgamma(n_d + K*alpha)                                       */
+/* ------------------------------------------------------------------------- */
+/* Exact-conditional yardstick (Section 3, Eq. 1; Section 4, Eq. 3).           */
+/*                                                                             */
+/* What the MH chain approximates with a few O(1) steps per token is one draw  */
+/* from the collapsed conditional of Eq. 1.  Two samplers draw it exactly:     */
+/*   - the frozen sweep: every token draws from Eq. 1 under the sweep-start    */
+/*     counts (the token's own contribution removed), the like-for-like        */
+/*     yardstick of the frozen MH sweep above;                                  */
+/*   - the sequential sweep: the textbook collapsed Gibbs sampler, counts      */
+/*     updated after every token (the samplers of Figures 12-14 work so).      */
+/* The frozen sweep splits Eq. 1 as Eq. 3 does,                                 */
+/*   p(k) ~ n_kd'(n_kw'+beta)/(n_k'+V beta)  +  alpha (n_kw'+beta)/(n_k'+V beta) */
+/* (primes: token removed), a term over the document's topics plus a term over  */
+/* all topics, and draws by inverse CDF over integer masses (each term floored  */
+/* at 2^-44), so that the draw is a function of the counts alone, whatever the  */
+/* order a second implementation adds the terms in.  One Philox word per        */
+/* token and sweep: counter (token, sweep, 0, 2) for the frozen sweep,          */
+/* (token, sweep, 0, 3) for the sequential one.  The paper is silent on all of  */
+/* this (its Gibbs samplers are other people's systems): these are readings.    */
+/* ------------------------------------------------------------------------- */
+
+/* floor(x * 2^44) of the document term and of the smoothing term of Eq. 3 */
+static uint64_t gibbs_doc_term(const ldaref_ctx *c, int32_t n_kd, int32_t n_kw, int64_t n_k)
+{
+    double x = ((double)n_kd * ((double)n_kw + c->beta)) / ((double)n_k + c->Vbeta);
+    return (uint64_t)(x * FIXED_ONE);
+}
+
+static uint64_t gibbs_prior_term(const ldaref_ctx *c, int32_t n_kw, int64_t n_k)
+{
+    double x = (c->alpha * ((double)n_kw + c->beta)) / ((double)n_k + c->Vbeta);
+    return (uint64_t)(x * FIXED_ONE);
+}
+
+/* Integer masses of token i under the frozen counts: doc_mass[k] (zero outside the document's
+ * topics) and prior_mass[k], k = 0..K-1; `tally` holds the document's n_kd (all K entries). */
+static void gibbs_masses(const ldaref_ctx *c, int64_t i, const int32_t *tally, uint64_t *doc_mass,
+                         uint64_t *prior_mass)
+{
+    int32_t w = c->word[i], z0 = c->z[i];
+    for (int32_t k = 0; k < c->K; ++k) {
+        int32_t own = (k == z0);
+        int32_t n_kd = tally[k] - own, n_kw = count_wk(c, w, k) - own;
+        int64_t n_k = c->nk[k] - own;
+        doc_mass[k] = n_kd > 0 ? gibbs_doc_term(c, n_kd, n_kw, n_k) : 0;
+        prior_mass[k] = gibbs_prior_term(c, n_kw, n_k);
+    }
+}
+
+/* Inverse CDF: the document term's topics first (ascending), then the smoothing term's. */
+static int32_t gibbs_pick(int32_t K, const uint64_t *doc_mass, const uint64_t *prior_mass, uint32_t r0)
+{
+    uint64_t sum_doc = 0, sum_prior = 0;
+    for (int32_t k = 0; k < K; ++k) { sum_doc += doc_mass[k]; sum_prior += prior_mass[k]; }
+    uint64_t total = sum_doc + sum_prior;
+    uint64_t x = (uint64_t)(((unsigned __int128)total * r0) >> 32); /* floor(total * r0 / 2^32) < total */
+    const uint64_t *m = doc_mass;
+    if (x >= sum_doc) { x -= sum_doc; m = prior_mass; }
+    uint64_t cum = 0;
+    for (int32_t k = 0; k < K; ++k) {
+        cum += m[k];
+        if (cum > x) return k;
+    }
+    return K - 1; /* not reached: x < the bucket's sum */
+}
+
+static int gibbs_limits(const ldaref_ctx *c)
+{
+    /* the document term is at most n_d * 2^44: sums stay below 2^63 for documents shorter than 2^19 */
+    for (int64_t d = 0; d < c->D; ++d)
+        if (c->doc_off[d + 1] - c->doc_off[d] >= (1 << 19)) return LDAREF_ERANGE;
+    return LDAREF_OK;
+}
+
+/* `iters` frozen exact-conditional sweeps, the documents shared among `threads` host threads. */
+int ldaref_gibbs_sweep(ldaref_ctx *c, int32_t iters, int32_t threads)
+{
+    if (!c || iters < 0 || threads < 1) return LDAREF_EINVAL;
+    if (!c->inited) return LDAREF_ESTATE;
+    int rc = gibbs_limits(c);
+    if (rc) return rc;
+    uint32_t key[2] = {(uint32_t)c->seed, (uint32_t)(c->seed >> 32)};
+    for (int32_t it = 0; it < iters; ++it) {
+        int failed = 0;
+#pragma omp parallel num_threads(threads)
+        {
+            int32_t *tally = (int32_t *)calloc((size_t)c->K, sizeof(int32_t));
+            uint64_t *dm = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)c->K);
+            uint64_t *pm = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)c->K);
+            if (!tally || !dm || !pm) {
+#pragma omp atomic write
+                failed = 1;
+            } else {
+#pragma omp for schedule(dynamic, 64)
+                for (int64_t d = 0; d < c->D; ++d) {
+                    int64_t lo = c->doc_off[d], hi = c->doc_off[d + 1];
+                    for (int64_t j = lo; j < hi; ++j) tally[c->z[j]] += 1;
+                    for (int64_t i = lo; i < hi; ++i) {
+                        uint32_t ctr[4] = {(uint32_t)i, c->sweep, 0u, 2u}, r[4];
+                        ldaref_philox4x32_10(ctr, key, r);
+                        gibbs_masses(c, i, tally, dm, pm);
+                        c->z_new[i] = gibbs_pick(c->K, dm, pm, r[0]);
+                    }
+                    for (int64_t j = lo; j < hi; ++j) tally[c->z[j]] = 0;
+                }
+            }
+            free(tally); free(dm); free(pm);
+        }
+        if (failed) return LDAREF_ENOMEM;
+        int32_t *tmp = c->z; c->z = c->z_new; c->z_new = tmp;
+        rc = rebuild_counts(c);
+        if (rc) return rc;
+        c->sweep += 1;
+    }
+    return LDAREF_OK;
+}
+
+/* The integer masses of one token under the current counts -- doc_mass_out[K] (document term) and
+ * prior_mass_out[K] (smoothing term) -- and the topic the frozen sweep would pick for it given the
+ * random word r0. */
+int ldaref_gibbs_masses(ldaref_ctx *c, int64_t token, uint64_t *doc_mass_out, uint64_t *prior_mass_out,
+                        uint32_t r0, int32_t *pick_out)
+{
+    if (!c || !doc_mass_out || !prior_mass_out) return LDAREF_EINVAL;
+    if (!c->inited) return LDAREF_ESTATE;
+    if (token < 0 || token >= c->N) return LDAREF_ERANGE;
+    int32_t *tally = (int32_t *)calloc((size_t)c->K, sizeof(int32_t));
+    uint64_t *dm = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)c->K);
+    uint64_t *pm = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)c->K);
+    if (!tally || !dm || !pm) { free(tally); free(dm); free(pm); return LDAREF_ENOMEM; }
+    int32_t d = c->doc_of[token];
+    for (int64_t j = c->doc_off[d]; j < c->doc_off[d + 1]; ++j) tally[c->z[j]] += 1;
+    gibbs_masses(c, token, tally, dm, pm);
+    for (int32_t k = 0; k < c->K; ++k) { doc_mass_out[k] = dm[k]; prior_mass_out[k] = pm[k]; }
+    if (pick_out) *pick_out = gibbs_pick(c->K, dm, pm, r0);
+    free(tally); free(dm); free(pm);
+    return LDAREF_OK;
+}
+
+/* `iters` sweeps of the sequential collapsed Gibbs sampler (Eq. 1): tokens in document order,
+ * every count updated as soon as a token is redrawn; plain floating-point inverse CDF. */
+int ldaref_gibbs_sweep_sequential(ldaref_ctx *c, int32_t iters)
+{
+    if (!c || iters < 0) return LDAREF_EINVAL;
+    if (!c->inited) return LDAREF_ESTATE;
+    if ((int64_t)c->V * c->K > ((int64_t)1 << 31)) return LDAREF_ERANGE; /* a dense n_kw is kept */
+    uint32_t key[2] = {(uint32_t)c->seed, (uint32_t)(c->seed >> 32)};
+    int32_t K = c->K;
+    int32_t *n_wk = (int32_t *)calloc((size_t)c->V * (size_t)K, sizeof(int32_t));
+    int32_t *n_dk = (int32_t *)calloc((size_t)K, sizeof(int32_t));
+    int64_t *n_k = (int64_t *)calloc((size_t)K, sizeof(int64_t));
+    double *cum = (double *)malloc(sizeof(double) * (size_t)K);
+    if (!n_wk || !n_dk || !n_k || !cum) { free(n_wk); free(n_dk); free(n_k); free(cum); return LDAREF_ENOMEM; }
+    for (int64_t i = 0; i < c->N; ++i) { n_wk[(size_t)c->word[i] * K + c->z[i]] += 1; n_k[c->z[i]] += 1; }
+    for (int32_t it = 0; it < iters; ++it) {
+        for (int64_t d = 0; d < c->D; ++d) {
+            int64_t lo = c->doc_off[d], hi = c->doc_off[d + 1];
+            for (int64_t j = lo; j < hi; ++j) n_dk[c->z[j]] += 1;
+            for (int64_t i = lo; i < hi; ++i) {
+                int32_t *row = n_wk + (size_t)c->word[i] * K;
+                int32_t s = c->z[i];
+                n_dk[s] -= 1; row[s] -= 1; n_k[s] -= 1;       /* the counts without token i */
+                double total = 0.0;
+                for (int32_t k = 0; k < K; ++k) {
+                    total += ((double)n_dk[k] + c->alpha) * ((double)row[k] + c->beta) /
+                             ((double)n_k[k] + c->Vbeta);      /* Eq. 1 */
+                    cum[k] = total;
+                }
+                uint32_t ctr[4] = {(uint32_t)i, c->sweep, 0u, 3u}, r[4];
+                ldaref_philox4x32_10(ctr, key, r);
+                double u = (double)r[0] * (1.0 / 4294967296.0) * total;
+                int32_t t = 0;
+                while (t < K - 1 && cum[t] <= u) ++t;
+                c->z[i] = t;
+                n_dk[t] += 1; row[t] += 1; n_k[t] += 1;
+            }
+            for (int64_t j = lo; j < hi; ++j) n_dk[c->z[j]] = 0;
+        }
+        c->sweep += 1;
+    }
+    free(n_wk); free(n_dk); free(n_k); free(cum);
+    return rebuild_counts(c);
+}
+
 /* Compensated sum (Neumaier's form of Kahan summation): `sum` plus the rounding errors collected in `err`. */
 typedef struct { double sum, err; } ksum;
 static void ksum_add(ksum *a, double x)

@@ -81,6 +81,10 @@ def lib():
             L.ldaref_get_assignments.argtypes = [vp, _p(np.int32)]
             L.ldaref_get_tables.argtypes = [vp, vp, vp, C.c_int64, vp, vp, vp,
                                             C.POINTER(C.c_uint64)]
+            L.ldaref_gibbs_sweep.argtypes = [vp, C.c_int32, C.c_int32]
+            L.ldaref_gibbs_sweep_sequential.argtypes = [vp, C.c_int32]
+            L.ldaref_gibbs_masses.argtypes = [vp, C.c_int64, _p(np.uint64), _p(np.uint64), C.c_uint32,
+                                              C.POINTER(C.c_int32)]
             L.ldaref_get_moves.argtypes = [vp, _p(np.int64)]
             L.ldaref_sweeps_done.argtypes = [vp]
             L.ldaref_sweeps_done.restype = C.c_uint32
@@ -245,6 +249,22 @@ class Oracle:
                                        C.byref(B)), "get_tables")
         return dict(row_off=off, sp_thr32=sp_thr[:nnz], sp_alias=sp_al[:nnz], mix32=mix,
                     dn_thr32=dthr, dn_alias=dal, dense_mass=B.value)
+
+    def gibbs_sweep(self, iters: int, threads: int = 1):
+        """Frozen exact-conditional sweeps (the yardstick of the frozen MH sweep)."""
+        _check(lib().ldaref_gibbs_sweep(self._h, iters, threads), "gibbs_sweep")
+
+    def gibbs_sweep_sequential(self, iters: int):
+        """Textbook collapsed Gibbs sweeps, counts updated token by token."""
+        _check(lib().ldaref_gibbs_sweep_sequential(self._h, iters), "gibbs_sweep_sequential")
+
+    def gibbs_masses(self, token: int, r0: int = 0):
+        """(document-term masses, smoothing-term masses, topic picked for the random word r0) of the
+        frozen exact-conditional draw of one token."""
+        dm, pm = np.zeros(self.K, np.uint64), np.zeros(self.K, np.uint64)
+        k = C.c_int32()
+        _check(lib().ldaref_gibbs_masses(self._h, token, dm, pm, r0, C.byref(k)), "gibbs_masses")
+        return dm, pm, k.value
 
     def moves(self):
         """(word-proposal steps, doc-proposal steps) of the last sweep call that moved a chain."""

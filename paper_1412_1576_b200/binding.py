@@ -21,7 +21,7 @@ LDA_NK, LDA_NWK, LDA_NDK = 0, 1, 2
 
 EXPORTS = [
     "lda_create", "lda_set_stream", "lda_set_option", "lda_set_proposals", "lda_load_corpus", "lda_load_corpus_device",
-    "lda_init", "lda_set_assignments", "lda_set_assignments_u16", "lda_sweep", "lda_loglik", "lda_get_counts",
+    "lda_init", "lda_set_assignments", "lda_set_assignments_u16", "lda_sweep", "lda_gibbs_sweep", "lda_loglik", "lda_get_counts",
     "lda_get_assignments", "lda_get_assignments_u16", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
     "lda_dense_table_noalloc",
 ]
@@ -79,6 +79,7 @@ def load_library(path: str | None = None):
     L.lda_set_assignments.argtypes = [vp, vp, u64, u32]
     L.lda_set_assignments_u16.argtypes = [vp, vp, u64, u32]
     L.lda_sweep.argtypes = [vp, i32, i32]
+    L.lda_gibbs_sweep.argtypes = [vp, i32]
     L.lda_loglik.argtypes = [vp, C.POINTER(dbl), C.POINTER(dbl), C.POINTER(dbl)]
     L.lda_get_counts.argtypes = [vp, C.c_int, vp, vp, vp, i64, C.POINTER(i64)]
     L.lda_get_assignments.argtypes = [vp, vp]
@@ -158,6 +159,10 @@ def lda_set_assignments_u16_ptr(h, z_host_ptr, seed, sweep=0):
 
 def lda_sweep(h, iters, mh_steps):
     return load_library().lda_sweep(h, iters, mh_steps)
+
+
+def lda_gibbs_sweep(h, iters):
+    return load_library().lda_gibbs_sweep(h, iters)
 
 
 def lda_loglik(h):
@@ -293,6 +298,10 @@ class LightLDA:
 
     def sweep(self, iters: int, mh_steps: int):
         self._ck(lda_sweep(self._h, iters, mh_steps), "lda_sweep")
+
+    def gibbs_sweep(self, iters: int):
+        """Frozen exact-conditional sweeps (yardstick for the MH sweep)."""
+        self._ck(lda_gibbs_sweep(self._h, iters), "lda_gibbs_sweep")
 
     def loglik(self):
         rc, v = lda_loglik(self._h)

@@ -11,6 +11,7 @@ void set_hist_smem_limits();
 void set_sample_smem_limits();
 void set_doc_smem_limits();
 void set_alias_smem_limits();
+void set_export_smem_limits();
 
 void* dev_alloc(Ctx& c, size_t bytes)
 {
@@ -327,6 +328,24 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         }
         close(D);
     }
+    // tiles of whole documents for the sorted n_kd rows: <= SORT_TILE tokens and <= SORT_TILE documents each
+    std::vector<int32_t> doc_sort_tiles, doc_sort_long;
+    {
+        int32_t s0 = 0;
+        int64_t tok = 0;
+        auto close = [&](int32_t s1) {
+            if (s1 > s0) { doc_sort_tiles.push_back(s0); doc_sort_tiles.push_back(s1); }
+        };
+        for (int32_t d = 0; d < D; ++d) {
+            const int64_t len = doc_off[d + 1] - doc_off[d];
+            if (len > SORT_TILE) { close(d); s0 = d + 1; tok = 0; doc_sort_long.push_back(d); continue; }
+            if (tok + len > SORT_TILE || d - s0 >= SORT_TILE) { close(d); s0 = d; tok = 0; }
+            tok += len;
+        }
+        close(D);
+    }
+    c.n_doc_sort_tiles = (int32_t)(doc_sort_tiles.size() / 2);
+    c.n_doc_sort_long = (int32_t)doc_sort_long.size();
     c.n_word_tiles = (int32_t)(word_tiles.size() / 2);
     c.n_doc_tiles = (int32_t)(doc_tiles.size() / 2);
     c.n_dense = (int32_t)dense_words.size();
@@ -353,12 +372,14 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.dense_words = upload(c, dense_words);
     c.hist_chunks = upload(c, hist_chunks);
     c.long_docs = upload(c, long_docs);
+    c.doc_sort_tiles = upload(c, doc_sort_tiles);
+    c.doc_sort_long = upload(c, doc_sort_long);
     c.alias_big = upload(c, alias_big);
     c.hot_tiles = upload(c, hot_tiles);
     c.hot_tiles_propose = upload(c, hot_tiles_propose);
     c.cold_tiles = upload(c, cold_tiles);
     ok = ok && v.row_start && v.dense_slot && c.word_tiles && c.doc_tiles && c.dense_words &&
-         c.hist_chunks && c.long_docs && c.alias_big && c.hot_tiles && c.hot_tiles_propose && c.cold_tiles;
+         c.hist_chunks && c.long_docs && c.doc_sort_tiles && c.doc_sort_long && c.alias_big && c.hot_tiles && c.hot_tiles_propose && c.cold_tiles;
     v.wk_nnz = (int32_t*)A((size_t)V * 4);
     v.wk_topic = (uint32_t*)A(cap1 * 4);
     v.wk_count = (uint32_t*)A(cap1 * 4);
@@ -462,6 +483,8 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
     set_sample_smem_limits();
     set_doc_smem_limits();
     set_alias_smem_limits();
+    set_export_smem_limits();
+    set_gibbs_smem_limits();
     *out = h;
     return LDA_OK;
 }
@@ -715,6 +738,30 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
     return LDA_OK;
 }
 
+int lda_gibbs_sweep(lda_ctx* h, int32_t iters)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (iters < 0) return fail(&c, LDA_EINVAL, "iters must be >= 0");
+    if (!c.inited) return fail(&c, LDA_ESTATE, "lda_gibbs_sweep before lda_init");
+    if (c.K > GIBBS_MAX_K) return fail(&c, LDA_ERANGE, "the exact-conditional sweep takes K <= 16384");
+    if ((long long)c.V * c.K * 8 > GIBBS_MAX_PREFIX_BYTES)
+        return fail(&c, LDA_ERANGE, "the exact-conditional sweep keeps V*K running sums: V*K*8 bytes must stay below 24 GiB");
+    if ((double)c.K * c.alpha >= 131072.0) return fail(&c, LDA_ERANGE, "the exact-conditional sweep needs K*alpha < 2^17");
+    if (c.v.count_bits > 19) return fail(&c, LDA_ERANGE, "the exact-conditional sweep takes documents shorter than 2^19 tokens");
+    int rc = check_device(c);
+    if (rc) return rc;
+    rc = gibbs_sweep(c, iters);
+    if (rc) return fail(&c, rc, "the exact-conditional sweep failed");
+    int bits = 0;
+    if ((rc = read_err(c, &bits))) { c.inited = false; return rc; }
+    if (bits) {
+        c.inited = false;
+        return fail(&c, LDA_EINTERNAL, "a kernel of the exact-conditional sweep raised the device error word");
+    }
+    return LDA_OK;
+}
+
 int lda_loglik(lda_ctx* h, double* total, double* word_ll, double* doc_ll)
 {
     if (!h) return LDA_EINVAL;
@@ -751,36 +798,24 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
         return LDA_OK;
     }
     if (which == LDA_NDK) {
-        if ((rc = ensure_dk(c))) return rc;
-        // every document's table is copied out and its filled slots sorted by topic on the host
-        std::vector<int32_t> start((size_t)c.D + 1);
-        if (cudaMemcpy(start.data(), v.doc_off, ((size_t)c.D + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
-            return cuda_fail(&c, "copying document offsets");
-        const int64_t spt = 4;  // slots per token (DK_SLOTS_PER_TOKEN of the device code)
-        std::vector<uint32_t> slots((size_t)std::max<int64_t>(spt * c.N, 1));
-        if (c.N && cudaMemcpy(slots.data(), v.dk_slots, (size_t)c.N * 4 * (size_t)spt, cudaMemcpyDeviceToHost) != cudaSuccess)
-            return cuda_fail(&c, "copying n_kd tables");
-        int64_t total = 0;
-        for (uint32_t e : slots) total += (c.N && e != DK_EMPTY);
+        // sorted rows are built on the device; only the row offsets and the nonzeros cross to the host
+        const bool sizes_only = !row_offsets && !topics && !counts;
+        DkCsr r;
+        if ((rc = build_dk_csr(c, r, sizes_only))) return fail(&c, rc, "building the n_kd rows failed");
+        int bits = 0;
+        if ((rc = read_err(c, &bits))) { free_dk_csr(r); return rc; }
+        if (bits) { free_dk_csr(r); return fail(&c, LDA_EINTERNAL, "the n_kd rows raised the device error word"); }
+        const int64_t total = (int64_t)r.total;
         if (nnz_out) *nnz_out = total;
-        if (!row_offsets && !topics && !counts) return LDA_OK;
-        if (capacity < total) return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros");
-        const uint32_t cmask = (1u << v.count_bits) - 1u;
-        std::vector<uint32_t> row;
-        int64_t o = 0;
-        for (int64_t d = 0; d < c.D; ++d) {
-            if (row_offsets) row_offsets[d] = o;
-            row.clear();
-            for (int64_t j = spt * (int64_t)start[(size_t)d]; j < spt * (int64_t)start[(size_t)d + 1]; ++j)
-                if (slots[(size_t)j] != DK_EMPTY) row.push_back(slots[(size_t)j]);
-            std::sort(row.begin(), row.end());
-            for (uint32_t e : row) {
-                if (topics) topics[o] = (int32_t)(e >> v.count_bits);
-                if (counts) counts[o] = (int32_t)(e & cmask);
-                ++o;
-            }
-        }
-        if (row_offsets) row_offsets[c.D] = o;
+        if (sizes_only) { free_dk_csr(r); return LDA_OK; }
+        if (capacity < total) { free_dk_csr(r); return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros"); }
+        static_assert(sizeof(long long) == sizeof(int64_t), "row offsets are copied as they are");
+        bool ok = true;
+        if (row_offsets) ok = ok && cudaMemcpy(row_offsets, r.row_off, ((size_t)c.D + 1) * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
+        if (topics && total) ok = ok && cudaMemcpy(topics, r.topic, (size_t)total * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+        if (counts && total) ok = ok && cudaMemcpy(counts, r.count, (size_t)total * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+        free_dk_csr(r);
+        if (!ok) return cuda_fail(&c, "copying the n_kd rows");
         return LDA_OK;
     }
     if (which != LDA_NWK) return fail(&c, LDA_EINVAL, "unknown table");

@@ -436,6 +436,41 @@ __global__ void k_count_filled(const uint32_t* __restrict__ slots, int64_t n, un
     if (threadIdx.x == 0 && s) atomicAdd(out, s);
 }
 
+struct EmitRowSizes {
+    int32_t* nnz;
+    __device__ __forceinline__ void entry(int32_t, int32_t, uint32_t, uint32_t) const {}
+    __device__ __forceinline__ void rows(int32_t seg, int32_t n) const { nnz[seg] = n; }
+};
+
+struct EmitRowEntries {
+    const long long* row_off;
+    int32_t* topic;
+    int32_t* count;
+    __device__ __forceinline__ void entry(int32_t seg, int32_t rank, uint32_t k, uint32_t n) const
+    {
+        const long long at = row_off[seg] + rank;
+        topic[at] = (int32_t)k;
+        count[at] = (int32_t)n;
+    }
+    __device__ __forceinline__ void rows(int32_t, int32_t) const {}
+};
+
+// Sorted rows of the segments (documents) of `tiles` from z given in segment order: sizes only, or
+// the entries at the row offsets (export.cu).
+template <typename T>
+void launch_doc_rows(Ctx& c, const int32_t* tiles, int32_t n_tiles, const T* z, int32_t* nnz, const long long* row_off,
+                     int32_t* topic, int32_t* count)
+{
+    if (nnz)
+        k_seg_count_sorted<T, EmitRowSizes><<<n_tiles, 256, 0, c.stream>>>(tiles, c.v.doc_off, z, c.v.topic_bits, c.K,
+                                                                            EmitRowSizes{nnz}, c.v.err);
+    else
+        k_seg_count_sorted<T, EmitRowEntries><<<n_tiles, 256, 0, c.stream>>>(
+            tiles, c.v.doc_off, z, c.v.topic_bits, c.K, EmitRowEntries{row_off, topic, count}, c.v.err);
+}
+template void launch_doc_rows<uint16_t>(Ctx&, const int32_t*, int32_t, const uint16_t*, int32_t*, const long long*, int32_t*, int32_t*);
+template void launch_doc_rows<int32_t>(Ctx&, const int32_t*, int32_t, const int32_t*, int32_t*, const long long*, int32_t*, int32_t*);
+
 static int hist_window(const Ctx& c) { return c.K < HIST_BINS ? c.K : HIST_BINS; }
 
 template <typename T>

@@ -174,6 +174,10 @@ struct Ctx {
     int32_t* dense_words = nullptr;  // [n_dense]
     int32_t* hist_chunks = nullptr;  // [n_hist_chunks*3] (word, first token, count)
     int32_t* long_docs = nullptr;    // [n_long_docs]
+    // sorted n_kd rows (export.cu): tiles of whole documents of at most SORT_TILE tokens, and the longer documents
+    int32_t n_doc_sort_tiles = 0, n_doc_sort_long = 0;
+    int32_t* doc_sort_tiles = nullptr;
+    int32_t* doc_sort_long = nullptr;
     int32_t* alias_big = nullptr;    // [n_alias_big] words whose row can exceed ALIAS_WARP_MAX; the first
                                      // n_alias_mid of them cannot exceed ALIAS_SMEM_ITEMS_MID
     int32_t* hot_tiles = nullptr;    // [n_hot_tiles*3] (word, first token, count): MH kernel, hot word (accept pass)
@@ -233,6 +237,24 @@ size_t doc_tile_smem_bytes(int tile_tokens);  // dynamic shared memory of the do
 int ensure_exchange(Ctx& c, int mh_steps);  // (re)allocates View::prop / View::dside; LDA_* status
 int launch_loglik(Ctx& c, double* out3_host);
 int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host);
+
+// n_kd as sorted rows in device memory (export.cu): row_off[D+1], and unless sizes_only the entries.
+// The caller releases the arrays with free_dk_csr().
+struct DkCsr {
+    long long* row_off = nullptr;
+    int32_t* nnz = nullptr;
+    int32_t* topic = nullptr;
+    int32_t* count = nullptr;
+    long long total = 0;
+};
+int build_dk_csr(Ctx& c, DkCsr& r, bool sizes_only);  // LDA_* status; queued on c.stream, rows complete after a sync
+void free_dk_csr(DkCsr& r);
+
+// Exact-conditional yardstick (gibbs.cu): `iters` frozen sweeps drawing from Eq. 1.  LDA_* status.
+constexpr int GIBBS_MAX_K = 16384;              // a word's dense n_kw row is staged in shared memory
+constexpr long long GIBBS_MAX_PREFIX_BYTES = 24ll << 30;  // V * K running sums of 8 bytes
+int gibbs_sweep(Ctx& c, int32_t iters);
+void set_gibbs_smem_limits();
 
 // load-time layout (sort + offsets); fills c.v token arrays. Returns LDA_* status.
 int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_host);

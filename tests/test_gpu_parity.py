@@ -346,6 +346,38 @@ def test_large_shape_sample_against_oracle():
         assert a == pytest.approx(b, rel=1e-9)
 
 
+def test_exact_conditional_sweep_matches_oracle(tiny_corpus, small_corpus):
+    """The yardstick sweep (every token drawn from Eq. 1 under frozen counts, split as Eq. 3, integer
+    masses): every token equal to the oracle's, on short and long documents, hot and tail words, and the
+    state it leaves is a state the MH sweep continues from on both sides alike."""
+    import os
+    cores = max(1, len(os.sched_getaffinity(0)))
+    long_docs = synth.generate(V=50, K=40, D=6, length=("fixed", 5000), zipf_s=1.0, alpha=0.1, beta=0.01, seed=5)
+    mid = synth.make("mid", seed=1, scale=0.01)
+    for c in (tiny_corpus, small_corpus, long_docs, mid):
+        g, o = _pair(c, seed=17)
+        g.sweep(2, 2)
+        o.sweep_threads(2, 2, cores)
+        for sweep in range(2):
+            g.gibbs_sweep(1)
+            o.gibbs_sweep(1, cores)
+            assert np.array_equal(g.get_assignments(), o.get_assignments()), sweep
+        assert g.stats()["sweeps_done"] == o.sweeps_done == 4
+        _assert_same_counts(g, o)
+        g.sweep(1, 2)
+        o.sweep_threads(1, 2, cores)
+        assert np.array_equal(g.get_assignments(), o.get_assignments())
+        for a, b in zip(g.loglik(), o.loglik()):
+            assert a == pytest.approx(b, rel=1e-10)
+    # beyond its limits the entry point refuses
+    w = binding.LightLDA(8, 20_000, 0.1, 0.1)
+    w.load_corpus(np.array([0, 1, 2], np.int32), np.array([0, 3], np.int64))
+    w.init(1)
+    with pytest.raises(binding.LdaError) as e:
+        w.gibbs_sweep(1)
+    assert e.value.status == binding.LDA_ERANGE
+
+
 def test_edge_cases():
     # empty documents, a single token, one topic, absent words
     w = np.array([3, 3, 0, 7, 7, 7], np.int32)

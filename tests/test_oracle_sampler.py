@@ -380,6 +380,99 @@ def test_move_counters_count_the_steps_that_changed_the_state(tiny_corpus):
     assert changed <= w + d <= 2 * c.n_tokens and w > 0 and d > 0
 
 
+# ---- exact-conditional yardstick (Eq. 1 / Eq. 3) --------------------------------------------------
+
+def _eq1_conditional(c, z, counts, i):
+    """Brute-force p(z_i = k | rest) of Eq. 1 from dense counts, the token's own contribution removed."""
+    n_wk, n_dk, n_k, doc = counts
+    w, d, s = c.word_ids.numpy()[i], doc[i], z[i]
+    own = np.zeros(c.K)
+    own[s] = 1.0
+    p = (n_dk[d] - own + c.alpha) * (n_wk[w] - own + c.beta) / (n_k - own + c.V * c.beta)
+    return p / p.sum()
+
+
+def test_gibbs_masses_are_eq1_and_the_pick_is_the_inverse_cdf(tiny):
+    c, o, z, counts = tiny
+    rng = np.random.default_rng(11)
+    for i in rng.integers(0, c.n_tokens, size=12):
+        dm, pm, _ = o.gibbs_masses(int(i))
+        mass = dm.astype(object) + pm.astype(object)          # exact integers
+        total = int(mass.sum())
+        pmf = np.array([int(m) / total for m in mass])
+        assert np.abs(pmf - _eq1_conditional(c, z, counts, i)).max() < 1e-10
+        # document-term masses sit on the document's other topics only
+        n_dk = counts[1][counts[3][i]].copy()
+        n_dk[z[i]] -= 1
+        assert np.array_equal(dm > 0, n_dk > 0)
+        # inverse CDF in exact integer arithmetic: document-term topics first, then all topics
+        order = [(int(m), k) for k, m in enumerate(dm)] + [(int(m), k) for k, m in enumerate(pm)]
+        for r0 in [0, 1, 2 ** 31, 2 ** 32 - 1] + [int(x) for x in rng.integers(0, 2 ** 32, size=40)]:
+            x, cum, want = (total * r0) >> 32, 0, None
+            for m, k in order:
+                cum += m
+                if cum > x:
+                    want = k
+                    break
+            assert o.gibbs_masses(int(i), r0)[2] == want
+        # and its law over uniform random words is the conditional
+        draws = np.array([o.gibbs_masses(int(i), int(r))[2] for r in rng.integers(0, 2 ** 32, size=4000)])
+        keep = pmf * 4000 >= 5
+        obs = np.bincount(draws, minlength=c.K)[keep]
+        exp = pmf[keep] * obs.sum() / pmf[keep].sum()
+        assert stats.chisquare(obs, exp).pvalue > 1e-4
+
+
+def test_frozen_gibbs_sweep_draws_every_token_from_the_sweep_start_state(tiny_corpus):
+    c = tiny_corpus
+    a, b = _oracle(c, 21), _oracle(c, 21)
+    a.sweep(2, 2)
+    b.sweep(2, 2)
+    z0 = a.get_assignments().copy()
+    picks = {}
+    for i in np.random.default_rng(3).integers(0, c.n_tokens, size=300):
+        r = ldaref.philox([int(i), a.sweeps_done, 0, 2], [21, 0])
+        picks[int(i)] = a.gibbs_masses(int(i), int(r[0]))[2]
+    a.gibbs_sweep(1, 1)
+    b.gibbs_sweep(1, 4)                                   # documents shared among threads: same sweep
+    z1 = a.get_assignments()
+    assert np.array_equal(z1, b.get_assignments()) and a.sweeps_done == 3
+    assert all(z1[i] == k for i, k in picks.items())
+    assert float(np.mean(z1 != z0)) > 0.2
+    n_wk, n_dk, n_k, _ = _dense_counts(c, z1)
+    assert np.array_equal(a.get_nk(), n_k)
+
+
+def test_sequential_gibbs_first_token_follows_eq1():
+    """The first token a sequential sweep redraws sees every other token at its old topic: over many
+    seeds its new topic is distributed as Eq. 1 says."""
+    c, o, z, counts = _toy(V=10, K=5, D=4, L=7)
+    p = _eq1_conditional(c, z, counts, 0)
+    draws = []
+    for seed in range(6000):
+        o.set_assignments(z, seed, 0)
+        o.gibbs_sweep_sequential(1)
+        draws.append(o.get_assignments()[0])
+    obs = np.bincount(np.array(draws), minlength=c.K)
+    assert stats.chisquare(obs, p * len(draws)).pvalue > 1e-4
+    # counts are those of the new assignments
+    z1 = o.get_assignments()
+    assert np.array_equal(o.get_nk(), np.bincount(z1, minlength=c.K))
+
+
+def test_yardsticks_order_on_tiny(tiny_corpus):
+    """Trend only (the paper prints no number: parity unpinned): after 30 sweeps from the same start the
+    sequential Gibbs sampler is ahead of the frozen exact-conditional sweep, which is ahead of (or level
+    with) the frozen two-step MH sweep it is the limit of."""
+    c = tiny_corpus
+    seq, fro, mh = _oracle(c, 3), _oracle(c, 3), _oracle(c, 3)
+    seq.gibbs_sweep_sequential(30)
+    fro.gibbs_sweep(30, 4)
+    mh.sweep(30, 2)
+    start = _oracle(c, 3).loglik()[0]
+    assert seq.loglik()[0] > fro.loglik()[0] > mh.loglik()[0] - 0.02 * abs(mh.loglik()[0]) and mh.loglik()[0] > start
+
+
 # ---- log-likelihood -----------------------------------------------------------------
 
 def _sequential_joint(c, z):
