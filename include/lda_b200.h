@@ -101,7 +101,14 @@ int lda_set_option(lda_ctx* ctx, const char* key, double value);
 #define LDA_PROPOSALS_DOC 2
 int lda_set_proposals(lda_ctx* ctx, int mode);
 
-/* Corpus in document order: token i has word word_ids[i]; document d owns tokens
+/* Storage of n_kw (Section 5): words with many tokens keep a dense row of K counters; the long tail
+ * keeps sparse rows.  The paper's sparse rows are hash tables because it updates them in place;
+ * here every row is rebuilt from the assignments each sweep, so a tail row is stored SORTED by
+ * topic (binary search instead of probing; the same order defines the items of the word's alias
+ * table).  Hashed rows in the paper's sense are what the document side uses for n_kd.  Which form a
+ * word gets never changes a result.
+ *
+ * Corpus in document order: token i has word word_ids[i]; document d owns tokens
  * [doc_offsets[d], doc_offsets[d+1]); doc_offsets has n_docs+1 entries, [0] = 0,
  * [n_docs] = n_tokens; empty documents are legal.  Builds the word-sorted token
  * layout once (Section 6, item 3) and chooses the dense/sparse class of every
@@ -187,7 +194,13 @@ int lda_get_tables(lda_ctx* ctx, uint32_t* sp_thr32, int32_t* sp_alias, int64_t 
  * LDA_NOALLOC_MAX_K topics (20 bytes per topic, about 2.6 MB); every GPU that loads the library
  * holds it until the process exits.  K above LDA_NOALLOC_MAX_K is refused with LDA_ERANGE.
  * The first call on each device looks up the array's device address (one runtime query, made
- * with that device current); make that first call before starting any stream capture.
+ * with that device current; the runtime may load the library's device code at that moment too, if
+ * nothing of it ran on the device before); make that first call before starting any stream capture.
+ * The looked-up address is cached per device without a lock: if two host threads may make the
+ * FIRST call on a device at the same time, serialise those two calls (later calls only read it).
+ * A caller that passes status_dev == NULL cannot learn of a failed construction (e.g. beta so small
+ * against n_k that every fixed-point weight is zero): the call still returns LDA_OK and the
+ * outputs stay unwritten.  Pass a status word wherever the inputs are not known to be sane.
  * All calls share the one array and it keeps the previous call's contents; nothing in it needs
  * clearing because each call overwrites what it later reads, and the status word is zeroed on
  * the stream before the kernel.  Two calls that overlap on the GPU (different streams, or

@@ -22,14 +22,29 @@ void* dev_alloc(Ctx& c, size_t bytes)
         return nullptr;
     }
     c.allocs.push_back(p);
+    c.alloc_bytes.push_back(bytes);
     c.device_bytes += (int64_t)bytes;
     return p;
+}
+
+void dev_free(Ctx& c, void* p)
+{
+    if (!p) return;
+    for (size_t i = 0; i < c.allocs.size(); ++i)
+        if (c.allocs[i] == p) {
+            c.device_bytes -= (int64_t)c.alloc_bytes[i];
+            c.allocs.erase(c.allocs.begin() + i);
+            c.alloc_bytes.erase(c.alloc_bytes.begin() + i);
+            break;
+        }
+    cudaFree(p);
 }
 
 void dev_free_all(Ctx& c)
 {
     for (void* p : c.allocs) cudaFree(p);
     c.allocs.clear();
+    c.alloc_bytes.clear();
     c.device_bytes = 0;
 }
 
@@ -81,11 +96,10 @@ static void free_corpus(Ctx& c)
 {
     int* err = c.v.err;
     // the error word is allocated in lda_create and outlives corpora
-    std::vector<void*> keep;
+    std::vector<void*> drop;
     for (void* p : c.allocs)
-        if (p == (void*)err) keep.push_back(p); else cudaFree(p);
-    c.allocs = keep;
-    c.device_bytes = keep.empty() ? 0 : 32;
+        if (p != (void*)err) drop.push_back(p);
+    for (void* p : drop) dev_free(c, p);
     View nv{};
     nv.V = c.V; nv.K = c.K; nv.alpha = c.alpha; nv.beta = c.beta;
     nv.Vbeta = (double)c.V * c.beta;
@@ -105,12 +119,6 @@ static void free_corpus(Ctx& c)
 int lda::ensure_exchange(Ctx& c, int mh_steps)
 {
     if (c.N == 0 || (mh_steps <= c.side_steps && c.side_mode == c.proposals && c.v.dside)) return LDA_OK;
-    auto drop = [&](void* p) {
-        if (!p) return;
-        for (size_t i = 0; i < c.allocs.size(); ++i)
-            if (c.allocs[i] == p) { c.allocs.erase(c.allocs.begin() + i); break; }
-        cudaFree(p);
-    };
     auto bytes_for = [&](int mode, int steps, size_t& prop_b, size_t& side_b, size_t& ua_b, int& stride) {
         const size_t zt = c.wide_topics ? 4 : 2, n = (size_t)c.N;
         const int n_word = mode == LDA_PROPOSALS_CYCLE ? (steps + 1) / 2 : mode == LDA_PROPOSALS_WORD ? steps : 0;
@@ -124,13 +132,9 @@ int lda::ensure_exchange(Ctx& c, int mh_steps)
     cudaStreamSynchronize(c.stream);
     size_t pb = 0, sb = 0, ub = 0;
     int stride = 0;
-    if (c.side_steps) {
-        bytes_for(c.side_mode, c.side_steps, pb, sb, ub, stride);
-        c.device_bytes -= (int64_t)(pb + sb + ub);
-    }
-    drop(c.v.prop);
-    drop(c.v.dside);
-    drop(c.v.ua_w);
+    dev_free(c, c.v.prop);
+    dev_free(c, c.v.dside);
+    dev_free(c, c.v.ua_w);
     c.v.prop = nullptr;
     c.v.dside = nullptr;
     c.v.ua_w = nullptr;

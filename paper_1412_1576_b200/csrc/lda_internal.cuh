@@ -191,6 +191,7 @@ struct Ctx {
     double* red = nullptr;                   // reduction partials for the log-likelihood
     int64_t* red_i = nullptr;
     std::vector<void*> allocs;
+    std::vector<size_t> alloc_bytes;  // size of every entry of `allocs`
     int64_t device_bytes = 0;
     lda_stats stats{};
     int64_t launches = 0;
@@ -260,6 +261,7 @@ void set_gibbs_smem_limits();
 int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_host);
 
 void* dev_alloc(Ctx& c, size_t bytes);  // tracked cudaMalloc; nullptr on failure
+void dev_free(Ctx& c, void* p);         // releases one tracked allocation (nullptr: nothing)
 void dev_free_all(Ctx& c);
 
 }  // namespace lda

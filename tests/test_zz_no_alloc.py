@@ -14,17 +14,20 @@ from paper_1412_1576_b200 import binding, synth
 pytestmark = pytest.mark.gpu
 
 
-def _tables_noalloc(torch, n_k, K, V, beta, stream):
+def _tables_noalloc(torch, n_k, K, V, beta, stream, check_free=False):
     nk_dev = torch.from_numpy(n_k).cuda()
     thr = torch.full((K,), -1, dtype=torch.int32, device="cuda")
     al = torch.full((K,), -1, dtype=torch.int32, device="cuda")
     mass = torch.zeros(1, dtype=torch.int64, device="cuda")
     status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
     torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     rc = binding.lda_dense_table_noalloc(nk_dev.data_ptr(), K, V, beta, thr.data_ptr(), al.data_ptr(),
                                          mass.data_ptr(), status.data_ptr(), stream)
     assert rc == binding.LDA_OK
     torch.cuda.synchronize()
+    if check_free:      # not on a device's first call: that one may load the library's device code
+        assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
     assert int(status.item()) == 0
     return (thr.cpu().numpy().view(np.uint32), al.cpu().numpy(), int(mass.item()) & (2 ** 64 - 1))
 
@@ -39,7 +42,7 @@ def test_noalloc_dense_table_equals_regular_entry_point_twice(K):
     g.init(1)
     for call in range(2):          # two calls in a row share the library's scratch array
         want = g.get_tables()
-        got = _tables_noalloc(torch, g.get_nk(), K, c.V, c.beta, stream)
+        got = _tables_noalloc(torch, g.get_nk(), K, c.V, c.beta, stream, check_free=call == 1)
         assert np.array_equal(got[0], want["dn_thr32"]), call
         assert np.array_equal(got[1], want["dn_alias"]), call
         assert got[2] == want["dense_mass"], call
