@@ -33,7 +33,7 @@ extern "C" {
 #endif
 
 #define LDA_OK 0
-#define LDA_EINVAL (-1)    /* NULL pointer, V/K <= 0, alpha/beta not finite and > 0, iters < 0, mh_steps < 1 */
+#define LDA_EINVAL (-1)    /* NULL pointer, V/K <= 0, alpha/beta not finite and > 0, iters < 0, mh_steps outside 1..1024 */
 #define LDA_ERANGE (-2)    /* word id outside [0,V), bad offsets, sizes beyond the limits, capacity too small */
 #define LDA_ESTATE (-3)    /* call order: load before init, init before sweep */
 #define LDA_ENOMEM (-4)    /* host or device allocation failed */

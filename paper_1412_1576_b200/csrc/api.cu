@@ -241,6 +241,10 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         // a dense row of K counters only pays for a word with a fair share of K tokens
         tf_cut = std::max<int32_t>({tmp[nth], (int32_t)std::max(1.0, c.dense_min_tf), K / 8});
     }
+    // K above the staging limit: only words with more than WARM_MAX_TF tokens get a dense row, the
+    // others with more tokens than a tail tile holds a sorted row built by a CTA of their own
+    const bool warm_class = K > HOT_STAGE_MAX_K;
+    std::vector<int32_t> warm_words;
     std::vector<int32_t> dense_slot((size_t)V, -1), dense_words, row_start((size_t)V + 1), alias_big, alias_mid;
     std::vector<int32_t> hist_chunks, word_tiles;
     int64_t cap_total = 0;
@@ -250,13 +254,16 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         cap_total += cap;
         if (cap > ALIAS_SMEM_ITEMS_MID) alias_big.push_back(w);
         else if (cap > ALIAS_WARP_MAX) alias_mid.push_back(w);
-        if (tf[w] > SORT_TILE || (tf[w] > 0 && tf[w] >= tf_cut)) {
+        if (warm_class && tf[w] > SORT_TILE && tf[w] <= WARM_MAX_TF) {
+            warm_words.push_back(w);
+        } else if (tf[w] > SORT_TILE || (tf[w] > 0 && tf[w] >= tf_cut)) {
             dense_slot[w] = (int32_t)dense_words.size();
             dense_words.push_back(w);
             for (int32_t o = 0; o < tf[w]; o += HIST_CHUNK) {
                 hist_chunks.push_back(w);
                 hist_chunks.push_back(word_off[w] + o);
                 hist_chunks.push_back(std::min(HIST_CHUNK, tf[w] - o));
+                hist_chunks.push_back(tf[w] <= HIST_CHUNK ? 1 : 0);
             }
         }
     }
@@ -268,7 +275,7 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
             if (s1 > s0) { word_tiles.push_back(s0); word_tiles.push_back(s1); }
         };
         for (int32_t w = 0; w < V; ++w) {
-            if (dense_slot[w] >= 0) { close(w); s0 = w + 1; tok = 0; continue; }
+            if (dense_slot[w] >= 0 || tf[w] > SORT_TILE) { close(w); s0 = w + 1; tok = 0; continue; }
             if (tok + tf[w] > SORT_TILE || w - s0 >= SORT_TILE) { close(w); s0 = w; tok = 0; }
             tok += tf[w];
         }
@@ -276,9 +283,9 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     }
     // MH kernel work lists: a hot word (more tokens than a tail tile holds; it has a dense row by
     // the rule above) is cut into runs of HOT_TILE tokens, tail words are packed whole into tiles
-    std::vector<int32_t> hot_tiles, hot_tiles_propose, cold_tiles;
+    std::vector<int32_t> hot_tiles, hot_tiles_warm, hot_tiles_propose, cold_tiles;
     {
-        static_assert(COLD_TILE >= SORT_TILE, "every word longer than a tail tile must have a dense row");
+        static_assert(COLD_TILE >= SORT_TILE, "every word longer than a tail tile must have a dense row or a warm one");
         int32_t s0 = 0, tok = 0;
         auto close = [&](int32_t s1) {
             if (s1 > s0 && tok > 0) { cold_tiles.push_back(s0); cold_tiles.push_back(s1); }
@@ -286,10 +293,11 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         for (int32_t w = 0; w < V; ++w) {
             if (tf[w] > COLD_TILE) {
                 close(w); s0 = w + 1; tok = 0;
+                std::vector<int32_t>& runs = dense_slot[w] >= 0 ? hot_tiles : hot_tiles_warm;
                 for (int32_t o = 0; o < tf[w]; o += HOT_TILE) {
-                    hot_tiles.push_back(w);
-                    hot_tiles.push_back(word_off[w] + o);
-                    hot_tiles.push_back(std::min(HOT_TILE, tf[w] - o));
+                    runs.push_back(w);
+                    runs.push_back(word_off[w] + o);
+                    runs.push_back(std::min(HOT_TILE, tf[w] - o));
                 }
                 for (int32_t o = 0; o < tf[w]; o += HOT_TILE_PROPOSE) {
                     hot_tiles_propose.push_back(w);
@@ -353,12 +361,14 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.n_word_tiles = (int32_t)(word_tiles.size() / 2);
     c.n_doc_tiles = (int32_t)(doc_tiles.size() / 2);
     c.n_dense = (int32_t)dense_words.size();
-    c.n_hist_chunks = (int32_t)(hist_chunks.size() / 3);
+    c.n_hist_chunks = (int32_t)(hist_chunks.size() / 4);
     c.n_long_docs = (int32_t)long_docs.size();
     c.n_alias_mid = (int32_t)alias_mid.size();
     alias_big.insert(alias_big.begin(), alias_mid.begin(), alias_mid.end());
     c.n_alias_big = (int32_t)alias_big.size();
     c.n_hot_tiles = (int32_t)(hot_tiles.size() / 3);
+    c.n_hot_tiles_warm = (int32_t)(hot_tiles_warm.size() / 3);
+    c.n_warm = (int32_t)warm_words.size();
     c.n_hot_tiles_propose = (int32_t)(hot_tiles_propose.size() / 3);
     c.n_cold_tiles = (int32_t)(cold_tiles.size() / 2);
 
@@ -380,10 +390,12 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.doc_sort_long = upload(c, doc_sort_long);
     c.alias_big = upload(c, alias_big);
     c.hot_tiles = upload(c, hot_tiles);
+    c.hot_tiles_warm = upload(c, hot_tiles_warm);
+    c.warm_words = upload(c, warm_words);
     c.hot_tiles_propose = upload(c, hot_tiles_propose);
     c.cold_tiles = upload(c, cold_tiles);
     ok = ok && v.row_start && v.dense_slot && c.word_tiles && c.doc_tiles && c.dense_words &&
-         c.hist_chunks && c.long_docs && c.doc_sort_tiles && c.doc_sort_long && c.alias_big && c.hot_tiles && c.hot_tiles_propose && c.cold_tiles;
+         c.hist_chunks && c.long_docs && c.doc_sort_tiles && c.doc_sort_long && c.alias_big && c.hot_tiles && c.hot_tiles_warm && c.warm_words && c.hot_tiles_propose && c.cold_tiles;
     v.wk_nnz = (int32_t*)A((size_t)V * 4);
     v.wk_topic = (uint32_t*)A(cap1 * 4);
     v.wk_count = (uint32_t*)A(cap1 * 4);
@@ -664,7 +676,8 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
 {
     if (!h) return LDA_EINVAL;
     Ctx& c = h->c;
-    if (iters < 0 || mh_steps < 1) return fail(&c, LDA_EINVAL, "iters must be >= 0 and mh_steps >= 1");
+    if (iters < 0 || mh_steps < 1 || mh_steps > 1024)
+        return fail(&c, LDA_EINVAL, "iters must be >= 0 and mh_steps in 1..1024");
     if (!c.inited) return fail(&c, LDA_ESTATE, "lda_sweep before lda_init");
     int rc = check_device(c);
     if (rc) return rc;

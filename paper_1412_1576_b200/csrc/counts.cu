@@ -189,37 +189,115 @@ k_word_rows(const int32_t* __restrict__ tiles, const int32_t* __restrict__ word_
     }
 }
 
-// Hot words: one CTA per chunk of a word's tokens; histogram of a window of
-// topics in shared memory, merged into the word's dense row with one global
-// add per nonzero bin.
+// Warm words (more tokens than a tail tile holds, no dense row): one CTA per word.  The word's
+// tokens are counted in 16-bit bins over a window of topics in shared memory (two bins per word of
+// shared memory; a warm word has fewer than 65536 tokens), and the nonzero bins, read in order,
+// are the sorted row: every warp owns a run of consecutive bin pairs, counts its nonzero bins, the
+// warps' totals are scanned, and a second walk writes the entries.
+template <typename T>
+__global__ void __launch_bounds__(512)
+k_warm_rows(const int32_t* __restrict__ words, const int32_t* __restrict__ word_off, const T* __restrict__ z,
+            const int32_t* __restrict__ row_start, uint32_t* __restrict__ wk_topic, uint32_t* __restrict__ wk_count,
+            int32_t* __restrict__ wk_nnz, int32_t K, int32_t window, int* err)
+{
+    extern __shared__ __align__(16) uint32_t bins2[];
+    __shared__ int32_t warp_total[17];
+    const int32_t w = words[blockIdx.x];
+    const int32_t first = word_off[w], cnt = word_off[w + 1] - first;
+    const int32_t out0 = row_start[w], cap = row_start[w + 1] - out0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    int32_t done = 0;
+    for (int32_t k0 = 0; k0 < K; k0 += window) {
+        const int32_t nb = min(window, K - k0), nw = (nb + 1) >> 1;
+        const int32_t nw4 = (nw + 3) >> 2;
+        for (int b = threadIdx.x; b < nw4; b += blockDim.x) reinterpret_cast<uint4*>(bins2)[b] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
+        for (int32_t j = threadIdx.x; j < cnt; j += blockDim.x) {
+            const uint32_t k = (uint32_t)__ldcs(z + first + j);
+            if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); continue; }
+            const uint32_t b = k - (uint32_t)k0;
+            if (b < (uint32_t)nb) atomicAdd(&bins2[b >> 1], (b & 1u) ? 0x10000u : 1u);
+        }
+        __syncthreads();
+        // a warp's run of bin pairs
+        const int32_t per_warp = ((nw + nwarps - 1) / nwarps + 31) & ~31;
+        const int32_t q0 = min(nw, warp * per_warp), q1 = min(nw, q0 + per_warp);
+        int32_t mine = 0;
+        for (int32_t q = q0 + lane; q < q1; q += 32) {
+            const uint32_t n2 = bins2[q];
+            mine += ((n2 & 0xFFFFu) != 0u) + ((n2 >> 16) != 0u);
+        }
+        mine = warp_reduce_sum<int32_t>(mine);
+        if (lane == 0) warp_total[warp] = mine;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int32_t run = 0;
+            for (int i = 0; i < nwarps; ++i) { const int32_t t = warp_total[i]; warp_total[i] = run; run += t; }
+            warp_total[16] = run;
+        }
+        __syncthreads();
+        int32_t at = done + warp_total[warp];
+        const int32_t total = warp_total[16];
+        if (done + total > cap) {
+            if (threadIdx.x == 0) atomicOr(err, ERR_ROW_OVERFLOW);
+        } else {
+            const uint32_t below = (1u << lane) - 1u;
+            for (int32_t q = q0 + lane; q - lane < q1; q += 32) {
+                const uint32_t n2 = q < q1 ? bins2[q] : 0u;
+                const bool lo = (n2 & 0xFFFFu) != 0u, hi = (n2 >> 16) != 0u;
+                const uint32_t m_lo = __ballot_sync(0xffffffffu, lo), m_hi = __ballot_sync(0xffffffffu, hi);
+                int32_t pos = at + __popc(m_lo & below) + __popc(m_hi & below);
+                if (lo) {
+                    wk_topic[out0 + pos] = (uint32_t)(k0 + 2 * q);
+                    wk_count[out0 + pos] = n2 & 0xFFFFu;
+                    ++pos;
+                }
+                if (hi) {
+                    wk_topic[out0 + pos] = (uint32_t)(k0 + 2 * q + 1);
+                    wk_count[out0 + pos] = n2 >> 16;
+                }
+                at += __popc(m_lo) + __popc(m_hi);
+            }
+        }
+        done += total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) wk_nnz[w] = done;
+}
+
+// Hot words: one CTA per run of a word's tokens (up to HIST_CHUNK of them); histogram of a window
+// of topics in shared memory (32-bit bins), merged into the word's dense row.  A word that fits
+// one run owns its row: its nonzero bins are stored.  A longer word's runs add theirs, one global
+// add per nonzero bin and run -- a few runs per word, so a row takes few adds per bin.
 template <typename T>
 __global__ void __launch_bounds__(512)
 k_hist_chunks(const int32_t* __restrict__ chunks, const T* __restrict__ z,
               const int32_t* __restrict__ dense_slot, int32_t* __restrict__ dense_rows, int32_t K,
               int32_t stride, int32_t window, int* err)
 {
-    // two 16-bit counters per word of shared memory: a chunk holds at most HIST_CHUNK < 65536 tokens
-    extern __shared__ uint32_t bins2[];
-    const int32_t w = chunks[3 * blockIdx.x], first = chunks[3 * blockIdx.x + 1],
-                  cnt = chunks[3 * blockIdx.x + 2];
+    extern __shared__ __align__(16) int32_t hist_bins[];
+    const int32_t w = chunks[4 * blockIdx.x], first = chunks[4 * blockIdx.x + 1],
+                  cnt = chunks[4 * blockIdx.x + 2];
+    const bool alone = chunks[4 * blockIdx.x + 3] != 0;  // the word's only run
     int32_t* row = dense_rows + (size_t)dense_slot[w] * stride;
     for (int32_t k0 = 0; k0 < K; k0 += window) {
-        const int32_t nb = min(window, K - k0), nw = (nb + 1) >> 1;
-        for (int b = threadIdx.x; b < nw; b += blockDim.x) bins2[b] = 0;
+        const int32_t nb = min(window, K - k0);
+        for (int b = threadIdx.x; b < (nb + 3) / 4; b += blockDim.x)
+            reinterpret_cast<int4*>(hist_bins)[b] = make_int4(0, 0, 0, 0);
         __syncthreads();
         auto add = [&](uint32_t k) {
             if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); return; }
             const uint32_t b = k - (uint32_t)k0;
-            if (b < (uint32_t)nb) atomicAdd(&bins2[b >> 1], (b & 1u) ? 0x10000u : 1u);
+            if (b < (uint32_t)nb) atomicAdd(&hist_bins[b], 1);
         };
-        // the chunk's topics are read 16 bytes at a time; what lies before the first and after the
+        // the run's topics are read 16 bytes at a time; what lies before the first and after the
         // last 16-byte boundary one by one
         constexpr int E = 16 / (int)sizeof(T);
         const int32_t head = min(cnt, (int32_t)((E - (first & (E - 1))) & (E - 1)));
         const int32_t nvec = (cnt - head) / E;
         const uint4* zv = reinterpret_cast<const uint4*>(z + first + head);
         for (int q = threadIdx.x; q < nvec; q += blockDim.x) {
-            const uint4 x = __ldcs(zv + q);
+            const uint4 x = k0 == 0 ? __ldcs(zv + q) : __ldg(zv + q);
             const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -234,10 +312,12 @@ k_hist_chunks(const int32_t* __restrict__ chunks, const T* __restrict__ z,
         for (int j = threadIdx.x; j < cnt - nvec * E; j += blockDim.x)
             add((uint32_t)z[first + (j < head ? j : nvec * E + j)]);
         __syncthreads();
-        for (int b = threadIdx.x; b < nw; b += blockDim.x) {
-            const uint32_t n2 = bins2[b];
-            if (n2 & 0xFFFFu) atomicAdd(&row[k0 + 2 * b], (int32_t)(n2 & 0xFFFFu));
-            if (n2 >> 16) atomicAdd(&row[k0 + 2 * b + 1], (int32_t)(n2 >> 16));
+        for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+            const int32_t n = hist_bins[b];
+            if (n) {
+                if (alone) row[k0 + b] = n;  // the row was cleared before the launch
+                else atomicAdd(&row[k0 + b], n);
+            }
         }
         __syncthreads();
     }
@@ -414,6 +494,22 @@ k_nk_from_sparse(const int32_t* __restrict__ row_start, const int32_t* __restric
     }
 }
 
+// The same sums when K is too large for bins in shared memory: one global add per row entry (the
+// adds of one warp go to different topics: a row holds a topic once).
+__global__ void __launch_bounds__(256)
+k_nk_from_sparse_direct(const int32_t* __restrict__ row_start, const int32_t* __restrict__ wk_nnz,
+                        const uint32_t* __restrict__ wk_topic, const uint32_t* __restrict__ wk_count,
+                        const int32_t* __restrict__ dense_slot, int32_t V, int32_t* __restrict__ nk)
+{
+    const int lane = threadIdx.x & 31;
+    const int32_t warps = (gridDim.x * blockDim.x) >> 5;
+    for (int32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < V; w += warps) {
+        if (dense_slot[w] >= 0) continue;
+        const int32_t r0 = row_start[w], n = wk_nnz[w];
+        for (int32_t j = lane; j < n; j += 32) atomicAdd(&nk[__ldcs(wk_topic + r0 + j)], (int32_t)__ldcs(wk_count + r0 + j));
+    }
+}
+
 __global__ void k_sum_i32(const int32_t* __restrict__ a, int64_t n, unsigned long long* out)
 {
     __shared__ unsigned long long tmp[32];
@@ -493,10 +589,16 @@ static int count_wk_t(Ctx& c)
         }
         ++launches;
     }
+    if (c.n_warm) {
+        const int win = c.K < HIST16_BINS ? c.K : HIST16_BINS;
+        k_warm_rows<T><<<c.n_warm, 512, (size_t)((win + 7) / 8) * 16, c.side[1]>>>(
+            c.warm_words, v.word_off, z, v.row_start, v.wk_topic, v.wk_count, v.wk_nnz, c.K, win, v.err);
+        ++launches;
+    }
     if (c.n_dense) {
         cudaMemsetAsync(v.dense_rows, 0, (size_t)c.n_dense * v.dense_stride * 4, c.stream);
-        const int win = c.K < HIST16_BINS ? c.K : HIST16_BINS;
-        k_hist_chunks<T><<<c.n_hist_chunks, 512, (size_t)((win + 1) / 2) * 4, c.stream>>>(
+        const int win = c.K < HIST32_BINS ? c.K : HIST32_BINS;
+        k_hist_chunks<T><<<c.n_hist_chunks, 512, (size_t)((win + 3) / 4) * 16, c.stream>>>(
             c.hist_chunks, z, v.dense_slot, v.dense_rows, c.K, v.dense_stride, win, v.err);
         k_compact_dense<<<c.n_dense, 256, 0, c.stream>>>(c.dense_words, v.dense_slot, v.dense_rows,
                                                          v.row_start, v.wk_topic, v.wk_count,
@@ -522,10 +624,16 @@ static int count_k(Ctx& c)
         ++launches;
     }
     if (c.n_dense < c.V) {
-        const int win = hist_window(c);
-        const int grid = std::min(148 * 4, (int)((c.V + 255) / 256));
-        k_nk_from_sparse<<<grid, 512, (size_t)win * 4, c.side[0]>>>(v.row_start, v.wk_nnz, v.wk_topic, v.wk_count,
-                                                                   v.dense_slot, c.V, v.nk, c.K, win);
+        if (c.K <= HIST_BINS) {
+            const int win = hist_window(c);
+            const int grid = std::min(148 * 4, (int)((c.V + 255) / 256));
+            k_nk_from_sparse<<<grid, 512, (size_t)win * 4, c.side[0]>>>(v.row_start, v.wk_nnz, v.wk_topic, v.wk_count,
+                                                                       v.dense_slot, c.V, v.nk, c.K, win);
+        } else {
+            const int grid = (int)std::min<int64_t>(148 * 16, ((int64_t)c.V * 32 + 255) / 256);
+            k_nk_from_sparse_direct<<<grid, 256, 0, c.side[0]>>>(v.row_start, v.wk_nnz, v.wk_topic, v.wk_count,
+                                                                v.dense_slot, c.V, v.nk);
+        }
         ++launches;
     }
     join_streams(c);
@@ -574,8 +682,10 @@ void set_hist_smem_limits()
     const int doc_bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
     cudaFuncSetAttribute(k_doc_hash<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
     cudaFuncSetAttribute(k_doc_hash<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
-    cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST16_BINS * 2);
-    cudaFuncSetAttribute(k_hist_chunks<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST16_BINS * 2);
+    cudaFuncSetAttribute(k_warm_rows<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST16_BINS * 2 + 16);
+    cudaFuncSetAttribute(k_warm_rows<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST16_BINS * 2 + 16);
+    cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST32_BINS * 4);
+    cudaFuncSetAttribute(k_hist_chunks<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST32_BINS * 4);
     cudaFuncSetAttribute(k_nk_from_sparse, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_BINS * 4);
 }
 

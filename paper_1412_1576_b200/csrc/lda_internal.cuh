@@ -64,12 +64,12 @@ static_assert(DOC_TILE_SLOTS % 4 == 0, "a tile's tables are cleared 16 bytes at 
 constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DOC_TILE_SLOTS + 4 + 4;
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (32-bit bins)
 constexpr int WORD_ROWS_BITMAP_MAX_K = 16384;  // tail rows: topic bitmap up to this K, key sort above
-constexpr int HIST16_BINS = 106496;  // window of the per-chunk n_kw histogram (16-bit bins, 208 KB)
+constexpr int HIST16_BINS = 106496;  // window of a warm word's n_kw histogram (16-bit bins, 208 KB)
+constexpr int HIST32_BINS = 49152;   // window of a hot word's n_kw histogram (32-bit bins, 192 KB)
 #ifndef LDA_HIST_CHUNK
-#define LDA_HIST_CHUNK 32768
+#define LDA_HIST_CHUNK 262144
 #endif
-constexpr int HIST_CHUNK = LDA_HIST_CHUNK;    // tokens per CTA in the histogram path
-static_assert(HIST_CHUNK < 65536, "the per-chunk histogram counts in 16 bits");
+constexpr int HIST_CHUNK = LDA_HIST_CHUNK;    // tokens per CTA (one run of a word) in the histogram path
 #ifndef LDA_HOT_TILE
 #define LDA_HOT_TILE 32768
 #endif
@@ -81,6 +81,11 @@ constexpr int HOT_TILE_PROPOSE = LDA_HOT_TILE_PROPOSE;  // propose pass: nothing
 constexpr int COLD_TILE = 2048;      // MH kernel: tokens of a tile of whole tail words
 constexpr int COLD_WORDS = 512;      // MH kernel: words per tail tile
 constexpr int HOT_STAGE_MAX_K = 16384;  // dense rows up to this many topics are staged in shared memory
+// Beyond that K a dense row (4 K bytes) only pays for frequent words.  Words with more tokens than
+// a tail tile holds but at most WARM_MAX_TF keep a sorted sparse row only ("warm" words): rebuilt by
+// one CTA per word from a 16-bit histogram over the topics, and staged whole in shared memory by
+// the accept pass (a row has at most as many entries as the word has tokens).
+constexpr int WARM_MAX_TF = 12288;
 #ifndef LDA_ALIAS_WARP_MAX
 #define LDA_ALIAS_WARP_MAX 512
 #endif
@@ -172,7 +177,7 @@ struct Ctx {
     int32_t* word_tiles = nullptr;   // [n_word_tiles*2] word ranges sorted per CTA
     int32_t* doc_tiles = nullptr;    // [n_doc_tiles*2]
     int32_t* dense_words = nullptr;  // [n_dense]
-    int32_t* hist_chunks = nullptr;  // [n_hist_chunks*3] (word, first token, count)
+    int32_t* hist_chunks = nullptr;  // [n_hist_chunks*4] (word, first token, count, 1 if the word's only run)
     int32_t* long_docs = nullptr;    // [n_long_docs]
     // sorted n_kd rows (export.cu): tiles of whole documents of at most SORT_TILE tokens, and the longer documents
     int32_t n_doc_sort_tiles = 0, n_doc_sort_long = 0;
@@ -180,7 +185,10 @@ struct Ctx {
     int32_t* doc_sort_long = nullptr;
     int32_t* alias_big = nullptr;    // [n_alias_big] words whose row can exceed ALIAS_WARP_MAX; the first
                                      // n_alias_mid of them cannot exceed ALIAS_SMEM_ITEMS_MID
-    int32_t* hot_tiles = nullptr;    // [n_hot_tiles*3] (word, first token, count): MH kernel, hot word (accept pass)
+    int32_t n_warm = 0, n_hot_tiles_warm = 0;
+    int32_t* warm_words = nullptr;      // [n_warm] words with a sorted row and more tokens than a tail tile holds
+    int32_t* hot_tiles_warm = nullptr;  // [n_hot_tiles_warm*3] their runs for the accept pass
+    int32_t* hot_tiles = nullptr;    // [n_hot_tiles*3] (word, first token, count): MH kernel, words with a dense row (accept pass)
     int32_t* hot_tiles_propose = nullptr;  // the same cut into the shorter runs of the propose passs
     int32_t* cold_tiles = nullptr;   // [n_cold_tiles*2] word ranges of whole tail words: MH kernel
     // alias-construction scratch

@@ -116,24 +116,22 @@ struct HotTile {
     uint32_t mix;
     void* bar;   // STAGED: barrier the bulk copy of the row completes on
     bool ready;  // the row has landed
-    bool gave_up;  // STAGED: the wait for the copy ran out; the rows are read from global memory instead
-    const int32_t* row_global;  // where the staged copies came from
-    const int32_t* nk_global;
+    bool gave_up;  // STAGED: the wait for the copy ran out
     __device__ __forceinline__ Ref ref(int32_t) const { return Ref{}; }
     // Called before the first lookup: the row must have landed by then.  If the bounded wait runs
-    // out, the error word is raised and this thread reads the (identical) rows in global memory, so
-    // nothing is ever read from shared memory the copy has not filled.
-    __device__ __forceinline__ void prepare(const View& v)
+    // out, the error word is raised and false returned: the caller must not touch the staged rows
+    // (it drops its remaining tokens; the host refuses to go on from a sweep that raised the word).
+    __device__ __forceinline__ bool prepare(const View& v)
     {
         if (STAGED && !ready) {
             if (!mbar_wait_bounded(bar, 0, STAGE_WAIT_LIMIT)) {
                 atomicOr(v.err, ERR_STAGE);
                 gave_up = true;
-                row = row_global;
-                nk_tab = nk_global;
+                return false;
             }
             ready = true;
         }
+        return true;
     }
     __device__ __forceinline__ int32_t count(const Ref&, uint32_t k) const
     {
@@ -196,7 +194,7 @@ struct ColdTile {
         }
         return Ref{rs[lo], nnz[lo], mix[lo]};
     }
-    __device__ __forceinline__ void prepare(const View&) {}
+    __device__ __forceinline__ bool prepare(const View&) { return true; }
     __device__ __forceinline__ int32_t count(const Ref& w, uint32_t k) const
     {
         int32_t lo = 0, hi = w.nnz;
@@ -227,6 +225,34 @@ struct ColdTile {
             t = (d.e.y == d.b || d.rz < d.e.x) ? d.b : d.e.y;
             n_tw = -1;
         }
+    }
+};
+
+// A warm word: sorted n_kw row without a dense one, staged in shared memory and looked up by binary
+// search inside one bucket of 2^shift consecutive topics: start[b] is the row position of bucket
+// b's first entry (WARM_BUCKETS + 1 positions, the last one the row's end).
+constexpr int WARM_BUCKETS = 1024;
+struct WarmTile {
+    struct Ref {};
+    const uint32_t* topic;
+    const uint32_t* cnt;
+    const int32_t* nk_tab;  // n_k in global memory
+    const uint32_t* start;
+    int shift;
+    static constexpr bool gave_up = false;
+    __device__ __forceinline__ Ref ref(int32_t) const { return Ref{}; }
+    __device__ __forceinline__ bool prepare(const View&) { return true; }
+    __device__ __forceinline__ int32_t nk(uint32_t k) const { return __ldg(nk_tab + k); }
+    __device__ __forceinline__ int32_t count(const Ref&, uint32_t k) const
+    {
+        int32_t lo = (int32_t)start[k >> shift];
+        const int32_t end = (int32_t)start[(k >> shift) + 1];
+        int32_t hi = end;
+        while (lo < hi) {
+            const int32_t mid = (lo + hi) >> 1;
+            if (topic[mid] < k) lo = mid + 1; else hi = mid;
+        }
+        return (lo < end && topic[lo] == k) ? (int32_t)cnt[lo] : 0;
     }
 };
 
@@ -322,7 +348,10 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
     const size_t N = (size_t)v.N;
     T* zw = reinterpret_cast<T*>(v.zw);
     bool bad = false;
-    uint32_t moved_w = 0, moved_d = 0;  // steps of this thread's tokens that moved the chain, by proposal
+    // steps of this thread's tokens that moved the chain: word-proposals in the low half, doc-proposals
+    // in the high half (a thread takes fewer than 65536 steps of either kind: lda_sweep bounds mh_steps)
+    uint32_t moved = 0;
+    bool staged_ok = true;
     // The reads of a token are issued ahead of its turn: its block-major index two iterations
     // early, the gathered record (which needs that index) one iteration early.
     const uint4* side4 = reinterpret_cast<const uint4*>(v.dside);
@@ -373,7 +402,8 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
             }
             if (m0 == 0) {
                 // counts at the start state s = z0, where all three are >= 1
-                tile.prepare(v);
+                staged_ok = tile.prepare(v);
+                if (!staged_ok) break;
                 z0 = s = own >> cb;
                 n_sd = (int32_t)(own & cmask);
                 n_sw = tile.count(w, z0);
@@ -412,7 +442,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 }
                 const double u = __dmul_rn(u32_to_double((uint32_t)ua[i]), INV_2_32);
                 if (live && __dmul_rn(u, den) < num) {
-                    if (step_is_doc<MODE>(i)) ++moved_d; else ++moved_w;
+                    moved += step_is_doc<MODE>(i) ? 0x10000u : 1u;
                     s = t[i];
                     n_sd = n_td;
                     n_sw = n_tw[i];
@@ -420,6 +450,7 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
                 }
             }
         }
+        if (!staged_ok) break;
         __stcs(zw + p, (T)s);
         store_topic_pair(reinterpret_cast<T*>(v.zbm), at, s);
     }
@@ -428,8 +459,8 @@ __device__ __forceinline__ void accept_tokens(const View& v, Tile& tile, const i
     __shared__ uint32_t moved_s[2];
     if (threadIdx.x == 0) moved_s[0] = moved_s[1] = 0u;
     __syncthreads();
-    moved_w = warp_reduce_sum<uint32_t>(moved_w);
-    moved_d = warp_reduce_sum<uint32_t>(moved_d);
+    const uint32_t moved_w = warp_reduce_sum<uint32_t>(moved & 0xFFFFu);
+    const uint32_t moved_d = warp_reduce_sum<uint32_t>(moved >> 16);
     if ((threadIdx.x & 31) == 0) {
         if (moved_w) atomicAdd(&moved_s[0], moved_w);
         if (moved_d) atomicAdd(&moved_s[1], moved_d);
@@ -483,14 +514,47 @@ k_word_hot(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
     tile.bar = &bar;
     tile.ready = !(STAGED && ACCEPT);
     tile.gave_up = false;
-    tile.row_global = row_g;
-    tile.nk_global = v.nk;
     if (ACCEPT) accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, accept_threads(FIXED), key, sweep, mh_steps);
     else propose_tokens<T, MODE, FIXED>(v, tile, p0, p0 + cnt, PROPOSE_THREADS, key, sweep, mh_steps);
     // ACCEPT: every thread that had a token waited for the copy; thread 0 always has one.  A thread
     // whose wait ran out waits once more (bounded again) before the CTA may retire: a bulk copy still
     // in flight must not land in shared memory that belongs to the next CTA.
     if (STAGED && ACCEPT && tile.gave_up) mbar_wait_bounded(&bar, 0, STAGE_WAIT_LIMIT);
+}
+
+// Warm words, accept pass: tile = (word, first token, count) like a hot word's, the sorted row
+// instead of a dense one.
+template <typename T, int CH, int MODE, int FIXED>
+__global__ void __launch_bounds__(accept_threads(FIXED), LDA_ACCEPT_MIN_CTAS)
+k_word_warm(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep, int32_t mh_steps_arg)
+{
+    const int32_t mh_steps = FIXED > 0 ? FIXED : mh_steps_arg;
+    extern __shared__ __align__(16) uint32_t warm_smem[];  // [2 * WARM_MAX_TF] topics, counts
+    __shared__ uint32_t start_s[WARM_BUCKETS + 1];
+    const int32_t w = tiles[3 * blockIdx.x], p0 = tiles[3 * blockIdx.x + 1], cnt = tiles[3 * blockIdx.x + 2];
+    const int32_t r0 = __ldg(v.row_start + w);
+    const int32_t nnz = min(__ldg(v.wk_nnz + w), WARM_MAX_TF);  // never more entries than tokens
+    uint32_t* topic_s = warm_smem;
+    uint32_t* count_s = warm_smem + WARM_MAX_TF;
+    for (int32_t j = threadIdx.x; j < nnz; j += blockDim.x) {
+        topic_s[j] = __ldg(v.wk_topic + r0 + j);
+        count_s[j] = __ldg(v.wk_count + r0 + j);
+    }
+    __syncthreads();
+    int shift = 0;
+    while (((v.K - 1) >> shift) >= WARM_BUCKETS) ++shift;
+    for (int32_t b = threadIdx.x; b <= WARM_BUCKETS; b += blockDim.x) {
+        const uint32_t k = (uint32_t)b << shift;
+        int32_t lo = 0, hi = nnz;
+        while (lo < hi) {
+            const int32_t mid = (lo + hi) >> 1;
+            if (topic_s[mid] < k) lo = mid + 1; else hi = mid;
+        }
+        start_s[b] = (uint32_t)lo;
+    }
+    __syncthreads();
+    WarmTile tile{topic_s, count_s, v.nk, start_s, shift};
+    accept_tokens<T, CH, MODE, FIXED>(v, tile, p0, p0 + cnt, accept_threads(FIXED), key, sweep, mh_steps);
 }
 
 // Tail words: tile = range of whole words [w0, w1) with at most COLD_TILE tokens.
@@ -609,6 +673,11 @@ static int launch_accept(Ctx& c, uint2 key, int mh_steps)
                 <<<c.n_hot_tiles, accept_threads(FIXED), 0, c.stream>>>(v, c.hot_tiles, key, c.sweep, mh_steps);
         ++launches;
     }
+    if (c.n_hot_tiles_warm) {
+        k_word_warm<T, CH, MODE, FIXED><<<c.n_hot_tiles_warm, accept_threads(FIXED), WARM_MAX_TF * 8, c.stream>>>(
+            v, c.hot_tiles_warm, key, c.sweep, mh_steps);
+        ++launches;
+    }
     if (c.n_cold_tiles) {
         k_word_cold<T, CH, true, MODE, FIXED><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key,
                                                                                            c.sweep, mh_steps);
@@ -690,6 +759,7 @@ static void set_hot_limit_one()
 {
     cudaFuncSetAttribute(k_word_hot<T, CH, true, true, MODE, FIXED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          HOT_STAGE_MAX_K * 8);
+    cudaFuncSetAttribute(k_word_warm<T, CH, MODE, FIXED>, cudaFuncAttributeMaxDynamicSharedMemorySize, WARM_MAX_TF * 8);
 }
 
 template <typename T, int CH>

@@ -236,19 +236,24 @@ def test_wide_topics_and_long_documents():
 
 def test_hot_words_with_unstaged_rows_and_odd_step_counts():
     """K above the shared-memory staging limit with words hot enough to get their own tiles, and
-    step counts that end on a word-proposal or exceed one group of four."""
-    c = synth.generate(V=40, K=20_000, D=300, length=("fixed", 400), zipf_s=1.0, alpha=0.05, beta=0.01, seed=8)
-    g, o = _pair(c, seed=5)
-    # rows of a few hundred to more than ten thousand items: every scratch placement of the alias build
-    nnz = np.diff(o.get_csr(ldaref.NWK)[0])
-    assert nnz.min() < 2048 < 4096 < np.sort(nnz)[-3] and nnz.max() > 10240
-    _assert_same_tables(g, o)
-    for mh_steps in (2, 5, 3):
-        g.sweep(1, mh_steps)
-        o.sweep(1, mh_steps)
-        assert np.array_equal(g.get_assignments(), o.get_assignments()), mh_steps
-    _assert_same_counts(g, o)
-    _assert_same_tables(g, o)
+    step counts that end on a word-proposal or exceed one group of four.  Words of 2049 to 12 288 tokens
+    are "warm" (sorted row only, staged by the accept pass), those above keep dense rows that the
+    accept pass reads in place."""
+    for D in (300, 1500):
+        c = synth.generate(V=40, K=20_000, D=D, length=("fixed", 400), zipf_s=1.0, alpha=0.05, beta=0.01, seed=8)
+        g, o = _pair(c, seed=5)
+        tf = np.bincount(c.word_ids.numpy(), minlength=c.V)
+        assert g.stats()["n_dense_words"] == int((tf > 12288).sum()) > 0 and int(((tf > 2048) & (tf <= 12288)).sum()) > 0
+        # rows of a few hundred to more than ten thousand items: every scratch placement of the alias build
+        nnz = np.diff(o.get_csr(ldaref.NWK)[0])
+        assert (D > 300 or nnz.min() < 2048) and 4096 < np.sort(nnz)[-3] and nnz.max() > 12288
+        _assert_same_tables(g, o)
+        for mh_steps in (2, 5, 3):
+            g.sweep(1, mh_steps)
+            o.sweep(1, mh_steps)
+            assert np.array_equal(g.get_assignments(), o.get_assignments()), mh_steps
+        _assert_same_counts(g, o)
+        _assert_same_tables(g, o)
 
 
 @pytest.mark.parametrize("mode", [binding.PROPOSALS_WORD, binding.PROPOSALS_DOC])
