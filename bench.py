@@ -355,9 +355,13 @@ def run_ours(args):
     if os.path.exists(prof):
         try:
             table = json.load(open(prof))
+            def per_token(entry):
+                # a kernel's measured DRAM bytes per token: the part that follows the tokens plus the
+                # part that follows the nonzeros of n_kw, at this run's rho
+                return entry.get("dram_bytes_per_token", 0.0) + entry.get("dram_bytes_per_nnz", 0.0) * rho
             tr = table.get(top, {})
             if tr.get("workload") == args.workload and tr.get("mh_steps") == M:
-                roofline["traffic"] = tr["dram_bytes_per_token"] * N
+                roofline["traffic"] = per_token(tr) * N
                 roofline["traffic_source"] = tr.get("source")
                 if "issue_active_pct" in tr:   # ncu smsp__issue_active of the same capture
                     roofline["issue_active_pct"] = tr["issue_active_pct"]
@@ -366,7 +370,7 @@ def run_ours(args):
             have = {k: table[k] for k in need if k in table and table[k].get("workload") == args.workload
                     and table[k].get("mh_steps") == M}
             if len(have) == len(need) and sweep_ms > 0:
-                moved = sum(v["dram_bytes_per_token"] for v in have.values())
+                moved = sum(per_token(v) for v in have.values())
                 roofline["bytes_moved_per_token"] = moved
                 roofline["bytes_moved_frac"] = moved * N / (sweep_ms * 1e-3) / 1e9 / peak
                 roofline["bytes_moved_what"] = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of every per-sweep "
