@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--sharded", action="store_true",
+                    help="document-sharded run of ONE corpus over the ranks (one all-reduce of n_kw per sweep) "
+                         "instead of independent replicas; strong scaling, off by default")
     ap.add_argument("--no-windows", action="store_true", help="skip the late-sweep and own-step-count windows")
     ap.add_argument("--late-sweep", type=int, default=50, help="first sweep of the late window")
     return ap.parse_args()
@@ -406,6 +409,86 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sharded(args):
+    """One corpus, its documents sharded over the ranks (paper_1412_1576_b200/sharded.py): per sweep
+    every rank sweeps its documents against the shared counts, then ONE all-reduce (NCCL) sums the
+    ranks' n_kw matrices.  Total work is fixed as the ranks grow: strong scaling."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_1412_1576_b200 import binding, sharded, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1 or "MASTER_ADDR" in os.environ:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        reduce = sharded.torch_all_reduce
+    else:
+        reduce = lambda m: None        # one shard: the sum over the shards is the matrix itself
+    cfg = workload_config(args)
+    M = args.mh_steps
+    corpus = synth.generate(seed=args.seed, device="cuda", **cfg)      # the same corpus on every rank
+    w = corpus.word_ids.cpu().numpy()
+    off = corpus.doc_offsets.cpu().numpy()
+    N = corpus.n_tokens
+    del corpus
+    torch.cuda.empty_cache()
+    stream = torch.cuda.current_stream()
+    matrix = torch.zeros(cfg["V"] * cfg["K"], dtype=torch.int32, device="cuda")
+    run = sharded.ShardedSweep(binding.LightLDA(cfg["V"], cfg["K"], cfg["alpha"], cfg["beta"], stream=stream.cuda_stream),
+                               matrix, all_reduce=reduce)
+    d0, d1 = sharded.shard_documents(off, world, rank)
+    run.load(w, off, d0, d1, sharded.term_frequencies(w, cfg["V"]))
+    n_local = int(off[d1] - off[d0])
+    del w
+    run.init(1234)
+    run.sweep(max(1, args.warmup), M)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist.is_initialized():
+            dist.barrier()
+        torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    ev0.record(stream)
+    run.sweep(args.steps, M)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist.is_initialized():
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    word, doc = run.loglik_parts()
+    if dist.is_initialized():
+        t = torch.tensor([doc], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t)
+        doc = float(t.item())
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    ms_per_step = ms / args.steps
+    print(json.dumps({
+        "metric": f"{METRIC} (mh_steps={M})", "value": N / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload} LDA" + (f" x{args.scale}" if args.scale != 1.0 else ""),
+                   "V": cfg["V"], "K": cfg["K"], "n_tokens": N, "tokens_on_rank_0": n_local, "mh_steps": M,
+                   "parallelism": f"documents sharded over {world} rank(s), one all-reduce of n_kw "
+                                  f"({cfg['V'] * cfg['K'] * 4} bytes) per sweep"},
+        "clocks": clocks, "loglik": word + doc,
+        "what": "lda_sweep + lda_word_counts_to_dense + all-reduce + lda_word_counts_from_dense per step"}))
+
+
 def host_cores() -> int:
     try:
         return max(1, len(os.sched_getaffinity(0)))
@@ -491,5 +574,7 @@ if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.sharded:
+        run_sharded(a)
     else:
         run_ours(a)

@@ -138,6 +138,34 @@ int lda_set_assignments_u16(lda_ctx* ctx, const uint16_t* z, uint64_t seed, uint
  * (token, sweep, step, 0). */
 int lda_sweep(lda_ctx* ctx, int32_t iters, int32_t mh_steps);
 
+/* Document-sharded data parallelism (Section 6, "Parameter Server and Data Placement": documents are
+ * partitioned over the workers, the word-topic table n_kw and its column sums n_k are shared and the
+ * workers' updates are aggregated after sampling).  A context may hold ONE SHARD of a corpus -- a
+ * run of consecutive documents.  Its n_kd is its own; n_kw and n_k must be the sums over all shards
+ * whenever a sweep starts.  The library does the local halves, the caller the sum (one all-reduce of
+ * a dense int32 matrix per sweep, e.g. ncclAllReduce / torch.distributed.all_reduce):
+ *
+ *   lda_set_shard(ctx, first_token, global_term_freq)      before lda_load_corpus
+ *   lda_load_corpus(shard's documents); lda_init(seed)      the same seed on every shard
+ *   repeat:  lda_word_counts_to_dense(ctx, M)               M = this shard's n_kw, DEVICE int32 [V*K]
+ *            M <- sum of M over the shards                  (the caller's collective)
+ *            lda_word_counts_from_dense(ctx, M)             n_kw, n_k := the sums
+ *            lda_sweep(ctx, 1, mh_steps)                    leaves the shard's own counts again
+ *
+ * first_token is the index of the shard's first token in the whole corpus: it offsets the Philox
+ * token key, so a sharded run draws exactly the random numbers of a single context holding all the
+ * documents and, the counts being frozen during a sweep, produces exactly its assignments.
+ * global_term_freq (HOST, V entries, copied; NULL = this corpus is the whole) is every word's token
+ * count over ALL shards: it sizes the rows and picks the dense/sparse class of a word.
+ * lda_word_counts_from_dense returns LDA_ERANGE (and the context must be initialised again) if a
+ * row of the matrix has more nonzeros than min(global_term_freq[w], K) or a negative entry.
+ * lda_loglik() on a shard gives the word part of the counts last imported and the document part of
+ * the shard's own documents: sum the document parts over the shards, take the word part once.
+ * Needs V*K*4 bytes per matrix (the caller's buffer). */
+int lda_set_shard(lda_ctx* ctx, int64_t first_token, const int32_t* global_term_freq);
+int lda_word_counts_to_dense(lda_ctx* ctx, int32_t* nwk_dev);
+int lda_word_counts_from_dense(lda_ctx* ctx, const int32_t* nwk_dev);
+
 /* Yardstick, not a fast path: `iters` frozen sweeps in which every token draws its new topic from the
  * collapsed conditional itself (Section 3, Eq. 1) under the sweep-start counts with the token's own
  * contribution removed -- the law the MH chain of lda_sweep() converges to as mh_steps grows

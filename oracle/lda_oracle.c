@@ -228,6 +228,8 @@ typedef struct ldaref_ctx {
     uint64_t seed;
     uint32_t sweep;      /* number of sweeps done since init */
     int proposals;       /* 0 cycle (word, doc, word, ...), 1 word-proposal only, 2 doc-proposal only */
+    uint32_t tok_base;   /* Philox token key of token 0 (nonzero when the corpus is one shard of a larger one) */
+    int64_t row_cap;     /* entries the four row arrays (row_*, sp_*) can hold */
     int64_t moves[2];    /* steps of the last sweep call that moved a chain: word-, doc-proposals */
     int loaded, inited;
 } ldaref_ctx;
@@ -299,6 +301,7 @@ int ldaref_load_corpus(ldaref_ctx *c, const int32_t *word_ids, int64_t n_tokens,
     int64_t N = n_tokens, D = n_docs;
     size_t n1 = (size_t)(N > 0 ? N : 1);
     c->N = N; c->D = D;
+    c->row_cap = (int64_t)n1;
     c->word = (int32_t *)malloc(sizeof(int32_t) * n1);
     c->doc_off = (int64_t *)malloc(sizeof(int64_t) * (size_t)(D + 1));
     c->doc_of = (int32_t *)malloc(sizeof(int32_t) * n1);
@@ -404,7 +407,7 @@ int ldaref_init(ldaref_ctx *c, uint64_t seed)
     c->sweep = 0;
     uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
     for (int64_t i = 0; i < c->N; ++i) {
-        uint32_t ctr[4] = {(uint32_t)i, 0u, 0u, 1u}, r[4];
+        uint32_t ctr[4] = {c->tok_base + (uint32_t)i, 0u, 0u, 1u}, r[4];
         ldaref_philox4x32_10(ctr, key, r);
         c->z[i] = (int32_t)scale_to_range(r[0], (uint32_t)c->K);
     }
@@ -537,7 +540,7 @@ static int32_t run_chain(const ldaref_ctx *c, int64_t i, uint32_t sweep, int32_t
     uint32_t key[2] = {(uint32_t)c->seed, (uint32_t)(c->seed >> 32)};
     int32_t s = c->z[i];
     for (int32_t m = 0; m < steps; ++m) {
-        uint32_t ctr[4] = {(uint32_t)i, sweep, (uint32_t)m, 0u}, r[4];
+        uint32_t ctr[4] = {c->tok_base + (uint32_t)i, sweep, (uint32_t)m, 0u}, r[4];
         ldaref_philox4x32_10(ctr, key, r);
         /* Section 4.3: the cycle alternates the two proposals; each alone is a valid MH kernel
          * for the same target (the variants compared in Figure 11) */
@@ -799,7 +802,7 @@ int ldaref_gibbs_sweep(ldaref_ctx *c, int32_t iters, int32_t threads)
                     int64_t lo = c->doc_off[d], hi = c->doc_off[d + 1];
                     for (int64_t j = lo; j < hi; ++j) tally[c->z[j]] += 1;
                     for (int64_t i = lo; i < hi; ++i) {
-                        uint32_t ctr[4] = {(uint32_t)i, c->sweep, 0u, 2u}, r[4];
+                        uint32_t ctr[4] = {c->tok_base + (uint32_t)i, c->sweep, 0u, 2u}, r[4];
                         ldaref_philox4x32_10(ctr, key, r);
                         gibbs_masses(c, i, tally, dm, pm);
                         c->z_new[i] = gibbs_pick(c->K, dm, pm, r[0]);
@@ -869,7 +872,7 @@ int ldaref_gibbs_sweep_sequential(ldaref_ctx *c, int32_t iters)
                              ((double)n_k[k] + c->Vbeta);      /* Eq. 1 */
                     cum[k] = total;
                 }
-                uint32_t ctr[4] = {(uint32_t)i, c->sweep, 0u, 3u}, r[4];
+                uint32_t ctr[4] = {c->tok_base + (uint32_t)i, c->sweep, 0u, 3u}, r[4];
                 ldaref_philox4x32_10(ctr, key, r);
                 double u = (double)r[0] * (1.0 / 4294967296.0) * total;
                 int32_t t = 0;
@@ -883,6 +886,73 @@ int ldaref_gibbs_sweep_sequential(ldaref_ctx *c, int32_t iters)
     }
     free(n_wk); free(n_dk); free(n_k); free(cum);
     return rebuild_counts(c);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Document shards (Section 6, "Parameter Server and Data Placement": the      */
+/* documents are partitioned over the workers, the word-topic table is        */
+/* shared).  An oracle context may hold a run of consecutive documents of a   */
+/* larger corpus: first_token is the index of its first token there and       */
+/* offsets the Philox token key; n_kw travels as a dense V x K matrix, the    */
+/* caller adds the shards' matrices up and hands the sum back before a sweep. */
+/* ------------------------------------------------------------------------- */
+int ldaref_set_shard(ldaref_ctx *c, int64_t first_token)
+{
+    if (!c || first_token < 0 || first_token >= ((int64_t)1 << 32)) return LDAREF_EINVAL;
+    c->tok_base = (uint32_t)first_token;
+    return LDAREF_OK;
+}
+
+int ldaref_word_counts_to_dense(const ldaref_ctx *c, int32_t *out)
+{
+    if (!c || !out) return LDAREF_EINVAL;
+    if (!c->inited) return LDAREF_ESTATE;
+    memset(out, 0, sizeof(int32_t) * (size_t)c->V * (size_t)c->K);
+    for (int32_t w = 0; w < c->V; ++w)
+        for (int64_t p = c->row_off[w]; p < c->row_off[w + 1]; ++p)
+            out[(size_t)w * c->K + c->row_topic[p]] = c->row_count[p];
+    return LDAREF_OK;
+}
+
+int ldaref_word_counts_from_dense(ldaref_ctx *c, const int32_t *in)
+{
+    if (!c || !in) return LDAREF_EINVAL;
+    if (!c->inited) return LDAREF_ESTATE;
+    int64_t nnz = 0;
+    for (size_t q = 0; q < (size_t)c->V * (size_t)c->K; ++q) {
+        if (in[q] < 0) return LDAREF_ERANGE;
+        nnz += in[q] > 0;
+    }
+    if (nnz > c->row_cap) {
+        size_t n = (size_t)nnz;
+        int32_t *a = (int32_t *)realloc(c->row_topic, sizeof(int32_t) * n);
+        if (a) c->row_topic = a;
+        int32_t *b = (int32_t *)realloc(c->row_count, sizeof(int32_t) * n);
+        if (b) c->row_count = b;
+        uint32_t *t = (uint32_t *)realloc(c->sp_thr32, sizeof(uint32_t) * n);
+        if (t) c->sp_thr32 = t;
+        int32_t *l = (int32_t *)realloc(c->sp_alias, sizeof(int32_t) * n);
+        if (l) c->sp_alias = l;
+        if (!a || !b || !t || !l) return LDAREF_ENOMEM;
+        c->row_cap = nnz;
+    }
+    memset(c->nk, 0, sizeof(int64_t) * (size_t)c->K);
+    nnz = 0;
+    for (int32_t w = 0; w < c->V; ++w) {
+        c->row_off[w] = nnz;
+        for (int32_t k = 0; k < c->K; ++k) {
+            int32_t n = in[(size_t)w * c->K + k];
+            if (n > 0) {
+                c->row_topic[nnz] = k;
+                c->row_count[nnz] = n;
+                c->nk[k] += n;          /* n_k = sum_w n_kw (Section 3) */
+                ++nnz;
+            }
+        }
+    }
+    c->row_off[c->V] = nnz;
+    c->tables_valid = 0;
+    return LDAREF_OK;
 }
 
 /* Compensated sum (Neumaier's form of Kahan summation): `sum` plus the rounding errors collected in `err`. */

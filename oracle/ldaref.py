@@ -85,6 +85,9 @@ def lib():
             L.ldaref_gibbs_sweep_sequential.argtypes = [vp, C.c_int32]
             L.ldaref_gibbs_masses.argtypes = [vp, C.c_int64, _p(np.uint64), _p(np.uint64), C.c_uint32,
                                               C.POINTER(C.c_int32)]
+            L.ldaref_set_shard.argtypes = [vp, C.c_int64]
+            L.ldaref_word_counts_to_dense.argtypes = [vp, _p(np.int32)]
+            L.ldaref_word_counts_from_dense.argtypes = [vp, _p(np.int32)]
             L.ldaref_get_moves.argtypes = [vp, _p(np.int64)]
             L.ldaref_sweeps_done.argtypes = [vp]
             L.ldaref_sweeps_done.restype = C.c_uint32
@@ -265,6 +268,19 @@ class Oracle:
         k = C.c_int32()
         _check(lib().ldaref_gibbs_masses(self._h, token, dm, pm, r0, C.byref(k)), "gibbs_masses")
         return dm, pm, k.value
+
+    def set_shard(self, first_token: int, global_term_freq=None):
+        """This context holds a run of documents of a larger corpus that starts at token first_token
+        (the term frequencies are accepted for symmetry with the library and not needed here)."""
+        _check(lib().ldaref_set_shard(self._h, first_token), "set_shard")
+
+    def word_counts_to_dense(self, matrix: np.ndarray):
+        assert matrix.dtype == np.int32 and matrix.size == self.V * self.K and matrix.flags.c_contiguous
+        _check(lib().ldaref_word_counts_to_dense(self._h, matrix.reshape(-1)), "word_counts_to_dense")
+
+    def word_counts_from_dense(self, matrix: np.ndarray):
+        assert matrix.dtype == np.int32 and matrix.size == self.V * self.K and matrix.flags.c_contiguous
+        _check(lib().ldaref_word_counts_from_dense(self._h, matrix.reshape(-1)), "word_counts_from_dense")
 
     def moves(self):
         """(word-proposal steps, doc-proposal steps) of the last sweep call that moved a chain."""

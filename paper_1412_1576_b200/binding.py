@@ -21,7 +21,7 @@ LDA_NK, LDA_NWK, LDA_NDK = 0, 1, 2
 
 EXPORTS = [
     "lda_create", "lda_set_stream", "lda_set_option", "lda_set_proposals", "lda_load_corpus", "lda_load_corpus_device",
-    "lda_init", "lda_set_assignments", "lda_set_assignments_u16", "lda_sweep", "lda_gibbs_sweep", "lda_loglik", "lda_get_counts",
+    "lda_set_shard", "lda_word_counts_to_dense", "lda_word_counts_from_dense", "lda_init", "lda_set_assignments", "lda_set_assignments_u16", "lda_sweep", "lda_gibbs_sweep", "lda_loglik", "lda_get_counts",
     "lda_get_assignments", "lda_get_assignments_u16", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
     "lda_dense_table_noalloc",
 ]
@@ -80,6 +80,9 @@ def load_library(path: str | None = None):
     L.lda_set_assignments_u16.argtypes = [vp, vp, u64, u32]
     L.lda_sweep.argtypes = [vp, i32, i32]
     L.lda_gibbs_sweep.argtypes = [vp, i32]
+    L.lda_set_shard.argtypes = [vp, i64, vp]
+    L.lda_word_counts_to_dense.argtypes = [vp, vp]
+    L.lda_word_counts_from_dense.argtypes = [vp, vp]
     L.lda_loglik.argtypes = [vp, C.POINTER(dbl), C.POINTER(dbl), C.POINTER(dbl)]
     L.lda_get_counts.argtypes = [vp, C.c_int, vp, vp, vp, i64, C.POINTER(i64)]
     L.lda_get_assignments.argtypes = [vp, vp]
@@ -159,6 +162,19 @@ def lda_set_assignments_u16_ptr(h, z_host_ptr, seed, sweep=0):
 
 def lda_sweep(h, iters, mh_steps):
     return load_library().lda_sweep(h, iters, mh_steps)
+
+
+def lda_set_shard(h, first_token, global_term_freq=None):
+    tf = None if global_term_freq is None else np.ascontiguousarray(global_term_freq, np.int32)
+    return load_library().lda_set_shard(h, int(first_token), None if tf is None else tf.ctypes.data)
+
+
+def lda_word_counts_to_dense(h, nwk_dev_ptr):
+    return load_library().lda_word_counts_to_dense(h, C.c_void_p(nwk_dev_ptr))
+
+
+def lda_word_counts_from_dense(h, nwk_dev_ptr):
+    return load_library().lda_word_counts_from_dense(h, C.c_void_p(nwk_dev_ptr))
 
 
 def lda_gibbs_sweep(h, iters):
@@ -298,6 +314,16 @@ class LightLDA:
 
     def sweep(self, iters: int, mh_steps: int):
         self._ck(lda_sweep(self._h, iters, mh_steps), "lda_sweep")
+
+    def set_shard(self, first_token: int, global_term_freq=None):
+        self._ck(lda_set_shard(self._h, first_token, global_term_freq), "lda_set_shard")
+
+    def word_counts_to_dense(self, matrix):
+        """matrix: CUDA int32 tensor of V*K elements (torch), filled with this context's n_kw."""
+        self._ck(lda_word_counts_to_dense(self._h, matrix.data_ptr()), "lda_word_counts_to_dense")
+
+    def word_counts_from_dense(self, matrix):
+        self._ck(lda_word_counts_from_dense(self._h, matrix.data_ptr()), "lda_word_counts_from_dense")
 
     def gibbs_sweep(self, iters: int):
         """Frozen exact-conditional sweeps (yardstick for the MH sweep)."""

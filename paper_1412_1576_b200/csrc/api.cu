@@ -215,6 +215,7 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     }
     v.topic_bits = tb;
     v.count_bits = cb;
+    v.tok_base = (uint32_t)c.shard_first_token;
 
     int rc = build_layout(c, words_dev, doc_off);
     if (rc != LDA_OK) { free_corpus(c); return fail(&c, rc, "building the word-sorted layout failed"); }
@@ -230,8 +231,14 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     }
 
     // --- dense / sparse class of every word (Section 5) ---------------------------------
-    std::vector<int32_t> tf((size_t)V);
-    for (int32_t w = 0; w < V; ++w) tf[w] = word_off[w + 1] - word_off[w];
+    // tf_here: the word's tokens in this corpus (its token range); tf: what the word's row and class
+    // are sized for -- the same, unless the corpus is one shard of a larger one (lda_set_shard), in
+    // which case the row has to hold the counts of all shards
+    std::vector<int32_t> tf_here((size_t)V), tf((size_t)V);
+    for (int32_t w = 0; w < V; ++w) {
+        tf_here[w] = word_off[w + 1] - word_off[w];
+        tf[w] = c.shard_global_tf.empty() ? tf_here[w] : std::max(tf_here[w], c.shard_global_tf[(size_t)w]);
+    }
     int32_t tf_cut = INT32_MAX;
     const int64_t n_top = (int64_t)std::floor(c.dense_frac * (double)V);
     if (n_top > 0) {
@@ -259,11 +266,11 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         } else if (tf[w] > SORT_TILE || (tf[w] > 0 && tf[w] >= tf_cut)) {
             dense_slot[w] = (int32_t)dense_words.size();
             dense_words.push_back(w);
-            for (int32_t o = 0; o < tf[w]; o += HIST_CHUNK) {
+            for (int32_t o = 0; o < tf_here[w]; o += HIST_CHUNK) {
                 hist_chunks.push_back(w);
                 hist_chunks.push_back(word_off[w] + o);
-                hist_chunks.push_back(std::min(HIST_CHUNK, tf[w] - o));
-                hist_chunks.push_back(tf[w] <= HIST_CHUNK ? 1 : 0);
+                hist_chunks.push_back(std::min(HIST_CHUNK, tf_here[w] - o));
+                hist_chunks.push_back(tf_here[w] <= HIST_CHUNK ? 1 : 0);
             }
         }
     }
@@ -294,15 +301,15 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
             if (tf[w] > COLD_TILE) {
                 close(w); s0 = w + 1; tok = 0;
                 std::vector<int32_t>& runs = dense_slot[w] >= 0 ? hot_tiles : hot_tiles_warm;
-                for (int32_t o = 0; o < tf[w]; o += HOT_TILE) {
+                for (int32_t o = 0; o < tf_here[w]; o += HOT_TILE) {
                     runs.push_back(w);
                     runs.push_back(word_off[w] + o);
-                    runs.push_back(std::min(HOT_TILE, tf[w] - o));
+                    runs.push_back(std::min(HOT_TILE, tf_here[w] - o));
                 }
-                for (int32_t o = 0; o < tf[w]; o += HOT_TILE_PROPOSE) {
+                for (int32_t o = 0; o < tf_here[w]; o += HOT_TILE_PROPOSE) {
                     hot_tiles_propose.push_back(w);
                     hot_tiles_propose.push_back(word_off[w] + o);
-                    hot_tiles_propose.push_back(std::min(HOT_TILE_PROPOSE, tf[w] - o));
+                    hot_tiles_propose.push_back(std::min(HOT_TILE_PROPOSE, tf_here[w] - o));
                 }
                 continue;
             }
@@ -751,6 +758,56 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
         s.doc_proposed = (int64_t)iters * c.N * (mh_steps - n_word);
         s.word_accepted = (int64_t)moves[0];
         s.doc_accepted = (int64_t)moves[1];
+    }
+    return LDA_OK;
+}
+
+int lda_set_shard(lda_ctx* h, int64_t first_token, const int32_t* global_term_freq)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (c.loaded) return fail(&c, LDA_ESTATE, "lda_set_shard must come before lda_load_corpus");
+    if (first_token < 0 || first_token >= 4294967296ll) return fail(&c, LDA_ERANGE, "first_token must be in [0, 2^32)");
+    c.shard_first_token = first_token;
+    c.shard_global_tf.clear();
+    if (global_term_freq) {
+        for (int32_t w = 0; w < c.V; ++w)
+            if (global_term_freq[w] < 0) return fail(&c, LDA_ERANGE, "negative term frequency");
+        c.shard_global_tf.assign(global_term_freq, global_term_freq + c.V);
+    }
+    return LDA_OK;
+}
+
+int lda_word_counts_to_dense(lda_ctx* h, int32_t* nwk_dev)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!nwk_dev) return fail(&c, LDA_EINVAL, "null matrix");
+    if (!c.inited) return fail(&c, LDA_ESTATE, "lda_word_counts_to_dense before lda_init");
+    int rc = check_device(c);
+    if (rc) return rc;
+    launch_word_counts_to_dense(c, nwk_dev);
+    if (cudaStreamSynchronize(c.stream) != cudaSuccess || cudaGetLastError() != cudaSuccess)
+        return cuda_fail(&c, "writing the count matrix");
+    return LDA_OK;
+}
+
+int lda_word_counts_from_dense(lda_ctx* h, const int32_t* nwk_dev)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (!nwk_dev) return fail(&c, LDA_EINVAL, "null matrix");
+    if (!c.inited) return fail(&c, LDA_ESTATE, "lda_word_counts_from_dense before lda_init");
+    int rc = check_device(c);
+    if (rc) return rc;
+    launch_word_counts_from_dense(c, nwk_dev);
+    c.tables_valid = false;
+    int bits = 0;
+    if ((rc = read_err(c, &bits))) { c.inited = false; return rc; }
+    if (bits) {
+        c.inited = false;
+        return fail(&c, LDA_ERANGE,
+                    "the matrix has negative entries or more nonzeros in a row than the term frequencies given to lda_set_shard allow");
     }
     return LDA_OK;
 }

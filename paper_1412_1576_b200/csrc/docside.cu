@@ -77,7 +77,7 @@ __device__ __forceinline__ void doc_side_token(const View& v, const uint32_t* ta
     };
     // doc-proposal of step st, the di-th of its kind
     auto doc_step = [&](int32_t st, int32_t di) {
-        const uint4 r = philox4x32_10(make_uint4(tok, sweep, (uint32_t)st, 0u), key);
+        const uint4 r = philox4x32_10(make_uint4(v.tok_base + tok, sweep, (uint32_t)st, 0u), key);
         const double uu = __dmul_rn((double)r.x, INV_2_32);
         uint32_t o2;
         if (__dmul_rn(uu, __dadd_rn(n_d, v.Kalpha)) < n_d) {

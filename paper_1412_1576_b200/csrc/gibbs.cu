@@ -116,7 +116,7 @@ k_gibbs_tokens(View v, const T* __restrict__ z, const int32_t* __restrict__ word
                                     (long long)gibbs_prior_term(v.alpha, v.beta, v.Vbeta, n_zw, n_z);
             const ull sum_prior = (ull)((long long)pre[K - 1] + delta);
             const ull total = sum_doc + sum_prior;
-            const uint4 r = philox4x32_10(make_uint4((uint32_t)i, sweep, 0u, 2u), key);
+            const uint4 r = philox4x32_10(make_uint4(v.tok_base + (uint32_t)i, sweep, 0u, 2u), key);
             ull x = __umul64hi(total, (ull)r.x << 32);  // floor(total * r.x / 2^32)
             uint32_t pick = (uint32_t)(K - 1);
             if (x < sum_doc) {

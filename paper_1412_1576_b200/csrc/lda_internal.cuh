@@ -102,6 +102,7 @@ constexpr int ALIAS_SMEM_ITEMS_BIG = 4096;   // ... and a 512-thread CTA
 struct View {
     int32_t V, K, N, D;
     double alpha, beta, Vbeta, Kalpha;
+    uint32_t tok_base;  // Philox token key of the corpus' first token (0 unless the corpus is a shard)
     int topic_bits;  // bits of K-1
     int count_bits;  // low bits of a packed n_kd entry that hold the count
     // tokens in word-sorted order (position p)
@@ -163,6 +164,8 @@ struct Ctx {
     int side_steps = 0;    // number of steps the exchange buffers are allocated for
     int side_mode = 0;     // ... and the proposal schedule they are laid out for
     int proposals = 0;     // LDA_PROPOSALS_*: which proposal each step of a chain draws
+    int64_t shard_first_token = 0;        // lda_set_shard(): global index of this corpus' first token
+    std::vector<int32_t> shard_global_tf;  // ... and the term frequencies over all shards (empty: this corpus alone)
     double dense_frac = 0.05;
     double dense_min_tf = 64;
     bool loaded = false, inited = false, tables_valid = false;
@@ -258,6 +261,11 @@ struct DkCsr {
 };
 int build_dk_csr(Ctx& c, DkCsr& r, bool sizes_only);  // LDA_* status; queued on c.stream, rows complete after a sync
 void free_dk_csr(DkCsr& r);
+
+// n_kw as a dense V x K matrix in device memory and back (shard.cu): the exchange format of the
+// document-sharded mode.  Return the number of kernels launched.
+int launch_word_counts_to_dense(Ctx& c, int32_t* nwk_dev);
+int launch_word_counts_from_dense(Ctx& c, const int32_t* nwk_dev);
 
 // Exact-conditional yardstick (gibbs.cu): `iters` frozen sweeps drawing from Eq. 1.  LDA_* status.
 constexpr int GIBBS_MAX_K = 16384;              // a word's dense n_kw row is staged in shared memory

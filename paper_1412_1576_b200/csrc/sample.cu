@@ -278,7 +278,7 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
             for (int u = 0; u < U; ++u) {
                 const int32_t p = p0 + u * nthreads;
                 const bool live = p < p_end;
-                tok[u] = live ? __ldcs(v.tok_orig + p) : 0u;
+                tok[u] = live ? v.tok_base + __ldcs(v.tok_orig + p) : 0u;
                 at[u] = live ? __ldcs(v.inv + p) : 0u;
             }
 #pragma unroll
@@ -302,7 +302,7 @@ __device__ __forceinline__ void propose_tokens(const View& v, const Tile& tile, 
         }
     } else {
         for (int32_t p = p_begin + (int32_t)threadIdx.x; p < p_end; p += nthreads) {
-            const uint32_t tok = __ldcs(v.tok_orig + p);
+            const uint32_t tok = v.tok_base + __ldcs(v.tok_orig + p);
             const uint32_t at = __ldcs(v.inv + p);  // the document-side pass reads block-major
             const typename Tile::Ref w = tile.ref(p - p_begin);
             for (int32_t m = 0; m < mh_steps; m += (MODE == LDA_PROPOSALS_CYCLE ? 2 : 1)) {
@@ -605,7 +605,7 @@ __global__ void k_init(View v, uint2 key)
     T* zbm = reinterpret_cast<T*>(v.zbm);
     for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < v.N;
          p += (int64_t)gridDim.x * blockDim.x) {
-        const uint32_t tok = v.tok_orig[p];
+        const uint32_t tok = v.tok_base + v.tok_orig[p];
         const uint4 r = philox4x32_10(make_uint4(tok, 0u, 0u, 1u), key);
         const T z = (T)scale_to_range(r.x, (uint32_t)v.K);
         zw[p] = z;
