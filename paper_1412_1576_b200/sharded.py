@@ -11,7 +11,7 @@ assignments of one context holding all the documents, whatever the number of sha
 
 This module is orchestration only (which call follows which, and the collective); every step of
 the sweep runs in the library's kernels.  The `engine` is a context object with the library's
-method names (``binding.LightLDA``); the tests also drive the CPU oracle through it.
+method names (``binding.LightLDA``); any object with the same methods can stand in for it.
 """
 
 from __future__ import annotations
@@ -50,7 +50,8 @@ class ShardedSweep:
 
     engine      context with set_shard / load_corpus / init / sweep / word_counts_to_dense /
                 word_counts_from_dense / loglik
-    matrix      the exchange buffer: V*K int32 (CUDA tensor for the library, numpy array for the oracle)
+    matrix      the exchange buffer: V*K int32 (a CUDA tensor for the library; whatever the engine's
+                word_counts_to_dense / _from_dense take)
     all_reduce  callable(matrix): sums the buffer over all shards in place
     """
 
