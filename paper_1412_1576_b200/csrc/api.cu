@@ -12,6 +12,7 @@ void set_sample_smem_limits();
 void set_doc_smem_limits();
 void set_alias_smem_limits();
 void set_export_smem_limits();
+void set_loglik_smem_limits();
 
 void* dev_alloc(Ctx& c, size_t bytes)
 {
@@ -108,7 +109,7 @@ static void free_corpus(Ctx& c)
     nv.err = err;
     nv.moves = c.v.moves;
     c.v = nv;
-    c.loaded = c.inited = c.tables_valid = c.dk_valid = false;
+    c.loaded = c.inited = c.tables_valid = false;
     c.N = c.D = 0;
     c.side_steps = 0;
 }
@@ -161,20 +162,6 @@ static int rebuild_counts(Ctx& c, int64_t* launches)
     n += launch_count_k(c);
     if (launches) *launches += n;
     c.tables_valid = false;
-    c.dk_valid = false;
-    return LDA_OK;
-}
-
-// The n_kd tables in device memory (the exported form; the MH step builds its own per tile).
-static int ensure_dk(Ctx& c)
-{
-    if (c.dk_valid) return LDA_OK;
-    launch_count_dk(c);
-    int bits = 0;
-    int rc = read_err(c, &bits);
-    if (rc) return rc;
-    if (bits) return fail(&c, LDA_EINTERNAL, "the n_kd rebuild raised the device error word");
-    c.dk_valid = true;
     return LDA_OK;
 }
 
@@ -416,12 +403,18 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     v.dn_idx = (uint32_t*)A((size_t)K * 4);
     v.dense_mass = (unsigned long long*)A(8);
     v.nk = (int32_t*)A((size_t)v.dense_stride * 4);  // padded like a dense row: copied in 16-byte units
-    v.dk_slots = (uint32_t*)A(n1 * 16 + 32);  // four slots per token, + one group past the end
+    // scratch tables of the documents longer than a tile: four slots per token, one document after the other
+    std::vector<long long> long_slot_off(long_docs.size() + 1, 0);
+    for (size_t i = 0; i < long_docs.size(); ++i)
+        long_slot_off[i + 1] = long_slot_off[i] + 4ll * (doc_off[long_docs[i] + 1] - doc_off[long_docs[i]]);
+    v.dk_slots = (uint32_t*)A((size_t)long_slot_off.back() * 4 + 32);
+    v.long_slot_off = upload(c, long_slot_off);
+    ok = ok && v.long_slot_off;
     c.sc_w = (unsigned long long*)A(cap1 * 8);
     c.sc_de = (unsigned long long*)A(cap1 * 8);
     c.sc_item = (uint32_t*)A(cap1 * 4);
     c.sc_dense = (unsigned long long*)A((size_t)K * 8 * 3);
-    c.red = (double*)A(sizeof(double) * 2 * 592);
+    c.red = (double*)A(sizeof(double) * (LL_WORD_PARTIALS + LL_DOC_PARTIALS));
     c.red_i = (int64_t*)A(16);
     if (!ok) { free_corpus(c); return fail(&c, LDA_ENOMEM, "device allocation failed"); }
     cudaMemsetAsync(v.wk_nnz, 0, (size_t)V * 4, c.stream);
@@ -432,6 +425,8 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.stats.n_tokens = N;
     c.stats.n_docs = D;
     c.stats.n_dense_words = c.n_dense;
+    c.n_nonempty_docs = 0;
+    for (int64_t d = 0; d < n_docs; ++d) c.n_nonempty_docs += doc_off[d + 1] > doc_off[d];
     c.loaded = true;
     return LDA_OK;
 }
@@ -469,6 +464,10 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
     if (!h) return LDA_ENOMEM;
     Ctx& c = h->c;
     c.V = V; c.K = K; c.alpha = alpha; c.beta = beta; c.device = dev;
+    if (cudaDeviceGetAttribute(&c.n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || c.n_sm < 1) {
+        cudaGetLastError();
+        c.n_sm = 148;
+    }
     c.wide_topics = K > 65536;
     c.v.V = V; c.v.K = K; c.v.alpha = alpha; c.v.beta = beta;
     c.v.Vbeta = (double)V * beta;
@@ -507,6 +506,7 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
     set_doc_smem_limits();
     set_alias_smem_limits();
     set_export_smem_limits();
+    set_loglik_smem_limits();
     set_gibbs_smem_limits();
     *out = h;
     return LDA_OK;
@@ -651,7 +651,6 @@ static int set_assignments(lda_ctx* h, const void* z, bool narrow, uint64_t seed
     // the record array (one word per token, only meaningful while the exported n_kd is valid)
     // doubles as the staging buffer: no allocation here
     void* zdev = c.v.rec;
-    c.dk_valid = false;
     if (c.N > 0 &&
         cudaMemcpyAsync(zdev, z, (size_t)c.N * (narrow ? 2 : 4), cudaMemcpyHostToDevice, c.stream) != cudaSuccess)
         return cuda_fail(&c, "copying assignments");
@@ -716,7 +715,6 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
             cudaEventRecord(c.ev[5], c.stream);
             cudaEventRecord(c.ev[6], c.stream);  // n_kd is rebuilt inside the next MH step, per tile
             c.tables_valid = false;
-            c.dk_valid = false;
             c.sweep += 1;
             s.kernel_launches += n;
         }
@@ -843,9 +841,11 @@ int lda_loglik(lda_ctx* h, double* total, double* word_ll, double* doc_ll)
     if (!c.inited) return fail(&c, LDA_ESTATE, "lda_loglik before lda_init");
     int rc = check_device(c);
     if (rc) return rc;
-    if ((rc = ensure_dk(c))) return rc;
     double out[3];
     if (launch_loglik(c, out) < 0) return cuda_fail(&c, "log-likelihood");
+    int bits = 0;
+    if ((rc = read_err(c, &bits))) return rc;
+    if (bits) return fail(&c, LDA_EINTERNAL, "the log-likelihood kernels raised the device error word");
     if (total) *total = out[0];
     if (word_ll) *word_ll = out[1];
     if (doc_ll) *doc_ll = out[2];
@@ -933,7 +933,6 @@ static int get_assignments(lda_ctx* h, void* z_out, bool narrow)
     int rc = check_device(c);
     if (rc) return rc;
     void* zdev = c.v.rec;  // staging, see set_assignments()
-    c.dk_valid = false;
     launch_export_assignments(c, zdev, narrow);
     cudaError_t e =
         cudaMemcpyAsync(z_out, zdev, (size_t)c.N * (narrow ? 2 : 4), cudaMemcpyDeviceToHost, c.stream);
@@ -989,7 +988,6 @@ int lda_get_stats(lda_ctx* h, lda_stats* out)
     Ctx& c = h->c;
     if (c.inited) {
         if (check_device(c)) return LDA_ECUDA;
-        if (ensure_dk(c)) return LDA_ECUDA;
         int64_t a = 0, b = 0;
         launch_count_nnz(c, &a, &b);
         c.stats.nnz_wk = a;

@@ -10,9 +10,8 @@
 //     the word's dense row, then compacted into the sorted row.
 // n_k: column sums of the rows just written.
 // n_kd (segments = documents): the MH step builds every document's table itself, per tile, in
-// shared memory (docside.cu); the kernels here write the same tables to device memory -- plus one
-// record (topic, its n_kd) per token -- when a caller asks for them (lda_get_counts, lda_loglik,
-// lda_get_stats).
+// shared memory (docside.cu), and so does the log-likelihood (loglik.cu); lda_get_counts gets
+// sorted rows from export.cu.
 // No per-token global atomics: a CTA touches global counters once per bin it
 // actually filled (documents longer than a tile are the one exception).
 #include <algorithm>
@@ -361,83 +360,6 @@ k_compact_dense(const int32_t* __restrict__ dense_words, const int32_t* __restri
     if (threadIdx.x == 0) wk_nnz[w] = done;
 }
 
-// n_kd as per-document open-addressing tables in device memory, for export (layout and probe
-// order: dk_insert in lda_device.cuh).  One CTA per tile of whole documents (`cap` tokens at
-// most): the tile's tables are built in shared memory by insertion and written out in one
-// coalesced pass, together with every token's record (topic, n_kd of its topic in its document).
-//
-template <typename T>
-__global__ void __launch_bounds__(1024)
-k_doc_hash(const int32_t* __restrict__ tiles, int32_t cap, const int32_t* __restrict__ doc_off,
-           const T* __restrict__ zbm, const uint32_t* __restrict__ bm_of_tok, uint32_t* __restrict__ rec,
-           uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
-{
-    extern __shared__ __align__(16) uint32_t doc_smem[];  // carved up for tiles of `cap` tokens
-    uint32_t* slots = doc_smem;
-    int32_t* soff = reinterpret_cast<int32_t*>(slots + DK_SLOTS_PER_TOKEN * cap);
-    uint32_t* topic = reinterpret_cast<uint32_t*>(soff + cap + 1);
-    const int tid = threadIdx.x;
-    const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
-    const int32_t nseg = s1 - s0;
-    const int32_t base = doc_off[s0];
-    const int32_t cnt = doc_off[s1] - base;
-    if (cnt == 0) return;
-    // the tile's documents lie in one or two blocks of the block-major order: these reads hit L2
-    for (int j = tid; j < cnt; j += blockDim.x) topic[j] = (uint32_t)__ldcg(zbm + 2 * (size_t)__ldcs(bm_of_tok + base + j));
-    for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = doc_off[s0 + j] - base;
-    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
-    __syncthreads();
-    // one warp per document: its lanes insert the document's tokens and note where each topic landed
-    const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-    for (int d = warp; d < nseg; d += nwarps) {
-        const int32_t first = soff[d], len = soff[d + 1] - first;
-        if (len == 0) continue;
-        for (int j = first + lane; j < first + len; j += 32) {
-            const uint32_t k = topic[j];
-            uint32_t slot = 0xFFFFFFFFu;
-            if (k < (uint32_t)K)
-                slot = dk_insert(slots + DK_SLOTS_PER_TOKEN * first, DK_SLOTS_PER_TOKEN * (uint32_t)len, k, count_bits);
-            if (slot == 0xFFFFFFFFu) atomicOr(err, k < (uint32_t)K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
-            else slot += DK_SLOTS_PER_TOKEN * (uint32_t)first;
-            topic[j] = slot;
-        }
-    }
-    __syncthreads();
-    uint32_t* out = slots_out + DK_SLOTS_PER_TOKEN * (size_t)base;
-    for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) out[j] = slots[j];
-    for (int j = tid; j < cnt; j += blockDim.x) {
-        const uint32_t slot = topic[j];
-        if (slot != 0xFFFFFFFFu) rec[base + j] = slots[slot];
-    }
-}
-
-// Documents longer than a tile: one CTA per document, the same insertion straight in global memory.
-template <typename T>
-__global__ void __launch_bounds__(512)
-k_long_doc_hash(const int32_t* __restrict__ long_docs, const int32_t* __restrict__ doc_off,
-                const T* __restrict__ zbm, const uint32_t* __restrict__ bm_of_tok, uint32_t* __restrict__ rec,
-                uint32_t* __restrict__ slots_out, int count_bits, int32_t K, int* err)
-{
-    const int32_t d = long_docs[blockIdx.x];
-    const int32_t first = doc_off[d], cnt = doc_off[d + 1] - first;
-    const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)cnt;
-    uint32_t* tab = slots_out + DK_SLOTS_PER_TOKEN * (size_t)first;
-    for (uint32_t j = threadIdx.x; j < cap; j += blockDim.x) tab[j] = DK_EMPTY;
-    __syncthreads();
-    for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-        const uint32_t k = (uint32_t)zbm[2 * (size_t)bm_of_tok[first + j]];
-        uint32_t at = 0xFFFFFFFFu;
-        if (k < (uint32_t)K) at = dk_insert(tab, cap, k, count_bits);
-        if (at == 0xFFFFFFFFu) atomicOr(err, k < (uint32_t)K ? ERR_ROW_OVERFLOW : ERR_TOPIC_RANGE);
-        rec[first + j] = at;  // parked here until every insertion is done
-    }
-    __syncthreads();
-    for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-        const uint32_t at = rec[first + j];
-        if (at != 0xFFFFFFFFu) rec[first + j] = tab[at];
-    }
-}
-
 // n_k = sum over words of n_kw (Section 3), taken from the rows the n_kw rebuild has just written
 // instead of from another pass over the assignments:
 //   - dense rows: column sums, one thread per topic and group of rows;
@@ -508,28 +430,6 @@ k_nk_from_sparse_direct(const int32_t* __restrict__ row_start, const int32_t* __
         const int32_t r0 = row_start[w], n = wk_nnz[w];
         for (int32_t j = lane; j < n; j += 32) atomicAdd(&nk[__ldcs(wk_topic + r0 + j)], (int32_t)__ldcs(wk_count + r0 + j));
     }
-}
-
-__global__ void k_sum_i32(const int32_t* __restrict__ a, int64_t n, unsigned long long* out)
-{
-    __shared__ unsigned long long tmp[32];
-    unsigned long long s = 0;
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
-         i += (int64_t)gridDim.x * blockDim.x)
-        s += (unsigned long long)a[i];
-    s = block_reduce_sum<unsigned long long>(s, tmp);
-    if (threadIdx.x == 0 && s) atomicAdd(out, s);
-}
-
-__global__ void k_count_filled(const uint32_t* __restrict__ slots, int64_t n, unsigned long long* out)
-{
-    __shared__ unsigned long long tmp[32];
-    unsigned long long s = 0;
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
-         i += (int64_t)gridDim.x * blockDim.x)
-        s += slots[i] != DK_EMPTY;
-    s = block_reduce_sum<unsigned long long>(s, tmp);
-    if (threadIdx.x == 0 && s) atomicAdd(out, s);
 }
 
 struct EmitRowSizes {
@@ -640,48 +540,11 @@ static int count_k(Ctx& c)
     return launches;
 }
 
-template <typename T>
-static int count_dk_t(Ctx& c)
-{
-    View& v = c.v;
-    int launches = 0;
-    const T* zbm = (const T*)v.zbm;
-    if (c.n_doc_tiles) {
-        k_doc_hash<T><<<c.n_doc_tiles, c.doc_threads, doc_tile_smem_bytes(c.doc_tile), c.stream>>>(
-            c.doc_tiles, c.doc_tile, v.doc_off, zbm, v.bm_of_tok, v.rec, v.dk_slots, v.count_bits, c.K, v.err);
-        ++launches;
-    }
-    if (c.n_long_docs) {
-        k_long_doc_hash<T><<<c.n_long_docs, 512, 0, c.stream>>>(c.long_docs, v.doc_off, zbm, v.bm_of_tok, v.rec, v.dk_slots,
-                                                               v.count_bits, c.K, v.err);
-        ++launches;
-    }
-    return launches;
-}
-
 int launch_count_wk(Ctx& c) { return c.wide_topics ? count_wk_t<int32_t>(c) : count_wk_t<uint16_t>(c); }
 int launch_count_k(Ctx& c) { return count_k(c); }
-int launch_count_dk(Ctx& c) { return c.wide_topics ? count_dk_t<int32_t>(c) : count_dk_t<uint16_t>(c); }
-
-int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host)
-{
-    unsigned long long* acc = (unsigned long long*)c.red_i;
-    cudaMemsetAsync(acc, 0, 16, c.stream);
-    k_sum_i32<<<296, 256, 0, c.stream>>>(c.v.wk_nnz, c.V, acc);
-    if (c.N) k_count_filled<<<592, 256, 0, c.stream>>>(c.v.dk_slots, (int64_t)DK_SLOTS_PER_TOKEN * c.N, acc + 1);
-    unsigned long long h[2] = {0, 0};
-    cudaMemcpyAsync(h, acc, 16, cudaMemcpyDeviceToHost, c.stream);
-    cudaStreamSynchronize(c.stream);
-    *nnz_wk_host = (int64_t)h[0];
-    *nnz_dk_host = (int64_t)h[1];
-    return 2;
-}
 
 void set_hist_smem_limits()
 {
-    const int doc_bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
-    cudaFuncSetAttribute(k_doc_hash<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
-    cudaFuncSetAttribute(k_doc_hash<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
     cudaFuncSetAttribute(k_warm_rows<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST16_BINS * 2 + 16);
     cudaFuncSetAttribute(k_warm_rows<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST16_BINS * 2 + 16);
     cudaFuncSetAttribute(k_hist_chunks<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST32_BINS * 4);

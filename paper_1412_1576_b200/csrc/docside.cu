@@ -191,8 +191,8 @@ k_doc_tile(View v, const int32_t* __restrict__ tiles, uint2 key, uint32_t sweep,
 }
 
 // Documents longer than a tile: one CTA per document; the table lives in the document's range of
-// the global slot array and the slot indices in its range of the record array (both are scratch
-// here: the exported n_kd tables are rebuilt on demand).
+// the scratch slots in device memory (long_slot_off: four slots per token of the long documents,
+// one after the other) and the slot indices in its range of the record array.
 template <typename T, int MODE, int FIXED>
 __global__ void __launch_bounds__(512)
 k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32_t sweep, int32_t mh_steps_arg)
@@ -202,7 +202,7 @@ k_long_doc_tile(View v, const int32_t* __restrict__ long_docs, uint2 key, uint32
     const int32_t first = v.doc_off[d], cnt = v.doc_off[d + 1] - first;
     const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)cnt;
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
-    uint32_t* tab = v.dk_slots + DK_SLOTS_PER_TOKEN * (size_t)first;
+    uint32_t* tab = v.dk_slots + v.long_slot_off[blockIdx.x];
     uint32_t* slot_of = v.rec + first;
     for (uint32_t j = threadIdx.x; j < cap; j += blockDim.x) tab[j] = DK_EMPTY;
     __syncthreads();

@@ -80,7 +80,6 @@ static int build_dk_csr_t(Ctx& c, DkCsr& r, bool sizes_only)
     cudaMemsetAsync(r.nnz, 0, ((size_t)D + 1) * 4, c.stream);
     // the assignments in document order, in the record array (scratch between calls)
     T* z = reinterpret_cast<T*>(v.rec);
-    c.dk_valid = false;
     launch_export_assignments(c, z, sizeof(T) == 2);
     const int win = c.K < HIST_BINS ? c.K : HIST_BINS;
     if (c.n_doc_sort_tiles)

@@ -174,8 +174,7 @@ int lda::gibbs_sweep(Ctx& c, int32_t iters)
         launch_count_wk(c);
         launch_count_k(c);
         c.tables_valid = false;
-        c.dk_valid = false;
-        c.sweep += 1;
+            c.sweep += 1;
         if (cudaStreamSynchronize(c.stream) != cudaSuccess) rc = LDA_ECUDA;
         free_dk_csr(r);
     }

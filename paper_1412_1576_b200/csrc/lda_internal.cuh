@@ -62,6 +62,9 @@ constexpr int DOC_TILE_MAX = DOC_TILE_ROUNDS * 1024;
 constexpr int DOC_TILE_SLOTS = LDA_DOC_TILE_SLOTS;  // slots per token of a tile's tables in shared memory
 static_assert(DOC_TILE_SLOTS % 4 == 0, "a tile's tables are cleared 16 bytes at a time");
 constexpr int DOC_TILE_SMEM_PER_TOKEN = 4 * DOC_TILE_SLOTS + 4 + 4;
+// partial sums of the log-likelihood kernels: word part; document part (tiles + long documents)
+constexpr int LL_WORD_PARTIALS = 592;
+constexpr int LL_DOC_PARTIALS = 148 * 16 + 592 + 1024;
 constexpr int HIST_BINS = 32768;     // shared-memory histogram window (32-bit bins)
 constexpr int WORD_ROWS_BITMAP_MAX_K = 16384;  // tail rows: topic bitmap up to this K, key sort above
 constexpr int HIST16_BINS = 106496;  // window of a warm word's n_kw histogram (16-bit bins, 208 KB)
@@ -122,8 +125,8 @@ struct View {
     void* zw;   // word-sorted order: read by the n_kw / n_k rebuild
     void* zbm;  // block-major order, two entries per token: its topic, read (through bm_of_tok) by everything
                 // that works per document, and beside it the first word-proposal of the running MH step
-    // Document order, valid after launch_count_dk() only (the exported form of n_kd):
-    // rec[i] = (z_i << count_bits) | n_kd[d][z_i].
+    // One word per token in document order: scratch (slot indices of long documents during the MH
+    // step, staging of assignments on their way in and out, z in document order for export.cu).
     uint32_t* rec;
     const int32_t* word_off;  // [V+1] token range of each word in word-sorted order
     const int32_t* doc_off;   // [D+1]
@@ -146,9 +149,11 @@ struct View {
     uint2* dn_pk;      // [K] (split point, alias) of the dense table in one word pair
     unsigned long long* dense_mass;
     int32_t* nk;  // [K]
-    // n_kd: document d owns the open-addressing table dk_slots[4*doc_off[d] .. 4*doc_off[d+1])
+    // n_kd of the documents longer than a tile (the others' tables only ever live in shared memory):
+    // the i-th long document owns the open-addressing table dk_slots[long_slot_off[i] .. long_slot_off[i+1])
     // (four slots per token, load <= 0.25); layout and probe order: dk_insert in lda_device.cuh.
     uint32_t* dk_slots;
+    const long long* long_slot_off;
     int* err;
     unsigned long long* moves;  // [2] steps of the running lda_sweep() that moved a chain: word-, doc-proposals
 };
@@ -157,6 +162,7 @@ struct Ctx {
     int32_t V = 0, K = 0;
     double alpha = 0, beta = 0;
     int device = 0;
+    int n_sm = 148;  // multiprocessors of the device
     cudaStream_t stream = nullptr;
     bool wide_topics = false;  // false: 16-bit topic storage, true: 32-bit
     int block_shift = 22;  // log2 of the tokens per block of the block-major order
@@ -169,7 +175,7 @@ struct Ctx {
     double dense_frac = 0.05;
     double dense_min_tf = 64;
     bool loaded = false, inited = false, tables_valid = false;
-    bool dk_valid = false;  // dk_slots / rec hold the n_kd tables of the current assignments
+    int64_t n_nonempty_docs = 0;
     uint64_t seed = 0;
     uint32_t sweep = 0;
     int64_t N = 0, D = 0;
@@ -240,7 +246,6 @@ int launch_spread_assignments(Ctx& c, const void* z_dev, bool narrow);  // z (do
 int launch_export_assignments(Ctx& c, void* z_dev, bool narrow);
 int launch_count_wk(Ctx& c);
 int launch_count_k(Ctx& c);
-int launch_count_dk(Ctx& c);
 int launch_alias_dense(Ctx& c);
 int launch_alias_sparse(Ctx& c);
 int launch_sample(Ctx& c, int mh_steps);   // all passes of the MH step; needs ensure_exchange()
