@@ -69,7 +69,10 @@ k_ll_doc_tiles(View v, const int32_t* __restrict__ tiles, int32_t n_tiles, int32
     uint32_t* slots = doc_smem;
     int32_t* soff = reinterpret_cast<int32_t*>(slots + DK_SLOTS_PER_TOKEN * cap);
     uint32_t* topic = reinterpret_cast<uint32_t*>(soff + cap + 1);
+    __shared__ double by_len[LL_TABLE];  // lgamma(n_d + K alpha) for documents shorter than LL_TABLE tokens
     fill_ll_table(small, v.alpha, lg_alpha);
+    for (int c = threadIdx.x; c < LL_TABLE; c += blockDim.x) by_len[c] = lgamma((double)c + v.Kalpha);
+    __syncthreads();
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
     const int tid = threadIdx.x;
     const uint32_t cmask = (1u << v.count_bits) - 1u;
@@ -96,7 +99,7 @@ k_ll_doc_tiles(View v, const int32_t* __restrict__ tiles, int32_t n_tiles, int32
                                    v.count_bits) == DK_EMPTY)
                     atomicOr(v.err, ERR_ROW_OVERFLOW);
             }
-            if (lane == 0 && len > 0) s -= lgamma((double)len + v.Kalpha);
+            if (lane == 0 && len > 0) s -= len < LL_TABLE ? by_len[len] : lgamma((double)len + v.Kalpha);
         }
         __syncthreads();
         for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) {
