@@ -26,6 +26,7 @@
 #ifndef LDA_B200_H
 #define LDA_B200_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -79,6 +80,19 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out);
 
 /* Run all later work of this context on `cuda_stream` (a cudaStream_t); NULL = default stream. */
 int lda_set_stream(lda_ctx* ctx, void* cuda_stream);
+
+/* Where the context's device memory comes from.  By default cudaMalloc / cudaFree; a caller that runs
+ * inside a framework with a memory pool of its own (PyTorch's caching allocator, say) hands the
+ * pool's routines in, and every later allocation of the context -- the corpus layout, the count and
+ * alias tables, the exchange buffers, transient buffers of lda_load_corpus / lda_get_counts /
+ * lda_gibbs_sweep -- goes through them.  alloc_fn returns DEVICE memory of at least `bytes` bytes,
+ * 256-byte aligned, usable on the context's stream, or NULL when it has none; free_fn takes such a
+ * pointer back (the library calls it only after the work that used the memory has finished on the
+ * context's stream).  Both or neither (NULL, NULL = back to cudaMalloc).  Must be called before
+ * lda_load_corpus (LDA_ESTATE afterwards); `user` is passed through. */
+typedef void* (*lda_alloc_fn)(size_t bytes, void* user);
+typedef void (*lda_free_fn)(void* ptr, void* user);
+int lda_set_allocator(lda_ctx* ctx, lda_alloc_fn alloc_fn, lda_free_fn free_fn, void* user);
 
 /* Tunables that never change results.  Must be set before lda_load_corpus().
  *   "dense_frac"   fraction of the vocabulary (by term frequency) whose n_kw rows are dense (Section 5)

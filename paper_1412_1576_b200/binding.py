@@ -20,7 +20,7 @@ LDA_OK, LDA_EINVAL, LDA_ERANGE, LDA_ESTATE, LDA_ENOMEM, LDA_ECUDA, LDA_EINTERNAL
 LDA_NK, LDA_NWK, LDA_NDK = 0, 1, 2
 
 EXPORTS = [
-    "lda_create", "lda_set_stream", "lda_set_option", "lda_set_proposals", "lda_load_corpus", "lda_load_corpus_device",
+    "lda_create", "lda_set_stream", "lda_set_allocator", "lda_set_option", "lda_set_proposals", "lda_load_corpus", "lda_load_corpus_device",
     "lda_set_shard", "lda_word_counts_to_dense", "lda_word_counts_from_dense", "lda_init", "lda_set_assignments", "lda_set_assignments_u16", "lda_sweep", "lda_gibbs_sweep", "lda_loglik", "lda_get_counts",
     "lda_get_assignments", "lda_get_assignments_u16", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
     "lda_dense_table_noalloc",
@@ -42,6 +42,11 @@ class lda_stats(C.Structure):
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+# lda_alloc_fn / lda_free_fn of the header
+ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
+FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
 
 
 class LdaError(RuntimeError):
@@ -71,6 +76,7 @@ def load_library(path: str | None = None):
     vp, i32, i64, u32, u64, dbl = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_double
     L.lda_create.argtypes = [i32, i32, dbl, dbl, C.POINTER(vp)]
     L.lda_set_stream.argtypes = [vp, vp]
+    L.lda_set_allocator.argtypes = [vp, ALLOC_FN, FREE_FN, vp]
     L.lda_set_option.argtypes = [vp, C.c_char_p, dbl]
     L.lda_set_proposals.argtypes = [vp, C.c_int]
     L.lda_load_corpus.argtypes = [vp, vp, i64, vp, i64]
@@ -112,6 +118,32 @@ def lda_create(V, K, alpha, beta):
 
 def lda_set_stream(h, cuda_stream):
     return load_library().lda_set_stream(h, C.c_void_p(cuda_stream))
+
+
+def lda_set_allocator(h, alloc_fn, free_fn):
+    """alloc_fn / free_fn: ALLOC_FN / FREE_FN objects (the caller keeps them alive), or None, None."""
+    return load_library().lda_set_allocator(h, alloc_fn or ALLOC_FN(0), free_fn or FREE_FN(0), None)
+
+
+def torch_caching_allocator(stream: int | None):
+    """(ALLOC_FN, FREE_FN) that take the context's device memory from PyTorch's caching allocator,
+    on the given stream (a raw cudaStream_t; None = the default stream)."""
+    import torch
+    device = torch.cuda.current_device()
+
+    def alloc(nbytes, _user):
+        try:
+            return torch.cuda.caching_allocator_alloc(int(nbytes), device, stream or 0)
+        except Exception:          # out of memory: the library reports LDA_ENOMEM
+            return None
+
+    def free(ptr, _user):
+        try:
+            if ptr:
+                torch.cuda.caching_allocator_delete(ptr)
+        except Exception:          # interpreter shutdown: the process's memory goes with it
+            pass
+    return ALLOC_FN(alloc), FREE_FN(free)
 
 
 def lda_set_option(h, key, value):
@@ -255,7 +287,9 @@ class LightLDA:
     """One sampler context on the current CUDA device."""
 
     def __init__(self, V: int, K: int, alpha: float, beta: float, stream: int | None = None,
-                 options: dict | None = None):
+                 options: dict | None = None, allocator: str = "torch"):
+        """allocator: "torch" takes the context's device memory from PyTorch's caching allocator (so it
+        shares one pool with the caller's tensors), "cuda" leaves the library on cudaMalloc."""
         self.V, self.K, self.alpha, self.beta = V, K, alpha, beta
         rc, self._h = lda_create(V, K, alpha, beta)
         if rc:
@@ -264,6 +298,12 @@ class LightLDA:
         self.N = self.D = 0
         if stream is not None:
             self._ck(lda_set_stream(self._h, stream), "lda_set_stream")
+        self._allocator = None
+        if allocator == "torch":
+            self._allocator = torch_caching_allocator(stream)    # kept alive as long as the context
+            self._ck(lda_set_allocator(self._h, *self._allocator), "lda_set_allocator")
+        elif allocator != "cuda":
+            raise ValueError("allocator must be 'torch' or 'cuda'")
         for k, val in (options or {}).items():
             self._ck(lda_set_option(self._h, k, val), f"lda_set_option({k})")
 

@@ -14,16 +14,32 @@ void set_alias_smem_limits();
 void set_export_smem_limits();
 void set_loglik_smem_limits();
 
-void* dev_alloc(Ctx& c, size_t bytes)
+void* raw_alloc(Ctx& c, size_t bytes)
 {
+    if (c.alloc_fn) return c.alloc_fn(bytes, c.alloc_user);
     void* p = nullptr;
-    if (bytes == 0) bytes = 16;
     if (cudaMalloc(&p, bytes) != cudaSuccess) {
         cudaGetLastError();
         return nullptr;
     }
+    return p;
+}
+
+void raw_free(Ctx& c, void* p)
+{
+    if (!p) return;
+    if (c.free_fn) c.free_fn(p, c.alloc_user);
+    else cudaFree(p);
+}
+
+void* dev_alloc(Ctx& c, size_t bytes)
+{
+    if (bytes == 0) bytes = 16;
+    void* p = raw_alloc(c, bytes);
+    if (!p) return nullptr;
     c.allocs.push_back(p);
     c.alloc_bytes.push_back(bytes);
+    c.alloc_own.push_back(c.alloc_fn ? 1 : 0);
     c.device_bytes += (int64_t)bytes;
     return p;
 }
@@ -34,18 +50,25 @@ void dev_free(Ctx& c, void* p)
     for (size_t i = 0; i < c.allocs.size(); ++i)
         if (c.allocs[i] == p) {
             c.device_bytes -= (int64_t)c.alloc_bytes[i];
+            const bool own = c.alloc_own[i] != 0;
             c.allocs.erase(c.allocs.begin() + i);
             c.alloc_bytes.erase(c.alloc_bytes.begin() + i);
-            break;
+            c.alloc_own.erase(c.alloc_own.begin() + i);
+            if (own && c.free_fn) c.free_fn(p, c.alloc_user);
+            else cudaFree(p);
+            return;
         }
-    cudaFree(p);
 }
 
 void dev_free_all(Ctx& c)
 {
-    for (void* p : c.allocs) cudaFree(p);
+    for (size_t i = 0; i < c.allocs.size(); ++i) {
+        if (c.alloc_own[i] && c.free_fn) c.free_fn(c.allocs[i], c.alloc_user);
+        else cudaFree(c.allocs[i]);
+    }
     c.allocs.clear();
     c.alloc_bytes.clear();
+    c.alloc_own.clear();
     c.device_bytes = 0;
 }
 
@@ -545,6 +568,17 @@ int lda_set_stream(lda_ctx* h, void* cuda_stream)
     return LDA_OK;
 }
 
+int lda_set_allocator(lda_ctx* h, lda_alloc_fn alloc_fn, lda_free_fn free_fn, void* user)
+{
+    if (!h || (alloc_fn == nullptr) != (free_fn == nullptr)) return LDA_EINVAL;
+    Ctx& c = h->c;
+    if (c.loaded) return fail(&c, LDA_ESTATE, "lda_set_allocator must come before lda_load_corpus");
+    c.alloc_fn = alloc_fn;
+    c.free_fn = free_fn;
+    c.alloc_user = user;
+    return LDA_OK;
+}
+
 int lda_set_option(lda_ctx* h, const char* key, double value)
 {
     if (!h || !key) return LDA_EINVAL;
@@ -589,18 +623,15 @@ int lda_load_corpus(lda_ctx* h, const int32_t* word_ids, int64_t n_tokens, const
     if (rc) return rc;
     if ((rc = check_device(c))) return rc;
     int32_t* wd = nullptr;
-    if (cudaMalloc(&wd, (size_t)std::max<int64_t>(n_tokens, 1) * 4) != cudaSuccess) {
-        cudaGetLastError();
-        return fail(&c, LDA_ENOMEM, "device allocation failed");
-    }
+    if (!tmp_alloc(c, &wd, (size_t)std::max<int64_t>(n_tokens, 1) * 4)) return fail(&c, LDA_ENOMEM, "device allocation failed");
     if (n_tokens > 0 &&
         cudaMemcpyAsync(wd, word_ids, (size_t)n_tokens * 4, cudaMemcpyHostToDevice, c.stream) != cudaSuccess) {
-        cudaFree(wd);
+        raw_free(c, wd);
         return cuda_fail(&c, "copying word ids");
     }
     rc = load_common(c, wd, n_tokens, doc_offsets, n_docs);
     cudaStreamSynchronize(c.stream);
-    cudaFree(wd);
+    raw_free(c, wd);
     return rc;
 }
 
@@ -877,18 +908,18 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
         DkCsr r;
         if ((rc = build_dk_csr(c, r, sizes_only))) return fail(&c, rc, "building the n_kd rows failed");
         int bits = 0;
-        if ((rc = read_err(c, &bits))) { free_dk_csr(r); return rc; }
-        if (bits) { free_dk_csr(r); return fail(&c, LDA_EINTERNAL, "the n_kd rows raised the device error word"); }
+        if ((rc = read_err(c, &bits))) { free_dk_csr(c, r); return rc; }
+        if (bits) { free_dk_csr(c, r); return fail(&c, LDA_EINTERNAL, "the n_kd rows raised the device error word"); }
         const int64_t total = (int64_t)r.total;
         if (nnz_out) *nnz_out = total;
-        if (sizes_only) { free_dk_csr(r); return LDA_OK; }
-        if (capacity < total) { free_dk_csr(r); return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros"); }
+        if (sizes_only) { free_dk_csr(c, r); return LDA_OK; }
+        if (capacity < total) { free_dk_csr(c, r); return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros"); }
         static_assert(sizeof(long long) == sizeof(int64_t), "row offsets are copied as they are");
         bool ok = true;
         if (row_offsets) ok = ok && cudaMemcpy(row_offsets, r.row_off, ((size_t)c.D + 1) * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
         if (topics && total) ok = ok && cudaMemcpy(topics, r.topic, (size_t)total * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
         if (counts && total) ok = ok && cudaMemcpy(counts, r.count, (size_t)total * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
-        free_dk_csr(r);
+        free_dk_csr(c, r);
         if (!ok) return cuda_fail(&c, "copying the n_kd rows");
         return LDA_OK;
     }

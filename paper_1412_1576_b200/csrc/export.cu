@@ -57,12 +57,12 @@ template <typename T>
 void launch_doc_rows(Ctx& c, const int32_t* tiles, int32_t n_tiles, const T* z, int32_t* nnz, const long long* row_off,
                      int32_t* topic, int32_t* count);  // counts.cu
 
-void free_dk_csr(DkCsr& r)
+void free_dk_csr(Ctx& c, DkCsr& r)
 {
-    cudaFree(r.row_off);
-    cudaFree(r.nnz);
-    cudaFree(r.topic);
-    cudaFree(r.count);
+    raw_free(c, r.row_off);
+    raw_free(c, r.nnz);
+    raw_free(c, r.topic);
+    raw_free(c, r.count);
     r = DkCsr{};
 }
 
@@ -72,9 +72,8 @@ static int build_dk_csr_t(Ctx& c, DkCsr& r, bool sizes_only)
     const View& v = c.v;
     const int32_t D = (int32_t)c.D;
     r = DkCsr{};
-    if (cudaMalloc(&r.row_off, ((size_t)D + 1) * 8) != cudaSuccess || cudaMalloc(&r.nnz, ((size_t)D + 1) * 4) != cudaSuccess) {
-        cudaGetLastError();
-        free_dk_csr(r);
+    if (!tmp_alloc(c, &r.row_off, ((size_t)D + 1) * 8) || !tmp_alloc(c, &r.nnz, ((size_t)D + 1) * 4)) {
+        free_dk_csr(c, r);
         return LDA_ENOMEM;
     }
     cudaMemsetAsync(r.nnz, 0, ((size_t)D + 1) * 4, c.stream);
@@ -91,9 +90,9 @@ static int build_dk_csr_t(Ctx& c, DkCsr& r, bool sizes_only)
     size_t temp_bytes = 0;
     // nnz(n_kd) <= n_tokens < 2^31: the 32-bit running sum cannot overflow
     if (cub::DeviceScan::ExclusiveSum(nullptr, temp_bytes, r.nnz, r.row_off, D + 1, c.stream) != cudaSuccess ||
-        cudaMalloc(&temp, temp_bytes ? temp_bytes : 1) != cudaSuccess) {
+        !tmp_alloc(c, &temp, temp_bytes)) {
         cudaGetLastError();
-        free_dk_csr(r);
+        free_dk_csr(c, r);
         return LDA_ENOMEM;
     }
     const cudaError_t e = cub::DeviceScan::ExclusiveSum(temp, temp_bytes, r.nnz, r.row_off, D + 1, c.stream);
@@ -102,17 +101,16 @@ static int build_dk_csr_t(Ctx& c, DkCsr& r, bool sizes_only)
         cudaMemcpyAsync(&total, r.row_off + D, 8, cudaMemcpyDeviceToHost, c.stream) != cudaSuccess ||
         cudaStreamSynchronize(c.stream) != cudaSuccess) {
         cudaGetLastError();
-        cudaFree(temp);
-        free_dk_csr(r);
+        raw_free(c, temp);
+        free_dk_csr(c, r);
         return LDA_ECUDA;
     }
-    cudaFree(temp);
+    raw_free(c, temp);
     r.total = total;
     if (sizes_only) return LDA_OK;
     const size_t cap = (size_t)(total > 0 ? total : 1);
-    if (cudaMalloc(&r.topic, cap * 4) != cudaSuccess || cudaMalloc(&r.count, cap * 4) != cudaSuccess) {
-        cudaGetLastError();
-        free_dk_csr(r);
+    if (!tmp_alloc(c, &r.topic, cap * 4) || !tmp_alloc(c, &r.count, cap * 4)) {
+        free_dk_csr(c, r);
         return LDA_ENOMEM;
     }
     if (c.n_doc_sort_tiles)

@@ -152,11 +152,8 @@ int lda::gibbs_sweep(Ctx& c, int32_t iters)
     int32_t* z_new = nullptr;
     ull* prefix = nullptr;
     int rc = LDA_OK;
-    if (cudaMalloc(&word_of, n1 * 4) != cudaSuccess || cudaMalloc(&z_new, n1 * 4) != cudaSuccess ||
-        cudaMalloc(&prefix, (size_t)c.V * c.K * 8) != cudaSuccess) {
-        cudaGetLastError();
+    if (!tmp_alloc(c, &word_of, n1 * 4) || !tmp_alloc(c, &z_new, n1 * 4) || !tmp_alloc(c, &prefix, (size_t)c.V * c.K * 8))
         rc = LDA_ENOMEM;
-    }
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     if (rc == LDA_OK && c.N > 0) k_word_of_tokens<<<1184, 256, 0, c.stream>>>(v, word_of);
     for (int32_t it = 0; rc == LDA_OK && it < iters && c.N > 0; ++it) {
@@ -176,13 +173,13 @@ int lda::gibbs_sweep(Ctx& c, int32_t iters)
         c.tables_valid = false;
             c.sweep += 1;
         if (cudaStreamSynchronize(c.stream) != cudaSuccess) rc = LDA_ECUDA;
-        free_dk_csr(r);
+        free_dk_csr(c, r);
     }
     if (iters > 0 && c.N == 0) c.sweep += (uint32_t)iters;
     cudaStreamSynchronize(c.stream);
-    cudaFree(word_of);
-    cudaFree(z_new);
-    cudaFree(prefix);
+    raw_free(c, word_of);
+    raw_free(c, z_new);
+    raw_free(c, prefix);
     if (rc == LDA_OK && cudaGetLastError() != cudaSuccess) rc = LDA_ECUDA;
     return rc;
 }

@@ -87,8 +87,8 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
     size_t temp_bytes = 0, temp2_bytes = 0;
     int rc = LDA_OK;
     do {
-        if (cudaMalloc(&keys_out, n1 * 4) != cudaSuccess || cudaMalloc(&iota, n1 * 4) != cudaSuccess ||
-            cudaMalloc(&keys_blk, n1 * 4) != cudaSuccess || cudaMalloc(&order, n1 * 4) != cudaSuccess) {
+        if (!tmp_alloc(c, &keys_out, n1 * 4) || !tmp_alloc(c, &iota, n1 * 4) || !tmp_alloc(c, &keys_blk, n1 * 4) ||
+            !tmp_alloc(c, &order, n1 * 4)) {
             rc = LDA_ENOMEM;
             break;
         }
@@ -101,7 +101,7 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
                 rc = LDA_ECUDA;
                 break;
             }
-            if (cudaMalloc(&temp, temp_bytes ? temp_bytes : 1) != cudaSuccess) {
+            if (!tmp_alloc(c, &temp, temp_bytes)) {
                 rc = LDA_ENOMEM;
                 break;
             }
@@ -121,7 +121,7 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
                 rc = LDA_ECUDA;
                 break;
             }
-            if (cudaMalloc(&temp2, temp2_bytes ? temp2_bytes : 1) != cudaSuccess) {
+            if (!tmp_alloc(c, &temp2, temp2_bytes)) {
                 rc = LDA_ENOMEM;
                 break;
             }
@@ -139,12 +139,12 @@ int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_hos
         if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess)
             rc = LDA_ECUDA;
     } while (0);
-    cudaFree(keys_out);
-    cudaFree(iota);
-    cudaFree(keys_blk);
-    cudaFree(order);
-    cudaFree(temp);
-    cudaFree(temp2);
+    raw_free(c, keys_out);
+    raw_free(c, iota);
+    raw_free(c, keys_blk);
+    raw_free(c, order);
+    raw_free(c, temp);
+    raw_free(c, temp2);
     if (rc != LDA_OK) return rc;
     c.v.inv = inv;
     c.v.bm_of_tok = bm_of_tok;

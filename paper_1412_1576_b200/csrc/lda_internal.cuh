@@ -207,8 +207,13 @@ struct Ctx {
     unsigned long long* sc_dense = nullptr;  // same three for the dense table, [3*K]
     double* red = nullptr;                   // reduction partials for the log-likelihood
     int64_t* red_i = nullptr;
+    // device memory comes from cudaMalloc / cudaFree unless lda_set_allocator() gave other routines
+    lda_alloc_fn alloc_fn = nullptr;
+    lda_free_fn free_fn = nullptr;
+    void* alloc_user = nullptr;
     std::vector<void*> allocs;
     std::vector<size_t> alloc_bytes;  // size of every entry of `allocs`
+    std::vector<char> alloc_own;      // 1: the entry came from the caller's allocator, 0: from cudaMalloc
     int64_t device_bytes = 0;
     lda_stats stats{};
     int64_t launches = 0;
@@ -265,7 +270,7 @@ struct DkCsr {
     long long total = 0;
 };
 int build_dk_csr(Ctx& c, DkCsr& r, bool sizes_only);  // LDA_* status; queued on c.stream, rows complete after a sync
-void free_dk_csr(DkCsr& r);
+void free_dk_csr(Ctx& c, DkCsr& r);
 
 // n_kw as a dense V x K matrix in device memory and back (shard.cu): the exchange format of the
 // document-sharded mode.  Return the number of kernels launched.
@@ -281,7 +286,15 @@ void set_gibbs_smem_limits();
 // load-time layout (sort + offsets); fills c.v token arrays. Returns LDA_* status.
 int build_layout(Ctx& c, const int32_t* word_ids_dev, const int64_t* doc_off_host);
 
-void* dev_alloc(Ctx& c, size_t bytes);  // tracked cudaMalloc; nullptr on failure
+void* raw_alloc(Ctx& c, size_t bytes);  // the context's allocator (cudaMalloc by default); nullptr on failure
+void raw_free(Ctx& c, void* p);
+template <typename P>
+inline bool tmp_alloc(Ctx& c, P** p, size_t bytes)  // transient buffer, released with raw_free()
+{
+    *p = static_cast<P*>(raw_alloc(c, bytes ? bytes : 1));
+    return *p != nullptr;
+}
+void* dev_alloc(Ctx& c, size_t bytes);  // tracked allocation held by the context; nullptr on failure
 void dev_free(Ctx& c, void* p);         // releases one tracked allocation (nullptr: nothing)
 void dev_free_all(Ctx& c);
 

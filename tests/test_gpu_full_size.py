@@ -19,7 +19,10 @@ CORES = max(1, len(os.sched_getaffinity(0)))
 
 
 def _free_gib():
+    import gc
     import torch
+    gc.collect()
+    torch.cuda.empty_cache()       # contexts of earlier tests gave their memory back to torch's pool
     return torch.cuda.mem_get_info()[0] / 2 ** 30
 
 
