@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--sharded", action="store_true",
                     help="document-sharded run of ONE corpus over the ranks (one all-reduce of n_kw per sweep) "
                          "instead of independent replicas; strong scaling, off by default")
+    ap.add_argument("--alias-slices", type=int, default=1,
+                    help="vocabulary slices whose word-proposal tables are in memory one at a time (default 1: all)")
     ap.add_argument("--no-windows", action="store_true", help="skip the late-sweep and own-step-count windows")
     ap.add_argument("--late-sweep", type=int, default=50, help="first sweep of the late window")
     return ap.parse_args()
@@ -193,7 +195,8 @@ def run_ours(args):
     gen_s = time.time() - t0
     N, D = corpus.n_tokens, corpus.n_docs
     stream = torch.cuda.current_stream()
-    lda = binding.LightLDA(cfg["V"], cfg["K"], cfg["alpha"], cfg["beta"], stream=stream.cuda_stream)
+    lda = binding.LightLDA(cfg["V"], cfg["K"], cfg["alpha"], cfg["beta"], stream=stream.cuda_stream,
+                           options={"alias_slices": args.alias_slices} if args.alias_slices != 1 else None)
     torch.cuda.empty_cache()
     t0 = time.time()
     lda.load_corpus(corpus.word_ids, corpus.doc_offsets)
@@ -394,6 +397,7 @@ def run_ours(args):
         "config": {"workload": f"{args.workload} LDA" + (f" x{args.scale}" if args.scale != 1.0 else ""),
                    "V": cfg["V"], "K": cfg["K"], "D": D, "n_tokens": N, "mh_steps": M,
                    "alpha": cfg["alpha"], "beta": cfg["beta"], "topic_bytes": topic_bytes,
+                   "alias_slices": args.alias_slices,
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "l2": "inputs larger than L2" if N * 14 > 126e6 else "inputs fit in L2",
                    "sweeps_timed": [st0["sweeps_done"], st0["sweeps_done"] + args.steps],

@@ -99,7 +99,16 @@ int lda_set_allocator(lda_ctx* ctx, lda_alloc_fn alloc_fn, lda_free_fn free_fn, 
  *   "dense_min_tf" words rarer than this (or than K/8) stay sparse even inside dense_frac
  *   "block_log2"   log2 of the tokens per block of documents in the block-major token order that the
  *                  document-side pass of the MH step walks (default 22: the exchange buffers
- *                  of one block, 20 bytes per token, stay in L2 while the document pass is on it)             */
+ *                  of one block, 20 bytes per token, stay in L2 while the document pass is on it)
+ *   "alias_slices" number of vocabulary slices (Section 3, Figure 1: the model is visited one slice at a
+ *                  time, and only that slice's alias tables are in memory; Section 6 "Pipelining").  Whole
+ *                  number in [1, 256], default 1.  The words are cut into runs of about equal row
+ *                  capacity; the word-proposal tables of Section 4.2 and their construction scratch
+ *                  (28-36 bytes per row slot, the largest part of the model's working set) are allocated
+ *                  for the largest slice only, and pass 1 of the MH step goes slice by slice: build the
+ *                  slice's tables, draw the word-proposals of its tokens.  The n_kw rows themselves stay
+ *                  resident (the accept pass and the rebuild need them).  No result depends on it; with
+ *                  more than one slice lda_stats.ms_alias_sparse is ~0 and ms_propose covers both.         */
 int lda_set_option(lda_ctx* ctx, const char* key, double value);
 
 /* Which proposal the steps of a token's chain draw (Section 4.3; the variants compared in

@@ -269,7 +269,7 @@ __device__ __forceinline__ uint32_t mixture_threshold(ull S, ull B)
 // One warp per word, rows of at most ALIAS_WARP_MAX items.  The two scratch arrays the binary
 // searches run over live in shared memory (12 bytes per item and warp), the third in the row's
 // range of the scratch array in device memory.
-__global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w)
+__global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w, int32_t w_lo, int32_t w_hi)
 {
     extern __shared__ __align__(16) unsigned char alias_scratch[];
     Group<false> g{nullptr};
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(256) k_alias_sparse_warp(View v, ull* sc_w)
     uint32_t* item_s = reinterpret_cast<uint32_t*>(reinterpret_cast<ull*>(alias_scratch) + 8 * ALIAS_WARP_MAX) +
                        (size_t)wic * ALIAS_WARP_MAX;
     const ull B = *v.dense_mass;
-    for (int32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < v.V; w += warps) {
+    for (int32_t w = w_lo + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); w < w_hi; w += warps) {
         const int32_t n = v.wk_nnz[w];
         if (n > ALIAS_WARP_MAX) continue;
         if (n == 0) {
@@ -343,23 +343,24 @@ int launch_alias_dense(Ctx& c)
 // longest rows (and the longest tail) first.
 int launch_alias_sparse(Ctx& c)
 {
+    const Ctx::Slice& q = c.slices[(size_t)c.cur_slice];
+    if (q.w_hi <= q.w_lo) return 0;
     int launches = 0;
     fork_streams(c);
     // words whose row cannot exceed ALIAS_SMEM_ITEMS_MID come first in the list
-    if (c.n_alias_big > c.n_alias_mid) {
-        k_alias_sparse_block<512>
-            <<<c.n_alias_big - c.n_alias_mid, 512, ALIAS_SMEM_ITEMS_BIG * ALIAS_SCRATCH_PER_ITEM, c.stream>>>(
-                c.v, c.alias_big + c.n_alias_mid, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_BIG);
+    if (q.big_n) {
+        k_alias_sparse_block<512><<<q.big_n, 512, ALIAS_SMEM_ITEMS_BIG * ALIAS_SCRATCH_PER_ITEM, c.stream>>>(
+            c.v, c.alias_big + c.n_alias_mid + q.big_lo, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_BIG);
         ++launches;
     }
-    if (c.n_alias_mid) {
-        k_alias_sparse_block<256><<<c.n_alias_mid, 256, ALIAS_SMEM_ITEMS_MID * ALIAS_SCRATCH_PER_ITEM, c.side[0]>>>(
-            c.v, c.alias_big, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_MID);
+    if (q.mid_n) {
+        k_alias_sparse_block<256><<<q.mid_n, 256, ALIAS_SMEM_ITEMS_MID * ALIAS_SCRATCH_PER_ITEM, c.side[0]>>>(
+            c.v, c.alias_big + q.mid_lo, c.sc_w, c.sc_de, c.sc_item, ALIAS_SMEM_ITEMS_MID);
         ++launches;
     }
-    int grid = (int)(((int64_t)c.V * 32 + 255) / 256);
+    int grid = (int)(((int64_t)(q.w_hi - q.w_lo) * 32 + 255) / 256);
     if (grid > 148 * 16) grid = 148 * 16;
-    k_alias_sparse_warp<<<grid, 256, ALIAS_WARP_SMEM, c.side[1]>>>(c.v, c.sc_w);
+    k_alias_sparse_warp<<<grid, 256, ALIAS_WARP_SMEM, c.side[1]>>>(c.v, c.sc_w, q.w_lo, q.w_hi);
     ++launches;
     join_streams(c);
     return launches;

@@ -135,6 +135,32 @@ static void free_corpus(Ctx& c)
     c.loaded = c.inited = c.tables_valid = false;
     c.N = c.D = 0;
     c.side_steps = 0;
+    c.slices.clear();
+    c.cur_slice = 0;
+    c.al_thr0 = c.al_idx0 = c.sc_item0 = c.sc_item = nullptr;
+    c.al_pk0 = nullptr;
+    c.sc_w0 = c.sc_de0 = c.sc_w = c.sc_de = nullptr;
+}
+
+// Row slot r of the running slice lives at entry r - row_lo of the slice-sized buffers: the pointers the
+// kernels index with row slots are the buffers' moved back by row_lo entries (and only ever used with
+// slots of that slice).
+template <typename P>
+static P* moved_back(P* base, int64_t entries)
+{
+    return base ? reinterpret_cast<P*>(reinterpret_cast<uintptr_t>(base) - (uintptr_t)entries * sizeof(P)) : nullptr;
+}
+
+void set_slice(Ctx& c, int slice)
+{
+    const Ctx::Slice& q = c.slices[(size_t)slice];
+    c.cur_slice = slice;
+    c.v.al_thr = moved_back(c.al_thr0, q.row_lo);
+    c.v.al_idx = moved_back(c.al_idx0, q.row_lo);
+    c.v.al_pk = moved_back(c.al_pk0, q.row_lo);
+    c.sc_w = moved_back(c.sc_w0, q.row_lo);
+    c.sc_de = moved_back(c.sc_de0, q.row_lo);
+    c.sc_item = moved_back(c.sc_item0, q.row_lo);
 }
 
 }  // namespace lda
@@ -192,7 +218,7 @@ static int ensure_tables(Ctx& c)
 {
     if (c.tables_valid) return LDA_OK;
     launch_alias_dense(c);
-    launch_alias_sparse(c);
+    launch_alias_sparse(c);  // the running slice's (lda_get_tables walks the slices itself)
     int bits = 0;
     int rc = read_err(c, &bits);
     if (rc) return rc;
@@ -285,6 +311,16 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
         }
     }
     row_start[V] = (int32_t)cap_total;
+    // vocabulary slices of about equal row capacity; slice_w[s] = first word of slice s
+    const int n_slices = std::max(1, c.alias_slices);
+    std::vector<int32_t> slice_w((size_t)n_slices + 1, V);
+    slice_w[0] = 0;
+    for (int sl = 1; sl < n_slices; ++sl) {
+        const int32_t target = (int32_t)(cap_total * sl / n_slices);
+        slice_w[sl] = (int32_t)(std::lower_bound(row_start.begin(), row_start.begin() + V, target) - row_start.begin());
+    }
+    std::vector<char> slice_starts((size_t)V + 1, 0);
+    for (int sl = 1; sl < n_slices; ++sl) slice_starts[(size_t)slice_w[sl]] = 1;
     // tiles of consecutive sparse words: <= SORT_TILE tokens and <= SORT_TILE words each
     {
         int32_t s0 = 0, tok = 0;
@@ -308,6 +344,7 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
             if (s1 > s0 && tok > 0) { cold_tiles.push_back(s0); cold_tiles.push_back(s1); }
         };
         for (int32_t w = 0; w < V; ++w) {
+            if (slice_starts[w]) { close(w); s0 = w; tok = 0; }  // no tile reaches across two slices
             if (tf[w] > COLD_TILE) {
                 close(w); s0 = w + 1; tok = 0;
                 std::vector<int32_t>& runs = dense_slot[w] >= 0 ? hot_tiles : hot_tiles_warm;
@@ -388,6 +425,37 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.n_warm = (int32_t)warm_words.size();
     c.n_hot_tiles_propose = (int32_t)(hot_tiles_propose.size() / 3);
     c.n_cold_tiles = (int32_t)(cold_tiles.size() / 2);
+    c.slices.assign((size_t)n_slices, Ctx::Slice{});
+    int64_t slice_rows_max = 1;
+    {
+        // every list is in ascending word order: a slice's part is a run of it
+        auto first_at = [](const std::vector<int32_t>& list, size_t lo, size_t hi, int stride, int32_t w) {
+            size_t a = lo, b = hi;  // first entry of [lo, hi) whose word is >= w
+            while (a < b) {
+                const size_t m = (a + b) / 2;
+                if (list[m * stride] < w) a = m + 1; else b = m;
+            }
+            return (int32_t)a;
+        };
+        const size_t n_mid = (size_t)c.n_alias_mid, n_big = (size_t)c.n_alias_big;
+        for (int sl = 0; sl < n_slices; ++sl) {
+            Ctx::Slice& q = c.slices[(size_t)sl];
+            q.w_lo = slice_w[(size_t)sl];
+            q.w_hi = slice_w[(size_t)sl + 1];
+            q.row_lo = row_start[(size_t)q.w_lo];
+            q.row_n = row_start[(size_t)q.w_hi] - q.row_lo;
+            slice_rows_max = std::max(slice_rows_max, q.row_n);
+            q.mid_lo = first_at(alias_big, 0, n_mid, 1, q.w_lo);
+            q.mid_n = first_at(alias_big, 0, n_mid, 1, q.w_hi) - q.mid_lo;
+            q.big_lo = first_at(alias_big, n_mid, n_big, 1, q.w_lo) - (int32_t)n_mid;
+            q.big_n = first_at(alias_big, n_mid, n_big, 1, q.w_hi) - (int32_t)n_mid - q.big_lo;
+            q.hotp_lo = first_at(hot_tiles_propose, 0, (size_t)c.n_hot_tiles_propose, 3, q.w_lo);
+            q.hotp_n = first_at(hot_tiles_propose, 0, (size_t)c.n_hot_tiles_propose, 3, q.w_hi) - q.hotp_lo;
+            q.cold_lo = first_at(cold_tiles, 0, (size_t)c.n_cold_tiles, 2, q.w_lo);
+            q.cold_n = first_at(cold_tiles, 0, (size_t)c.n_cold_tiles, 2, q.w_hi) - q.cold_lo;
+        }
+    }
+    const size_t cap_alias = (size_t)slice_rows_max;
 
     const size_t n1 = (size_t)std::max<int64_t>(N, 1), cap1 = (size_t)std::max<int64_t>(cap_total, 1);
     const size_t zt = c.wide_topics ? 4 : 2;
@@ -417,9 +485,9 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     v.wk_topic = (uint32_t*)A(cap1 * 4);
     v.wk_count = (uint32_t*)A(cap1 * 4);
     v.dense_rows = (int32_t*)A(std::max<size_t>((size_t)c.n_dense * v.dense_stride, 1) * 4);
-    v.al_thr = (uint32_t*)A(cap1 * 4);
-    v.al_idx = (uint32_t*)A(cap1 * 4);
-    v.al_pk = c.wide_topics ? nullptr : (uint2*)A(cap1 * 8);
+    c.al_thr0 = (uint32_t*)A(cap_alias * 4);
+    c.al_idx0 = (uint32_t*)A(cap_alias * 4);
+    c.al_pk0 = c.wide_topics ? nullptr : (uint2*)A(cap_alias * 8);
     v.dn_pk = (uint2*)A((size_t)K * 8);
     v.mix32 = (uint32_t*)A((size_t)V * 4);
     v.dn_thr = (uint32_t*)A((size_t)K * 4);
@@ -433,13 +501,14 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     v.dk_slots = (uint32_t*)A((size_t)long_slot_off.back() * 4 + 32);
     v.long_slot_off = upload(c, long_slot_off);
     ok = ok && v.long_slot_off;
-    c.sc_w = (unsigned long long*)A(cap1 * 8);
-    c.sc_de = (unsigned long long*)A(cap1 * 8);
-    c.sc_item = (uint32_t*)A(cap1 * 4);
+    c.sc_w0 = (unsigned long long*)A(cap_alias * 8);
+    c.sc_de0 = (unsigned long long*)A(cap_alias * 8);
+    c.sc_item0 = (uint32_t*)A(cap_alias * 4);
     c.sc_dense = (unsigned long long*)A((size_t)K * 8 * 3);
     c.red = (double*)A(sizeof(double) * (LL_WORD_PARTIALS + LL_DOC_PARTIALS));
     c.red_i = (int64_t*)A(16);
     if (!ok) { free_corpus(c); return fail(&c, LDA_ENOMEM, "device allocation failed"); }
+    set_slice(c, 0);
     cudaMemsetAsync(v.wk_nnz, 0, (size_t)V * 4, c.stream);
     cudaMemsetAsync(v.mix32, 0, (size_t)V * 4, c.stream);
     cudaMemsetAsync(v.nk, 0, (size_t)K * 4, c.stream);
@@ -589,6 +658,12 @@ int lda_set_option(lda_ctx* h, const char* key, double value)
         c.dense_frac = value;
         return LDA_OK;
     }
+    if (!std::strcmp(key, "alias_slices")) {
+        if (!(value >= 1.0 && value <= 256.0) || value != std::floor(value))
+            return fail(&c, LDA_EINVAL, "alias_slices must be a whole number in [1,256]");
+        c.alias_slices = (int)value;
+        return LDA_OK;
+    }
     if (!std::strcmp(key, "dense_min_tf")) {
         if (!(value >= 1.0)) return fail(&c, LDA_EINVAL, "dense_min_tf must be >= 1");
         c.dense_min_tf = value;
@@ -736,7 +811,7 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
             cudaEventRecord(c.ev[0], c.stream);
             n += launch_alias_dense(c);
             cudaEventRecord(c.ev[1], c.stream);
-            n += launch_alias_sparse(c);
+            if (c.slices.size() == 1) n += launch_alias_sparse(c);  // else slice by slice inside pass 1
             cudaEventRecord(c.ev[2], c.stream);
             n += launch_sample(c, mh_steps);
             cudaEventRecord(c.ev[3], c.stream);
@@ -984,26 +1059,49 @@ int lda_get_tables(lda_ctx* h, uint32_t* sp_thr32, int32_t* sp_alias, int64_t ca
     if (!c.inited) return fail(&c, LDA_ESTATE, "lda_get_tables before lda_init");
     int rc = check_device(c);
     if (rc) return rc;
-    if ((rc = ensure_tables(c))) return rc;
     const View& v = c.v;
     const size_t V = (size_t)c.V, K = (size_t)c.K;
+    const bool want_sparse = sp_thr32 || sp_alias;
+    std::vector<int32_t> nnz(V), start(V + 1);
+    std::vector<uint32_t> a, b;
+    if (want_sparse) {
+        if (cudaMemcpy(nnz.data(), v.wk_nnz, V * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+            cudaMemcpy(start.data(), v.row_start, (V + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+            return cuda_fail(&c, "copy");
+        int64_t total = 0;
+        for (size_t w = 0; w < V; ++w) total += nnz[w];
+        if (capacity < total) return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros");
+        a.resize(std::max<size_t>((size_t)start[V], 1));
+        b.resize(a.size());
+    }
+    // The device holds the sparse tables of one vocabulary slice at a time: build slice after slice
+    // (one slice: the whole vocabulary, built once and kept until the counts change).
+    const bool one = c.slices.size() == 1;
+    if (one) {
+        if ((rc = ensure_tables(c))) return rc;
+    } else {
+        c.tables_valid = false;
+        launch_alias_dense(c);
+    }
+    for (size_t sl = 0; sl < c.slices.size(); ++sl) {
+        const Ctx::Slice& q = c.slices[sl];
+        if (!one) {
+            set_slice(c, (int)sl);
+            launch_alias_sparse(c);
+            int bits = 0;
+            if ((rc = read_err(c, &bits))) return rc;
+            if (bits) return fail(&c, LDA_EINTERNAL, "alias construction raised the device error word");
+        }
+        if (want_sparse && q.row_n &&
+            (cudaMemcpy(a.data() + q.row_lo, c.al_thr0, (size_t)q.row_n * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+             cudaMemcpy(b.data() + q.row_lo, c.al_idx0, (size_t)q.row_n * 4, cudaMemcpyDeviceToHost) != cudaSuccess))
+            return cuda_fail(&c, "copy");
+    }
     if (mix32 && cudaMemcpy(mix32, v.mix32, V * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail(&c, "copy");
     if (dn_thr32 && cudaMemcpy(dn_thr32, v.dn_thr, K * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail(&c, "copy");
     if (dn_alias && cudaMemcpy(dn_alias, v.dn_idx, K * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail(&c, "copy");
     if (dense_mass && cudaMemcpy(dense_mass, v.dense_mass, 8, cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail(&c, "copy");
-    if (!sp_thr32 && !sp_alias) return LDA_OK;
-    std::vector<int32_t> nnz(V), start(V + 1);
-    if (cudaMemcpy(nnz.data(), v.wk_nnz, V * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
-        cudaMemcpy(start.data(), v.row_start, (V + 1) * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
-        return cuda_fail(&c, "copy");
-    int64_t total = 0;
-    for (size_t w = 0; w < V; ++w) total += nnz[w];
-    if (capacity < total) return fail(&c, LDA_ERANGE, "capacity below the number of nonzeros");
-    const size_t cap = (size_t)start[V];
-    std::vector<uint32_t> a(std::max<size_t>(cap, 1)), b(std::max<size_t>(cap, 1));
-    if (cap && (cudaMemcpy(a.data(), v.al_thr, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
-                cudaMemcpy(b.data(), v.al_idx, cap * 4, cudaMemcpyDeviceToHost) != cudaSuccess))
-        return cuda_fail(&c, "copy");
+    if (!want_sparse) return LDA_OK;
     int64_t o = 0;
     for (size_t w = 0; w < V; ++w)
         for (int32_t j = 0; j < nnz[w]; ++j, ++o) {

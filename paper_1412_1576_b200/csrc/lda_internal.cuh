@@ -174,6 +174,7 @@ struct Ctx {
     std::vector<int32_t> shard_global_tf;  // ... and the term frequencies over all shards (empty: this corpus alone)
     double dense_frac = 0.05;
     double dense_min_tf = 64;
+    int alias_slices = 1;  // vocabulary slices whose word-proposal tables are alive one at a time
     bool loaded = false, inited = false, tables_valid = false;
     int64_t n_nonempty_docs = 0;
     uint64_t seed = 0;
@@ -200,6 +201,26 @@ struct Ctx {
     int32_t* hot_tiles = nullptr;    // [n_hot_tiles*3] (word, first token, count): MH kernel, words with a dense row (accept pass)
     int32_t* hot_tiles_propose = nullptr;  // the same cut into the shorter runs of the propose passs
     int32_t* cold_tiles = nullptr;   // [n_cold_tiles*2] word ranges of whole tail words: MH kernel
+    // Vocabulary slices (Section 3, Fig. 1: the model is visited slice by slice): the words are cut into
+    // runs of about equal row capacity; the sparse alias tables and their construction scratch hold one
+    // slice at a time (entry of row slot r of the running slice: r - row_lo), so pass 1 goes slice by
+    // slice: build the slice's tables, draw the word-proposals of its tokens.  One slice = everything.
+    struct Slice {
+        int32_t w_lo = 0, w_hi = 0;        // words [w_lo, w_hi)
+        int64_t row_lo = 0, row_n = 0;     // their row slots [row_lo, row_lo + row_n)
+        int32_t mid_lo = 0, mid_n = 0;     // their part of alias_big[0 .. n_alias_mid)
+        int32_t big_lo = 0, big_n = 0;     // ... of alias_big[n_alias_mid .. n_alias_big), relative to n_alias_mid
+        int32_t hotp_lo = 0, hotp_n = 0;   // ... of hot_tiles_propose
+        int32_t cold_lo = 0, cold_n = 0;   // ... of cold_tiles
+    };
+    std::vector<Slice> slices;
+    int cur_slice = 0;
+    uint32_t* al_thr0 = nullptr;  // the slice-sized buffers View::al_thr, al_idx, al_pk and sc_w, sc_de, sc_item
+    uint32_t* al_idx0 = nullptr;  // point into, shifted by the running slice's row_lo
+    uint2* al_pk0 = nullptr;
+    unsigned long long* sc_w0 = nullptr;
+    unsigned long long* sc_de0 = nullptr;
+    uint32_t* sc_item0 = nullptr;
     // alias-construction scratch
     unsigned long long* sc_w = nullptr;   // [row capacity total] scaled masses
     unsigned long long* sc_de = nullptr;  // deficits prefix (front) / surpluses prefix (back)
@@ -252,7 +273,8 @@ int launch_export_assignments(Ctx& c, void* z_dev, bool narrow);
 int launch_count_wk(Ctx& c);
 int launch_count_k(Ctx& c);
 int launch_alias_dense(Ctx& c);
-int launch_alias_sparse(Ctx& c);
+int launch_alias_sparse(Ctx& c);            // the running slice's tables
+void set_slice(Ctx& c, int slice);          // makes `slice` the running one (moves the table pointers)
 int launch_sample(Ctx& c, int mh_steps);   // all passes of the MH step; needs ensure_exchange()
 int launch_doc_side(Ctx& c, int mh_steps);  // pass 2 of the MH step
 size_t doc_tile_smem_bytes(int tile_tokens);  // dynamic shared memory of the document-tile kernels

@@ -689,16 +689,18 @@ static int launch_accept(Ctx& c, uint2 key, int mh_steps)
 template <typename T, int CH, int MODE, int FIXED>
 static int launch_propose(Ctx& c, uint2 key, int mh_steps)
 {
+    // the running vocabulary slice's tokens (its tables are the ones in memory)
     const View& v = c.v;
+    const Ctx::Slice& q = c.slices[(size_t)c.cur_slice];
     int launches = 0;
-    if (c.n_hot_tiles_propose) {
-        k_word_hot<T, CH, false, false, MODE, FIXED><<<c.n_hot_tiles_propose, PROPOSE_THREADS, 0, c.stream>>>(
-            v, c.hot_tiles_propose, key, c.sweep, mh_steps);
+    if (q.hotp_n) {
+        k_word_hot<T, CH, false, false, MODE, FIXED><<<q.hotp_n, PROPOSE_THREADS, 0, c.stream>>>(
+            v, c.hot_tiles_propose + 3 * (size_t)q.hotp_lo, key, c.sweep, mh_steps);
         ++launches;
     }
-    if (c.n_cold_tiles) {
-        k_word_cold<T, CH, false, MODE, FIXED><<<c.n_cold_tiles, COLD_THREADS, 0, c.stream>>>(v, c.cold_tiles, key,
-                                                                                            c.sweep, mh_steps);
+    if (q.cold_n) {
+        k_word_cold<T, CH, false, MODE, FIXED><<<q.cold_n, COLD_THREADS, 0, c.stream>>>(
+            v, c.cold_tiles + 2 * (size_t)q.cold_lo, key, c.sweep, mh_steps);
         ++launches;
     }
     return launches;
@@ -709,12 +711,21 @@ static int sample_tc(Ctx& c, int mh_steps)
 {
     const uint2 key = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
     int launches = 0;
-    // pass 1: word-proposals (none in a doc-proposal-only chain)
+    // pass 1: word-proposals (none in a doc-proposal-only chain).  With more than one vocabulary
+    // slice the sparse alias tables exist for one slice at a time: build a slice's, draw from them,
+    // go on to the next (one slice: the caller has built them already).
     if (MODE != LDA_PROPOSALS_DOC) {
-        if (CH == 2 && mh_steps == 2)
-            launches += launch_propose<T, 2, MODE, 2>(c, key, mh_steps);
-        else
-            launches += launch_propose<T, CH, MODE, 0>(c, key, mh_steps);
+        const int n_slices = (int)c.slices.size();
+        for (int sl = 0; sl < n_slices; ++sl) {
+            if (n_slices > 1) {
+                set_slice(c, sl);
+                launches += launch_alias_sparse(c);
+            }
+            if (CH == 2 && mh_steps == 2)
+                launches += launch_propose<T, 2, MODE, 2>(c, key, mh_steps);
+            else
+                launches += launch_propose<T, CH, MODE, 0>(c, key, mh_steps);
+        }
     }
     // pass 2: document side
     cudaEventRecord(c.ev[8], c.stream);

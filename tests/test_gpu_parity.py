@@ -310,6 +310,46 @@ def test_block_size_is_invisible(small_corpus, block_log2):
         assert a == pytest.approx(b, rel=1e-10)
 
 
+@pytest.mark.parametrize("slices", [2, 5])
+def test_vocabulary_slices_are_invisible(small_corpus, slices):
+    """Pass 1 slice by slice (only one slice's alias tables in memory): same sweeps, same tables, every
+    schedule and step count; less device memory."""
+    c = small_corpus
+    whole = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
+    whole.load_corpus(c.word_ids.numpy(), c.doc_offsets.numpy())
+    g, o = _pair(c, seed=8, options={"alias_slices": slices})
+    assert g.stats()["device_bytes"] < whole.stats()["device_bytes"]
+    whole.close()
+    _assert_same_tables(g, o)
+    for mode, steps in ((binding.PROPOSALS_CYCLE, 2), (binding.PROPOSALS_CYCLE, 4),
+                        (binding.PROPOSALS_WORD, 3), (binding.PROPOSALS_DOC, 2)):
+        g.set_proposals(mode)
+        o.set_proposals(mode)
+        g.sweep(2, steps)
+        o.sweep(2, steps)
+        assert np.array_equal(g.get_assignments(), o.get_assignments()), (mode, steps)
+        assert g.stats()["ms_alias_sparse"] < 0.05     # nothing between its two events
+    _assert_same_counts(g, o)
+    _assert_same_tables(g, o)
+    g.sweep(1, 2)           # a sweep after the tables were read slice by slice
+    o.sweep(1, 2)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+
+
+def test_vocabulary_slices_large_and_big_shapes():
+    """Slices on the benchmark shapes: hot words with dense rows and rows of up to K items (large x0.01),
+    32-bit topics with warm words (big x0.003); more slices than some of them have words of a class."""
+    for name, scale, slices in (("large", 0.01, 4), ("big", 0.003, 7)):
+        c = synth.make(name, seed=0, scale=scale)
+        g, o = _pair(c, seed=17, options={"alias_slices": slices})
+        for sweep in range(2):
+            g.sweep(1, 2)
+            o.sweep(1, 2)
+            assert np.array_equal(g.get_assignments(), o.get_assignments()), (name, sweep)
+        assert np.array_equal(g.get_nk(), o.get_nk())
+        _assert_same_tables(g, o)
+
+
 def test_mid_shape_documents_and_lognormal_lengths():
     """Documents of ~330 tokens (a larger document-tile shape than the 90-token configs pick) and a
     heavy-tailed length law whose longest documents get a CTA of their own."""
@@ -406,6 +446,18 @@ def test_edge_cases():
     g.init(0)
     g.sweep(2, 2)
     assert g.get_assignments().size == 0
+
+
+def test_alias_slices_option_range(tiny_corpus):
+    c = tiny_corpus
+    for bad in (0, 2.5, 257):
+        with pytest.raises(binding.LdaError):
+            binding.LightLDA(c.V, c.K, c.alpha, c.beta, options={"alias_slices": bad})
+    g, o = _pair(c, seed=2, options={"alias_slices": 256})     # far more slices than words with tables
+    g.sweep(2, 2)
+    o.sweep(2, 2)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_tables(g, o)
 
 
 def test_error_paths():
