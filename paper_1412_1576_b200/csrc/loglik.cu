@@ -78,15 +78,47 @@ k_ll_doc_tiles(View v, const int32_t* __restrict__ tiles, int32_t n_tiles, int32
     const uint32_t cmask = (1u << v.count_bits) - 1u;
     double s = 0.0;
     unsigned long long filled = 0;
+    // A thread's tokens of a tile (cap = DOC_TILE_ROUNDS x blockDim.x): their block-major indices are
+    // read one tile ahead, so that a tile starts with its gathers already issued side by side.
+    uint32_t bm[DOC_TILE_ROUNDS];
+    auto tile_range = [&](int32_t t, int32_t& s0, int32_t& s1, int32_t& base, int32_t& cnt) {
+        s0 = tiles[2 * t];
+        s1 = tiles[2 * t + 1];
+        base = v.doc_off[s0];
+        cnt = v.doc_off[s1] - base;
+    };
+    auto read_bm = [&](int32_t base, int32_t cnt) {
+#pragma unroll
+        for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
+            const int j = tid + r * (int)blockDim.x;
+            bm[r] = j < cnt ? __ldcs(v.bm_of_tok + base + j) : 0u;
+        }
+    };
+    int32_t s0 = 0, s1 = 0, base = 0, cnt = 0;
+    if ((int32_t)blockIdx.x < n_tiles) {
+        tile_range(blockIdx.x, s0, s1, base, cnt);
+        read_bm(base, cnt);
+    }
     for (int32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-        const int32_t s0 = tiles[2 * t], s1 = tiles[2 * t + 1];
         const int32_t nseg = s1 - s0;
-        const int32_t base = v.doc_off[s0];
-        const int32_t cnt = v.doc_off[s1] - base;
-        for (int j = tid; j < cnt; j += blockDim.x)
-            topic[j] = (uint32_t)__ldcg(zbm + 2 * (size_t)__ldcs(v.bm_of_tok + base + j));
-        for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = v.doc_off[s0 + j] - base;
-        for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) slots[j] = DK_EMPTY;
+        const int32_t first_doc = s0, tile_base = base, tile_cnt = cnt;
+        uint32_t zt[DOC_TILE_ROUNDS];
+#pragma unroll
+        for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
+            const int j = tid + r * (int)blockDim.x;
+            zt[r] = j < tile_cnt ? (uint32_t)__ldcg(zbm + 2 * (size_t)bm[r]) : 0u;
+        }
+        if (t + (int32_t)gridDim.x < n_tiles) {
+            tile_range(t + gridDim.x, s0, s1, base, cnt);
+            read_bm(base, cnt);
+        }
+#pragma unroll
+        for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
+            const int j = tid + r * (int)blockDim.x;
+            if (j < tile_cnt) topic[j] = zt[r];
+        }
+        for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = v.doc_off[first_doc + j] - tile_base;
+        for (int j = tid; j < DK_SLOTS_PER_TOKEN * tile_cnt; j += blockDim.x) slots[j] = DK_EMPTY;
         __syncthreads();
         // one warp per document: its lanes insert the document's tokens
         const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -102,7 +134,7 @@ k_ll_doc_tiles(View v, const int32_t* __restrict__ tiles, int32_t n_tiles, int32
             if (lane == 0 && len > 0) s -= len < LL_TABLE ? by_len[len] : lgamma((double)len + v.Kalpha);
         }
         __syncthreads();
-        for (int j = tid; j < DK_SLOTS_PER_TOKEN * cnt; j += blockDim.x) {
+        for (int j = tid; j < DK_SLOTS_PER_TOKEN * tile_cnt; j += blockDim.x) {
             const uint32_t e = slots[j];
             if (e != DK_EMPTY) {
                 const uint32_t c = e & cmask;
@@ -164,8 +196,23 @@ k_ll_doc_long(View v, const int32_t* __restrict__ long_docs, int32_t n_long, dou
     if (threadIdx.x == 0 && filled) atomicAdd(nnz_out, filled);
 }
 
-// Grids of the document part: as many CTAs as fit the GPU at once, each taking tiles in turns.
-static int doc_ll_grid(const Ctx& c) { return std::max(1, std::min<int>(c.n_doc_tiles, c.n_sm * (2048 / c.doc_threads))); }
+// Grids of the document part: as many CTAs as the GPU holds at once (a CTA that had to wait for a
+// free slot would run its whole share of the tiles after the others, at low occupancy), each taking
+// tiles in turns.
+template <typename T>
+static int doc_ll_resident(const Ctx& c)
+{
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_ll_doc_tiles<T>, c.doc_threads,
+                                                      doc_tile_smem_bytes(c.doc_tile)) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    return c.n_sm * per_sm;
+}
+static int doc_ll_grid(const Ctx& c)
+{
+    const int resident = c.wide_topics ? doc_ll_resident<int32_t>(c) : doc_ll_resident<uint16_t>(c);
+    return std::max(1, std::min<int>(c.n_doc_tiles, resident));
+}
 static int long_ll_grid(const Ctx& c) { return std::max(1, std::min<int>(c.n_long_docs, LL_BLOCKS)); }
 
 // Queues the document part: partial sums to part[0 .. number returned), nnz(n_kd) to *nnz_dev (cleared here).
