@@ -100,6 +100,9 @@ int lda_set_allocator(lda_ctx* ctx, lda_alloc_fn alloc_fn, lda_free_fn free_fn, 
  *   "block_log2"   log2 of the tokens per block of documents in the block-major token order that the
  *                  document-side pass of the MH step walks (default 22: the exchange buffers
  *                  of one block, 20 bytes per token, stay in L2 while the document pass is on it)
+ *   "copy_chunk_log2" log2 of the tokens per chunk in which assignments cross the host link (default 25):
+ *                  a chunk is copied on the context's copy stream while its neighbour is spread into, or
+ *                  collected from, the device layout.  Whole number in [10, 30]; no result depends on it.
  *   "alias_slices" number of vocabulary slices (Section 3, Figure 1: the model is visited one slice at a
  *                  time, and only that slice's alias tables are in memory; Section 6 "Pipelining").  Whole
  *                  number in [1, 256], default 1.  The words are cut into runs of about equal row
@@ -217,6 +220,22 @@ int lda_get_assignments(lda_ctx* ctx, int32_t* z_out);
 
 /* The same as 16-bit topics; needs K <= 65536, LDA_ERANGE otherwise. */
 int lda_get_assignments_u16(lda_ctx* ctx, uint16_t* z_out);
+
+/* The two calls above without the wait at the end (the paper has no counterpart: Section 6 overlaps
+ * its transfers by pipelining data blocks; here the one transfer of a sweep's result is overlapped
+ * with what the caller does next).  The assignments are collected and copied to z_out (host memory;
+ * pinned, or the copy is not asynchronous) chunk by chunk on a stream of the context's own; the call
+ * returns once that is queued.  z_out is complete, and may be read, after lda_wait() has returned
+ * LDA_OK.  Calls made in between are legal: lda_loglik(), lda_get_stats() and lda_get_tables() run
+ * beside the transfer; a call that changes the state (lda_sweep, lda_set_assignments, lda_init, ...)
+ * is ordered after it on the device.  z_out stays owned by the caller and must stay valid until
+ * lda_wait() or lda_destroy(). */
+int lda_get_assignments_async(lda_ctx* ctx, int32_t* z_out);
+int lda_get_assignments_u16_async(lda_ctx* ctx, uint16_t* z_out);
+
+/* Waits for everything the context has queued (its stream and its copy stream).  LDA_ECUDA if the
+ * device reports an error. */
+int lda_wait(lda_ctx* ctx);
 
 /* Word-proposal tables built from the current counts (Section 4.2): per-word sparse
  * alias tables indexed like the LDA_NWK rows (split point as a 32-bit fraction,

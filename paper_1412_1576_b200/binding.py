@@ -22,7 +22,7 @@ LDA_NK, LDA_NWK, LDA_NDK = 0, 1, 2
 EXPORTS = [
     "lda_create", "lda_set_stream", "lda_set_allocator", "lda_set_option", "lda_set_proposals", "lda_load_corpus", "lda_load_corpus_device",
     "lda_set_shard", "lda_word_counts_to_dense", "lda_word_counts_from_dense", "lda_init", "lda_set_assignments", "lda_set_assignments_u16", "lda_sweep", "lda_gibbs_sweep", "lda_loglik", "lda_get_counts",
-    "lda_get_assignments", "lda_get_assignments_u16", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
+    "lda_get_assignments", "lda_get_assignments_u16", "lda_get_assignments_async", "lda_get_assignments_u16_async", "lda_wait", "lda_get_tables", "lda_get_stats", "lda_last_error", "lda_destroy",
     "lda_dense_table_noalloc",
 ]
 
@@ -93,6 +93,9 @@ def load_library(path: str | None = None):
     L.lda_get_counts.argtypes = [vp, C.c_int, vp, vp, vp, i64, C.POINTER(i64)]
     L.lda_get_assignments.argtypes = [vp, vp]
     L.lda_get_assignments_u16.argtypes = [vp, vp]
+    L.lda_get_assignments_async.argtypes = [vp, vp]
+    L.lda_get_assignments_u16_async.argtypes = [vp, vp]
+    L.lda_wait.argtypes = [vp]
     L.lda_get_tables.argtypes = [vp, vp, vp, i64, vp, vp, vp, C.POINTER(u64)]
     L.lda_get_stats.argtypes = [vp, C.POINTER(lda_stats)]
     L.lda_dense_table_noalloc.argtypes = [vp, i32, i32, dbl, vp, vp, vp, vp, vp]
@@ -247,6 +250,19 @@ def lda_get_assignments_u16_ptr(h, z_host_ptr):
     return load_library().lda_get_assignments_u16(h, C.c_void_p(z_host_ptr))
 
 
+def lda_get_assignments_async_ptr(h, z_host_ptr):
+    """Queues the export into (pinned) host memory at this address; complete after lda_wait()."""
+    return load_library().lda_get_assignments_async(h, C.c_void_p(z_host_ptr))
+
+
+def lda_get_assignments_u16_async_ptr(h, z_host_ptr):
+    return load_library().lda_get_assignments_u16_async(h, C.c_void_p(z_host_ptr))
+
+
+def lda_wait(h):
+    return load_library().lda_wait(h)
+
+
 def lda_get_tables(h, sp_thr32, sp_alias, mix32, dn_thr32, dn_alias):
     B = C.c_uint64()
     p = lambda a: None if a is None else a.ctypes.data
@@ -395,6 +411,17 @@ class LightLDA:
         out = np.zeros(max(self.N, 1), np.int32)
         self._ck(lda_get_assignments(self._h, out), "lda_get_assignments")
         return out[:self.N]
+
+    def get_assignments_async(self, host_tensor):
+        """Starts copying the assignments into a pinned CPU tensor (int32, or uint16/int16 for 16-bit topics) and
+        returns; the tensor is complete after wait().  lda_loglik and lda_get_stats may run meanwhile."""
+        narrow = host_tensor.element_size() == 2
+        fn = lda_get_assignments_u16_async_ptr if narrow else lda_get_assignments_async_ptr
+        assert host_tensor.numel() >= self.N and host_tensor.is_contiguous() and not host_tensor.is_cuda
+        self._ck(fn(self._h, host_tensor.data_ptr()), "lda_get_assignments_async")
+
+    def wait(self):
+        self._ck(lda_wait(self._h), "lda_wait")
 
     def get_assignments_u16(self) -> np.ndarray:
         out = np.zeros(max(self.N, 1), np.uint16)

@@ -106,6 +106,24 @@ static int check_device(Ctx& c)
     return LDA_OK;
 }
 
+// An export started by lda_get_assignments*_async() may still be copying out of the staging buffer:
+// whatever is queued on the context's stream from here on starts after it (no host wait).
+static void order_after_export(Ctx& c)
+{
+    if (!c.export_pending) return;
+    cudaStreamWaitEvent(c.stream, c.ev_export, 0);
+    c.export_pending = false;
+}
+
+// Host wait for everything the context has queued, the copy stream included.
+static int wait_all(Ctx& c)
+{
+    cudaError_t e = cudaStreamSynchronize(c.stream);
+    if (e == cudaSuccess && c.copy) e = cudaStreamSynchronize(c.copy);
+    c.export_pending = false;
+    return e == cudaSuccess ? LDA_OK : cuda_fail(&c, "waiting for the context's streams");
+}
+
 template <typename T>
 static T* upload(Ctx& c, const std::vector<T>& h)
 {
@@ -118,6 +136,8 @@ static T* upload(Ctx& c, const std::vector<T>& h)
 
 static void free_corpus(Ctx& c)
 {
+    if (c.copy) cudaStreamSynchronize(c.copy);  // an export may still read the staging buffer
+    c.export_pending = false;
     int* err = c.v.err;
     // the error word is allocated in lda_create and outlives corpora
     std::vector<void*> drop;
@@ -587,6 +607,9 @@ int lda_create(int32_t V, int32_t K, double alpha, double beta, lda_ctx** out)
         for (int i = 0; i < 2 && ok; ++i)
             ok = cudaEventCreateWithFlags(&c.ev_join[i], cudaEventDisableTiming) == cudaSuccess &&
                  cudaStreamCreateWithFlags(&c.side[i], cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaStreamCreateWithFlags(&c.copy, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c.ev_chunk, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c.ev_export, cudaEventDisableTiming) == cudaSuccess;
         c.have_side = true;  // lda_destroy() releases whatever was created
         if (!ok) {
             lda_destroy(h);
@@ -619,6 +642,12 @@ void lda_destroy(lda_ctx* h)
             if (c.ev_join[i]) cudaEventDestroy(c.ev_join[i]);
         }
         if (c.ev_fork) cudaEventDestroy(c.ev_fork);
+        if (c.copy) {
+            cudaStreamSynchronize(c.copy);
+            cudaStreamDestroy(c.copy);
+        }
+        if (c.ev_chunk) cudaEventDestroy(c.ev_chunk);
+        if (c.ev_export) cudaEventDestroy(c.ev_export);
     }
     if (c.have_events)
         for (int i = 0; i < Ctx::EV_RING * 10; ++i) cudaEventDestroy(c.ev_ring[i / 10][i % 10]);
@@ -662,6 +691,12 @@ int lda_set_option(lda_ctx* h, const char* key, double value)
         if (!(value >= 1.0 && value <= 256.0) || value != std::floor(value))
             return fail(&c, LDA_EINVAL, "alias_slices must be a whole number in [1,256]");
         c.alias_slices = (int)value;
+        return LDA_OK;
+    }
+    if (!std::strcmp(key, "copy_chunk_log2")) {
+        if (!(value >= 10.0 && value <= 30.0) || value != std::floor(value))
+            return fail(&c, LDA_EINVAL, "copy_chunk_log2 must be a whole number in [10,30]");
+        c.copy_chunk = (int64_t)1 << (int)value;
         return LDA_OK;
     }
     if (!std::strcmp(key, "dense_min_tf")) {
@@ -734,6 +769,7 @@ int lda_init(lda_ctx* h, uint64_t seed)
     if (!c.loaded) return fail(&c, LDA_ESTATE, "lda_init before lda_load_corpus");
     int rc = check_device(c);
     if (rc) return rc;
+    order_after_export(c);
     c.seed = seed;
     c.sweep = 0;
     launch_init(c);
@@ -756,11 +792,23 @@ static int set_assignments(lda_ctx* h, const void* z, bool narrow, uint64_t seed
     if (rc) return rc;
     // the record array (one word per token, only meaningful while the exported n_kd is valid)
     // doubles as the staging buffer: no allocation here
-    void* zdev = c.v.rec;
-    if (c.N > 0 &&
-        cudaMemcpyAsync(zdev, z, (size_t)c.N * (narrow ? 2 : 4), cudaMemcpyHostToDevice, c.stream) != cudaSuccess)
-        return cuda_fail(&c, "copying assignments");
-    launch_spread_assignments(c, zdev, narrow);
+    char* zdev = reinterpret_cast<char*>(c.v.rec);
+    order_after_export(c);
+    // chunk by chunk on the copy stream, each chunk spread into the block-major order (on the context's
+    // stream) while the next one is on its way
+    const size_t zt = narrow ? 2 : 4;
+    cudaEventRecord(c.ev_chunk, c.stream);
+    cudaStreamWaitEvent(c.copy, c.ev_chunk, 0);  // the staging buffer's earlier users are done
+    for (int64_t first = 0; first < c.N; first += c.copy_chunk) {
+        const int64_t count = std::min<int64_t>(c.copy_chunk, c.N - first);
+        if (cudaMemcpyAsync(zdev + (size_t)first * zt, reinterpret_cast<const char*>(z) + (size_t)first * zt,
+                            (size_t)count * zt, cudaMemcpyHostToDevice, c.copy) != cudaSuccess)
+            return cuda_fail(&c, "copying assignments");
+        cudaEventRecord(c.ev_chunk, c.copy);
+        cudaStreamWaitEvent(c.stream, c.ev_chunk, 0);
+        launch_spread_chunk(c, zdev, narrow, first, count);
+    }
+    launch_word_order_topics(c);
     int bits = 0;
     rc = read_err(c, &bits);
     if (rc) return rc;
@@ -793,6 +841,7 @@ int lda_sweep(lda_ctx* h, int32_t iters, int32_t mh_steps)
     if (!c.inited) return fail(&c, LDA_ESTATE, "lda_sweep before lda_init");
     int rc = check_device(c);
     if (rc) return rc;
+    order_after_export(c);
     if ((rc = ensure_exchange(c, mh_steps))) return rc;
     lda_stats& s = c.stats;
     s.ms_alias_dense = s.ms_alias_sparse = s.ms_sample = s.ms_count_wk = s.ms_count_k = s.ms_count_dk =
@@ -929,6 +978,7 @@ int lda_gibbs_sweep(lda_ctx* h, int32_t iters)
     if (c.v.count_bits > 19) return fail(&c, LDA_ERANGE, "the exact-conditional sweep takes documents shorter than 2^19 tokens");
     int rc = check_device(c);
     if (rc) return rc;
+    order_after_export(c);
     rc = gibbs_sweep(c, iters);
     if (rc) return fail(&c, rc, "the exact-conditional sweep failed");
     int bits = 0;
@@ -966,6 +1016,7 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
     if (!c.inited) return fail(&c, LDA_ESTATE, "lda_get_counts before lda_init");
     int rc = check_device(c);
     if (rc) return rc;
+    order_after_export(c);
     const View& v = c.v;
     cudaStreamSynchronize(c.stream);
     if (which == LDA_NK) {
@@ -1028,7 +1079,7 @@ int lda_get_counts(lda_ctx* h, int which, int64_t* row_offsets, int32_t* topics,
     return LDA_OK;
 }
 
-static int get_assignments(lda_ctx* h, void* z_out, bool narrow)
+static int get_assignments(lda_ctx* h, void* z_out, bool narrow, bool wait)
 {
     if (!h) return LDA_EINVAL;
     Ctx& c = h->c;
@@ -1038,18 +1089,41 @@ static int get_assignments(lda_ctx* h, void* z_out, bool narrow)
     if (c.N == 0) return LDA_OK;
     int rc = check_device(c);
     if (rc) return rc;
-    void* zdev = c.v.rec;  // staging, see set_assignments()
-    launch_export_assignments(c, zdev, narrow);
-    cudaError_t e =
-        cudaMemcpyAsync(z_out, zdev, (size_t)c.N * (narrow ? 2 : 4), cudaMemcpyDeviceToHost, c.stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
-    if (e != cudaSuccess) return cuda_fail(&c, "copying assignments");
-    return LDA_OK;
+    order_after_export(c);
+    char* zdev = reinterpret_cast<char*>(c.v.rec);  // staging, see set_assignments()
+    // chunk by chunk: collected into document order on the context's stream, copied out on the copy
+    // stream while the next chunk is collected
+    const size_t zt = narrow ? 2 : 4;
+    for (int64_t first = 0; first < c.N; first += c.copy_chunk) {
+        const int64_t count = std::min<int64_t>(c.copy_chunk, c.N - first);
+        launch_export_chunk(c, zdev, narrow, first, count);
+        cudaEventRecord(c.ev_chunk, c.stream);
+        cudaStreamWaitEvent(c.copy, c.ev_chunk, 0);
+        if (cudaMemcpyAsync(reinterpret_cast<char*>(z_out) + (size_t)first * zt, zdev + (size_t)first * zt,
+                            (size_t)count * zt, cudaMemcpyDeviceToHost, c.copy) != cudaSuccess)
+            return cuda_fail(&c, "copying assignments");
+    }
+    cudaEventRecord(c.ev_export, c.copy);
+    c.export_pending = true;
+    return wait ? wait_all(c) : LDA_OK;
 }
 
-int lda_get_assignments(lda_ctx* h, int32_t* z_out) { return get_assignments(h, z_out, false); }
+int lda_get_assignments(lda_ctx* h, int32_t* z_out) { return get_assignments(h, z_out, false, true); }
 
-int lda_get_assignments_u16(lda_ctx* h, uint16_t* z_out) { return get_assignments(h, z_out, true); }
+int lda_get_assignments_u16(lda_ctx* h, uint16_t* z_out) { return get_assignments(h, z_out, true, true); }
+
+int lda_get_assignments_async(lda_ctx* h, int32_t* z_out) { return get_assignments(h, z_out, false, false); }
+
+int lda_get_assignments_u16_async(lda_ctx* h, uint16_t* z_out) { return get_assignments(h, z_out, true, false); }
+
+int lda_wait(lda_ctx* h)
+{
+    if (!h) return LDA_EINVAL;
+    Ctx& c = h->c;
+    int rc = check_device(c);
+    if (rc) return rc;
+    return wait_all(c);
+}
 
 int lda_get_tables(lda_ctx* h, uint32_t* sp_thr32, int32_t* sp_alias, int64_t capacity, uint32_t* mix32,
                    uint32_t* dn_thr32, int32_t* dn_alias, uint64_t* dense_mass)

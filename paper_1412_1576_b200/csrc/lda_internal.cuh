@@ -249,6 +249,14 @@ struct Ctx {
     cudaStream_t side[2] = {};
     cudaEvent_t ev_fork = nullptr, ev_join[2] = {};
     bool have_side = false;
+    // Assignments travel between host and device in chunks on a stream of their own, so that the copy
+    // of one chunk runs beside the kernel that spreads (or collects) its neighbour.  ev_chunk orders a
+    // chunk's two halves; ev_export completes when the last chunk of an export has reached the host:
+    // whatever touches the staging buffer next waits for it on the device (order_after_export()).
+    int64_t copy_chunk = 1 << 25;  // tokens per chunk (option "copy_chunk_log2")
+    cudaStream_t copy = nullptr;
+    cudaEvent_t ev_chunk = nullptr, ev_export = nullptr;
+    bool export_pending = false;
     std::string err;
 };
 
@@ -269,7 +277,10 @@ inline void join_streams(Ctx& c)
 // --- launchers (each returns the number of kernels it launched) -----------------
 int launch_init(Ctx& c);
 int launch_spread_assignments(Ctx& c, const void* z_dev, bool narrow);  // z (doc order; u16 if narrow, else i32) -> both layouts
+int launch_spread_chunk(Ctx& c, const void* z_dev, bool narrow, int64_t first, int64_t count);  // ... tokens [first, first+count) -> block-major
+int launch_word_order_topics(Ctx& c);                                  // block-major -> word order, all tokens
 int launch_export_assignments(Ctx& c, void* z_dev, bool narrow);
+int launch_export_chunk(Ctx& c, void* z_dev, bool narrow, int64_t first, int64_t count);
 int launch_count_wk(Ctx& c);
 int launch_count_k(Ctx& c);
 int launch_alias_dense(Ctx& c);

@@ -617,13 +617,13 @@ __global__ void k_init(View v, uint2 key)
 // steps that each stay coalesced on one side: document order -> block-major order (the scattered
 // writes stay inside one block of that order at a time), then block-major -> word order.
 template <typename T, typename IN>
-__global__ void k_spread(View v, const IN* __restrict__ z_in)
+__global__ void k_spread(View v, const IN* __restrict__ z_in, int64_t first, int64_t count)
 {
     // one token per thread, CTAs in document order: the scattered writes of the CTAs in flight stay
     // inside one block of the block-major order (a grid-stride loop would let them drift apart)
     T* zbm = reinterpret_cast<T*>(v.zbm);
-    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (i >= v.N) return;
+    const int64_t i = first + blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i >= first + count) return;
     int64_t a = (int64_t)z_in[i];
     if (a < 0 || a >= v.K) {
         atomicOr(v.err, ERR_TOPIC_RANGE);
@@ -643,12 +643,12 @@ __global__ void k_word_order_topics(View v)
 }
 
 template <typename T, typename OUT>
-__global__ void k_export(View v, OUT* __restrict__ out)
+__global__ void k_export(View v, OUT* __restrict__ out, int64_t first, int64_t count)
 {
     // one token per thread, CTAs in document order (see k_spread)
     const T* zbm = reinterpret_cast<const T*>(v.zbm);
-    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (i < v.N) out[i] = (OUT)zbm[2 * (size_t)__ldcs(v.bm_of_tok + i)];
+    const int64_t i = first + blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i < first + count) out[i] = (OUT)zbm[2 * (size_t)__ldcs(v.bm_of_tok + i)];
 }
 
 static int grid_for(int64_t n, int block)
@@ -806,30 +806,44 @@ int launch_init(Ctx& c)
 }
 
 // `narrow`: the caller's array holds 16-bit topics (only with 16-bit topic storage), else int32.
-int launch_spread_assignments(Ctx& c, const void* z_dev, bool narrow)
+int launch_spread_chunk(Ctx& c, const void* z_dev, bool narrow, int64_t first, int64_t count)
+{
+    if (count <= 0) return 0;
+    const unsigned full = (unsigned)((count + 255) / 256);  // one token per thread
+    if (c.wide_topics) k_spread<int32_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev, first, count);
+    else if (narrow) k_spread<uint16_t, uint16_t><<<full, 256, 0, c.stream>>>(c.v, (const uint16_t*)z_dev, first, count);
+    else k_spread<uint16_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev, first, count);
+    return 1;
+}
+
+int launch_word_order_topics(Ctx& c)
 {
     if (c.N == 0) return 0;
     const int g = grid_for(c.N, 256);
-    const unsigned full = (unsigned)((c.N + 255) / 256);  // one token per thread
-    if (c.wide_topics) {
-        k_spread<int32_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev);
-        k_word_order_topics<int32_t><<<g, 256, 0, c.stream>>>(c.v);
-    } else {
-        if (narrow) k_spread<uint16_t, uint16_t><<<full, 256, 0, c.stream>>>(c.v, (const uint16_t*)z_dev);
-        else k_spread<uint16_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (const int32_t*)z_dev);
-        k_word_order_topics<uint16_t><<<g, 256, 0, c.stream>>>(c.v);
-    }
-    return 2;
+    if (c.wide_topics) k_word_order_topics<int32_t><<<g, 256, 0, c.stream>>>(c.v);
+    else k_word_order_topics<uint16_t><<<g, 256, 0, c.stream>>>(c.v);
+    return 1;
+}
+
+int launch_spread_assignments(Ctx& c, const void* z_dev, bool narrow)
+{
+    if (c.N == 0) return 0;
+    return launch_spread_chunk(c, z_dev, narrow, 0, c.N) + launch_word_order_topics(c);
+}
+
+int launch_export_chunk(Ctx& c, void* z_dev, bool narrow, int64_t first, int64_t count)
+{
+    if (count <= 0) return 0;
+    const unsigned full = (unsigned)((count + 255) / 256);  // one token per thread
+    if (c.wide_topics) k_export<int32_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev, first, count);
+    else if (narrow) k_export<uint16_t, uint16_t><<<full, 256, 0, c.stream>>>(c.v, (uint16_t*)z_dev, first, count);
+    else k_export<uint16_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev, first, count);
+    return 1;
 }
 
 int launch_export_assignments(Ctx& c, void* z_dev, bool narrow)
 {
-    if (c.N == 0) return 0;
-    const unsigned full = (unsigned)((c.N + 255) / 256);  // one token per thread
-    if (c.wide_topics) k_export<int32_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev);
-    else if (narrow) k_export<uint16_t, uint16_t><<<full, 256, 0, c.stream>>>(c.v, (uint16_t*)z_dev);
-    else k_export<uint16_t, int32_t><<<full, 256, 0, c.stream>>>(c.v, (int32_t*)z_dev);
-    return 1;
+    return launch_export_chunk(c, z_dev, narrow, 0, c.N);
 }
 
 }  // namespace lda

@@ -497,3 +497,38 @@ def test_device_resident_load_matches_host_load(tiny_corpus):
     a.sweep(2, 2)
     b.sweep(2, 2)
     assert np.array_equal(a.get_assignments(), b.get_assignments())
+
+
+def test_chunked_transfers_and_async_export(small_corpus):
+    """Assignments cross the host link in chunks on the context's copy stream.  The asynchronous export
+    delivers what the blocking one does, the log-likelihood may be taken while it runs, and a sweep
+    called before lda_wait() is ordered after the copy."""
+    import torch
+    c = small_corpus
+    g, o = _pair(c, seed=41, options={"copy_chunk_log2": 12})      # some 500 chunks with a ragged last one
+    g.sweep(1, 2)
+    o.sweep(1, 2)
+    want = o.get_assignments()
+    for dtype in (torch.int32, torch.int16):
+        host = torch.full((g.N,), -1, dtype=dtype).pin_memory()
+        g.get_assignments_async(host)
+        ll = g.loglik()
+        g.wait()
+        assert np.array_equal(host.numpy().astype(np.int64) & 0xFFFF, want)
+        assert ll[0] == pytest.approx(o.loglik()[0], rel=1e-10)
+    # a sweep queued right behind the export must not disturb it, nor be disturbed by it
+    host = torch.full((g.N,), -1, dtype=torch.int32).pin_memory()
+    g.get_assignments_async(host)
+    g.sweep(1, 2)
+    o.sweep(1, 2)
+    g.wait()
+    assert np.array_equal(host.numpy(), want)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    # import through the chunked path, then go on
+    z = o.get_assignments()
+    g.set_assignments(z, 41, 2)
+    o.set_assignments(z, 41, 2)
+    g.sweep(1, 2)
+    o.sweep(1, 2)
+    assert np.array_equal(g.get_assignments(), o.get_assignments())
+    _assert_same_counts(g, o)
