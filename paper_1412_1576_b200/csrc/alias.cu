@@ -21,6 +21,11 @@ namespace lda {
 
 typedef unsigned long long ull;
 
+#ifndef LDA_ALIAS_BINS_AT_ONCE
+#define LDA_ALIAS_BINS_AT_ONCE 2
+#endif
+constexpr int ALIAS_BINS_AT_ONCE = LDA_ALIAS_BINS_AT_ONCE;  // bins a thread finishes side by side
+
 template <bool BLOCK>
 struct Group {
     ull* smem;  // CTA groups only: >= 99 entries
@@ -131,16 +136,29 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
                                uint2* __restrict__ out_pk, const uint32_t* __restrict__ pk_topic, int* err)
 {
     const int r = g.rank(), gs = g.size();
+    // Items are taken four (weights) or two (bins) at a time per thread, their loads issued side by
+    // side: a row is built by one warp or one CTA, so what a pass costs is the latency of its chain of
+    // dependent reads, not the number of instructions.
     ull s = 0;
-    for (int32_t i = r; i < n; i += gs) {
-        const ull wt = weight(i);
-        sc_w[i] = wt;
-        s += wt;
+    for (int32_t i0 = r; i0 < n; i0 += 4 * gs) {
+        ull wt[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t i = i0 + u * gs;
+            wt[u] = i < n ? weight(i) : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t i = i0 + u * gs;
+            if (i < n) sc_w[i] = wt[u];
+            s += wt[u];
+        }
     }
     const ull W44 = g.reduce(s);
     int sh = bit_length(W44) + bit_length((ull)n) - 62;
     if (sh < 0) sh = 0;
     s = 0;
+#pragma unroll 4
     for (int32_t i = r; i < n; i += gs) s += sc_w[i] >> sh;
     const ull W = g.reduce(s);
     if (W == 0) {
@@ -149,11 +167,13 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
     }
     // Every thread takes a run of consecutive items (lights and heavies are numbered in ascending
     // item order): one pass to count them and add up their deficits and surpluses, one scan of the
-    // threads' totals, one pass to write the prefix of every item.
+    // threads' totals, one pass to write the prefix of every item.  An odd run length keeps the
+    // threads of a warp on different shared-memory banks.
     g.sync();  // the weights were written item by item across the group
-    const int32_t seg = (n + gs - 1) / gs;
+    const int32_t seg = ((n + gs - 1) / gs) | 1;
     const int32_t i_first = min(n, r * seg), i_last = min(n, i_first + seg);
     ull cnt = 0, d_mine = 0, e_mine = 0;
+#pragma unroll 4
     for (int32_t i = i_first; i < i_last; ++i) {
         const ull a = (ull)n * (sc_w[i] >> sh);
         if (a <= W) { cnt += 1ull; d_mine += W - a; } else { cnt += 1ull << 32; e_mine += a - W; }
@@ -163,6 +183,7 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
     {
         uint32_t l = (uint32_t)pre[0], m = (uint32_t)(pre[0] >> 32);
         ull d_at = pre[1], e_at = pre[2];
+#pragma unroll 2
         for (int32_t i = i_first; i < i_last; ++i) {
             const ull a = (ull)n * (sc_w[i] >> sh);
             sc_w[i] = a;
@@ -183,44 +204,81 @@ __device__ ull build_alias_row(const Group<BLOCK>& g, int32_t n, Weight weight, 
     const ull d_sum = tot[1];
     g.sync();
     const Frac32 frac(W);
-    for (uint32_t l = r; l < L; l += gs) {
-        const uint32_t i = sc_item[l];
-        const ull a = sc_w[i];
-        uint32_t al = i;
-        if (a != W) {
-            const ull D = sc_de[l];
-            uint32_t lo = 0, hi = H;  // number of heavies with E_m <= D
-            while (lo < hi) {
-                const uint32_t mid = (lo + hi) >> 1;
-                if (sc_de[n - 1 - mid] <= D) lo = mid + 1; else hi = mid;
+    // The searches below count the entries of a sorted prefix array under a bound, one bit of the
+    // answer per step from the top: the same number of steps for every item, so two items' searches
+    // run in one loop.
+    constexpr int U = ALIAS_BINS_AT_ONCE;
+    const uint32_t top_h = H ? 1u << (31 - __clz((int)H)) : 0u;
+    const uint32_t top_l = L ? 1u << (31 - __clz((int)L)) : 0u;
+    for (uint32_t l0 = r; l0 < L; l0 += U * gs) {
+        uint32_t it[U], pos[U];
+        ull a[U], D[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t l = l0 + u * gs;
+            it[u] = l < L ? sc_item[l] : 0u;
+            D[u] = l < L ? sc_de[l] : 0ull;
+            pos[u] = 0;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) a[u] = l0 + u * gs < L ? sc_w[it[u]] : W;
+        for (uint32_t step = top_h; step; step >>= 1) {  // number of heavies with E_m <= D
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t q = pos[u] + step;
+                if (q <= H && sc_de[n - q] <= D[u]) pos[u] = q;
             }
-            if (lo >= H) { atomicOr(err, ERR_ALIAS); lo = H ? H - 1 : 0; }
-            al = H ? sc_item[n - 1 - lo] : i;
         }
-        const uint32_t thr32 = frac(a);
-        out_thr[i] = thr32;
-        out_idx[i] = al;
-        store_packed_bin(out_pk, pk_topic, i, thr32, al);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (l0 + u * gs >= L) continue;
+            const uint32_t i = it[u];
+            uint32_t al = i;
+            if (a[u] != W) {
+                uint32_t lo = pos[u];
+                if (lo >= H) { atomicOr(err, ERR_ALIAS); lo = H ? H - 1 : 0; }
+                al = H ? sc_item[n - 1 - lo] : i;
+            }
+            const uint32_t thr32 = frac(a[u]);
+            out_thr[i] = thr32;
+            out_idx[i] = al;
+            store_packed_bin(out_pk, pk_topic, i, thr32, al);
+        }
     }
-    for (uint32_t m = r; m < H; m += gs) {
-        const uint32_t i = sc_item[n - 1 - m];
-        const ull E = sc_de[n - 1 - m];
-        uint32_t lo = 0, hi = L;  // first light l with D_l >= E; l == L stands for the total deficit
-        while (lo < hi) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (sc_de[mid] >= E) hi = mid; else lo = mid + 1;
+    for (uint32_t m0 = r; m0 < H; m0 += U * gs) {
+        uint32_t it[U], pos[U];
+        ull E[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t m = m0 + u * gs;
+            it[u] = m < H ? sc_item[n - 1 - m] : 0u;
+            E[u] = m < H ? sc_de[n - 1 - m] : 0ull;
+            pos[u] = 0;
         }
-        const ull Dl = lo < L ? sc_de[lo] : d_sum;
-        const ull thr = W + E - Dl;
-        uint32_t al = i;
-        if (thr != W) {
-            if (m + 1 >= H) atomicOr(err, ERR_ALIAS);
-            else al = sc_item[n - 1 - (m + 1)];
+        for (uint32_t step = top_l; step; step >>= 1) {  // number of lights with D_l < E: the first light with D_l >= E
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t q = pos[u] + step;
+                if (q <= L && sc_de[q - 1] < E[u]) pos[u] = q;
+            }
         }
-        const uint32_t thr32 = frac(thr);
-        out_thr[i] = thr32;
-        out_idx[i] = al;
-        store_packed_bin(out_pk, pk_topic, i, thr32, al);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t m = m0 + u * gs;
+            if (m >= H) continue;
+            const uint32_t i = it[u], lo = pos[u];  // lo == L stands for the total deficit
+            const ull Dl = lo < L ? sc_de[lo] : d_sum;
+            const ull thr = W + E[u] - Dl;
+            uint32_t al = i;
+            if (thr != W) {
+                if (m + 1 >= H) atomicOr(err, ERR_ALIAS);
+                else al = sc_item[n - 1 - (m + 1)];
+            }
+            const uint32_t thr32 = frac(thr);
+            out_thr[i] = thr32;
+            out_idx[i] = al;
+            store_packed_bin(out_pk, pk_topic, i, thr32, al);
+        }
     }
     return W44;
 }
