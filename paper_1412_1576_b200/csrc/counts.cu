@@ -144,12 +144,38 @@ k_word_rows(const int32_t* __restrict__ tiles, const int32_t* __restrict__ word_
     uint32_t* before = word_smem + bw;  // [bw] set bits before each bitmap word
     const int tid = threadIdx.x;
     const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
+    // Words of at most 32 tokens (most of the vocabulary) take one warp each and no barrier: a lane
+    // holds a token, lanes with the same topic find each other, the lowest of them writes the entry at
+    // the rank of its topic among the word's distinct topics.
+    {
+        const int lane = tid & 31;
+        for (int32_t w = s0 + (tid >> 5); w < s1; w += (int32_t)(blockDim.x >> 5)) {
+            const int32_t first = word_off[w], n = word_off[w + 1] - first;
+            if (n > 32) continue;
+            uint32_t k = 0xFFFFFFFFu;
+            if (lane < n) {
+                k = (uint32_t)__ldcs(z + first + lane);
+                if (k >= (uint32_t)K) { atomicOr(err, ERR_TOPIC_RANGE); k = 0xFFFFFFFFu; }
+            }
+            const uint32_t same = __match_any_sync(0xFFFFFFFFu, k);
+            const bool lead = k != 0xFFFFFFFFu && (uint32_t)(__ffs((int)same) - 1) == (uint32_t)lane;
+            const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, lead);
+            int32_t rank = 0;
+            for (uint32_t m = leaders; m; m &= m - 1u) {
+                const uint32_t other = __shfl_sync(0xFFFFFFFFu, k, __ffs((int)m) - 1);
+                rank += other < k ? 1 : 0;
+            }
+            if (lead) {
+                const int32_t r = row_start[w] + rank;
+                wk_topic[r] = k;
+                wk_count[r] = (uint32_t)__popc(same);
+            }
+            if (lane == 0) wk_nnz[w] = __popc(leaders);
+        }
+    }
     for (int32_t w = s0; w < s1; ++w) {
         const int32_t first = word_off[w], n = word_off[w + 1] - first;
-        if (n == 0) {
-            if (tid == 0) wk_nnz[w] = 0;
-            continue;
-        }
+        if (n <= 32) continue;  // done above
         const uint32_t cap = DK_SLOTS_PER_TOKEN * (uint32_t)n;
         for (int32_t i = tid; i < bw; i += blockDim.x) bitmap[i] = 0;
         for (uint32_t i = tid; i < cap; i += blockDim.x) table[i] = DK_EMPTY;
