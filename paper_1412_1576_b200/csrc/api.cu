@@ -527,6 +527,10 @@ static int load_common(Ctx& c, const int32_t* words_dev, int64_t n_tokens, const
     c.sc_dense = (unsigned long long*)A((size_t)K * 8 * 3);
     c.red = (double*)A(sizeof(double) * (LL_WORD_PARTIALS + LL_DOC_PARTIALS));
     c.red_i = (int64_t*)A(16);
+    c.ll_tab = (double*)A(sizeof(double) * 2 * 512);
+    c.ll_tile_part = (double*)A(sizeof(double) * std::max<size_t>((size_t)c.n_doc_tiles, 1));
+    c.ll_tile_nnz = (uint32_t*)A(4 * std::max<size_t>((size_t)c.n_doc_tiles, 1));
+    c.ll_tables_ready = false;
     if (!ok) { free_corpus(c); return fail(&c, LDA_ENOMEM, "device allocation failed"); }
     set_slice(c, 0);
     cudaMemsetAsync(v.wk_nnz, 0, (size_t)V * 4, c.stream);

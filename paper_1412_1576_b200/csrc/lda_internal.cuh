@@ -226,6 +226,10 @@ struct Ctx {
     unsigned long long* sc_de = nullptr;  // deficits prefix (front) / surpluses prefix (back)
     uint32_t* sc_item = nullptr;          // light items (front) / heavy items (back)
     unsigned long long* sc_dense = nullptr;  // same three for the dense table, [3*K]
+    double* ll_tab = nullptr;        // [2 * 512] lgamma tables of the log-likelihood's document part
+    double* ll_tile_part = nullptr;  // [n_doc_tiles] its partial sums, one per tile of documents
+    uint32_t* ll_tile_nnz = nullptr; // [n_doc_tiles] filled table slots of the tile: its share of nnz(n_kd)
+    bool ll_tables_ready = false;
     double* red = nullptr;                   // reduction partials for the log-likelihood
     int64_t* red_i = nullptr;
     // device memory comes from cudaMalloc / cudaFree unless lda_set_allocator() gave other routines

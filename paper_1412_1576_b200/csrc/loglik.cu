@@ -52,97 +52,109 @@ __global__ void k_sum_nnz(const int32_t* __restrict__ a, int64_t n, unsigned lon
     if (threadIdx.x == 0 && s) atomicAdd(out, s);
 }
 
-// Document part.  n_kd is not kept between sweeps (the MH step builds it per tile of documents
-// and drops it), so it is built here the same way: a CTA takes tiles of whole documents in turns
-// (tile t, t + gridDim.x, ...: a fixed assignment, so a CTA's partial sum is the same on every
-// run), inserts the tile's topics into the documents' hashed tables in shared memory, and adds up
-// lgamma(n_kd + alpha) - lgamma(alpha) over the filled slots and -lgamma(n_d + K alpha) per document.
-// It also counts the filled slots: nnz(n_kd).
-template <typename T>
-__global__ void __launch_bounds__(1024)
-k_ll_doc_tiles(View v, const int32_t* __restrict__ tiles, int32_t n_tiles, int32_t cap, double lg_alpha,
-               double* __restrict__ out, unsigned long long* __restrict__ nnz_out)
+// Tables of the document part in device memory, filled once per corpus: [0, LL_TABLE) holds
+// lgamma(c + alpha) - lgamma(alpha), [LL_TABLE, 2 LL_TABLE) holds lgamma(n + K alpha).
+__global__ void k_ll_fill_tables(View v, double lg_alpha, double* __restrict__ tab)
 {
-    extern __shared__ __align__(16) uint32_t doc_smem[];  // carved up for tiles of `cap` tokens
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < LL_TABLE; c += gridDim.x * blockDim.x) {
+        tab[c] = lgamma((double)c + v.alpha) - lg_alpha;
+        tab[LL_TABLE + c] = lgamma((double)c + v.Kalpha);
+    }
+}
+
+// lgamma() for the rare count beyond the tables, kept out of line so that the kernel below fits the
+// register budget of a full multiprocessor.
+__device__ __noinline__ double lgamma_out_of_line(double x) { return lgamma(x); }
+
+// Document part.  n_kd is not kept between sweeps (the MH step builds it per tile of documents
+// and drops it), so it is built here the same way and by the same shape of kernel as pass 2 of the
+// MH step: one CTA per tile of whole documents, a thread owns DOC_TILE_ROUNDS tokens, inserts their
+// topics into the documents' hashed tables in shared memory, and the CTA then adds up
+// lgamma(n_kd + alpha) - lgamma(alpha) over the filled slots and -lgamma(n_d + K alpha) per document.
+// One partial sum per tile (a second kernel adds them in a fixed order) and the number of filled
+// slots, nnz(n_kd).
+template <typename T, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1536 / THREADS)
+k_ll_doc_tiles(View v, const int32_t* __restrict__ tiles, double lg_alpha, const double* __restrict__ tab,
+               double* __restrict__ tile_part, uint32_t* __restrict__ tile_nnz)
+{
+    constexpr int cap = DOC_TILE_ROUNDS * THREADS;
+    extern __shared__ __align__(16) uint32_t doc_smem[];
     __shared__ double tmp[32];
-    __shared__ double small[LL_TABLE];
-    uint32_t* slots = doc_smem;
-    int32_t* soff = reinterpret_cast<int32_t*>(slots + DK_SLOTS_PER_TOKEN * cap);
-    uint32_t* topic = reinterpret_cast<uint32_t*>(soff + cap + 1);
-    __shared__ double by_len[LL_TABLE];  // lgamma(n_d + K alpha) for documents shorter than LL_TABLE tokens
-    fill_ll_table(small, v.alpha, lg_alpha);
-    for (int c = threadIdx.x; c < LL_TABLE; c += blockDim.x) by_len[c] = lgamma((double)c + v.Kalpha);
-    __syncthreads();
-    const T* zbm = reinterpret_cast<const T*>(v.zbm);
+    uint32_t* slots = doc_smem;                                                            // [DK_SLOTS_PER_TOKEN * cap]
+    int32_t* soff = reinterpret_cast<int32_t*>(slots + DK_SLOTS_PER_TOKEN * cap);          // [cap + 1]
     const int tid = threadIdx.x;
+    const int32_t s0 = tiles[2 * blockIdx.x], s1 = tiles[2 * blockIdx.x + 1];
+    const int32_t nseg = s1 - s0;
+    const int32_t base = v.doc_off[s0];
+    const int32_t cnt = v.doc_off[s1] - base;
+    const T* zbm = reinterpret_cast<const T*>(v.zbm);
+    uint32_t z[DOC_TILE_ROUNDS];
+#pragma unroll
+    for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
+        const int j = tid + r * THREADS;
+        z[r] = 0;
+        if (j < cnt) z[r] = (uint32_t)__ldcg(zbm + 2 * (size_t)__ldcs(v.bm_of_tok + base + j));
+    }
+    for (int j = tid; j <= nseg; j += THREADS) soff[j] = v.doc_off[s0 + j] - base;
+    const uint4 empty4 = make_uint4(DK_EMPTY, DK_EMPTY, DK_EMPTY, DK_EMPTY);
+    for (int j = tid; j < cnt * (DK_SLOTS_PER_TOKEN / 4); j += THREADS) reinterpret_cast<uint4*>(slots)[j] = empty4;
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
+        const int j = tid + r * THREADS;
+        if (j < cnt) {
+            int lo = 0, hi = nseg;  // last document with soff[doc] <= j
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (soff[mid] <= j) lo = mid; else hi = mid;
+            }
+            const int32_t first = soff[lo], len = soff[lo + 1] - first;
+            if (z[r] >= (uint32_t)v.K) atomicOr(v.err, ERR_TOPIC_RANGE);
+            else if (dk_insert(slots + DK_SLOTS_PER_TOKEN * first, DK_SLOTS_PER_TOKEN * (uint32_t)len, z[r],
+                               v.count_bits) == DK_EMPTY)
+                atomicOr(v.err, ERR_ROW_OVERFLOW);
+        }
+    }
+    __syncthreads();
     const uint32_t cmask = (1u << v.count_bits) - 1u;
     double s = 0.0;
-    unsigned long long filled = 0;
-    // A thread's tokens of a tile (cap = DOC_TILE_ROUNDS x blockDim.x): their block-major indices are
-    // read one tile ahead, so that a tile starts with its gathers already issued side by side.
-    uint32_t bm[DOC_TILE_ROUNDS];
-    auto tile_range = [&](int32_t t, int32_t& s0, int32_t& s1, int32_t& base, int32_t& cnt) {
-        s0 = tiles[2 * t];
-        s1 = tiles[2 * t + 1];
-        base = v.doc_off[s0];
-        cnt = v.doc_off[s1] - base;
-    };
-    auto read_bm = [&](int32_t base, int32_t cnt) {
+    uint32_t filled = 0;
+    for (int j = tid; j < cnt; j += THREADS) {  // a token's worth of slots at a time
+        const uint4 e4 = reinterpret_cast<const uint4*>(slots)[j];
+        const uint32_t e[4] = {e4.x, e4.y, e4.z, e4.w};
 #pragma unroll
-        for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
-            const int j = tid + r * (int)blockDim.x;
-            bm[r] = j < cnt ? __ldcs(v.bm_of_tok + base + j) : 0u;
-        }
-    };
-    int32_t s0 = 0, s1 = 0, base = 0, cnt = 0;
-    if ((int32_t)blockIdx.x < n_tiles) {
-        tile_range(blockIdx.x, s0, s1, base, cnt);
-        read_bm(base, cnt);
-    }
-    for (int32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-        const int32_t nseg = s1 - s0;
-        const int32_t first_doc = s0, tile_base = base, tile_cnt = cnt;
-        uint32_t zt[DOC_TILE_ROUNDS];
-#pragma unroll
-        for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
-            const int j = tid + r * (int)blockDim.x;
-            zt[r] = j < tile_cnt ? (uint32_t)__ldcg(zbm + 2 * (size_t)bm[r]) : 0u;
-        }
-        if (t + (int32_t)gridDim.x < n_tiles) {
-            tile_range(t + gridDim.x, s0, s1, base, cnt);
-            read_bm(base, cnt);
-        }
-#pragma unroll
-        for (int r = 0; r < DOC_TILE_ROUNDS; ++r) {
-            const int j = tid + r * (int)blockDim.x;
-            if (j < tile_cnt) topic[j] = zt[r];
-        }
-        for (int j = tid; j <= nseg; j += blockDim.x) soff[j] = v.doc_off[first_doc + j] - tile_base;
-        for (int j = tid; j < DK_SLOTS_PER_TOKEN * tile_cnt; j += blockDim.x) slots[j] = DK_EMPTY;
-        __syncthreads();
-        // one warp per document: its lanes insert the document's tokens
-        const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-        for (int d = warp; d < nseg; d += nwarps) {
-            const int32_t first = soff[d], len = soff[d + 1] - first;
-            for (int j = first + lane; j < first + len; j += 32) {
-                const uint32_t k = topic[j];
-                if (k >= (uint32_t)v.K) atomicOr(v.err, ERR_TOPIC_RANGE);
-                else if (dk_insert(slots + DK_SLOTS_PER_TOKEN * first, DK_SLOTS_PER_TOKEN * (uint32_t)len, k,
-                                   v.count_bits) == DK_EMPTY)
-                    atomicOr(v.err, ERR_ROW_OVERFLOW);
-            }
-            if (lane == 0 && len > 0) s -= len < LL_TABLE ? by_len[len] : lgamma((double)len + v.Kalpha);
-        }
-        __syncthreads();
-        for (int j = tid; j < DK_SLOTS_PER_TOKEN * tile_cnt; j += blockDim.x) {
-            const uint32_t e = slots[j];
-            if (e != DK_EMPTY) {
-                const uint32_t c = e & cmask;
-                s += c < (uint32_t)LL_TABLE ? small[c] : lgamma((double)c + v.alpha) - lg_alpha;
+        for (int q = 0; q < 4; ++q) {
+            if (e[q] != DK_EMPTY) {
+                const uint32_t c = e[q] & cmask;
+                s += c < (uint32_t)LL_TABLE ? __ldg(tab + c) : lgamma_out_of_line((double)c + v.alpha) - lg_alpha;
                 ++filled;
             }
         }
-        __syncthreads();
+    }
+    for (int d = tid; d < nseg; d += THREADS) {
+        const int32_t len = soff[d + 1] - soff[d];
+        if (len > 0) s -= len < LL_TABLE ? __ldg(tab + LL_TABLE + len) : lgamma_out_of_line((double)len + v.Kalpha);
+    }
+    s = block_reduce_sum<double>(s, tmp);
+    if (tid == 0) tile_part[blockIdx.x] = s;
+    __syncthreads();
+    filled = block_reduce_sum<uint32_t>(filled, reinterpret_cast<uint32_t*>(tmp));
+    if (tid == 0) tile_nnz[blockIdx.x] = filled;
+}
+
+// Adds the tiles' partial sums: CTA b takes the b-th run of `per` consecutive tiles, always in the same order.
+__global__ void __launch_bounds__(256) k_ll_sum_tiles(const double* __restrict__ tile_part,
+                                                      const uint32_t* __restrict__ tile_nnz, int32_t n_tiles, int32_t per,
+                                                      double* __restrict__ out, unsigned long long* __restrict__ nnz_out)
+{
+    __shared__ double tmp[32];
+    const int32_t t0 = blockIdx.x * per, t1 = min(n_tiles, t0 + per);
+    double s = 0.0;
+    unsigned long long filled = 0;
+    for (int32_t t = t0 + threadIdx.x; t < t1; t += blockDim.x) {
+        s += tile_part[t];
+        filled += tile_nnz[t];
     }
     s = block_reduce_sum<double>(s, tmp);
     if (threadIdx.x == 0) out[blockIdx.x] = s;
@@ -196,24 +208,25 @@ k_ll_doc_long(View v, const int32_t* __restrict__ long_docs, int32_t n_long, dou
     if (threadIdx.x == 0 && filled) atomicAdd(nnz_out, filled);
 }
 
-// Grids of the document part: as many CTAs as the GPU holds at once (a CTA that had to wait for a
-// free slot would run its whole share of the tiles after the others, at low occupancy), each taking
-// tiles in turns.
-template <typename T>
-static int doc_ll_resident(const Ctx& c)
-{
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_ll_doc_tiles<T>, c.doc_threads,
-                                                      doc_tile_smem_bytes(c.doc_tile)) != cudaSuccess || per_sm < 1)
-        per_sm = 1;
-    return c.n_sm * per_sm;
-}
-static int doc_ll_grid(const Ctx& c)
-{
-    const int resident = c.wide_topics ? doc_ll_resident<int32_t>(c) : doc_ll_resident<uint16_t>(c);
-    return std::max(1, std::min<int>(c.n_doc_tiles, resident));
-}
+constexpr int LL_TILE_SUMS = 1024;  // partial sums the tiles' sums are folded into
+
 static int long_ll_grid(const Ctx& c) { return std::max(1, std::min<int>(c.n_long_docs, LL_BLOCKS)); }
+
+template <typename T>
+static void launch_ll_tiles_t(Ctx& c, size_t smem, double lg_alpha)
+{
+    switch (c.doc_threads) {
+        case 128: k_ll_doc_tiles<T, 128><<<c.n_doc_tiles, 128, smem, c.stream>>>(c.v, c.doc_tiles, lg_alpha, c.ll_tab, c.ll_tile_part, c.ll_tile_nnz); break;
+        case 256: k_ll_doc_tiles<T, 256><<<c.n_doc_tiles, 256, smem, c.stream>>>(c.v, c.doc_tiles, lg_alpha, c.ll_tab, c.ll_tile_part, c.ll_tile_nnz); break;
+        case 512: k_ll_doc_tiles<T, 512><<<c.n_doc_tiles, 512, smem, c.stream>>>(c.v, c.doc_tiles, lg_alpha, c.ll_tab, c.ll_tile_part, c.ll_tile_nnz); break;
+        default: k_ll_doc_tiles<T, 1024><<<c.n_doc_tiles, 1024, smem, c.stream>>>(c.v, c.doc_tiles, lg_alpha, c.ll_tab, c.ll_tile_part, c.ll_tile_nnz); break;
+    }
+}
+static void launch_ll_tiles(Ctx& c, size_t smem, double lg_alpha)
+{
+    if (c.wide_topics) launch_ll_tiles_t<int32_t>(c, smem, lg_alpha);
+    else launch_ll_tiles_t<uint16_t>(c, smem, lg_alpha);
+}
 
 // Queues the document part: partial sums to part[0 .. number returned), nnz(n_kd) to *nnz_dev (cleared here).
 static int queue_doc_part(Ctx& c, double* part, unsigned long long* nnz_dev)
@@ -222,14 +235,15 @@ static int queue_doc_part(Ctx& c, double* part, unsigned long long* nnz_dev)
     const double lg_alpha = std::lgamma(c.alpha);
     int n = 0;
     if (c.n_doc_tiles) {
-        const int g = std::min(doc_ll_grid(c), LL_DOC_PARTIALS - LL_BLOCKS);
+        if (!c.ll_tables_ready) {
+            k_ll_fill_tables<<<2, 256, 0, c.stream>>>(c.v, lg_alpha, c.ll_tab);
+            c.ll_tables_ready = true;
+        }
         const size_t smem = doc_tile_smem_bytes(c.doc_tile);
-        if (c.wide_topics)
-            k_ll_doc_tiles<int32_t><<<g, c.doc_threads, smem, c.stream>>>(c.v, c.doc_tiles, c.n_doc_tiles, c.doc_tile,
-                                                                         lg_alpha, part, nnz_dev);
-        else
-            k_ll_doc_tiles<uint16_t><<<g, c.doc_threads, smem, c.stream>>>(c.v, c.doc_tiles, c.n_doc_tiles, c.doc_tile,
-                                                                          lg_alpha, part, nnz_dev);
+        launch_ll_tiles(c, smem, lg_alpha);
+        const int per = (c.n_doc_tiles + LL_TILE_SUMS - 1) / LL_TILE_SUMS;
+        const int g = (c.n_doc_tiles + per - 1) / per;
+        k_ll_sum_tiles<<<g, 256, 0, c.stream>>>(c.ll_tile_part, c.ll_tile_nnz, c.n_doc_tiles, per, part, nnz_dev);
         n += g;
     }
     if (c.n_long_docs) {
@@ -259,7 +273,7 @@ int launch_loglik(Ctx& c, double* out3_host)
     out3_host[0] = lw + ld;
     out3_host[1] = lw;
     out3_host[2] = ld;
-    return 2 + (c.n_doc_tiles ? 1 : 0) + (c.n_long_docs ? 1 : 0);
+    return 2 + (c.n_doc_tiles ? 2 : 0) + (c.n_long_docs ? 1 : 0);
 }
 
 // nnz(n_kw) and nnz(n_kd) of the current assignments (the latter by the document part's kernels).
@@ -280,8 +294,8 @@ int launch_count_nnz(Ctx& c, int64_t* nnz_wk_host, int64_t* nnz_dk_host)
 void set_loglik_smem_limits()
 {
     const int doc_bytes = (int)doc_tile_smem_bytes(DOC_TILE_MAX);
-    cudaFuncSetAttribute(k_ll_doc_tiles<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
-    cudaFuncSetAttribute(k_ll_doc_tiles<int32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
+    cudaFuncSetAttribute(k_ll_doc_tiles<uint16_t, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
+    cudaFuncSetAttribute(k_ll_doc_tiles<int32_t, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, doc_bytes);
 }
 
 }  // namespace lda
