@@ -37,10 +37,10 @@ def _host_gib():
     return 0.0
 
 
-def _gpu_and_oracle(c, seed):
+def _gpu_and_oracle(c, seed, options=None):
     """The library loaded from device tensors, the oracle from host copies of the same arrays."""
     import torch
-    g = binding.LightLDA(c.V, c.K, c.alpha, c.beta)
+    g = binding.LightLDA(c.V, c.K, c.alpha, c.beta, options=options)
     g.load_corpus(c.word_ids, c.doc_offsets)
     g.init(seed)
     w = c.word_ids.cpu().numpy()
@@ -114,12 +114,13 @@ def test_large_full_size_sampled_tokens_against_oracle():
 
 def test_mid_full_size_two_whole_sweeps():
     """Config 3 at its full size (99 M tokens, K = 1000, documents of ~330 tokens): two whole oracle sweeps;
-    every token, every count, every alias table and the move counters equal."""
+    every token, every count, every alias table and the move counters equal.  The library runs pass 1 in three
+    vocabulary slices (one slice's alias tables in memory at a time), which must not show."""
     import torch
     if _free_gib() < 12 or _host_gib() < 12:
         pytest.skip("needs 12 GB of device and of host memory")
     c = synth.make("mid", seed=0, device="cuda")
-    g, o, w, off = _gpu_and_oracle(c, 77)
+    g, o, w, off = _gpu_and_oracle(c, 77, options={"alias_slices": 3})
     del c
     torch.cuda.empty_cache()
     for sweep in range(2):
