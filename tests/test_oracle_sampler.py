@@ -591,3 +591,42 @@ def test_each_single_proposal_neglects_one_part_of_the_likelihood():
     assert parts[2, "doc"] > parts[0, "doc"] > parts[1, "doc"]
     # the neglected part is far behind, the other one only a little ahead
     assert parts[0, "word"] - parts[2, "word"] > 5 * (parts[2, "doc"] - parts[0, "doc"])
+
+
+def test_set_assignments_installs_z_and_its_counts(tiny_corpus):
+    """ldaref_set_assignments: the assignments become exactly the given z, every count table becomes the
+    brute-force count of z, the Philox position becomes (seed, sweep) -- shown by continuing, draw for draw, a
+    context that REACHED that position by sweeping -- and a topic outside [0, K) is refused."""
+    c = tiny_corpus
+    rng = np.random.default_rng(17)
+    z = rng.integers(0, c.K, size=c.n_tokens).astype(np.int32)
+    o = _oracle(c, 5)
+    o.sweep(2, 2)                                  # some other state first
+    o.set_assignments(z, 99, 3)
+    assert np.array_equal(o.get_assignments(), z)
+    n_wk, n_dk, n_k, _ = _dense_counts(c, z)
+    assert np.array_equal(o.get_nk(), n_k)
+    for which, dense in ((ldaref.NWK, n_wk), (ldaref.NDK, n_dk)):
+        off, top, cnt = o.get_csr(which)
+        rebuilt = np.zeros_like(dense)
+        for r in range(dense.shape[0]):
+            assert np.all(np.diff(top[off[r]:off[r + 1]]) > 0)          # topics ascending, no duplicates
+            rebuilt[r, top[off[r]:off[r + 1]]] = cnt[off[r]:off[r + 1]]
+        assert np.array_equal(rebuilt, dense) and int(cnt[:off[-1]].min()) >= 1
+    # the counter: a context seeded 99 that has done three sweeps stands at sweep 3 of the same streams; handing
+    # its assignments, seed and sweep number to another context must continue it draw for draw
+    p = _oracle(c, 99)
+    p.sweep(3, 2)
+    zp = p.get_assignments()
+    o.set_assignments(zp, 99, 3)
+    o.sweep(1, 2)
+    p.sweep(1, 2)
+    assert np.array_equal(o.get_assignments(), p.get_assignments())
+    q = _oracle(c, 5)
+    q.set_assignments(zp, 99, 4)                   # another sweep number: other draws
+    q.sweep(1, 2)
+    assert not np.array_equal(q.get_assignments(), p.get_assignments())
+    bad = z.copy()
+    bad[7] = c.K
+    with pytest.raises(Exception):
+        o.set_assignments(bad, 1, 0)
