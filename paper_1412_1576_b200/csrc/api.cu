@@ -188,7 +188,7 @@ void set_slice(Ctx& c, int slice)
 // Buffers the passes of the MH step hand results to each other in; sized by the number of steps.
 int lda::ensure_exchange(Ctx& c, int mh_steps)
 {
-    if (c.N == 0 || (mh_steps <= c.side_steps && c.side_mode == c.proposals && c.v.dside)) return LDA_OK;
+    if (c.N == 0) return LDA_OK;
     auto bytes_for = [&](int mode, int steps, size_t& prop_b, size_t& side_b, size_t& ua_b, int& stride) {
         const size_t zt = c.wide_topics ? 4 : 2, n = (size_t)c.N;
         const int n_word = mode == LDA_PROPOSALS_CYCLE ? (steps + 1) / 2 : mode == LDA_PROPOSALS_WORD ? steps : 0;
@@ -199,9 +199,17 @@ int lda::ensure_exchange(Ctx& c, int mh_steps)
         side_b = 4 * (size_t)stride * n;
         ua_b = 4 * planes * n;
     };
-    cudaStreamSynchronize(c.stream);
     size_t pb = 0, sb = 0, ub = 0;
     int stride = 0;
+    if (mh_steps <= c.side_steps && c.side_mode == c.proposals && c.v.dside) {
+        // buffers laid out for more steps of the same schedule are large enough: only the record
+        // stride follows the step count (a chain of two steps keeps its 16-byte records after a
+        // chain of four has run)
+        bytes_for(c.proposals, mh_steps, pb, sb, ub, stride);
+        c.v.side_stride = stride;
+        return LDA_OK;
+    }
+    cudaStreamSynchronize(c.stream);
     dev_free(c, c.v.prop);
     dev_free(c, c.v.dside);
     dev_free(c, c.v.ua_w);

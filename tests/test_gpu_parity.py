@@ -532,3 +532,15 @@ def test_chunked_transfers_and_async_export(small_corpus):
     o.sweep(1, 2)
     assert np.array_equal(g.get_assignments(), o.get_assignments())
     _assert_same_counts(g, o)
+
+
+def test_step_count_down_and_up_again(small_corpus):
+    """The exchange buffers are laid out for the largest step count seen; a shorter chain afterwards uses the
+    same buffers with its own record size: four steps, two, one, five, two."""
+    c = small_corpus
+    g, o = _pair(c, seed=23)
+    for steps in (4, 2, 1, 5, 2):
+        g.sweep(1, steps)
+        o.sweep(1, steps)
+        assert np.array_equal(g.get_assignments(), o.get_assignments()), steps
+    _assert_same_counts(g, o)
